@@ -1,0 +1,173 @@
+/*
+ * spla.h — C ABI of the SPLA decode-step attention library for NVIDIA B200 (sm_100a).
+ *
+ * SPLA = block Sparse Plus Linear Attention (arXiv 2601.22379).  For every
+ * (sequence, KV head) "unit" one decode step
+ *   1. scores every KV block with the second-order Taylor estimate of its
+ *      attention mass, from the block's key mean and diagonal covariance
+ *      (Section 3.1, Eq. block-score-expand, Eq. taylor-2nd), summed over the
+ *      G query heads of the GQA group after per-head normalisation
+ *      (Section 2.2, grouped BlockScore equation);
+ *   2. selects top_k blocks: forced sink/local blocks plus the best others
+ *      (Section 2.1, Eq. sparse-attn; Section 4 "Sparsity Specifications");
+ *   3. runs exact softmax attention over the selected blocks only
+ *      (Section 2.2, Eq. gqa-sparse);
+ *   4. adds residual linear attention over the unselected blocks by
+ *      subtraction: o_rla = phi(q) S_bar - phi(q) S_tilde, S_bar the global
+ *      recurrent state, S_tilde rebuilt from the selected K/V already on chip
+ *      (Section 3.2, Eq. rla-impl-1..3), phi = softmax over features;
+ *   5. merges: out = o_sparse + RMSNorm(o_rla) (Section 3.3).
+ *
+ * General rules
+ *   - All device buffers are owned by the caller.  The library allocates no
+ *     device memory, frees none, and never synchronises the device except in
+ *     spla_sync_status.  Every call enqueues its work on the given stream
+ *     (a cudaStream_t passed as void*; NULL = the legacy default stream) and
+ *     returns; results are ready when that stream reaches them.
+ *   - Pointers marked DEVICE must be device memory of the current device,
+ *     16-byte aligned (k_cache, v_cache, stats, rla_state, tok_lse and the
+ *     workspace: 256-byte aligned).  Pointers marked HOST are ordinary host
+ *     memory and are read before the call returns.
+ *   - Every function returns SPLA_OK (0) or a negative spla_status_t.
+ *     Argument errors are detected on the host before anything is launched.
+ *     A condition only the device can see (a sequence that would exceed
+ *     max_context) skips the offending work without faulting and latches a
+ *     status word that spla_sync_status reports.
+ *   - Query head m belongs to KV head m / G, G = n_q_heads / n_kv_heads.
+ *   - Order per decode step: spla_append_tokens(k_t, v_t) then
+ *     spla_decode(q_t): the query attends to every cached token, its own
+ *     position included (Section 2, problem statement), and S_bar_t includes
+ *     token t (Eq. rla-impl-1).
+ */
+#ifndef SPLA_H_
+#define SPLA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SPLA_OK = 0,
+  SPLA_ERR_INVALID_ARG = -1,  /* NULL pointer, bad shape, misaligned buffer, workspace too small */
+  SPLA_ERR_CAPACITY = -2,     /* an append would exceed max_context (host- or device-detected) */
+  SPLA_ERR_CUDA = -3,         /* a CUDA runtime call or launch failed; see spla_last_cuda_error */
+  SPLA_ERR_UNSUPPORTED = -4   /* valid request outside what the kernels are built for */
+} spla_status_t;
+
+typedef enum { SPLA_F32 = 0, SPLA_BF16 = 1 } spla_dtype_t;
+
+/* flags */
+#define SPLA_ADOPT_CONTENTS 1u /* spla_init_cache keeps stats / rla_state / tok_lse / seq_lens as they are */
+#define SPLA_FIRST_ORDER 2u    /* block score without the covariance term (Eq. taylor-1st) */
+#define SPLA_NO_RLA 4u         /* out = o_sparse; the residual branch is skipped (the paper's SPA ablation) */
+
+typedef struct {
+  int32_t batch;          /* sequences per call, >= 1 */
+  int32_t n_q_heads;      /* H_q */
+  int32_t n_kv_heads;     /* H_kv; G = H_q / H_kv must be an integer in [1, 16] */
+  int32_t head_dim;       /* d: 64 or 128 */
+  int32_t block_size;     /* B: 16, 32, 64 or 128 tokens */
+  int32_t top_k;          /* k: blocks read per unit per step, 1..64 */
+  int32_t max_context;    /* capacity in tokens per sequence; ceil(max_context / B) <= 32768 */
+  int32_t n_sink_blocks;  /* always-selected initial blocks (paper: 1) */
+  int32_t n_local_blocks; /* always-selected most recent blocks (paper: 4); n_sink + n_local <= top_k */
+  int32_t kv_dtype;       /* spla_dtype_t of k_cache, v_cache, k_new, v_new */
+  int32_t q_dtype;        /* spla_dtype_t of q */
+  float sm_scale;         /* multiplies q in the block score and in exact attention; 0 -> 1/sqrt(d) */
+  float phi_scale;        /* multiplies q and k inside the feature map phi = softmax; 0 -> 1 */
+  float rms_eps;          /* epsilon of the RMSNorm; 0 -> 1e-6 */
+  uint32_t flags;
+} spla_config_t;
+
+/* Device buffers of one cache, all caller-owned.  max_blocks = ceil(max_context / B). */
+typedef struct {
+  void *k_cache;      /* DEVICE [batch][H_kv][max_blocks][B][d] kv_dtype; token t of a unit lives in block t / B */
+  void *v_cache;      /* DEVICE same layout */
+  float *stats;       /* DEVICE [batch][H_kv][max_blocks][2][d] fp32: key mean, then population variance */
+  float *rla_state;   /* DEVICE [batch][H_kv][d][d] fp32 S_bar: row = feature of phi(k), column = value dim */
+  float *tok_lse;     /* DEVICE [batch][H_kv][max_blocks * B] fp32: logsumexp_c(phi_scale * k_t[c]) per token */
+  int32_t *seq_lens;  /* DEVICE [batch]: tokens cached per sequence */
+  void *workspace;    /* DEVICE scratch of at least spla_sizes_t.workspace bytes; contents are the library's */
+  size_t workspace_bytes;
+} spla_buffers_t;
+
+typedef struct {
+  size_t k_cache, v_cache, stats, rla_state, tok_lse, seq_lens, workspace; /* bytes */
+} spla_sizes_t;
+
+typedef struct spla_cache spla_cache_t; /* opaque host-side descriptor */
+
+/* Byte size of every buffer for a configuration.  HOST pointers.  Validates the configuration. */
+int spla_query_sizes(const spla_config_t *config, spla_sizes_t *sizes_out);
+
+/*
+ * Bind caller-owned buffers to a descriptor (the paper's KV cache k_{1:N}, v_{1:N} "retained in memory to be
+ * attended to by all future query vectors", Section 2, together with the block statistics of Section 3.1 and
+ * the recurrent state of Eq. rla-impl-1).  Unless SPLA_ADOPT_CONTENTS is set, stats, rla_state, tok_lse,
+ * seq_lens are zeroed on `stream`; the workspace is always initialised.  K/V contents are never cleared.
+ * config, buffers: HOST, copied.  *cache_out: HOST, receives a descriptor to release with spla_destroy_cache.
+ */
+int spla_init_cache(const spla_config_t *config, const spla_buffers_t *buffers, void *stream, spla_cache_t **cache_out);
+
+/*
+ * Append tokens to every sequence (the cache growth of Section 2 plus the state update of Eq. rla-impl-1 and
+ * the statistics of Eq. taylor-2nd).  For sequence b the first n_new[b] of the max_new provided tokens are
+ * stored at positions seq_lens[b]..; the mean and population variance of every touched block are recomputed
+ * from the cached keys; S_bar += phi(k_t)^T v_t for each new token in fp32; tok_lse is filled; seq_lens[b]
+ * grows by n_new[b].
+ *   k_new, v_new: DEVICE [batch][H_kv][max_new][d] kv_dtype.
+ *   n_new: DEVICE int32 [batch], each in [0, max_new]; NULL means max_new for every sequence.
+ *   max_new >= 1.  Returns SPLA_ERR_CAPACITY (nothing enqueued) if the host-side bound on the longest
+ *   sequence plus max_new exceeds max_context; a sequence that overflows on the device only is skipped and
+ *   reported by spla_sync_status.
+ */
+int spla_append_tokens(spla_cache_t *cache, const void *k_new, const void *v_new, const int32_t *n_new,
+                       int32_t max_new, void *stream);
+
+/*
+ * One decode step for every sequence: steps 1-5 of the file comment.
+ *   q:          DEVICE [batch][H_q][d] q_dtype, unscaled.
+ *   rms_weight: DEVICE [H_q][d] fp32 RMSNorm scale (the only parameters the method adds, Section 3.3);
+ *               may be NULL with SPLA_NO_RLA.
+ *   out:        DEVICE [batch][H_q][d] fp32.
+ *   sel_idx:    DEVICE int32 [batch][H_kv][top_k] or NULL: selected block indices, ascending, padded with -1.
+ *   dbg_o_sparse, dbg_o_rla: DEVICE fp32 [batch][H_q][d] or NULL: the exact-attention output and the
+ *               residual o_bar - o_tilde before the RMSNorm.
+ * A sequence of length 0 yields out = 0.  Unselected blocks' K/V are never read.
+ */
+int spla_decode(spla_cache_t *cache, const void *q, const float *rms_weight, float *out, int32_t *sel_idx,
+                float *dbg_o_sparse, float *dbg_o_rla, void *stream);
+
+/*
+ * Same as spla_decode with the selection given instead of computed (steps 3-5 only): sel_in DEVICE int32
+ * [batch][H_kv][top_k], ascending valid block indices padded with -1.  For testing against an oracle when a
+ * tie makes several index sets correct, and for callers that select elsewhere.
+ */
+int spla_decode_selected(spla_cache_t *cache, const void *q, const float *rms_weight, const int32_t *sel_in,
+                         float *out, float *dbg_o_sparse, float *dbg_o_rla, void *stream);
+
+/* Block scores of the last spla_decode: DEVICE fp32 [batch][H_kv][max_blocks] copy-out (entries >= nblk are 0). */
+int spla_copy_scores(spla_cache_t *cache, float *scores_out, void *stream);
+
+/* Waits for `stream`, then returns and clears the device-latched status (SPLA_OK or SPLA_ERR_CAPACITY). */
+int spla_sync_status(spla_cache_t *cache, void *stream);
+
+/* Tells the library an upper bound of the current sequence lengths after adopting contents (HOST value). */
+int spla_set_length_bound(spla_cache_t *cache, int32_t max_seq_len);
+
+/* Releases the descriptor only; caller buffers are untouched.  NULL is allowed. */
+int spla_destroy_cache(spla_cache_t *cache);
+
+/* Static, NUL-terminated description of a status code. */
+const char *spla_status_string(int status);
+
+/* Text of the last CUDA error this library saw on the calling thread ("" if none). */
+const char *spla_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPLA_H_ */

@@ -1,0 +1,249 @@
+// C ABI of the library: argument validation, workspace carve-up and kernel launches.  Host code only.
+#include <math.h>
+#include <new>
+#include <stdio.h>
+#include <string.h>
+
+#include "../../include/spla.h"
+#include "spla_internal.h"
+
+using namespace spla;
+
+struct spla_cache {
+  spla_config_t cfg;
+  spla_buffers_t buf;
+  Params p;
+  int64_t len_bound;   // host-side upper bound of the longest sequence
+};
+
+static thread_local char g_cuda_err[256] = "";
+
+static int cuda_fail(cudaError_t e, const char* where) {
+  snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", where, cudaGetErrorString(e));
+  return SPLA_ERR_CUDA;
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static int validate_config(const spla_config_t* c) {
+  if (!c) return SPLA_ERR_INVALID_ARG;
+  if (c->batch < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->top_k < 1 || c->max_context < 1)
+    return SPLA_ERR_INVALID_ARG;
+  if (c->n_q_heads % c->n_kv_heads) return SPLA_ERR_INVALID_ARG;
+  if (c->n_sink_blocks < 0 || c->n_local_blocks < 0 || c->n_sink_blocks + c->n_local_blocks > c->top_k)
+    return SPLA_ERR_INVALID_ARG;
+  if ((c->kv_dtype != SPLA_F32 && c->kv_dtype != SPLA_BF16) || (c->q_dtype != SPLA_F32 && c->q_dtype != SPLA_BF16))
+    return SPLA_ERR_INVALID_ARG;
+  if (c->sm_scale < 0.f || c->phi_scale < 0.f || c->rms_eps < 0.f) return SPLA_ERR_INVALID_ARG;
+  if (c->flags & ~(SPLA_ADOPT_CONTENTS | SPLA_FIRST_ORDER | SPLA_NO_RLA)) return SPLA_ERR_INVALID_ARG;
+  const int G = c->n_q_heads / c->n_kv_heads;
+  if (G > kMaxGroup) return SPLA_ERR_UNSUPPORTED;
+  if (c->head_dim != 64 && c->head_dim != 128) return SPLA_ERR_UNSUPPORTED;
+  if (c->block_size != 16 && c->block_size != 32 && c->block_size != 64 && c->block_size != 128)
+    return SPLA_ERR_UNSUPPORTED;
+  if (c->top_k > kMaxTopK) return SPLA_ERR_UNSUPPORTED;
+  const int64_t max_blocks = ((int64_t)c->max_context + c->block_size - 1) / c->block_size;
+  if (max_blocks > kMaxBlocks) return SPLA_ERR_UNSUPPORTED;
+  if ((int64_t)c->batch * c->n_kv_heads > 65535) return SPLA_ERR_UNSUPPORTED;
+  return SPLA_OK;
+}
+
+struct WorkspaceLayout {
+  size_t ell, chunk_part, scores, obar_part, sel, n_sel, att_acc, att_ml, score_ticket, attend_ticket, status, total;
+  int max_chunks;
+};
+
+static WorkspaceLayout workspace_layout(const spla_config_t* c) {
+  WorkspaceLayout w;
+  const size_t U = (size_t)c->batch * c->n_kv_heads, G = c->n_q_heads / c->n_kv_heads, d = c->head_dim;
+  const size_t max_blocks = ((size_t)c->max_context + c->block_size - 1) / c->block_size;
+  w.max_chunks = (int)((max_blocks + kScoreChunk - 1) / kScoreChunk);
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  w.ell = take(U * G * max_blocks * 4);
+  w.chunk_part = take(U * w.max_chunks * G * 2 * 4);
+  w.scores = take(U * max_blocks * 4);
+  w.obar_part = take(U * kStateSplits * G * d * 4);
+  w.sel = take(U * c->top_k * 4);
+  w.n_sel = take(U * 4);
+  w.att_acc = take(U * c->top_k * 2 * G * d * 4);
+  w.att_ml = take(U * c->top_k * G * 2 * 4);
+  w.score_ticket = take(U * 4);
+  w.attend_ticket = take(U * 4);
+  w.status = take(256);
+  w.total = off;
+  return w;
+}
+
+extern "C" int spla_query_sizes(const spla_config_t* config, spla_sizes_t* sizes_out) {
+  int rc = validate_config(config);
+  if (rc) return rc;
+  if (!sizes_out) return SPLA_ERR_INVALID_ARG;
+  const size_t U = (size_t)config->batch * config->n_kv_heads, d = config->head_dim, B = config->block_size;
+  const size_t max_blocks = ((size_t)config->max_context + B - 1) / B;
+  const size_t e = config->kv_dtype == SPLA_BF16 ? 2 : 4;
+  sizes_out->k_cache = U * max_blocks * B * d * e;
+  sizes_out->v_cache = sizes_out->k_cache;
+  sizes_out->stats = U * max_blocks * 2 * d * 4;
+  sizes_out->rla_state = U * d * d * 4;
+  sizes_out->tok_lse = U * max_blocks * B * 4;
+  sizes_out->seq_lens = (size_t)config->batch * 4;
+  sizes_out->workspace = workspace_layout(config).total;
+  return SPLA_OK;
+}
+
+static bool aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+
+extern "C" int spla_init_cache(const spla_config_t* config, const spla_buffers_t* b, void* stream,
+                               spla_cache_t** cache_out) {
+  int rc = validate_config(config);
+  if (rc) return rc;
+  if (!b || !cache_out) return SPLA_ERR_INVALID_ARG;
+  if (!b->k_cache || !b->v_cache || !b->stats || !b->rla_state || !b->tok_lse || !b->seq_lens || !b->workspace)
+    return SPLA_ERR_INVALID_ARG;
+  if (!aligned(b->k_cache, 256) || !aligned(b->v_cache, 256) || !aligned(b->stats, 256) ||
+      !aligned(b->rla_state, 256) || !aligned(b->tok_lse, 256) || !aligned(b->workspace, 256) ||
+      !aligned(b->seq_lens, 4))
+    return SPLA_ERR_INVALID_ARG;
+  spla_sizes_t sz;
+  spla_query_sizes(config, &sz);
+  if (b->workspace_bytes < sz.workspace) return SPLA_ERR_INVALID_ARG;
+
+  spla_cache* c = new (std::nothrow) spla_cache;
+  if (!c) return SPLA_ERR_INVALID_ARG;
+  c->cfg = *config;
+  c->buf = *b;
+  if (c->cfg.sm_scale == 0.f) c->cfg.sm_scale = 1.0f / sqrtf((float)config->head_dim);
+  if (c->cfg.phi_scale == 0.f) c->cfg.phi_scale = 1.0f;
+  if (c->cfg.rms_eps == 0.f) c->cfg.rms_eps = 1e-6f;
+
+  Params& p = c->p;
+  memset(&p, 0, sizeof(p));
+  p.batch = config->batch; p.Hq = config->n_q_heads; p.Hkv = config->n_kv_heads; p.G = p.Hq / p.Hkv;
+  p.d = config->head_dim; p.B = config->block_size; p.top_k = config->top_k;
+  p.max_context = config->max_context;
+  p.max_blocks = (config->max_context + config->block_size - 1) / config->block_size;
+  p.n_sink = config->n_sink_blocks; p.n_local = config->n_local_blocks;
+  p.flags = config->flags; p.kv_bf16 = config->kv_dtype == SPLA_BF16;
+  p.sm_scale = c->cfg.sm_scale; p.phi_scale = c->cfg.phi_scale; p.rms_eps = c->cfg.rms_eps;
+  p.k_cache = b->k_cache; p.v_cache = b->v_cache; p.stats = b->stats; p.state = b->rla_state;
+  p.tok_lse = b->tok_lse; p.seq_lens = b->seq_lens;
+  const WorkspaceLayout w = workspace_layout(config);
+  char* ws = reinterpret_cast<char*>(b->workspace);
+  p.ell = (float*)(ws + w.ell); p.chunk_part = (float*)(ws + w.chunk_part); p.scores = (float*)(ws + w.scores);
+  p.obar_part = (float*)(ws + w.obar_part); p.sel = (int*)(ws + w.sel); p.n_sel = (int*)(ws + w.n_sel);
+  p.att_acc = (float*)(ws + w.att_acc); p.att_ml = (float*)(ws + w.att_ml);
+  p.score_ticket = (int*)(ws + w.score_ticket); p.attend_ticket = (int*)(ws + w.attend_ticket);
+  p.status = (int*)(ws + w.status);
+  p.max_chunks = w.max_chunks;
+
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaError_t e = cudaMemsetAsync(b->workspace, 0, w.total, s);
+  if (e == cudaSuccess && !(config->flags & SPLA_ADOPT_CONTENTS)) {
+    e = cudaMemsetAsync(b->stats, 0, sz.stats, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(b->rla_state, 0, sz.rla_state, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(b->tok_lse, 0, sz.tok_lse, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(b->seq_lens, 0, sz.seq_lens, s);
+    c->len_bound = 0;
+  } else {
+    c->len_bound = config->max_context;   // adopted contents: lengths unknown to the host until told
+  }
+  if (e != cudaSuccess) {
+    delete c;
+    return cuda_fail(e, "spla_init_cache");
+  }
+  *cache_out = c;
+  return SPLA_OK;
+}
+
+extern "C" int spla_set_length_bound(spla_cache_t* c, int32_t max_seq_len) {
+  if (!c || max_seq_len < 0 || max_seq_len > c->cfg.max_context) return SPLA_ERR_INVALID_ARG;
+  c->len_bound = max_seq_len;
+  return SPLA_OK;
+}
+
+extern "C" int spla_append_tokens(spla_cache_t* c, const void* k_new, const void* v_new, const int32_t* n_new,
+                                  int32_t max_new, void* stream) {
+  if (!c || !k_new || !v_new || max_new < 1) return SPLA_ERR_INVALID_ARG;
+  if (!aligned(k_new, 16) || !aligned(v_new, 16)) return SPLA_ERR_INVALID_ARG;
+  if (c->len_bound + max_new > c->cfg.max_context) return SPLA_ERR_CAPACITY;
+  cudaError_t e = launch_append(c->p, k_new, v_new, n_new, max_new, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e, "spla_append_tokens");
+  c->len_bound += max_new;
+  return SPLA_OK;
+}
+
+static int chunks_for_bound(const spla_cache* c) {
+  const int64_t blocks = (c->len_bound + c->cfg.block_size - 1) / c->cfg.block_size;
+  const int64_t ch = (blocks + kScoreChunk - 1) / kScoreChunk;
+  return (int)(ch < 1 ? 1 : ch);
+}
+
+extern "C" int spla_decode(spla_cache_t* c, const void* q, const float* rms_weight, float* out, int32_t* sel_idx,
+                           float* dbg_o_sparse, float* dbg_o_rla, void* stream) {
+  if (!c || !q || !out) return SPLA_ERR_INVALID_ARG;
+  if (!rms_weight && !(c->cfg.flags & SPLA_NO_RLA)) return SPLA_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(out, 16)) return SPLA_ERR_INVALID_ARG;
+  Params p = c->p;
+  p.n_chunks_cap = chunks_for_bound(c);
+  const int qb = c->cfg.q_dtype == SPLA_BF16;
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaError_t e = launch_score_select(p, q, qb, sel_idx, s);
+  if (e != cudaSuccess) return cuda_fail(e, "spla_decode/score_select");
+  e = launch_attend_merge(p, q, qb, rms_weight, nullptr, out, dbg_o_sparse, dbg_o_rla, s);
+  if (e != cudaSuccess) return cuda_fail(e, "spla_decode/attend_merge");
+  return SPLA_OK;
+}
+
+extern "C" int spla_decode_selected(spla_cache_t* c, const void* q, const float* rms_weight, const int32_t* sel_in,
+                                    float* out, float* dbg_o_sparse, float* dbg_o_rla, void* stream) {
+  if (!c || !q || !out || !sel_in) return SPLA_ERR_INVALID_ARG;
+  if (!rms_weight && !(c->cfg.flags & SPLA_NO_RLA)) return SPLA_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(out, 16)) return SPLA_ERR_INVALID_ARG;
+  Params p = c->p;
+  p.n_chunks_cap = 0;                      // only the o_bar CTAs of the first kernel run
+  const int qb = c->cfg.q_dtype == SPLA_BF16;
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaError_t e = cudaSuccess;
+  if (!(c->cfg.flags & SPLA_NO_RLA)) e = launch_score_select(p, q, qb, nullptr, s);
+  if (e != cudaSuccess) return cuda_fail(e, "spla_decode_selected/o_bar");
+  e = launch_attend_merge(p, q, qb, rms_weight, sel_in, out, dbg_o_sparse, dbg_o_rla, s);
+  if (e != cudaSuccess) return cuda_fail(e, "spla_decode_selected/attend_merge");
+  return SPLA_OK;
+}
+
+extern "C" int spla_copy_scores(spla_cache_t* c, float* scores_out, void* stream) {
+  if (!c || !scores_out) return SPLA_ERR_INVALID_ARG;
+  const size_t bytes = (size_t)c->p.batch * c->p.Hkv * c->p.max_blocks * sizeof(float);
+  cudaError_t e = cudaMemcpyAsync(scores_out, c->p.scores, bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)stream);
+  return e == cudaSuccess ? SPLA_OK : cuda_fail(e, "spla_copy_scores");
+}
+
+extern "C" int spla_sync_status(spla_cache_t* c, void* stream) {
+  if (!c) return SPLA_ERR_INVALID_ARG;
+  int st = 0;
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaError_t e = cudaMemcpyAsync(&st, c->p.status, sizeof(int), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e == cudaSuccess && st != 0) e = cudaMemsetAsync(c->p.status, 0, sizeof(int), s);
+  if (e != cudaSuccess) return cuda_fail(e, "spla_sync_status");
+  return st;
+}
+
+extern "C" int spla_destroy_cache(spla_cache_t* c) {
+  delete c;
+  return SPLA_OK;
+}
+
+extern "C" const char* spla_status_string(int status) {
+  switch (status) {
+    case SPLA_OK: return "ok";
+    case SPLA_ERR_INVALID_ARG: return "invalid argument";
+    case SPLA_ERR_CAPACITY: return "cache capacity exceeded";
+    case SPLA_ERR_CUDA: return "CUDA error";
+    case SPLA_ERR_UNSUPPORTED: return "unsupported configuration";
+    default: return "unknown status";
+  }
+}
+
+extern "C" const char* spla_last_cuda_error(void) { return g_cuda_err; }

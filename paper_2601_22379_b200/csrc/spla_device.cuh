@@ -1,0 +1,158 @@
+// Device-side helpers shared by the SPLA kernels: parameter block, type loads,
+// warp reductions, mbarrier + bulk-copy (TMA) wrappers for sm_100a.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace spla {
+
+constexpr int kScoreThreads = 256;      // block-score kernel: 8 warps, one block record per warp at a time
+constexpr int kScoreChunk = 64;         // block records per CTA
+constexpr int kStateSplits = 4;         // CTAs per unit that compute o_bar = phi(q) S_bar
+constexpr int kAttendThreads = 128;     // sparse-attend kernel: 4 warps per selected block
+constexpr int kMaxGroup = 16;
+constexpr int kMaxTopK = 64;
+constexpr int kMaxBlocks = 32768;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// Everything a kernel needs, passed by value.
+struct Params {
+  int batch, Hq, Hkv, G, d, B, top_k, max_blocks, max_context, n_sink, n_local;
+  unsigned flags;
+  int kv_bf16;                          // K/V cache element type: 1 = bf16, 0 = fp32
+  float sm_scale, phi_scale, rms_eps;
+  int n_chunks_cap;                     // score-kernel chunks launched per unit
+  // caller buffers
+  void* k_cache;
+  void* v_cache;
+  float* stats;
+  float* state;
+  float* tok_lse;
+  int* seq_lens;
+  // workspace regions
+  float* ell;          // [U][G][max_blocks]      Taylor log-mass per head and block
+  float* chunk_part;   // [U][max_chunks][G][2]   per-chunk (max, sum exp) of ell, natural log domain
+  float* scores;       // [U][max_blocks]         aggregated BlockScore
+  float* obar_part;    // [U][kStateSplits][G][d] partial phi(q) S_bar
+  int* sel;            // [U][top_k]
+  int* n_sel;          // [U]
+  float* att_acc;      // [U][top_k][2][G][d]     per selected block: softmax numerator, then linear term
+  float* att_ml;       // [U][top_k][G][2]        per selected block: (max, sum) in log2 domain
+  int* score_ticket;   // [U]
+  int* attend_ticket;  // [U]
+  int* status;         // [1]
+  int max_chunks;
+};
+
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// Loads VEC consecutive elements starting at p (aligned to VEC * sizeof(T)) as floats.
+template <int VEC>
+__device__ __forceinline__ void load_vec(const float* p, float (&out)[VEC]) {
+  if constexpr (VEC == 4) {
+    float4 v = *reinterpret_cast<const float4*>(p);
+    out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+  } else if constexpr (VEC == 2) {
+    float2 v = *reinterpret_cast<const float2*>(p);
+    out[0] = v.x; out[1] = v.y;
+  } else {
+    out[0] = *p;
+  }
+}
+template <int VEC>
+__device__ __forceinline__ void load_vec(const __nv_bfloat16* p, float (&out)[VEC]) {
+  if constexpr (VEC == 4) {
+    uint2 raw = *reinterpret_cast<const uint2*>(p);
+    out[0] = __uint_as_float(raw.x << 16); out[1] = __uint_as_float(raw.x & 0xffff0000u);
+    out[2] = __uint_as_float(raw.y << 16); out[3] = __uint_as_float(raw.y & 0xffff0000u);
+  } else if constexpr (VEC == 2) {
+    uint32_t raw = *reinterpret_cast<const uint32_t*>(p);
+    out[0] = __uint_as_float(raw << 16); out[1] = __uint_as_float(raw & 0xffff0000u);
+  } else {
+    out[0] = __bfloat162float(*p);
+  }
+}
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Sums N (a power of two, <= 32) per-lane values across the warp with N - 1 + log2(32 / N) shuffles instead
+// of 5 N: each halving step keeps one half of the values and hands the other half to the partner lane.
+// On return v[0] of lane l holds the warp total of the input value with index l / (32 / N).
+template <int N>
+__device__ __forceinline__ void warp_reduce_multi(float (&v)[N], int lane) {
+  static_assert(N >= 1 && N <= 32 && (N & (N - 1)) == 0, "N must be a power of two <= 32");
+  int off = 16;
+#pragma unroll
+  for (int n = N; n > 1; n >>= 1) {
+    const bool upper = (lane & off) != 0;
+#pragma unroll
+    for (int i = 0; i < n / 2; ++i) {
+      const float send = upper ? v[i] : v[i + n / 2];
+      const float keep = upper ? v[i + n / 2] : v[i];
+      v[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+    }
+    off >>= 1;
+  }
+#pragma unroll
+  for (; off > 0; off >>= 1) v[0] += __shfl_xor_sync(0xffffffffu, v[0], off);
+}
+
+// ---- mbarrier + bulk async copy (TMA, untiled) -------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Global -> shared bulk copy; src, dst 16-byte aligned, bytes a multiple of 16.  Never multicast.
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+// Bounded wait: returns false if the phase did not complete within the iteration limit.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  const uint32_t addr = smem_u32(bar);
+  for (int it = 0; it < (1 << 22); ++it) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(addr), "r"(parity)
+        : "memory");
+    if (done) return true;
+    if (it > 64) __nanosleep(64);
+  }
+  return false;
+}
+
+// Programmatic dependent launch: wait for the preceding grid's memory, allow the next grid to start.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+}  // namespace spla

@@ -1,0 +1,26 @@
+// Host-side declarations shared by the translation units of the library (not part of the public ABI).
+#pragma once
+
+#include "spla_device.cuh"
+
+namespace spla {
+
+// GQA group sizes are padded to the next power of two inside the kernels; padded heads carry zero queries
+// and are never written out.
+inline int padded_group(int G) {
+  int gp = 1;
+  while (gp < G) gp <<= 1;
+  return gp;
+}
+
+// score_select.cu
+cudaError_t launch_score_select(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream);
+// attend_merge.cu
+cudaError_t launch_attend_merge(const Params& p, const void* q, int q_is_bf16, const float* rms_weight,
+                                const int* sel_in, float* out, float* dbg_o_sparse, float* dbg_o_rla,
+                                cudaStream_t stream);
+// append.cu
+cudaError_t launch_append(const Params& p, const void* k_new, const void* v_new, const int* n_new, int max_new,
+                          cudaStream_t stream);
+
+}  // namespace spla

@@ -1,0 +1,361 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the float64 oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import spla_oracle as O
+from paper_2601_22379_b200 import binding, runner, synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _decode_all(cache, w, q, gamma):
+    cfg = cache.cfg
+    sel = cache.new_sel_buffer()
+    osp = torch.empty(cfg.batch, cfg.n_q_heads, cfg.head_dim, dtype=torch.float32, device=DEV)
+    orla = torch.empty_like(osp)
+    out = cache.decode(q, gamma, sel_idx=sel, dbg_o_sparse=osp, dbg_o_rla=orla)
+    torch.cuda.synchronize()
+    assert cache.sync_status() == 0
+    return out.cpu().numpy(), osp.cpu().numpy(), orla.cpu().numpy(), sel.cpu().numpy()
+
+
+def _check_units(w, cache, q, gamma, K, V, lens, units, n_sink, n_local, extra=None, order=2, use_rla=True):
+    """extra: optional dict (b,h) -> (K_tail, V_tail) of appended tokens."""
+    out, osp, orla, sel = _decode_all(cache, w, q, gamma)
+    n_exact = 0
+    for (b, h) in units:
+        L = int(lens[b])
+        Ku, Vu = K[b, h, :L], V[b, h, :L]
+        if extra is not None:
+            Ku = torch.cat([Ku, extra[(b, h)][0]], dim=0)
+            Vu = torch.cat([Vu, extra[(b, h)][1]], dim=0)
+
+        def run(override=None):
+            return parity.oracle_unit(w, q[b], Ku, Vu, gamma, h, n_sink=n_sink, n_local=n_local, override=override,
+                                      order=order, use_rla=use_rla)
+        res = run()
+        n_exact += parity.compare_unit(w, res, out[b], osp[b], orla[b], sel[b, h], h, n_sink=n_sink, n_local=n_local,
+                                       rerun=run)
+    return n_exact
+
+
+def _all_units(w):
+    return [(b, h) for b in range(w.batch) for h in range(w.n_kv_heads)]
+
+
+# ---------------------------------------------------------------------------------------------------------
+# append: statistics, state, per-token lse, lengths
+# ---------------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name,ctx", [("tiny_ref", 64 * 9 + 17), ("gqa_32k", 64 * 11 + 5)])
+def test_append_statistics_and_state_match_oracle(name, ctx):
+    w = synth.BY_NAME[name].scaled(batch=2, context=ctx, n_needles=0)
+    cache, K, V, lens = runner.build_cache(w, DEV)
+    torch.cuda.synchronize()
+    assert cache.sync_status() == 0
+    assert cache.bufs.seq_lens.cpu().tolist() == [ctx, ctx]
+    nblk = -(-ctx // w.block_size)
+    for b in range(w.batch):
+        for h in range(w.n_kv_heads):
+            Kd, Vd = K[b, h].double().cpu().numpy(), V[b, h].double().cpu().numpy()
+            mean, var, n = O.block_statistics(Kd, w.block_size)
+            st = cache.bufs.stats[b, h, :nblk].cpu().numpy()
+            assert parity.rel_l2(st[:, 0], mean) < 2e-6 and parity.rel_l2(st[:, 1], var) < 2e-6
+            S = cache.bufs.rla_state[b, h].cpu().numpy()
+            assert parity.rel_l2(S, O.rla_global_state(Kd, Vd)) < 2e-6
+            lse = cache.bufs.tok_lse[b, h, :ctx].cpu().numpy()
+            ref = np.log(np.sum(np.exp(Kd - Kd.max(axis=1, keepdims=True)), axis=1)) + Kd.max(axis=1)
+            assert np.max(np.abs(lse - ref)) < 2e-5
+            kc = cache.bufs.k_cache[b, h].reshape(-1, w.head_dim)[:ctx]
+            assert torch.equal(kc, K[b, h]) and torch.equal(cache.bufs.v_cache[b, h].reshape(-1, w.head_dim)[:ctx], V[b, h])
+    # chunked and token-by-token appends give the same statistics bit for bit, and the same state to rounding
+    cache2, _, _, _ = runner.build_cache(w, DEV, chunk=100, prefill=(K, V, lens))
+    torch.cuda.synchronize()
+    assert torch.equal(cache2.bufs.stats[:, :, :nblk], cache.bufs.stats[:, :, :nblk])
+    assert torch.equal(cache2.bufs.tok_lse[:, :, :ctx], cache.bufs.tok_lse[:, :, :ctx])
+    assert parity.rel_l2(cache2.bufs.rla_state.cpu().numpy(), cache.bufs.rla_state.cpu().numpy()) < 2e-6
+
+
+def test_ragged_append_with_device_lengths():
+    w = synth.BY_NAME["ragged_serving"].scaled(batch=5, context=1500, context_min=1, n_steps=4)
+    cache, K, V, lens = runner.build_cache(w, DEV, chunk=333)
+    torch.cuda.synchronize()
+    assert torch.equal(cache.bufs.seq_lens, lens)
+    for b in range(w.batch):
+        L = int(lens[b])
+        nblk = -(-L // w.block_size)
+        mean, var, _ = O.block_statistics(K[b, 3, :L].double().cpu().numpy(), w.block_size)
+        st = cache.bufs.stats[b, 3, :nblk].cpu().numpy()
+        assert parity.rel_l2(st[:, 0], mean) < 2e-6 and parity.rel_l2(st[:, 1], var) < 2e-6
+
+
+# ---------------------------------------------------------------------------------------------------------
+# decode on scaled-down versions of the five configurations: every unit, ragged tails, forced-block variants
+# ---------------------------------------------------------------------------------------------------------
+SMALL = [
+    ("tiny_ref", dict(context=64 * 20 + 13)),
+    ("gqa_32k", dict(batch=2, context=64 * 70 + 31)),
+    ("long_128k", dict(batch=1, context=64 * 150 + 1, n_steps=2)),
+    ("very_long_1m", dict(context=128 * 140 + 77, n_needles=4)),
+    ("ragged_serving", dict(batch=6, context=6000, context_min=300, n_steps=2)),
+]
+
+
+@pytest.mark.parametrize("name,over", SMALL)
+@pytest.mark.parametrize("forced", [(1, 4), (0, 0), (1, 1)])
+def test_decode_matches_oracle_small(name, over, forced):
+    w = synth.BY_NAME[name].scaled(**over)
+    n_sink, n_local = forced
+    cache, K, V, lens = runner.build_cache(w, DEV, n_sink=n_sink, n_local=n_local)
+    gamma = synth.gamma(w).to(DEV)
+    q = synth.step_queries(w, 0, DEV)
+    lens_h = lens.cpu().numpy()
+    n_exact = _check_units(w, cache, q, gamma, K, V, lens_h, _all_units(w), n_sink, n_local)
+    assert n_exact >= 0.9 * w.batch * w.n_kv_heads        # tie-band swaps are rare
+
+
+def test_decode_steps_with_append_small():
+    """Append one token then decode, across a block boundary; every unit checked at every step."""
+    w = synth.BY_NAME["long_128k"].scaled(batch=2, context=64 * 40 + 62, n_steps=5)
+    cache, K, V, lens = runner.build_cache(w, DEV)
+    gamma = synth.gamma(w).to(DEV)
+    lens_h = lens.cpu().numpy()
+    extra = {u: (torch.zeros(0, w.head_dim, dtype=w.torch_dtype, device=DEV),) * 2 for u in _all_units(w)}
+    for step in range(w.n_steps):
+        k1, v1 = synth.step_kv(w, step, DEV)
+        cache.append_tokens(k1, v1)
+        for (b, h) in extra:
+            extra[(b, h)] = (torch.cat([extra[(b, h)][0], k1[b, h]]), torch.cat([extra[(b, h)][1], v1[b, h]]))
+        q = synth.step_queries(w, step, DEV)
+        _check_units(w, cache, q, gamma, K, V, lens_h, _all_units(w), w.n_sink, w.n_local, extra=extra)
+    assert cache.bufs.seq_lens.cpu().tolist() == [w.context + w.n_steps] * w.batch
+
+
+# ---------------------------------------------------------------------------------------------------------
+# the five configurations at full size, in the launch configuration the benchmark times; sampled units
+# ---------------------------------------------------------------------------------------------------------
+def _sample_units(w, n, seed=0):
+    rng = np.random.default_rng(seed)
+    allu = _all_units(w)
+    idx = rng.permutation(len(allu))[:n]
+    return [allu[i] for i in idx]
+
+
+def test_config1_tiny_ref_full_16_steps():
+    w = synth.CONFIGS[0]
+    cache, K, V, lens = runner.build_cache(w, DEV)
+    gamma = synth.gamma(w).to(DEV)
+    lens_h = lens.cpu().numpy()
+    extra = {(0, 0): (torch.zeros(0, w.head_dim, device=DEV), torch.zeros(0, w.head_dim, device=DEV))}
+    needles = set(synth.needle_blocks(w)[0, 0].tolist())
+    for step in range(w.n_steps):
+        k1, v1 = synth.step_kv(w, step, DEV)
+        cache.append_tokens(k1, v1)
+        extra[(0, 0)] = (torch.cat([extra[(0, 0)][0], k1[0, 0]]), torch.cat([extra[(0, 0)][1], v1[0, 0]]))
+        q = synth.step_queries(w, step, DEV)
+        _check_units(w, cache, q, gamma, K, V, lens_h, [(0, 0)], w.n_sink, w.n_local, extra=extra)
+        sel = cache.new_sel_buffer()
+        cache.decode(q, gamma, sel_idx=sel)
+        assert needles <= set(sel.cpu().numpy()[0, 0].tolist())
+
+
+def test_config2_gqa_32k_full_three_query_seeds():
+    w = synth.CONFIGS[1]
+    cache, K, V, lens = runner.build_cache(w, DEV)
+    gamma = synth.gamma(w).to(DEV)
+    lens_h = lens.cpu().numpy()
+    nb = synth.needle_blocks(w)
+    for seed in range(3):
+        q = synth.step_queries(w, seed, DEV)
+        units = _sample_units(w, 4, seed)
+        _check_units(w, cache, q, gamma, K, V, lens_h, units, w.n_sink, w.n_local)
+        sel = cache.new_sel_buffer()
+        cache.decode(q, gamma, sel_idx=sel)
+        sel = sel.cpu().numpy()
+        for b in range(w.batch):
+            for h in range(w.n_kv_heads):
+                assert set(nb[b, h].tolist()) <= set(sel[b, h].tolist())
+
+
+def _stepped_full(w, n_units, check_steps):
+    cache, K, V, lens = runner.build_cache(w, DEV)
+    gamma = synth.gamma(w).to(DEV)
+    gam = gamma.double().cpu().numpy()
+    lens_h = lens.cpu().numpy()
+    units = _sample_units(w, n_units, 1)
+    G = w.group
+    orc = {}
+    for (b, h) in units:
+        L = int(lens_h[b])
+        orc[(b, h)] = O.UnitCache.from_prefill(K[b, h, :L].double().cpu().numpy(), V[b, h, :L].double().cpu().numpy(),
+                                               w.block_size)
+    del K, V
+    for step in range(w.n_steps):
+        k1, v1 = synth.step_kv(w, step, DEV)
+        cache.append_tokens(k1, v1)
+        for (b, h), oc in orc.items():
+            oc.append(k1[b, h].double().cpu().numpy(), v1[b, h].double().cpu().numpy())
+        if step not in check_steps:
+            continue
+        q = synth.step_queries(w, step, DEV)
+        out, osp, orla, sel = _decode_all(cache, w, q, gamma)
+        qh = q.double().cpu().numpy()
+        for (b, h), oc in orc.items():
+            def run(override=None):
+                return oc.decode(qh[b, h * G:(h + 1) * G], gam[h * G:(h + 1) * G], top_k=w.top_k, n_sink=w.n_sink,
+                                 n_local=w.n_local, override_selection=override)
+            parity.compare_unit(w, run(), out[b], osp[b], orla[b], sel[b, h], h, n_sink=w.n_sink, n_local=w.n_local,
+                                rerun=run)
+    torch.cuda.synchronize()
+    assert cache.sync_status() == 0
+    assert torch.equal(cache.bufs.seq_lens.cpu(), torch.as_tensor(lens_h) + w.n_steps)
+
+
+def test_config3_long_128k_full_64_steps():
+    _stepped_full(synth.CONFIGS[2], n_units=3, check_steps={0, 1, 31, 62, 63})
+
+
+def test_config4_very_long_1m_full():
+    w = synth.CONFIGS[3]
+    cache, K, V, lens = runner.build_cache(w, DEV)
+    gamma = synth.gamma(w).to(DEV)
+    q = synth.step_queries(w, 0, DEV)
+    _check_units(w, cache, q, gamma, K, V, lens.cpu().numpy(), _sample_units(w, 2, 4), w.n_sink, w.n_local)
+
+
+def test_config5_ragged_serving_full_256_steps():
+    _stepped_full(synth.CONFIGS[4], n_units=4, check_steps={0, 63, 64, 255})
+
+
+# ---------------------------------------------------------------------------------------------------------
+# edge and degenerate cases
+# ---------------------------------------------------------------------------------------------------------
+def test_fewer_blocks_than_top_k_is_dense_attention():
+    w = synth.BY_NAME["gqa_32k"].scaled(batch=1, context=64 * 5 + 9, n_needles=0, top_k=16)
+    cache, K, V, lens = runner.build_cache(w, DEV)
+    gamma = synth.gamma(w).to(DEV)
+    q = synth.step_queries(w, 0, DEV)
+    out, osp, orla, sel = _decode_all(cache, w, q, gamma)
+    assert sel[0, 0].tolist() == [0, 1, 2, 3, 4, 5] + [-1] * 10
+    G = w.group
+    for h in range(w.n_kv_heads):
+        dense = torch.nn.functional.scaled_dot_product_attention(
+            q[0, h * G:(h + 1) * G].double()[None], K[0, h].double()[None], V[0, h].double()[None])[0].cpu().numpy()
+        parity.check_outputs("o_sparse", osp[0, h * G:(h + 1) * G], dense, "bf16")
+        obar = parity.oracle_unit(w, q[0], K[0, h], V[0, h], gamma, h, n_sink=1, n_local=4)["o_bar"]
+        # everything selected: the residual is rounding noise relative to the global term
+        assert np.abs(orla[0, h * G:(h + 1) * G]).max() < 5e-3 * np.abs(obar).max()
+
+
+def test_empty_and_one_token_sequences():
+    w = synth.BY_NAME["ragged_serving"].scaled(batch=3, context=200, context_min=200, n_steps=2)
+    cache = binding.SplaCache(runner.config_for(w), DEV)
+    gamma = synth.gamma(w).to(DEV)
+    q = synth.step_queries(w, 0, DEV)
+    out, osp, orla, sel = _decode_all(cache, w, q, gamma)
+    assert np.all(out == 0) and np.all(sel == -1)
+    # sequence 0 stays empty, 1 gets one token, 2 gets 130 tokens
+    K, V, _ = runner.generate_prefill(w, DEV)
+    n_new = torch.tensor([0, 1, 130], dtype=torch.int32, device=DEV)
+    cache.append_tokens(K, V, n_new)
+    out, osp, orla, sel = _decode_all(cache, w, q, gamma)
+    assert np.all(out[0] == 0) and np.all(sel[0] == -1)
+    assert np.all(sel[1, :, 0] == 0) and np.all(sel[1, :, 1:] == -1)
+    # one token: softmax over a single token returns its value; the residual branch vanishes
+    np.testing.assert_allclose(osp[1].reshape(8, 4, -1), np.repeat(V[1, :, :1].float().cpu().numpy(), 4, axis=1), atol=1e-6)
+    lens = np.array([0, 1, 130])
+    _check_units(w, cache, q, gamma, K, V, lens, [(2, h) for h in range(8)], w.n_sink, w.n_local)
+
+
+@pytest.mark.parametrize("hq,hkv", [(1, 1), (2, 1), (5, 1), (8, 1), (16, 1), (6, 2)])
+def test_group_sizes(hq, hkv):
+    w = synth.BY_NAME["gqa_32k"].scaled(batch=1, n_q_heads=hq, n_kv_heads=hkv, context=64 * 40 + 3, n_needles=3)
+    cache, K, V, lens = runner.build_cache(w, DEV)
+    gamma = synth.gamma(w).to(DEV)
+    q = synth.step_queries(w, 0, DEV)
+    _check_units(w, cache, q, gamma, K, V, lens.cpu().numpy(), _all_units(w), w.n_sink, w.n_local)
+
+
+@pytest.mark.parametrize("B,d,dt", [(16, 64, "bf16"), (32, 128, "f32"), (128, 64, "f32"), (128, 128, "bf16"), (64, 64, "bf16")])
+def test_block_sizes_head_dims_dtypes(B, d, dt):
+    w = synth.BY_NAME["gqa_32k"].scaled(batch=1, n_q_heads=4, n_kv_heads=2, head_dim=d, block_size=B, kv_dtype=dt,
+                                       context=B * 33 + B // 2, n_needles=2, top_k=8, n_outlier_channels=2)
+    cache, K, V, lens = runner.build_cache(w, DEV)
+    gamma = synth.gamma(w).to(DEV)
+    q = synth.step_queries(w, 0, DEV)
+    _check_units(w, cache, q, gamma, K, V, lens.cpu().numpy(), _all_units(w), w.n_sink, w.n_local)
+
+
+def test_first_order_and_no_rla_flags():
+    w = synth.BY_NAME["gqa_32k"].scaled(batch=1, context=64 * 60 + 20, n_needles=3)
+    gamma = synth.gamma(w).to(DEV)
+    q = synth.step_queries(w, 0, DEV)
+    cache, K, V, lens = runner.build_cache(w, DEV, flags=binding.SPLA_FIRST_ORDER)
+    _check_units(w, cache, q, gamma, K, V, lens.cpu().numpy(), _all_units(w), w.n_sink, w.n_local, order=1)
+    cache2, _, _, _ = runner.build_cache(w, DEV, flags=binding.SPLA_NO_RLA, prefill=(K, V, lens))
+    out, osp, orla, sel = _decode_all(cache2, w, q, gamma)
+    assert np.array_equal(out, osp)
+    for h in range(w.n_kv_heads):
+        res = parity.oracle_unit(w, q[0], K[0, h], V[0, h], gamma, h, n_sink=w.n_sink, n_local=w.n_local, use_rla=False)
+        if parity.check_selection(sel[0, h], res, w.top_k, w.n_sink, w.n_local):
+            parity.check_outputs("out", out[0, h * 4:(h + 1) * 4], res["out"], "bf16")
+
+
+def test_decode_selected_uses_the_given_blocks():
+    w = synth.BY_NAME["gqa_32k"].scaled(batch=2, context=64 * 30 + 7, n_needles=0, top_k=6)
+    cache, K, V, lens = runner.build_cache(w, DEV)
+    gamma = synth.gamma(w).to(DEV)
+    q = synth.step_queries(w, 0, DEV)
+    rng = np.random.default_rng(5)
+    sel = np.full((w.batch, w.n_kv_heads, w.top_k), -1, dtype=np.int32)
+    for b in range(w.batch):
+        for h in range(w.n_kv_heads):
+            n = int(rng.integers(1, w.top_k + 1))
+            sel[b, h, :n] = np.sort(rng.permutation(31)[:n])
+    osp = torch.empty(w.batch, w.n_q_heads, w.head_dim, device=DEV)
+    orla = torch.empty_like(osp)
+    out = cache.decode_selected(q, gamma, torch.as_tensor(sel, device=DEV), dbg_o_sparse=osp, dbg_o_rla=orla)
+    out, osp, orla = out.cpu().numpy(), osp.cpu().numpy(), orla.cpu().numpy()
+    for b in range(w.batch):
+        for h in range(w.n_kv_heads):
+            res = parity.oracle_unit(w, q[b], K[b, h], V[b, h], gamma, h, n_sink=1, n_local=4,
+                                     override=[int(i) for i in sel[b, h] if i >= 0])
+            sl = slice(h * 4, (h + 1) * 4)
+            parity.check_outputs("o_sparse", osp[b, sl], res["o_sparse"], "bf16")
+            parity.check_outputs("o_rla", orla[b, sl], res["o_rla"], "bf16")
+            parity.check_outputs("out", out[b, sl], res["out"], "bf16")
+
+
+def test_scores_are_normalised_and_match_oracle():
+    w = synth.BY_NAME["gqa_32k"].scaled(batch=1, context=64 * 100 + 40, n_needles=4)
+    cache, K, V, lens = runner.build_cache(w, DEV)
+    gamma = synth.gamma(w).to(DEV)
+    q = synth.step_queries(w, 0, DEV)
+    cache.decode(q, gamma)
+    sc = cache.scores().cpu().numpy()
+    nblk = 101
+    for h in range(w.n_kv_heads):
+        res = parity.oracle_unit(w, q[0], K[0, h], V[0, h], gamma, h, n_sink=1, n_local=4)
+        np.testing.assert_allclose(sc[0, h, :nblk], res["score"], rtol=2e-5)
+        assert abs(sc[0, h, :nblk].sum() - w.group) < 1e-4
+
+
+def test_capacity_overflow_is_reported_not_faulted():
+    w = synth.BY_NAME["gqa_32k"].scaled(batch=2, context=256, n_needles=0, n_steps=3)
+    cache, K, V, lens = runner.build_cache(w, DEV)
+    k1, v1 = synth.step_kv(w, 0, DEV)
+    for _ in range(3):
+        cache.append_tokens(k1, v1)
+    with pytest.raises(binding.SplaError) as e:          # host-side bound: 256 + 3 is full
+        cache.append_tokens(k1, v1)
+    assert e.value.status == binding.SPLA_ERR_CAPACITY
+    # device-side: lie to the host bound, the kernel skips the overflowing sequences and latches the status
+    cache.set_length_bound(0)
+    before = cache.bufs.rla_state.clone()
+    cache.append_tokens(k1, v1)
+    torch.cuda.synchronize()
+    assert cache.sync_status() == binding.SPLA_ERR_CAPACITY
+    assert cache.sync_status() == 0
+    assert cache.bufs.seq_lens.cpu().tolist() == [259, 259] and torch.equal(before, cache.bufs.rla_state)
