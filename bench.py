@@ -1,0 +1,392 @@
+#!/usr/bin/env python
+"""Benchmark of the SPLA decode step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One *step* = one pass of the whole hot path over one batch of synthetic input: append one token per
+sequence (cache write, block statistics, recurrent state) and decode (block score, top-k, sparse attention,
+residual linear attention, merge).  Metric: decode-attention queries x heads per second (batch * H_q per step),
+whole job, at the 128K-context configuration, plus the HBM roofline of the dominant kernel.
+
+Timing: W warm-up steps, then exactly K steps between barrier + synchronize, timed with CUDA events on the
+launching stream, max over ranks.  The steps rotate over R independent caches so that the bytes touched per
+rotation exceed three times the L2 size (cold-L2 protocol).  Steps are replayed from a CUDA graph of 64 steps
+so that the Python launch path is not what is measured.  One JSON line is printed by rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode_attention_query_heads_per_s"
+UNIT = "query_heads/s"
+L2_BYTES = 126 * 1024 * 1024
+GRAPH_STEPS = 64
+
+
+# ------------------------------------------------------------------------------------------------------------
+# CPU baseline: the float64 oracle, as it stands, on the host cores (also the --impl reference arm)
+# ------------------------------------------------------------------------------------------------------------
+_ORACLE_UNITS = None
+
+
+def _oracle_worker(args):
+    """Times incremental-form oracle decodes of one unit (block statistics and state cached, as a server would)."""
+    idx, n_dec, cfg = args
+    from threadpoolctl import threadpool_limits
+    from oracle import spla_oracle as O
+    K, V, qs, gam = _ORACLE_UNITS[idx]
+    with threadpool_limits(limits=1):
+        cache = O.UnitCache.from_prefill(K, V, cfg["block_size"])
+        t0 = time.perf_counter()
+        for i in range(n_dec):
+            cache.decode(qs[i % len(qs)], gam, top_k=cfg["top_k"], n_sink=cfg["n_sink"], n_local=cfg["n_local"])
+        return time.perf_counter() - t0
+
+
+def oracle_throughput(w, n_dec_per_unit: int, repeats: int = 1):
+    """Runs the oracle on one sequence's KV heads (one unit per process).  Returns (query_heads/s list, cores, sample)."""
+    global _ORACLE_UNITS
+    import multiprocessing as mp
+    import numpy as np
+    from paper_2601_22379_b200 import synth
+    cores = len(os.sched_getaffinity(0))
+    n_units = max(1, min(cores, w.n_kv_heads))
+    K, V = synth.prefill_kv(w, 0, "cpu")
+    G = w.group
+    gam = synth.gamma(w).double().numpy()
+    qs = [synth.step_queries(w, s, "cpu")[0].double().numpy() for s in range(8)]
+    _ORACLE_UNITS = [(K[h].double().numpy(), V[h].double().numpy(), [q[h * G:(h + 1) * G] for q in qs],
+                      gam[h * G:(h + 1) * G]) for h in range(n_units)]
+    del K, V
+    cfg = dict(block_size=w.block_size, top_k=w.top_k, n_sink=w.n_sink, n_local=w.n_local)
+    values = []
+    ctx = mp.get_context("fork")
+    with ctx.Pool(n_units) as pool:
+        for _ in range(repeats):
+            times = pool.map(_oracle_worker, [(i, n_dec_per_unit, cfg) for i in range(n_units)])
+            values.append(n_units * n_dec_per_unit * G / max(times))
+    _ORACLE_UNITS = None
+    sample = (f"{n_units} units (sequence 0, KV heads 0..{n_units - 1}) of {w.name}, {n_dec_per_unit} decode calls each, "
+              f"float64 numpy oracle with cached block statistics and state, one process per unit")
+    return values, n_units, sample
+
+
+def run_reference(args, w):
+    """--impl reference: the oracle timed on the host cores, same metric and config."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps, warmup = args.steps, max(args.warmup, 0)
+    n_dec = 24
+    t0 = time.perf_counter()
+    vals, cores, sample = oracle_throughput(w, n_dec, repeats=max(1, min(steps + warmup, 6)))
+    vals = vals[min(warmup, len(vals) - 1):] or vals
+    value = statistics.mean(vals)
+    line = base_line(args, w, value, ms_per_step=1e3 * w.batch * w.n_q_heads / value)
+    line.update({"impl": "reference", "dtype": "f64", "n_gpus": args.gpus,
+                 "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+                 "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                 "gpu_launches": 0, "wall_s": time.perf_counter() - t0})
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------------------
+def base_line(args, w, value, ms_per_step):
+    from paper_2601_22379_b200 import synth
+    by = synth.algorithmic_bytes_per_step(w)
+    return {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if w.kv_dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": w.name, "batch": w.batch, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads,
+                   "head_dim": w.head_dim, "context": w.context, "block_size": w.block_size, "top_k": w.top_k,
+                   "n_sink": w.n_sink, "n_local": w.n_local, "kv_dtype": w.kv_dtype,
+                   "algorithmic_bytes_per_step": by["total"], "dense_kv_bytes_per_step": by["dense_kv"],
+                   "parallelism": f"replicas x{args.gpus} (units are independent; no collective)"},
+    }
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.perf_counter(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.05)
+        self.proc.terminate()
+        rows = [r for t, r in self.rows if t0 <= t <= t1] or [r for _, r in self.rows[-3:]]
+        sm, smax, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            try:
+                sm.append(float(f[0])); smax.append(float(f[1])); power.append(float(f[2]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2601_22379_b200 import build, runner, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    cpu_base = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        vals, cores, sample = oracle_throughput(w, 24, repeats=2)      # before CUDA is initialised (fork)
+        cpu_base = {"value": vals[-1], "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+
+    build.build()
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    steps, warmup = args.steps, max(args.warmup, 3)
+    by = synth.algorithmic_bytes_per_step(w)
+    R = 2                                                             # caches to rotate over (cold-L2 protocol)
+    while R * by["total"] < 3 * L2_BYTES and R < GRAPH_STEPS:
+        R *= 2
+    n_e2e = max(8, min(steps, 256))
+    per_cache = -(-(steps + warmup + 2 * GRAPH_STEPS + n_e2e) // R) + 2 * GRAPH_STEPS
+    wl = w.scaled(n_steps=per_cache)
+    prefill = runner.generate_prefill(wl, dev)
+    caches = []
+    for _ in range(R):
+        c, _, _, _ = runner.build_cache(wl, dev, prefill=prefill)
+        caches.append(c)
+    del prefill
+    n_app = [0] * R                                                   # tokens appended per cache so far
+
+    def set_bounds(exact: bool):
+        # The library sizes its grids from a host-side bound of the sequence lengths.  Graph replays append
+        # without the host seeing it, so the bound is raised to the capacity while graphs run and put back after.
+        for ci, c in enumerate(caches):
+            c.set_length_bound(w.context + n_app[ci] if exact else wl.max_context - GRAPH_STEPS)
+    gamma = synth.gamma(w).to(dev)
+    n_in = GRAPH_STEPS
+    qs = [synth.step_queries(w, s, dev) for s in range(n_in)]
+    kvs = [synth.step_kv(w, s, dev) for s in range(n_in)]
+    outs = [torch.empty(w.batch, w.n_q_heads, w.head_dim, dtype=torch.float32, device=dev) for _ in range(R)]
+    stream = torch.cuda.Stream(device=dev)
+    counter = {"i": 0}
+
+    def one_step():
+        i = counter["i"]
+        counter["i"] += 1
+        c = caches[i % R]
+        k1, v1 = kvs[i % n_in]
+        c.append_tokens(k1, v1)
+        n_app[i % R] += 1
+        c.decode(qs[i % n_in], gamma, out=outs[i % R])
+
+    def decode_only(i):
+        caches[i % R].decode(qs[i % n_in], gamma, out=outs[i % R])
+
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        for _ in range(warmup):
+            one_step()
+        graph = None
+        saved = list(n_app)
+        set_bounds(exact=False)
+        if steps >= GRAPH_STEPS:
+            counter["i"] = 0
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                for _ in range(GRAPH_STEPS):
+                    one_step()
+            n_app[:] = saved                                           # capture enqueued nothing
+            graph.replay()                                             # one untimed replay
+            for ci in range(R):
+                n_app[ci] += GRAPH_STEPS // R
+        graph_dec = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph_dec, stream=stream):
+            for i in range(GRAPH_STEPS):
+                decode_only(i)
+        graph_dec.replay()
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- the timed region: exactly `steps` steps ----------------------------------------------------------
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.15)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t0 = time.perf_counter()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        n_rep = steps // GRAPH_STEPS if graph is not None else 0
+        for _ in range(n_rep):
+            graph.replay()
+        for ci in range(R):
+            n_app[ci] += n_rep * (GRAPH_STEPS // R)
+        set_bounds(exact=True)
+        for _ in range(steps - n_rep * GRAPH_STEPS):
+            one_step()
+        e1.record(stream)
+    barrier()
+    t1 = time.perf_counter()
+    total_ms = e0.elapsed_time(e1)
+    clocks = sampler.stop(t0, t1)
+    for c in caches:
+        st = c.sync_status()
+        if st != 0:
+            raise RuntimeError(f"device status {st} after the timed region")
+
+    # ---- decode-only (no append) for context, same rotation ---------------------------------------------------
+    with torch.cuda.stream(stream):
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_dec_rep = max(1, min(steps // GRAPH_STEPS, 64))
+        d0.record(stream)
+        for _ in range(n_dec_rep):
+            graph_dec.replay()
+        d1.record(stream)
+    torch.cuda.synchronize()
+    dec_ms = d0.elapsed_time(d1) / (n_dec_rep * GRAPH_STEPS)
+
+    # ---- per-kernel durations of the decode, CUDA events between the two kernels -----------------------------
+    n_prof = max(8, min(steps, 128))
+    sc_ms, at_ms = [], []
+    with torch.cuda.stream(stream):
+        for i in range(n_prof):
+            a, b = caches[i % R].decode_profile(qs[i % n_in], gamma, outs[i % R])
+            sc_ms.append(a)
+            at_ms.append(b)
+    sc, at = statistics.mean(sc_ms), statistics.mean(at_ms)
+
+    # ---- end to end through the public call with host buffers --------------------------------------------------
+    hq = [q.cpu().pin_memory() for q in qs[:8]]
+    hk = [(k.cpu().pin_memory(), v.cpu().pin_memory()) for k, v in kvs[:8]]
+    dq, dk, dv = torch.empty_like(qs[0]), torch.empty_like(kvs[0][0]), torch.empty_like(kvs[0][1])
+    hout = torch.empty(w.batch, w.n_q_heads, w.head_dim, dtype=torch.float32).pin_memory()
+    h2d = hq[0].numel() * hq[0].element_size() + 2 * hk[0][0].numel() * hk[0][0].element_size()
+    d2h = hout.numel() * 4
+    barrier()
+    with torch.cuda.stream(stream):
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record(stream)
+        for i in range(n_e2e):
+            c = caches[i % R]
+            dq.copy_(hq[i % 8], non_blocking=True)
+            dk.copy_(hk[i % 8][0], non_blocking=True)
+            dv.copy_(hk[i % 8][1], non_blocking=True)
+            c.append_tokens(dk, dv)
+            n_app[i % R] += 1
+            c.decode(dq, gamma, out=outs[i % R])
+            hout.copy_(outs[i % R], non_blocking=True)
+            stream.synchronize()                                       # the caller reads the result before the next step
+        g1.record(stream)
+    barrier()
+    e2e_ms = g0.elapsed_time(g1) / n_e2e
+
+    t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = float(t[0]), float(t[1])
+    qh_per_step = w.batch * w.n_q_heads * world
+    value = qh_per_step * steps / (total_ms * 1e-3)
+
+    peak, peak_kind = measured_peaks()
+    score_bytes = by["stats"] + by["state"]
+    achieved = score_bytes / (sc * 1e-3) / 1e9
+    line = base_line(args, w, value, ms_per_step=total_ms / steps)
+    line["warmup"] = warmup
+    line["config"].update({"l2_protocol": f"rotation over {R} independent caches ({R * by['total'] / 2**20:.0f} MiB per "
+                                          f"rotation, > 3x L2) - cold L2", "context_growth_tokens_per_cache": per_cache,
+                           "launch": f"CUDA graph of {GRAPH_STEPS} steps replayed" if graph is not None else "eager"})
+    line.update({
+        "clocks": clocks,
+        "e2e": {"value": w.batch * w.n_q_heads * world / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+        "gpu_launches": 6 * steps,
+        "roofline": {"bound": "hbm", "kernel": "score_select_kernel", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                     "bytes_per_launch": score_bytes, "ms_per_launch": sc, "traffic": args.traffic},
+        "kernels": {"score_select_ms": sc, "attend_merge_ms": at,
+                    "attend_merge_GBps": by["selected_kv"] / (at * 1e-3) / 1e9,
+                    "decode_only_ms": dec_ms, "decode_only_GBps": by["total"] / (dec_ms * 1e-3) / 1e9,
+                    "decode_only_frac_of_peak": by["total"] / (dec_ms * 1e-3) / 1e9 / peak,
+                    "decode_only_frac_of_8TBps": by["total"] / (dec_ms * 1e-3) / 8e12,
+                    "decode_only_query_heads_per_s": w.batch * w.n_q_heads / (dec_ms * 1e-3)},
+    })
+    if cpu_base is not None:
+        line["cpu_baseline"] = cpu_base
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=8192)
+    ap.add_argument("--warmup", type=int, default=64)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="long_128k")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--traffic", type=float, default=None,
+                    help="DRAM bytes per launch of the dominant kernel from an ncu capture (reported as roofline.traffic)")
+    args = ap.parse_args()
+    from paper_2601_22379_b200 import synth
+    w = synth.BY_NAME[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

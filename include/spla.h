@@ -149,6 +149,15 @@ int spla_decode(spla_cache_t *cache, const void *q, const float *rms_weight, flo
 int spla_decode_selected(spla_cache_t *cache, const void *q, const float *rms_weight, const int32_t *sel_in,
                          float *out, float *dbg_o_sparse, float *dbg_o_rla, void *stream);
 
+/*
+ * Measurement aid: spla_decode with a CUDA event recorded on `stream` before, between and after its two
+ * kernels, followed by a wait for the last event.  stage_ms: HOST float[2], receives the device time in
+ * milliseconds of the score+select kernel and of the attend+merge kernel.  Unlike every other call this one
+ * blocks the calling thread, and it may create three CUDA events on its first use for a cache.
+ */
+int spla_decode_profile(spla_cache_t *cache, const void *q, const float *rms_weight, float *out, float *stage_ms,
+                        void *stream);
+
 /* Block scores of the last spla_decode: DEVICE fp32 [batch][H_kv][max_blocks] copy-out (entries >= nblk are 0). */
 int spla_copy_scores(spla_cache_t *cache, float *scores_out, void *stream);
 

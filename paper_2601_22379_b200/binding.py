@@ -19,6 +19,7 @@ SPLA_ADOPT_CONTENTS, SPLA_FIRST_ORDER, SPLA_NO_RLA = 1, 2, 4
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libspla.so")
 
 EXPORTS = ["spla_query_sizes", "spla_init_cache", "spla_append_tokens", "spla_decode", "spla_decode_selected",
+           "spla_decode_profile",
            "spla_copy_scores", "spla_sync_status", "spla_set_length_bound", "spla_destroy_cache",
            "spla_status_string", "spla_last_cuda_error"]
 
@@ -61,6 +62,7 @@ def load(path: str | None = None) -> C.CDLL:
     lib.spla_append_tokens.argtypes = [vp, vp, vp, vp, i32, vp]
     lib.spla_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.spla_decode_selected.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.spla_decode_profile.argtypes = [vp, vp, vp, vp, C.POINTER(C.c_float), vp]
     lib.spla_copy_scores.argtypes = [vp, vp, vp]
     lib.spla_sync_status.argtypes = [vp, vp]
     lib.spla_set_length_bound.argtypes = [vp, i32]
@@ -201,6 +203,14 @@ class SplaCache:
                                                  out.data_ptr(), _ptr(dbg_o_sparse), _ptr(dbg_o_rla), _stream()),
                    "spla_decode_selected")
         return out
+
+    def decode_profile(self, q, rms_weight, out: torch.Tensor):
+        """Blocking decode that returns (score_select_ms, attend_merge_ms) measured with CUDA events."""
+        ms = (C.c_float * 2)()
+        with torch.cuda.device(self.device):
+            _check(self.lib.spla_decode_profile(self.handle, q.data_ptr(), _ptr(rms_weight), out.data_ptr(), ms,
+                                                _stream()), "spla_decode_profile")
+        return float(ms[0]), float(ms[1])
 
     # -- helpers ------------------------------------------------------------------------------------------
     def scores(self) -> torch.Tensor:

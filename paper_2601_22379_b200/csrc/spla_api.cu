@@ -14,6 +14,8 @@ struct spla_cache {
   spla_buffers_t buf;
   Params p;
   int64_t len_bound;   // host-side upper bound of the longest sequence
+  cudaEvent_t ev[3];   // created on first use by spla_decode_profile
+  bool have_ev;
 };
 
 static thread_local char g_cuda_err[256] = "";
@@ -113,6 +115,7 @@ extern "C" int spla_init_cache(const spla_config_t* config, const spla_buffers_t
   if (!c) return SPLA_ERR_INVALID_ARG;
   c->cfg = *config;
   c->buf = *b;
+  c->have_ev = false;
   if (c->cfg.sm_scale == 0.f) c->cfg.sm_scale = 1.0f / sqrtf((float)config->head_dim);
   if (c->cfg.phi_scale == 0.f) c->cfg.phi_scale = 1.0f;
   if (c->cfg.rms_eps == 0.f) c->cfg.rms_eps = 1e-6f;
@@ -195,6 +198,33 @@ extern "C" int spla_decode(spla_cache_t* c, const void* q, const float* rms_weig
   return SPLA_OK;
 }
 
+extern "C" int spla_decode_profile(spla_cache_t* c, const void* q, const float* rms_weight, float* out,
+                                   float* stage_ms, void* stream) {
+  if (!c || !q || !out || !stage_ms) return SPLA_ERR_INVALID_ARG;
+  if (!rms_weight && !(c->cfg.flags & SPLA_NO_RLA)) return SPLA_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(out, 16)) return SPLA_ERR_INVALID_ARG;
+  cudaError_t e = cudaSuccess;
+  if (!c->have_ev) {
+    for (int i = 0; i < 3 && e == cudaSuccess; ++i) e = cudaEventCreate(&c->ev[i]);
+    if (e != cudaSuccess) return cuda_fail(e, "spla_decode_profile/events");
+    c->have_ev = true;
+  }
+  Params p = c->p;
+  p.n_chunks_cap = chunks_for_bound(c);
+  const int qb = c->cfg.q_dtype == SPLA_BF16;
+  cudaStream_t s = (cudaStream_t)stream;
+  e = cudaEventRecord(c->ev[0], s);
+  if (e == cudaSuccess) e = launch_score_select(p, q, qb, nullptr, s);
+  if (e == cudaSuccess) e = cudaEventRecord(c->ev[1], s);
+  if (e == cudaSuccess) e = launch_attend_merge(p, q, qb, rms_weight, nullptr, out, nullptr, nullptr, s);
+  if (e == cudaSuccess) e = cudaEventRecord(c->ev[2], s);
+  if (e == cudaSuccess) e = cudaEventSynchronize(c->ev[2]);
+  if (e == cudaSuccess) e = cudaEventElapsedTime(&stage_ms[0], c->ev[0], c->ev[1]);
+  if (e == cudaSuccess) e = cudaEventElapsedTime(&stage_ms[1], c->ev[1], c->ev[2]);
+  if (e != cudaSuccess) return cuda_fail(e, "spla_decode_profile");
+  return SPLA_OK;
+}
+
 extern "C" int spla_decode_selected(spla_cache_t* c, const void* q, const float* rms_weight, const int32_t* sel_in,
                                     float* out, float* dbg_o_sparse, float* dbg_o_rla, void* stream) {
   if (!c || !q || !out || !sel_in) return SPLA_ERR_INVALID_ARG;
@@ -231,6 +261,8 @@ extern "C" int spla_sync_status(spla_cache_t* c, void* stream) {
 }
 
 extern "C" int spla_destroy_cache(spla_cache_t* c) {
+  if (c && c->have_ev)
+    for (int i = 0; i < 3; ++i) cudaEventDestroy(c->ev[i]);
   delete c;
   return SPLA_OK;
 }
