@@ -164,6 +164,33 @@ int spla_copy_scores(spla_cache_t *cache, float *scores_out, void *stream);
 /* Waits for `stream`, then returns and clears the device-latched status (SPLA_OK or SPLA_ERR_CAPACITY). */
 int spla_sync_status(spla_cache_t *cache, void *stream);
 
+/*
+ * Block scoring + top-k selection (steps 1-2 of spla_decode) for callers that cannot allocate device memory.
+ * The paper has no counterpart to this call; it exists for deployment reasons only.  Some code that wants a
+ * selection has no way to provide the workspace the regular path needs: it runs inside a memory pool that was
+ * sized and frozen up front, or it is a plug-in that receives tensors but no allocator, or it sits in a loop where
+ * cudaMalloc (which synchronises the device) is off limits.  This variant therefore takes only inputs and
+ * outputs and keeps the kernel's scratch in a fixed array inside the library's device image.
+ *   config:     HOST; batch, heads, head_dim, block_size, top_k, max_context, sink/local counts, q_dtype,
+ *               sm_scale and SPLA_FIRST_ORDER are used.  The scratch needed, about
+ *               batch * H_kv * max_blocks * (G + 1) * 4 bytes, must fit SPLA_NOALLOC_SCRATCH_BYTES, otherwise
+ *               SPLA_ERR_UNSUPPORTED is returned and nothing is launched.
+ *   stats:      DEVICE fp32 [batch][H_kv][max_blocks][2][d], as maintained by spla_append_tokens.
+ *   seq_lens:   DEVICE int32 [batch].
+ *   q:          DEVICE [batch][H_q][d] q_dtype.
+ *   sel_idx:    DEVICE int32 [batch][H_kv][top_k] output, ascending, padded with -1.
+ *   scores_out: DEVICE fp32 [batch][H_kv][max_blocks] output or NULL (entries past the last block are 0).
+ * The call allocates nothing: no cudaMalloc / cudaFree and no allocating library routine.  Every GPU that loads
+ * the library carries the SPLA_NOALLOC_SCRATCH_BYTES array until the process exits.  The first call on each
+ * device looks up the array's device address (with that device current); make that first call outside any
+ * stream capture.  All calls share the one array, which still holds the previous call's contents (what must
+ * start at zero is cleared on `stream` first): two of these calls that overlap on the GPU - different streams,
+ * or different threads - race on it and give wrong selections.  Issue them on one stream, or order them yourself.
+ */
+#define SPLA_NOALLOC_SCRATCH_BYTES (4u << 20)
+int spla_select_blocks_noalloc(const spla_config_t *config, const float *stats, const int32_t *seq_lens,
+                               const void *q, int32_t *sel_idx, float *scores_out, void *stream);
+
 /* Tells the library an upper bound of the current sequence lengths after adopting contents (HOST value). */
 int spla_set_length_bound(spla_cache_t *cache, int32_t max_seq_len);
 

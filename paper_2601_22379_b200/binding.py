@@ -19,7 +19,7 @@ SPLA_ADOPT_CONTENTS, SPLA_FIRST_ORDER, SPLA_NO_RLA = 1, 2, 4
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libspla.so")
 
 EXPORTS = ["spla_query_sizes", "spla_init_cache", "spla_append_tokens", "spla_decode", "spla_decode_selected",
-           "spla_decode_profile",
+           "spla_decode_profile", "spla_select_blocks_noalloc",
            "spla_copy_scores", "spla_sync_status", "spla_set_length_bound", "spla_destroy_cache",
            "spla_status_string", "spla_last_cuda_error"]
 
@@ -63,6 +63,7 @@ def load(path: str | None = None) -> C.CDLL:
     lib.spla_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.spla_decode_selected.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.spla_decode_profile.argtypes = [vp, vp, vp, vp, C.POINTER(C.c_float), vp]
+    lib.spla_select_blocks_noalloc.argtypes = [C.POINTER(SplaConfig), vp, vp, vp, vp, vp, vp]
     lib.spla_copy_scores.argtypes = [vp, vp, vp]
     lib.spla_sync_status.argtypes = [vp, vp]
     lib.spla_set_length_bound.argtypes = [vp, i32]
@@ -123,6 +124,22 @@ class _Bufs:
     tok_lse: torch.Tensor
     seq_lens: torch.Tensor
     workspace: torch.Tensor
+
+
+NOALLOC_SCRATCH_BYTES = 4 << 20
+
+
+def select_blocks_noalloc(cfg: SplaConfig, stats: torch.Tensor, seq_lens: torch.Tensor, q: torch.Tensor,
+                          sel_idx: torch.Tensor, scores_out: torch.Tensor | None = None) -> int:
+    """Score + select for callers that may not allocate on the device: every tensor is passed in, the kernel's
+    scratch is a fixed array inside the library.  Returns the status code (0 = ok) instead of raising, so that a
+    caller can fall back to `SplaCache.decode` when the configuration exceeds the fixed scratch.  Calls share
+    that scratch: never let two of them overlap on the GPU."""
+    assert stats.is_cuda and stats.dtype == torch.float32 and stats.is_contiguous()
+    assert seq_lens.dtype == torch.int32 and sel_idx.dtype == torch.int32 and q.is_contiguous()
+    with torch.cuda.device(stats.device):
+        return load().spla_select_blocks_noalloc(C.byref(cfg), stats.data_ptr(), seq_lens.data_ptr(), q.data_ptr(),
+                                                 sel_idx.data_ptr(), _ptr(scores_out), _stream())
 
 
 class SplaCache:
