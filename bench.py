@@ -193,6 +193,8 @@ def run_ours(args, w):
     R = 2                                                             # caches to rotate over (cold-L2 protocol)
     while R * by["total"] < 3 * L2_BYTES and R < GRAPH_STEPS:
         R *= 2
+    if args.caches > 0:                                               # profiling aid: fewer caches, less device memory
+        R = args.caches
     n_e2e = max(8, min(steps, 256))
     per_cache = -(-(steps + warmup + 2 * GRAPH_STEPS + n_e2e) // R) + 2 * GRAPH_STEPS
     wl = w.scaled(n_steps=per_cache)
@@ -246,11 +248,13 @@ def run_ours(args, w):
             graph.replay()                                             # one untimed replay
             for ci in range(R):
                 n_app[ci] += GRAPH_STEPS // R
-        graph_dec = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph_dec, stream=stream):
-            for i in range(GRAPH_STEPS):
-                decode_only(i)
-        graph_dec.replay()
+        graph_dec = None
+        if steps >= GRAPH_STEPS:
+            graph_dec = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph_dec, stream=stream):
+                for i in range(GRAPH_STEPS):
+                    decode_only(i)
+            graph_dec.replay()
     torch.cuda.synchronize()
 
     def barrier():
@@ -290,8 +294,12 @@ def run_ours(args, w):
         d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         n_dec_rep = max(1, min(steps // GRAPH_STEPS, 64))
         d0.record(stream)
-        for _ in range(n_dec_rep):
-            graph_dec.replay()
+        for r in range(n_dec_rep):
+            if graph_dec is not None:
+                graph_dec.replay()
+            else:
+                for i in range(GRAPH_STEPS):
+                    decode_only(i)
         d1.record(stream)
     torch.cuda.synchronize()
     dec_ms = d0.elapsed_time(d1) / (n_dec_rep * GRAPH_STEPS)
@@ -377,6 +385,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="long_128k")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--caches", type=int, default=0, help="rotate over this many caches instead of the cold-L2 count "
+                    "(for profiler captures, which must hold little device memory)")
     ap.add_argument("--traffic", type=float, default=None,
                     help="DRAM bytes per launch of the dominant kernel from an ncu capture (reported as roofline.traffic)")
     args = ap.parse_args()

@@ -4,7 +4,9 @@
 //   ell^m_i = ln n_i + q_hat^m . mean_i + ln(1 + 1/2 sum_c (q_hat^m_c)^2 var_i[c])
 // is the log of the second-order Taylor estimate of the block's attention mass; per head the masses are
 // normalised over all blocks and the G heads are summed (Section 2.2).  One warp consumes one 2d-float
-// statistics record with a single 128-bit load per lane for the mean and one for the variance.
+// statistics record with a single 128-bit load per lane for the mean and one for the variance; a CTA streams
+// `chunk` consecutive records, 32 at a time, with the next 32 already in flight (register double buffer), and
+// the grid is sized to about one resident wave so that the per-CTA fixed cost is paid once.
 //
 // Selection (Section 2.1 Select; Section 4 forced sink/local blocks): the last CTA of a unit to finish
 // (atomic ticket, no waiting) reduces the per-chunk normalisers, forms the aggregated score, and picks the
@@ -13,12 +15,48 @@
 
 namespace spla {
 
+namespace {
+
+constexpr int UNR = 4;                                  // records per warp per round
+constexpr int kRound = (kScoreThreads / 32) * UNR;      // records per CTA per round (32)
+
+template <int VEC>
+__device__ __forceinline__ void load_record(const float* rec, int D, int lane, bool valid, float (&mean)[VEC],
+                                            float (&var)[VEC]) {
+  if (valid) {
+    if constexpr (VEC == 4) {
+      const float4 a = __ldcs(reinterpret_cast<const float4*>(rec + lane * 4));
+      const float4 b = __ldcs(reinterpret_cast<const float4*>(rec + D + lane * 4));
+      mean[0] = a.x; mean[1] = a.y; mean[2] = a.z; mean[3] = a.w;
+      var[0] = b.x; var[1] = b.y; var[2] = b.z; var[3] = b.w;
+    } else {
+      const float2 a = __ldcs(reinterpret_cast<const float2*>(rec + lane * 2));
+      const float2 b = __ldcs(reinterpret_cast<const float2*>(rec + D + lane * 2));
+      mean[0] = a.x; mean[1] = a.y;
+      var[0] = b.x; var[1] = b.y;
+    }
+  } else {
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) { mean[v] = 0.f; var[v] = 0.f; }
+  }
+}
+
+// Merge two (max, sum-of-exp) pairs.
+__device__ __forceinline__ void lse_merge(float& m, float& s, float m2, float s2) {
+  const float nm = fmaxf(m, m2);
+  if (nm > -INFINITY) s = s * __expf(m - nm) + s2 * __expf(m2 - nm);
+  m = nm;
+}
+
+}  // namespace
+
 template <int D, int GP>
-__global__ void __launch_bounds__(kScoreThreads) score_select_kernel(const Params p, const void* __restrict__ q_raw,
-                                                                     int q_is_bf16, int* __restrict__ sel_user) {
+__global__ void __launch_bounds__(kScoreThreads, 2) score_select_kernel(const Params p, const void* __restrict__ q_raw,
+                                                                        int q_is_bf16, int* __restrict__ sel_user) {
   constexpr int VEC = D / 32;
   constexpr int NV = 2 * GP;             // values reduced per record: GP mean dots, GP variance dots
   constexpr int LPV = 32 / NV > 0 ? 32 / NV : 1;  // lanes holding a copy of each reduced value
+  constexpr int FB = LPV < UNR ? LPV : UNR;       // records finalised together, one per copy lane
   constexpr int NWARP = kScoreThreads / 32;
   extern __shared__ __align__(16) unsigned char smem_raw[];
 
@@ -26,9 +64,6 @@ __global__ void __launch_bounds__(kScoreThreads) score_select_kernel(const Param
   const int b = u / p.Hkv, h = u % p.Hkv;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = p.G;
-  const int L = p.seq_lens[b];
-  const int nblk = (L + p.B - 1) / p.B;
-  const int n_chunks = max(1, (nblk + kScoreChunk - 1) / kScoreChunk);
   const int c = blockIdx.x;
 
   // ------------------------------------------------------------------ o_bar role ----------------------
@@ -37,6 +72,13 @@ __global__ void __launch_bounds__(kScoreThreads) score_select_kernel(const Param
     float* phiq = reinterpret_cast<float*>(smem_raw);      // [GP][D]
     float* red = phiq + GP * D;                            // [kScoreThreads / D][GP][D]
     const float a2 = p.phi_scale * kLog2e;
+    constexpr int RG = kScoreThreads / D;                  // row groups working side by side
+    constexpr int ROWS = D / kStateSplits / RG;            // rows per thread
+    const int rg = tid / D, j = tid % D;
+    const float* S = p.state + (size_t)u * D * D + (size_t)(s * (D / kStateSplits) + rg) * D + j;
+    float sv[ROWS];
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) sv[r] = __ldcs(S + (size_t)r * RG * D);     // all loads in flight before use
     for (int g = warp; g < G; g += NWARP) {
       float x[VEC];
       const size_t qoff = ((size_t)b * p.Hq + (size_t)h * G + g) * D + lane * VEC;
@@ -55,18 +97,15 @@ __global__ void __launch_bounds__(kScoreThreads) score_select_kernel(const Param
       for (int v = 0; v < VEC; ++v) phiq[g * D + lane * VEC + v] = x[v] * inv;
     }
     __syncthreads();
-    constexpr int RG = kScoreThreads / D;                  // row groups working side by side
-    const int rg = tid / D, j = tid % D;
-    const int rows = D / kStateSplits;
-    const float* S = p.state + (size_t)u * D * D;
     float acc[GP];
 #pragma unroll
     for (int g = 0; g < GP; ++g) acc[g] = 0.f;
-    for (int r = s * rows + rg; r < (s + 1) * rows; r += RG) {
-      const float sv = S[(size_t)r * D + j];
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+      const int row = s * (D / kStateSplits) + rg + r * RG;
 #pragma unroll
       for (int g = 0; g < GP; ++g)
-        if (g < G) acc[g] = fmaf(phiq[g * D + r], sv, acc[g]);
+        if (g < G) acc[g] = fmaf(phiq[g * D + row], sv[r], acc[g]);
     }
 #pragma unroll
     for (int g = 0; g < GP; ++g) red[(rg * GP + g) * D + j] = acc[g];
@@ -82,6 +121,10 @@ __global__ void __launch_bounds__(kScoreThreads) score_select_kernel(const Param
   }
 
   // ------------------------------------------------------------------ score role ----------------------
+  const int L = p.seq_lens[b];
+  const int nblk = (L + p.B - 1) / p.B;
+  const int chunk = p.chunk;
+  const int n_chunks = max(1, (nblk + chunk - 1) / chunk);
   if (c >= n_chunks) return;
 
   // q_hat slices for the mean dot and 1/2 q_hat^2 for the variance dot, in registers.
@@ -106,61 +149,83 @@ __global__ void __launch_bounds__(kScoreThreads) score_select_kernel(const Param
 
   const float* stats_u = p.stats + (size_t)u * p.max_blocks * 2 * D;
   float* ell_u = p.ell + (size_t)u * G * p.max_blocks;
-  // Lanes 0..15 end up with the mean dots, lanes 16..31 with the variance dots; value index = lane / LPV.
+  // After the warp reduction lanes 0..15 hold the mean dots and lanes 16..31 the variance dots, value index
+  // lane / LPV, each replicated on LPV lanes.  Copy lane `sub` finalises record `sub` of the batch, so the
+  // log / exp work of FB records runs side by side instead of one record at a time.
   const int my_g = (lane & 15) / LPV;
-  const bool writer = lane < 16 && (lane % LPV) == 0 && my_g < G;
+  const int sub = lane % LPV;
+  const bool fin_lane = lane < 16 && sub < FB && my_g < G;
+  const float ln_full = logf((float)p.B);
+  const float ln_last = logf((float)max(1, L - (nblk - 1) * p.B));
   float run_max = -INFINITY, run_sum = 0.f;
 
-  constexpr int RPW = kScoreChunk / NWARP;   // records per warp
-  constexpr int UNR = 4;                     // records in flight per warp
-  const int rec0 = c * kScoreChunk + warp * RPW;
-#pragma unroll 1
-  for (int r0 = 0; r0 < RPW; r0 += UNR) {
-    float mean[UNR][VEC], var[UNR][VEC];
+  const int rounds = chunk / kRound;
+  const int base = c * chunk + warp * UNR;                 // record of (round 0, r = 0) for this warp
+
+  float mean[2][UNR][VEC], var[2][UNR][VEC];
+  auto load_round = [&](int round, int buf) {
 #pragma unroll
     for (int r = 0; r < UNR; ++r) {
-      const int i = rec0 + r0 + r;
-      if (i < nblk) {
-        const float* rec = stats_u + (size_t)i * 2 * D;
-        load_vec<VEC>(rec + lane * VEC, mean[r]);
-        load_vec<VEC>(rec + D + lane * VEC, var[r]);
-      } else {
-#pragma unroll
-        for (int v = 0; v < VEC; ++v) { mean[r][v] = 0.f; var[r][v] = 0.f; }
-      }
+      const int i = base + round * kRound + r;
+      load_record<VEC>(stats_u + (size_t)i * 2 * D, D, lane, i < nblk, mean[buf][r], var[buf][r]);
     }
+  };
+  auto compute_round = [&](int round, int buf) {
+    const int i0 = base + round * kRound;
+    if (i0 >= nblk) return;                                // warp-uniform
 #pragma unroll
-    for (int r = 0; r < UNR; ++r) {
-      const int i = rec0 + r0 + r;
-      float vals[NV];
+    for (int r0 = 0; r0 < UNR; r0 += FB) {
+      float dm_keep = 0.f, dv_keep = 0.f;
 #pragma unroll
-      for (int g = 0; g < GP; ++g) {
-        float dm = 0.f, dv = 0.f;
+      for (int rr = 0; rr < FB; ++rr) {
+        const int r = r0 + rr;
+        float vals[NV];
 #pragma unroll
-        for (int v = 0; v < VEC; ++v) {
-          dm = fmaf(qm[g][v], mean[r][v], dm);
-          dv = fmaf(qv[g][v], var[r][v], dv);
+        for (int g = 0; g < GP; ++g) {
+          float dm = 0.f, dv = 0.f;
+#pragma unroll
+          for (int v = 0; v < VEC; ++v) {
+            dm = fmaf(qm[g][v], mean[buf][r][v], dm);
+            dv = fmaf(qv[g][v], var[buf][r][v], dv);
+          }
+          vals[g] = dm;
+          vals[GP + g] = dv;
         }
-        vals[g] = dm;
-        vals[GP + g] = dv;
+        warp_reduce_multi<NV>(vals, lane);
+        const float other = __shfl_xor_sync(0xffffffffu, vals[0], 16);   // variance dot of the same head
+        if (sub == rr) { dm_keep = vals[0]; dv_keep = other; }
       }
-      warp_reduce_multi<NV>(vals, lane);
-      const float other = __shfl_xor_sync(0xffffffffu, vals[0], 16);   // variance dot of the same head
-      if (writer && i < nblk) {
-        const int n_i = min(p.B, L - i * p.B);
-        const float ell = __logf((float)n_i) + vals[0] + log1pf(other);
+      const int i = i0 + r0 + sub;
+      if (fin_lane && i < nblk) {
+        const float ell = (i == nblk - 1 ? ln_last : ln_full) + dm_keep + __logf(1.f + dv_keep);
         ell_u[(size_t)my_g * p.max_blocks + i] = ell;
         const float nm = fmaxf(run_max, ell);
         run_sum = run_sum * __expf(run_max - nm) + __expf(ell - nm);
         run_max = nm;
       }
     }
+  };
+
+  load_round(0, 0);
+#pragma unroll 1
+  for (int round = 0; round < rounds; round += 2) {
+    if (round + 1 < rounds) load_round(round + 1, 1);
+    compute_round(round, 0);
+    if (round + 1 < rounds) {
+      if (round + 2 < rounds) load_round(round + 2, 0);
+      compute_round(round + 1, 1);
+    }
   }
 
-  // per-chunk (max, sum exp) per head
+  // per-chunk (max, sum exp) per head: fold the FB finalising lanes, then the warps
+#pragma unroll
+  for (int o = 1; o < FB; o <<= 1) {
+    const float m2 = __shfl_xor_sync(0xffffffffu, run_max, o), s2 = __shfl_xor_sync(0xffffffffu, run_sum, o);
+    lse_merge(run_max, run_sum, m2, s2);
+  }
   float* wred = reinterpret_cast<float*>(smem_raw);     // [NWARP][GP][2]
   __shared__ int is_last_s;
-  if (writer) {
+  if (fin_lane && sub == 0) {
     wred[(warp * GP + my_g) * 2 + 0] = run_max;
     wred[(warp * GP + my_g) * 2 + 1] = run_sum;
   }
@@ -168,12 +233,7 @@ __global__ void __launch_bounds__(kScoreThreads) score_select_kernel(const Param
   if (tid < G) {
     float m = -INFINITY, s = 0.f;
 #pragma unroll
-    for (int w = 0; w < NWARP; ++w) {
-      const float wm = wred[(w * GP + tid) * 2], ws = wred[(w * GP + tid) * 2 + 1];
-      const float nm = fmaxf(m, wm);
-      if (nm > -INFINITY) s = s * __expf(m - nm) + ws * __expf(wm - nm);
-      m = nm;
-    }
+    for (int w = 0; w < NWARP; ++w) lse_merge(m, s, wred[(w * GP + tid) * 2], wred[(w * GP + tid) * 2 + 1]);
     float* cp = p.chunk_part + (((size_t)u * p.max_chunks + c) * G + tid) * 2;
     cp[0] = m;
     cp[1] = s;
@@ -199,12 +259,10 @@ __global__ void __launch_bounds__(kScoreThreads) score_select_kernel(const Param
 
   for (int g = warp; g < G; g += NWARP) {
     float m = -INFINITY, s = 0.f;
+#pragma unroll 4
     for (int cc = lane; cc < n_chunks; cc += 32) {
-      const float* cp = p.chunk_part + (((size_t)u * p.max_chunks + cc) * G + g) * 2;
-      const float cm = __ldcg(cp), cs = __ldcg(cp + 1);
-      const float nm = fmaxf(m, cm);
-      if (nm > -INFINITY) s = s * __expf(m - nm) + cs * __expf(cm - nm);
-      m = nm;
+      const float2 ms = __ldcg(reinterpret_cast<const float2*>(p.chunk_part + (((size_t)u * p.max_chunks + cc) * G + g) * 2));
+      lse_merge(m, s, ms.x, ms.y);
     }
     const float M = warp_max(m);
     s = (m > -INFINITY) ? s * __expf(m - M) : 0.f;
@@ -215,16 +273,35 @@ __global__ void __launch_bounds__(kScoreThreads) score_select_kernel(const Param
 
   const int k_eff = min(p.top_k, nblk);
   float* scores_u = p.scores + (size_t)u * p.max_blocks;
-  for (int i = tid; i < nblk; i += kScoreThreads) {
-    float sc = 0.f;
-    for (int g = 0; g < G; ++g) sc += __expf(__ldcg(ell_u + (size_t)g * p.max_blocks + i) - lse_s[g]);
-    scores_u[i] = sc;
-    const bool forced = (i < p.n_sink) || (i >= nblk - p.n_local);
-    keys[i] = forced ? 0xffffffffu : __float_as_uint(sc);
+  float lse_r[GP];
+#pragma unroll
+  for (int g = 0; g < GP; ++g) lse_r[g] = g < G ? lse_s[g] : 0.f;
+  constexpr int SB = 4;                                             // blocks per thread with loads in flight together
+  for (int i0 = 0; i0 < nblk; i0 += kScoreThreads * SB) {
+    float e[SB][GP];
+#pragma unroll
+    for (int j = 0; j < SB; ++j) {
+      const int i = i0 + j * kScoreThreads + tid;
+#pragma unroll
+      for (int g = 0; g < GP; ++g) e[j][g] = (g < G && i < nblk) ? __ldcg(ell_u + (size_t)g * p.max_blocks + i) : -INFINITY;
+    }
+#pragma unroll
+    for (int j = 0; j < SB; ++j) {
+      const int i = i0 + j * kScoreThreads + tid;
+      if (i < nblk) {
+        float sc = 0.f;
+#pragma unroll
+        for (int g = 0; g < GP; ++g)
+          if (g < G) sc += __expf(e[j][g] - lse_r[g]);
+        scores_u[i] = sc;
+        const bool forced = (i < p.n_sink) || (i >= nblk - p.n_local);
+        keys[i] = forced ? 0xffffffffu : __float_as_uint(sc);
+      }
+    }
   }
   __syncthreads();
 
-  // radix select: the k_eff-th largest key
+  // radix select: the k_eff-th largest key.  Equal digits inside a warp are counted with one atomic.
   uint32_t prefix = 0, mask = 0;
   int kk = k_eff;
   if (k_eff > 0) {
@@ -232,9 +309,16 @@ __global__ void __launch_bounds__(kScoreThreads) score_select_kernel(const Param
     for (int shift = 24; shift >= 0; shift -= 8) {
       hist[tid] = 0;                                                   // kScoreThreads == 256 bins
       __syncthreads();
-      for (int i = tid; i < nblk; i += kScoreThreads) {
-        const uint32_t key = keys[i];
-        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+      for (int i0 = 0; i0 < nblk; i0 += kScoreThreads) {
+        const int i = i0 + tid;
+        const uint32_t key = i < nblk ? keys[i] : 0u;
+        const bool in = i < nblk && (key & mask) == prefix;
+        const unsigned act = __ballot_sync(0xffffffffu, in);
+        if (in) {
+          const uint32_t digit = (key >> shift) & 255u;
+          const unsigned peers = __match_any_sync(act, digit);
+          if (lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
+        }
       }
       __syncthreads();
       if (warp == 0) {
@@ -261,7 +345,6 @@ __global__ void __launch_bounds__(kScoreThreads) score_select_kernel(const Param
       prefix |= sel_digit_s << shift;
       mask |= 0xffu << shift;
       kk = sel_k_s;
-      __syncthreads();
     }
   }
   const uint32_t T = prefix;   // threshold key; kk = how many keys equal to T are taken (lowest indices first)
@@ -287,7 +370,7 @@ __global__ void __launch_bounds__(kScoreThreads) score_select_kernel(const Param
   for (int w = 0; w < warp; ++w) { gt_before += wtot[0][w]; eq_before += wtot[1][w]; }
   int* sel_u = p.sel + (size_t)u * p.top_k;
   int* sel_o = sel_user ? sel_user + (size_t)u * p.top_k : nullptr;
-  if (k_eff > 0) {
+  if (k_eff > 0 && n_gt + n_eq > 0) {
     for (int i = i0; i < i1; ++i) {
       const uint32_t key = keys[i];
       const bool take = key > T || (key == T && eq_before < kk);
@@ -333,6 +416,14 @@ static cudaError_t launch_d(const Params& p, int GP, const void* q, int qb, int*
     case 8: return launch_one<D, 8>(p, q, qb, sel_user, s);
     default: return launch_one<D, 16>(p, q, qb, sel_user, s);
   }
+}
+
+int score_chunk_for(long long units, long long max_seq_blocks, int sm_count) {
+  // Smallest chunk (a multiple of the 32 records a CTA consumes per round) for which all score CTAs are
+  // resident at once (two CTAs per SM); long ragged batches simply take several waves of the largest chunk.
+  int chunk = kScoreChunkMin;
+  while (chunk < kScoreChunkMax && units * ((max_seq_blocks + chunk - 1) / chunk) > 2LL * sm_count) chunk *= 2;
+  return chunk;
 }
 
 cudaError_t launch_score_select(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream) {

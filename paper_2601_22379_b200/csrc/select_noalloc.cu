@@ -62,7 +62,7 @@ extern "C" int spla_select_blocks_noalloc(const spla_config_t* cfg, const float*
   // Carve the selection kernel's scratch out of the fixed array; refuse what does not fit.
   const size_t U = (size_t)cfg->batch * cfg->n_kv_heads, G = cfg->n_q_heads / cfg->n_kv_heads;
   const size_t max_blocks = ((size_t)cfg->max_context + cfg->block_size - 1) / cfg->block_size;
-  const size_t max_chunks = (max_blocks + kScoreChunk - 1) / kScoreChunk;
+  const size_t max_chunks = (max_blocks + kScoreChunkMin - 1) / kScoreChunkMin;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align256(off + bytes); return o; };
   const size_t o_ticket = take(U * 4);                      // must be zero when the kernel starts
@@ -90,7 +90,8 @@ extern "C" int spla_select_blocks_noalloc(const spla_config_t* cfg, const float*
   p.kv_bf16 = cfg->kv_dtype == SPLA_BF16;
   p.sm_scale = cfg->sm_scale == 0.f ? 1.0f / sqrtf((float)cfg->head_dim) : cfg->sm_scale;
   p.phi_scale = 1.f; p.rms_eps = 1e-6f;
-  p.n_chunks_cap = (int)max_chunks;
+  p.chunk = score_chunk_for((long long)U, (long long)max_blocks, 148);
+  p.n_chunks_cap = (int)((max_blocks + p.chunk - 1) / p.chunk);
   p.stats = const_cast<float*>(stats);
   p.seq_lens = const_cast<int*>(seq_lens);
   p.score_ticket = (int*)(base + o_ticket); p.status = (int*)(base + o_status);

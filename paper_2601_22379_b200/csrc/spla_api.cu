@@ -16,6 +16,7 @@ struct spla_cache {
   int64_t len_bound;   // host-side upper bound of the longest sequence
   cudaEvent_t ev[3];   // created on first use by spla_decode_profile
   bool have_ev;
+  int sm_count;
 };
 
 static thread_local char g_cuda_err[256] = "";
@@ -59,7 +60,7 @@ static WorkspaceLayout workspace_layout(const spla_config_t* c) {
   WorkspaceLayout w;
   const size_t U = (size_t)c->batch * c->n_kv_heads, G = c->n_q_heads / c->n_kv_heads, d = c->head_dim;
   const size_t max_blocks = ((size_t)c->max_context + c->block_size - 1) / c->block_size;
-  w.max_chunks = (int)((max_blocks + kScoreChunk - 1) / kScoreChunk);
+  w.max_chunks = (int)((max_blocks + kScoreChunkMin - 1) / kScoreChunkMin);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   w.ell = take(U * G * max_blocks * 4);
@@ -116,6 +117,13 @@ extern "C" int spla_init_cache(const spla_config_t* config, const spla_buffers_t
   c->cfg = *config;
   c->buf = *b;
   c->have_ev = false;
+  c->sm_count = 148;
+  {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+      c->sm_count = n;
+  }
   if (c->cfg.sm_scale == 0.f) c->cfg.sm_scale = 1.0f / sqrtf((float)config->head_dim);
   if (c->cfg.phi_scale == 0.f) c->cfg.phi_scale = 1.0f;
   if (c->cfg.rms_eps == 0.f) c->cfg.rms_eps = 1e-6f;
@@ -176,10 +184,12 @@ extern "C" int spla_append_tokens(spla_cache_t* c, const void* k_new, const void
   return SPLA_OK;
 }
 
-static int chunks_for_bound(const spla_cache* c) {
-  const int64_t blocks = (c->len_bound + c->cfg.block_size - 1) / c->cfg.block_size;
-  const int64_t ch = (blocks + kScoreChunk - 1) / kScoreChunk;
-  return (int)(ch < 1 ? 1 : ch);
+// Sizes the score grid from the host-side bound of the sequence lengths.
+static void plan_score_grid(const spla_cache* c, Params* p) {
+  int64_t blocks = (c->len_bound + c->cfg.block_size - 1) / c->cfg.block_size;
+  if (blocks < 1) blocks = 1;
+  p->chunk = score_chunk_for((long long)p->batch * p->Hkv, blocks, c->sm_count);
+  p->n_chunks_cap = (int)((blocks + p->chunk - 1) / p->chunk);
 }
 
 extern "C" int spla_decode(spla_cache_t* c, const void* q, const float* rms_weight, float* out, int32_t* sel_idx,
@@ -188,7 +198,7 @@ extern "C" int spla_decode(spla_cache_t* c, const void* q, const float* rms_weig
   if (!rms_weight && !(c->cfg.flags & SPLA_NO_RLA)) return SPLA_ERR_INVALID_ARG;
   if (!aligned(q, 16) || !aligned(out, 16)) return SPLA_ERR_INVALID_ARG;
   Params p = c->p;
-  p.n_chunks_cap = chunks_for_bound(c);
+  plan_score_grid(c, &p);
   const int qb = c->cfg.q_dtype == SPLA_BF16;
   cudaStream_t s = (cudaStream_t)stream;
   cudaError_t e = launch_score_select(p, q, qb, sel_idx, s);
@@ -210,7 +220,7 @@ extern "C" int spla_decode_profile(spla_cache_t* c, const void* q, const float* 
     c->have_ev = true;
   }
   Params p = c->p;
-  p.n_chunks_cap = chunks_for_bound(c);
+  plan_score_grid(c, &p);
   const int qb = c->cfg.q_dtype == SPLA_BF16;
   cudaStream_t s = (cudaStream_t)stream;
   e = cudaEventRecord(c->ev[0], s);
@@ -232,6 +242,7 @@ extern "C" int spla_decode_selected(spla_cache_t* c, const void* q, const float*
   if (!aligned(q, 16) || !aligned(out, 16)) return SPLA_ERR_INVALID_ARG;
   Params p = c->p;
   p.n_chunks_cap = 0;                      // only the o_bar CTAs of the first kernel run
+  p.chunk = kScoreChunkMin;
   const int qb = c->cfg.q_dtype == SPLA_BF16;
   cudaStream_t s = (cudaStream_t)stream;
   cudaError_t e = cudaSuccess;

@@ -9,7 +9,8 @@
 namespace spla {
 
 constexpr int kScoreThreads = 256;      // block-score kernel: 8 warps, one block record per warp at a time
-constexpr int kScoreChunk = 64;         // block records per CTA
+constexpr int kScoreChunkMin = 32;      // block records per CTA: a power of two in [32, 512], chosen per launch
+constexpr int kScoreChunkMax = 512;
 constexpr int kStateSplits = 4;         // CTAs per unit that compute o_bar = phi(q) S_bar
 constexpr int kAttendThreads = 128;     // sparse-attend kernel: 4 warps per selected block
 constexpr int kMaxGroup = 16;
@@ -25,6 +26,7 @@ struct Params {
   int kv_bf16;                          // K/V cache element type: 1 = bf16, 0 = fp32
   float sm_scale, phi_scale, rms_eps;
   int n_chunks_cap;                     // score-kernel chunks launched per unit
+  int chunk;                            // block records per score CTA
   // caller buffers
   void* k_cache;
   void* v_cache;

@@ -14,6 +14,7 @@ inline int padded_group(int G) {
 }
 
 // score_select.cu
+int score_chunk_for(long long units, long long max_seq_blocks, int sm_count);
 cudaError_t launch_score_select(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream);
 // attend_merge.cu
 cudaError_t launch_attend_merge(const Params& p, const void* q, int q_is_bf16, const float* rms_weight,
