@@ -9,6 +9,7 @@
 // so the selected linear term costs no extra memory traffic and unselected blocks are never read.
 // The last CTA of the unit (atomic ticket, nobody waits) merges the partials, subtracts o_tilde from
 // o_bar = phi(q) S_bar (Eq. rla-impl-3), applies the RMSNorm and adds the two branches (Section 3.3).
+#include "attend_common.cuh"
 #include "spla_internal.h"
 
 namespace spla {
@@ -33,14 +34,7 @@ __global__ void __launch_bounds__(kAttendThreads) attend_merge_kernel(const Para
 
   const int nsel = p.n_sel[u];
   if (item >= nsel) {
-    if (nsel == 0 && item == 0) {               // empty sequence: the output is zero
-      for (int idx = tid; idx < G * D; idx += kAttendThreads) {
-        const size_t o = ((size_t)b * p.Hq + (size_t)h * G) * D + idx;
-        out[o] = 0.f;
-        if (dbg_sparse) dbg_sparse[o] = 0.f;
-        if (dbg_rla) dbg_rla[o] = 0.f;
-      }
-    }
+    if (nsel == 0 && item == 0) write_zero_unit<D>(p, u, out, dbg_sparse, dbg_rla);   // empty sequence
     return;
   }
   const int blk = p.sel[(size_t)u * p.top_k + item];
@@ -206,68 +200,10 @@ __global__ void __launch_bounds__(kAttendThreads) attend_merge_kernel(const Para
     ml[0] = m_s[tid];
     ml[1] = l_s[tid];
   }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const int t = atomicAdd(&p.attend_ticket[u], 1);
-    flag_s = (t == nsel - 1);
-    if (flag_s) p.attend_ticket[u] = 0;
-  }
-  __syncthreads();
-  if (!flag_s) return;
-  __threadfence();
+  if (!arrive_last(&p.attend_ticket[u], nsel, &flag_s)) return;
 
   // ---- merge (last CTA of the unit) ---------------------------------------------------------------------
-  float* wt_s = reinterpret_cast<float*>(smem_raw);          // [nsel][G] weights exp2(m_it - M) / L
-  float* red_s = wt_s + kMaxTopK * kMaxGroup;                // [NWARP]
-  if (tid < G) {
-    const float* ml = p.att_ml + ((size_t)u * p.top_k * G + tid) * 2;
-    float M = -INFINITY;
-    for (int it = 0; it < nsel; ++it) M = fmaxf(M, __ldcg(ml + (size_t)it * G * 2));
-    float Ls = 0.f;
-    for (int it = 0; it < nsel; ++it) {
-      const float wgt = ex2(__ldcg(ml + (size_t)it * G * 2) - M);
-      wt_s[it * G + tid] = wgt;
-      Ls += wgt * __ldcg(ml + (size_t)it * G * 2 + 1);
-    }
-    const float inv = 1.f / Ls;
-    for (int it = 0; it < nsel; ++it) wt_s[it * G + tid] *= inv;
-  }
-  __syncthreads();
-  const float* parts = p.att_acc + (size_t)u * p.top_k * 2 * G * D;
-  for (int g = 0; g < G; ++g) {
-    float o_sp = 0.f, o_til = 0.f, o_bar = 0.f;
-    if (tid < D) {
-      for (int it = 0; it < nsel; ++it) {
-        const float* pp = parts + (size_t)it * 2 * G * D;
-        o_sp = fmaf(wt_s[it * G + g], __ldcg(pp + (size_t)g * D + tid), o_sp);
-        if (rla) o_til += __ldcg(pp + (size_t)(G + g) * D + tid);
-      }
-      if (rla) {
-#pragma unroll
-        for (int s = 0; s < kStateSplits; ++s)
-          o_bar += __ldcg(p.obar_part + (((size_t)u * kStateSplits + s) * G + g) * D + tid);
-      }
-    }
-    const float r = o_bar - o_til;
-    const size_t o = ((size_t)b * p.Hq + (size_t)h * G + g) * D + tid;
-    float res = o_sp;
-    if (rla) {
-      float sq = warp_sum(tid < D ? r * r : 0.f);
-      __syncthreads();
-      if (lane == 0) red_s[warp] = sq;
-      __syncthreads();
-      float tot = 0.f;
-#pragma unroll
-      for (int w2 = 0; w2 < NWARP; ++w2) tot += red_s[w2];
-      if (tid < D) res += rms_weight[((size_t)h * G + g) * D + tid] * r * rsqrtf(tot / D + p.rms_eps);
-    }
-    if (tid < D) {
-      out[o] = res;
-      if (dbg_sparse) dbg_sparse[o] = o_sp;
-      if (dbg_rla) dbg_rla[o] = r;
-    }
-  }
+  merge_unit<D>(p, u, nsel, rms_weight, out, dbg_sparse, dbg_rla, reinterpret_cast<float*>(smem_raw));
 }
 
 // Copies a caller-given selection into the workspace and counts its valid entries.
@@ -292,7 +228,7 @@ static cudaError_t launch_one(const Params& p, const void* q, int qb, const floa
   constexpr int NWARP = kAttendThreads / 32;
   size_t smem = (size_t)2 * p.B * D * sizeof(T) + (size_t)p.B * sizeof(float) + (size_t)p.B * NV * sizeof(float) +
                 (size_t)(4 * GP + 2 * NWARP * GP) * sizeof(float) + 16;
-  const size_t smem_merge = (size_t)(kMaxTopK * kMaxGroup + NWARP) * sizeof(float);
+  const size_t smem_merge = (size_t)(kMaxTopK * kMaxGroup) * sizeof(float);
   if (smem_merge > smem) smem = smem_merge;
   const size_t smem_red = (size_t)(kAttendThreads / D) * NV * D * sizeof(float);
   if (smem_red > smem) smem = smem_red;
@@ -324,6 +260,8 @@ cudaError_t launch_attend_merge(const Params& p, const void* q, int q_is_bf16, c
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
+  if (p.kv_bf16 && q_is_bf16 && p.G <= 8)
+    return launch_attend_mma(p, q, rms_weight, out, dbg_o_sparse, dbg_o_rla, stream);
   const int GP = padded_group(p.G);
   if (p.kv_bf16) {
     return p.d == 128 ? launch_g<__nv_bfloat16, 128>(p, GP, q, q_is_bf16, rms_weight, out, dbg_o_sparse, dbg_o_rla, stream)

@@ -238,16 +238,16 @@ __global__ void __launch_bounds__(kScoreThreads, 2) score_select_kernel(const Pa
     cp[0] = m;
     cp[1] = s;
   }
-  __threadfence();
-  __syncthreads();
+  __syncthreads();                                       // every thread's stores precede thread 0's fence
   if (tid == 0) {
+    __threadfence();
     const int t = atomicAdd(&p.score_ticket[u], 1);
     is_last_s = (t == n_chunks - 1);
     if (is_last_s) p.score_ticket[u] = 0;                // ready for the next decode step
+    __threadfence();
   }
   __syncthreads();
   if (!is_last_s) return;
-  __threadfence();
 
   // ------------------------------------------------------------------ selection (one CTA per unit) ----
   uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw);           // [max_blocks]
@@ -256,6 +256,20 @@ __global__ void __launch_bounds__(kScoreThreads, 2) score_select_kernel(const Pa
   __shared__ int wtot[2][NWARP];
   __shared__ uint32_t sel_digit_s;
   __shared__ int sel_k_s;
+
+  // The first batch of log masses is requested before the normalisers are reduced: the two do not depend on
+  // each other and each is one L2 round trip.
+  constexpr int SB = 4;                                             // blocks per thread with loads in flight together
+  float e[SB][GP];
+  auto load_batch = [&](int i0) {
+#pragma unroll
+    for (int j = 0; j < SB; ++j) {
+      const int i = i0 + j * kScoreThreads + tid;
+#pragma unroll
+      for (int g = 0; g < GP; ++g) e[j][g] = (g < G && i < nblk) ? __ldcg(ell_u + (size_t)g * p.max_blocks + i) : -INFINITY;
+    }
+  };
+  load_batch(0);
 
   for (int g = warp; g < G; g += NWARP) {
     float m = -INFINITY, s = 0.f;
@@ -276,15 +290,8 @@ __global__ void __launch_bounds__(kScoreThreads, 2) score_select_kernel(const Pa
   float lse_r[GP];
 #pragma unroll
   for (int g = 0; g < GP; ++g) lse_r[g] = g < G ? lse_s[g] : 0.f;
-  constexpr int SB = 4;                                             // blocks per thread with loads in flight together
   for (int i0 = 0; i0 < nblk; i0 += kScoreThreads * SB) {
-    float e[SB][GP];
-#pragma unroll
-    for (int j = 0; j < SB; ++j) {
-      const int i = i0 + j * kScoreThreads + tid;
-#pragma unroll
-      for (int g = 0; g < GP; ++g) e[j][g] = (g < G && i < nblk) ? __ldcg(ell_u + (size_t)g * p.max_blocks + i) : -INFINITY;
-    }
+    if (i0 > 0) load_batch(i0);
 #pragma unroll
     for (int j = 0; j < SB; ++j) {
       const int i = i0 + j * kScoreThreads + tid;
@@ -301,7 +308,8 @@ __global__ void __launch_bounds__(kScoreThreads, 2) score_select_kernel(const Pa
   }
   __syncthreads();
 
-  // radix select: the k_eff-th largest key.  Equal digits inside a warp are counted with one atomic.
+  // radix select: the k_eff-th largest key, 8 bits per pass.  A warp whose active lanes all hold the same
+  // digit (the rule in the exponent pass) adds its count once; otherwise each lane adds for itself.
   uint32_t prefix = 0, mask = 0;
   int kk = k_eff;
   if (k_eff > 0) {
@@ -309,15 +317,21 @@ __global__ void __launch_bounds__(kScoreThreads, 2) score_select_kernel(const Pa
     for (int shift = 24; shift >= 0; shift -= 8) {
       hist[tid] = 0;                                                   // kScoreThreads == 256 bins
       __syncthreads();
+#pragma unroll 4
       for (int i0 = 0; i0 < nblk; i0 += kScoreThreads) {
         const int i = i0 + tid;
         const uint32_t key = i < nblk ? keys[i] : 0u;
         const bool in = i < nblk && (key & mask) == prefix;
         const unsigned act = __ballot_sync(0xffffffffu, in);
-        if (in) {
+        if (act) {
           const uint32_t digit = (key >> shift) & 255u;
-          const unsigned peers = __match_any_sync(act, digit);
-          if (lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
+          const uint32_t first = __shfl_sync(0xffffffffu, digit, __ffs(act) - 1);
+          const unsigned same = __ballot_sync(0xffffffffu, in && digit == first);
+          if (same == act) {
+            if (lane == __ffs(act) - 1) atomicAdd(&hist[first], __popc(act));
+          } else if (in) {
+            atomicAdd(&hist[digit], 1);
+          }
         }
       }
       __syncthreads();

@@ -147,6 +147,7 @@ extern "C" int spla_init_cache(const spla_config_t* config, const spla_buffers_t
   p.score_ticket = (int*)(ws + w.score_ticket); p.attend_ticket = (int*)(ws + w.attend_ticket);
   p.status = (int*)(ws + w.status);
   p.max_chunks = w.max_chunks;
+  p.bpc = 1;
 
   cudaStream_t s = (cudaStream_t)stream;
   cudaError_t e = cudaMemsetAsync(b->workspace, 0, w.total, s);
@@ -192,6 +193,16 @@ static void plan_score_grid(const spla_cache* c, Params* p) {
   p->n_chunks_cap = (int)((blocks + p->chunk - 1) / p->chunk);
 }
 
+// Selected blocks per CTA of the tensor-core attend kernel: more blocks per CTA means fewer split-K partials
+// to merge, as long as the grid still fills the machine.
+static int attend_bpc(const spla_cache* c) {
+  const long long items = (long long)c->p.batch * c->p.Hkv * c->p.top_k;
+  const size_t tile = (size_t)c->p.B * c->p.d * 2 * 2 + (size_t)c->p.B * 4;
+  int bpc = 1;
+  while (bpc < 4 && items / (bpc * 2) >= 3LL * c->sm_count && tile * bpc * 2 <= 100 * 1024) bpc *= 2;
+  return bpc;
+}
+
 extern "C" int spla_decode(spla_cache_t* c, const void* q, const float* rms_weight, float* out, int32_t* sel_idx,
                            float* dbg_o_sparse, float* dbg_o_rla, void* stream) {
   if (!c || !q || !out) return SPLA_ERR_INVALID_ARG;
@@ -199,6 +210,7 @@ extern "C" int spla_decode(spla_cache_t* c, const void* q, const float* rms_weig
   if (!aligned(q, 16) || !aligned(out, 16)) return SPLA_ERR_INVALID_ARG;
   Params p = c->p;
   plan_score_grid(c, &p);
+  p.bpc = attend_bpc(c);
   const int qb = c->cfg.q_dtype == SPLA_BF16;
   cudaStream_t s = (cudaStream_t)stream;
   cudaError_t e = launch_score_select(p, q, qb, sel_idx, s);
@@ -221,6 +233,7 @@ extern "C" int spla_decode_profile(spla_cache_t* c, const void* q, const float* 
   }
   Params p = c->p;
   plan_score_grid(c, &p);
+  p.bpc = attend_bpc(c);
   const int qb = c->cfg.q_dtype == SPLA_BF16;
   cudaStream_t s = (cudaStream_t)stream;
   e = cudaEventRecord(c->ev[0], s);
@@ -243,6 +256,7 @@ extern "C" int spla_decode_selected(spla_cache_t* c, const void* q, const float*
   Params p = c->p;
   p.n_chunks_cap = 0;                      // only the o_bar CTAs of the first kernel run
   p.chunk = kScoreChunkMin;
+  p.bpc = attend_bpc(c);
   const int qb = c->cfg.q_dtype == SPLA_BF16;
   cudaStream_t s = (cudaStream_t)stream;
   cudaError_t e = cudaSuccess;

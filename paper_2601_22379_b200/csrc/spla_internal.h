@@ -20,6 +20,9 @@ cudaError_t launch_score_select(const Params& p, const void* q, int q_is_bf16, i
 cudaError_t launch_attend_merge(const Params& p, const void* q, int q_is_bf16, const float* rms_weight,
                                 const int* sel_in, float* out, float* dbg_o_sparse, float* dbg_o_rla,
                                 cudaStream_t stream);
+// attend_mma.cu (bf16 K/V and q, G <= 8)
+cudaError_t launch_attend_mma(const Params& p, const void* q, const float* rms_weight, float* out, float* dbg_o_sparse,
+                              float* dbg_o_rla, cudaStream_t stream);
 // append.cu
 cudaError_t launch_append(const Params& p, const void* k_new, const void* v_new, const int* n_new, int max_new,
                           cudaStream_t stream);
