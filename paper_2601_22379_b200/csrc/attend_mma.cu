@@ -97,6 +97,7 @@ __global__ void __launch_bounds__(kAttendThreads) attend_mma_kernel(const Params
     if (nsel == 0 && item == 0) write_zero_unit<D>(p, u, out, dbg_sparse, dbg_rla);
     return;
   }
+  SPLA_MARK(p, u, 32 + item, 0);
   const int L = p.seq_lens[b];
   const int j0 = item * bpc;
   const int nb = min(bpc, nsel - j0);
@@ -162,6 +163,7 @@ __global__ void __launch_bounds__(kAttendThreads) attend_mma_kernel(const Params
     }
   }
 
+  SPLA_MARK(p, u, 32 + item, 1);
   // ---- per-warp running state over its slices -----------------------------------------------------------
   float m_run = -INFINITY, l_run = 0.f;      // row g of the exact branch (l: this lane's share)
   float o[NT][4];
@@ -176,6 +178,7 @@ __global__ void __launch_bounds__(kAttendThreads) attend_mma_kernel(const Params
   for (int j = 0; j < nb; ++j) {
     cp_async_wait_pending(4 - 1 - j);        // four groups were committed; block j is group j
     __syncthreads();
+    if (j == 0) SPLA_MARK(p, u, 32 + item, 2);
     const uint32_t ks = smem_u32(smem_raw + (size_t)j * 2 * tile_bytes);
     const uint32_t vs = ks + tile_bytes;
     const float* lse_s = reinterpret_cast<const float*>(lse_base + (size_t)j * B * 4);
@@ -253,6 +256,7 @@ __global__ void __launch_bounds__(kAttendThreads) attend_mma_kernel(const Params
   }
   cp_async_wait_pending(0);
 
+  SPLA_MARK(p, u, 32 + item, 3);
   // ---- fold the four warps together ------------------------------------------------------------------------
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
@@ -296,8 +300,11 @@ __global__ void __launch_bounds__(kAttendThreads) attend_mma_kernel(const Params
     ml[1] = Lg;
   }
 
+  SPLA_MARK(p, u, 32 + item, 4);
   if (!arrive_last(&p.attend_ticket[u], n_items, &flag_s)) return;
+  SPLA_MARK(p, u, 32 + item, 5);
   merge_unit<D>(p, u, n_items, rms_weight, out, dbg_sparse, dbg_rla, reinterpret_cast<float*>(smem_raw));
+  SPLA_MARK(p, u, 32 + item, 6);
 }
 
 template <int D>

@@ -1,5 +1,6 @@
 // C ABI of the library: argument validation, workspace carve-up and kernel launches.  Host code only.
 #include <math.h>
+#include <stdlib.h>
 #include <new>
 #include <stdio.h>
 #include <string.h>
@@ -147,6 +148,9 @@ extern "C" int spla_init_cache(const spla_config_t* config, const spla_buffers_t
   p.score_ticket = (int*)(ws + w.score_ticket); p.attend_ticket = (int*)(ws + w.attend_ticket);
   p.status = (int*)(ws + w.status);
   p.max_chunks = w.max_chunks;
+#ifdef SPLA_TRACE
+  p.trace = getenv("SPLA_TRACE_PTR") ? (unsigned long long*)strtoull(getenv("SPLA_TRACE_PTR"), nullptr, 0) : nullptr;
+#endif
   p.bpc = 1;
 
   cudaStream_t s = (cudaStream_t)stream;

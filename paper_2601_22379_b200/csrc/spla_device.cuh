@@ -48,6 +48,9 @@ struct Params {
   int* attend_ticket;  // [U]
   int* status;         // [1]
   int max_chunks;
+#ifdef SPLA_TRACE
+  unsigned long long* trace;  // development builds only: [unit][64 CTAs][8 marks] of %globaltimer values
+#endif
 };
 
 __device__ __forceinline__ float to_float(float x) { return x; }
@@ -153,6 +156,21 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   }
   return false;
 }
+
+// Development aid, compiled in only with -DSPLA_TRACE (python -m paper_2601_22379_b200.build --trace): thread 0 of
+// a CTA stores %globaltimer at numbered marks so that the phases of a kernel can be laid out on a time line.
+#ifdef SPLA_TRACE
+#define SPLA_MARK(p, unit, cta, k)                                                        \
+  do {                                                                                    \
+    if ((p).trace && threadIdx.x == 0 && (cta) < 64) {                                    \
+      unsigned long long t_;                                                              \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                              \
+      (p).trace[((size_t)(unit) * 64 + (cta)) * 8 + (k)] = t_;                            \
+    }                                                                                     \
+  } while (0)
+#else
+#define SPLA_MARK(p, unit, cta, k) do { } while (0)
+#endif
 
 // Programmatic dependent launch: wait for the preceding grid's memory, allow the next grid to start.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
