@@ -1,0 +1,463 @@
+// Block score + selection, cluster edition: the CTAs that score one (sequence, KV head) unit form a thread-block
+// cluster, so the selection no longer runs as a serial tail in one CTA behind a global-memory hand-off.
+//
+//   phase A  every CTA streams its share of the unit's statistics records through a ring of shared-memory
+//            stages filled by bulk asynchronous copies (a producer warp, full/empty mbarriers) and keeps the
+//            Taylor log masses ell^m_i (Section 3.1 of the paper, Eq. taylor-2nd, diagonal covariance) and its
+//            per-head (max, sum exp) in shared memory;
+//   sync 1   hardware cluster barrier;
+//   phase B  every CTA reads the partial normalisers of its siblings over distributed shared memory, forms the
+//            aggregated BlockScore of its own blocks (Section 2.2: per-head softmax over blocks, summed over the
+//            group), picks its best min(k, n) blocks and pushes them into the leader CTA's memory;
+//   sync 2   hardware cluster barrier;
+//   phase C  the leader picks the top k of the <= 16 x 64 candidates (forced sink / local blocks carry the
+//            maximal key; Section 4 "Sparsity Specifications") and writes them in ascending order, while its
+//            siblings compute o_bar = phi(q) S_bar, the part of the residual branch that needs no selection.
+// Ordering everywhere is (score descending, block index ascending).  The only waits are the two hardware
+// barriers and bounded mbarrier polls.  No multicast is used.
+#include "spla_internal.h"
+#include "state_role.cuh"
+#include "topk_select.cuh"
+
+namespace spla {
+
+namespace {
+
+constexpr int kCsConsumers = 8;                          // consumer warps
+constexpr int kCsThreads = (kCsConsumers + 1) * 32;      // + one producer warp
+constexpr int kStageRec = 32;                            // statistics records per ring stage
+constexpr int kStages = 3;
+constexpr int kMaxCluster = 16;
+constexpr int UNR = kStageRec / kCsConsumers;            // records per warp per stage (4)
+
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float ld_dsmem_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_dsmem_u32(uint32_t addr, uint32_t v) {
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void lse_merge(float& m, float& s, float m2, float s2) {
+  const float nm = fmaxf(m, m2);
+  if (nm > -INFINITY) s = s * __expf(m - nm) + s2 * __expf(m2 - nm);
+  m = nm;
+}
+
+// Sums N per-lane values over aligned groups of W lanes (W = 16 or 32, N <= W a power of two) by halving:
+// afterwards v[0] of lane l holds the group total of the value with index (l % W) / (W / N).
+template <int N, int W>
+__device__ __forceinline__ void group_reduce_multi(float (&v)[N], int lane) {
+  int off = W / 2;
+#pragma unroll
+  for (int n = N; n > 1; n >>= 1) {
+    const bool upper = (lane & off) != 0;
+#pragma unroll
+    for (int i = 0; i < n / 2; ++i) {
+      const float send = upper ? v[i] : v[i + n / 2];
+      const float keep = upper ? v[i + n / 2] : v[i];
+      v[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+    }
+    off >>= 1;
+  }
+#pragma unroll
+  for (; off > 0; off >>= 1) v[0] += __shfl_xor_sync(0xffffffffu, v[0], off);
+}
+
+// Layout of the dynamic shared memory (identical in every CTA, which distributed shared memory relies on).
+template <int D, int GP>
+struct Smem {
+  static constexpr int kRecBytes = 2 * D * 4;
+  static constexpr int kStageBytes = kStageRec * kRecBytes;
+  static constexpr int kRingBytes = kStages * kStageBytes;
+  // after streaming the ring is dead and holds the selection's work arrays:
+  static constexpr int kKeys = 0;                                   // uint32 [1024]        this CTA's block keys
+  static constexpr int kCandKey = kKeys + 1024 * 4;                 // uint32 [16][64]      (the leader's copy is the live one)
+  static constexpr int kCandIdx = kCandKey + kMaxCluster * kMaxTopK * 4;
+  static constexpr int kCandCnt = kCandIdx + kMaxCluster * kMaxTopK * 4;   // int [16]
+  static constexpr int kFlatKey = kCandCnt + 64;                    // uint32 [1024]
+  static constexpr int kFlatIdx = kFlatKey + kMaxCluster * kMaxTopK * 4;
+  static constexpr int kSelTmp = kFlatIdx + kMaxCluster * kMaxTopK * 4;    // int [64]
+  static constexpr int kScratch = (kSelTmp + kMaxTopK * 4 + 15) / 16 * 16; // TopkScratch
+  static constexpr int kWorkEnd = kScratch + (int)sizeof(TopkScratch);
+  static_assert(kWorkEnd <= kRingBytes, "selection work arrays must fit in the dead ring");
+  // fixed region after the ring:
+  static constexpr int kPart = kRingBytes;                          // float [GP][2]  this CTA's (max, sum)
+  static constexpr int kAllPart = kPart + GP * 2 * 4;               // float [16][GP][2]
+  static constexpr int kLse = kAllPart + kMaxCluster * GP * 2 * 4;  // float [GP]
+  static constexpr int kWred = kLse + GP * 4;                       // float [8][GP][2]
+  static constexpr int kBars = (kWred + kCsConsumers * GP * 2 * 4 + 7) / 8 * 8;   // uint64 [2 * kStages]
+  static constexpr int kEll = (kBars + 2 * kStages * 8 + 15) / 16 * 16;            // float [G][chunk]
+};
+
+}  // namespace
+
+template <int D, int GP>
+__global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Params p, const void* __restrict__ q_raw,
+                                                                      int q_is_bf16, int* __restrict__ sel_user) {
+  using SM = Smem<D, GP>;
+  constexpr int W = GP <= 4 ? 16 : 32;          // lanes that share one record
+  constexpr int NGRP = 32 / W;                  // records a warp works on side by side
+  constexpr int PASSES = UNR / NGRP;
+  constexpr int VECW = D / W;                   // floats of the mean (and of the variance) per lane
+  constexpr int NV = 2 * GP;
+  constexpr int LPV = W / NV;                   // lanes holding a copy of each reduced value
+  constexpr int FB = LPV < PASSES ? LPV : PASSES;
+  static_assert(LPV >= 1, "group too large for the lane layout");
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int CS = gridDim.x;
+  const int rank = blockIdx.x;
+  const int G = p.G;
+  const int u = blockIdx.y;
+  const int b = u / p.Hkv, h = u % p.Hkv;
+
+  float* part_s = reinterpret_cast<float*>(smem_raw + SM::kPart);
+  float* all_part = reinterpret_cast<float*>(smem_raw + SM::kAllPart);
+  float* lse_s = reinterpret_cast<float*>(smem_raw + SM::kLse);
+  float* wred = reinterpret_cast<float*>(smem_raw + SM::kWred);
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw + SM::kBars);
+  uint64_t* empty = full + kStages;
+  float* ell_s = reinterpret_cast<float*>(smem_raw + SM::kEll);          // [G][chunk]
+  __shared__ int err_s;
+
+  // ---- queries first: the streaming below saturates the memory system, and a small load issued into that
+  // traffic takes several microseconds.  Lane layout: `hl` of W lanes covers d = c * 4 W + 4 hl .. + 3.
+  const int hl = lane % W, grp = lane / W;
+  float qm[GP][VECW], qv[GP][VECW];
+  if (warp < kCsConsumers) {
+#pragma unroll
+    for (int g = 0; g < GP; ++g) {
+      if (g < G) {
+        const size_t qrow = ((size_t)b * p.Hq + (size_t)h * G + g) * D;
+#pragma unroll
+        for (int c = 0; c < (VECW >= 4 ? VECW / 4 : 1); ++c) {
+          constexpr int CW = VECW >= 4 ? 4 : VECW;
+          float x[CW];
+          const size_t qoff = qrow + (size_t)c * W * 4 + hl * CW;
+          if (q_is_bf16) load_vec<CW>(reinterpret_cast<const __nv_bfloat16*>(q_raw) + qoff, x);
+          else load_vec<CW>(reinterpret_cast<const float*>(q_raw) + qoff, x);
+#pragma unroll
+          for (int v = 0; v < CW; ++v) {
+            qm[g][c * CW + v] = x[v] * p.sm_scale;
+            qv[g][c * CW + v] = (p.flags & 2u) ? 0.f : 0.5f * qm[g][c * CW + v] * qm[g][c * CW + v];
+          }
+        }
+      } else {
+#pragma unroll
+        for (int v = 0; v < VECW; ++v) { qm[g][v] = 0.f; qv[g][v] = 0.f; }
+      }
+    }
+  }
+  const int L = p.seq_lens[b];
+  const int nblk = (L + p.B - 1) / p.B;
+  const int chunk = p.chunk;
+  const int rec_begin = min(nblk, rank * chunk);
+  const int rec_end = min(nblk, rec_begin + chunk);
+  const int n_my = rec_end - rec_begin;
+  const int n_rounds = (n_my + kStageRec - 1) / kStageRec;
+  SPLA_MARK(p, u, rank, 0);
+
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kCsConsumers); }
+    err_s = 0;
+  }
+  __syncthreads();
+  SPLA_MARK(p, u, rank, 1);
+
+  const float* stats_u = p.stats + (size_t)u * p.max_blocks * 2 * D;
+
+  if (warp == kCsConsumers) {
+    // ---------------------------------------------------------------- producer warp ------------------------
+    if (lane == 0) {
+      for (int r = 0; r < n_rounds; ++r) {
+        const int s = r % kStages;
+        if (r >= kStages && !mbar_wait(&empty[s], ((r / kStages) - 1) & 1)) { atomicExch(&err_s, 1); break; }
+        const int nrec = min(kStageRec, n_my - r * kStageRec);
+        const uint32_t bytes = (uint32_t)nrec * SM::kRecBytes;
+        mbar_expect_tx(&full[s], bytes);
+        bulk_g2s(smem_raw + (size_t)s * SM::kStageBytes, stats_u + (size_t)(rec_begin + r * kStageRec) * 2 * D, bytes, &full[s]);
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- consumer warps -----------------------
+    // After the group reduction the first W/2 lanes of a group hold the mean dots and the others the variance
+    // dots, value index (hl % (W/2)) / LPV, each on LPV lanes.  Copy lane `sub` keeps the result of pass `sub`,
+    // so the log / exp work of FB passes runs side by side.
+    const int my_g = (hl % (W / 2)) / LPV;
+    const int sub = hl % LPV;
+    const bool fin_lane = hl < W / 2 && sub < FB && my_g < G;
+    const float ln_full = logf((float)p.B);
+    const float ln_last = logf((float)max(1, L - (nblk - 1) * p.B));
+    float run_max = -INFINITY, run_sum = 0.f;
+
+#pragma unroll 1
+    for (int r = 0; r < n_rounds; ++r) {
+      const int s = r % kStages;
+      if (!mbar_wait(&full[s], (r / kStages) & 1)) { if (lane == 0) atomicExch(&err_s, 1); break; }
+      const int l0 = r * kStageRec + warp * UNR;                       // first record of this warp, CTA-local
+      const float* st = reinterpret_cast<const float*>(smem_raw + (size_t)s * SM::kStageBytes) + (size_t)(warp * UNR) * 2 * D;
+      float mean[PASSES][VECW], var[PASSES][VECW];
+#pragma unroll
+      for (int ps = 0; ps < PASSES; ++ps) {
+        const int rec = ps * NGRP + grp;
+        if (l0 + rec < n_my) {
+#pragma unroll
+          for (int c = 0; c < (VECW >= 4 ? VECW / 4 : 1); ++c) {
+            constexpr int CW = VECW >= 4 ? 4 : VECW;
+            float a[CW], bb[CW];
+            load_vec<CW>(st + (size_t)rec * 2 * D + c * W * 4 + hl * CW, a);
+            load_vec<CW>(st + (size_t)rec * 2 * D + D + c * W * 4 + hl * CW, bb);
+#pragma unroll
+            for (int v = 0; v < CW; ++v) { mean[ps][c * CW + v] = a[v]; var[ps][c * CW + v] = bb[v]; }
+          }
+        } else {
+#pragma unroll
+          for (int v = 0; v < VECW; ++v) { mean[ps][v] = 0.f; var[ps][v] = 0.f; }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty[s]);                            // the stage is in registers: hand it back
+      if (l0 < n_my) {
+#pragma unroll
+        for (int p0 = 0; p0 < PASSES; p0 += FB) {
+          float dm_keep = 0.f, dv_keep = 0.f;
+#pragma unroll
+          for (int pp = 0; pp < FB; ++pp) {
+            float vals[NV];
+#pragma unroll
+            for (int g = 0; g < GP; ++g) {
+              float dm = 0.f, dv = 0.f;
+#pragma unroll
+              for (int v = 0; v < VECW; ++v) {
+                dm = fmaf(qm[g][v], mean[p0 + pp][v], dm);
+                dv = fmaf(qv[g][v], var[p0 + pp][v], dv);
+              }
+              vals[g] = dm;
+              vals[GP + g] = dv;
+            }
+            group_reduce_multi<NV, W>(vals, lane);
+            const float other = __shfl_xor_sync(0xffffffffu, vals[0], W / 2);   // variance dot of the same head
+            if (sub == pp) { dm_keep = vals[0]; dv_keep = other; }
+          }
+          const int li = l0 + (p0 + sub) * NGRP + grp;
+          if (fin_lane && li < n_my) {
+            const float ell = (rec_begin + li == nblk - 1 ? ln_last : ln_full) + dm_keep + __logf(1.f + dv_keep);
+            ell_s[my_g * chunk + li] = ell;
+            const float nm = fmaxf(run_max, ell);
+            run_sum = run_sum * __expf(run_max - nm) + __expf(ell - nm);
+            run_max = nm;
+          }
+        }
+      }
+    }
+    SPLA_MARK(p, u, rank, 2);
+    // fold the finalising lanes of a head: copy lanes (xor < LPV), then the record groups of the warp (xor W)
+#pragma unroll
+    for (int o = 1; o < FB; o <<= 1) {
+      const float m2 = __shfl_xor_sync(0xffffffffu, run_max, o), s2 = __shfl_xor_sync(0xffffffffu, run_sum, o);
+      lse_merge(run_max, run_sum, m2, s2);
+    }
+    if constexpr (NGRP == 2) {
+      const float m2 = __shfl_xor_sync(0xffffffffu, run_max, 16), s2 = __shfl_xor_sync(0xffffffffu, run_sum, 16);
+      lse_merge(run_max, run_sum, m2, s2);
+    }
+    if (fin_lane && sub == 0 && grp == 0) {
+      wred[(warp * GP + my_g) * 2 + 0] = run_max;
+      wred[(warp * GP + my_g) * 2 + 1] = run_sum;
+    }
+  }
+  __syncthreads();
+  if (tid < G) {
+    float m = -INFINITY, s = 0.f;
+#pragma unroll
+    for (int w = 0; w < kCsConsumers; ++w) lse_merge(m, s, wred[(w * GP + tid) * 2], wred[(w * GP + tid) * 2 + 1]);
+    part_s[tid * 2] = m;
+    part_s[tid * 2 + 1] = s;
+  }
+  if (tid == 0 && err_s) atomicExch(p.status, -3);
+
+  cluster_sync_all();                                                   // ---- sync 1: partial normalisers visible
+
+  // ------------------------------------------------------------------ phase B -------------------------------
+  SPLA_MARK(p, u, rank, 3);
+  if (tid < CS * G) {
+    const int r = tid / G, g = tid % G;
+    const uint32_t remote = map_to_rank(smem_u32(part_s + g * 2), (uint32_t)r);
+    all_part[(r * GP + g) * 2] = ld_dsmem_f32(remote);
+    all_part[(r * GP + g) * 2 + 1] = ld_dsmem_f32(remote + 4);
+  }
+  __syncthreads();
+  if (tid < G) {
+    float m = -INFINITY, s = 0.f;
+    for (int r = 0; r < CS; ++r) lse_merge(m, s, all_part[(r * GP + tid) * 2], all_part[(r * GP + tid) * 2 + 1]);
+    lse_s[tid] = m + __logf(s);
+  }
+  __syncthreads();
+
+  uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw + SM::kKeys);
+  TopkScratch* scratch = reinterpret_cast<TopkScratch*>(smem_raw + SM::kScratch);
+  const int k_eff = min(p.top_k, nblk);
+  {
+    float lse_r[GP];
+#pragma unroll
+    for (int g = 0; g < GP; ++g) lse_r[g] = g < G ? lse_s[g] : 0.f;
+    float* scores_u = p.scores + (size_t)u * p.max_blocks;
+    for (int li = tid; li < n_my; li += kCsThreads) {
+      float sc = 0.f;
+#pragma unroll
+      for (int g = 0; g < GP; ++g)
+        if (g < G) sc += __expf(ell_s[g * chunk + li] - lse_r[g]);
+      const int i = rec_begin + li;
+      scores_u[i] = sc;
+      const bool forced = (i < p.n_sink) || (i >= nblk - p.n_local);
+      keys[li] = forced ? 0xffffffffu : __float_as_uint(sc);
+    }
+  }
+  __syncthreads();
+  SPLA_MARK(p, u, rank, 4);
+
+  // this CTA's best min(k_eff, n_my) blocks go to the leader's candidate table
+  {
+    const uint32_t cand_key0 = map_to_rank(smem_u32(smem_raw + SM::kCandKey), 0u) + (uint32_t)rank * kMaxTopK * 4;
+    const uint32_t cand_idx0 = map_to_rank(smem_u32(smem_raw + SM::kCandIdx), 0u) + (uint32_t)rank * kMaxTopK * 4;
+    const int cnt = select_topk(
+        keys, n_my, k_eff, [&](int li) { return rec_begin + li; },
+        [&](int slot, uint32_t key, int idx) {
+          st_dsmem_u32(cand_key0 + (uint32_t)slot * 4, key);
+          st_dsmem_u32(cand_idx0 + (uint32_t)slot * 4, (uint32_t)idx);
+        },
+        scratch);
+    if (tid == 0) st_dsmem_u32(map_to_rank(smem_u32(smem_raw + SM::kCandCnt), 0u) + (uint32_t)rank * 4, (uint32_t)cnt);
+  }
+  SPLA_MARK(p, u, rank, 5);
+
+  cluster_sync_all();                                                   // ---- sync 2: candidates are in the leader
+  SPLA_MARK(p, u, rank, 6);
+  const bool rla = !(p.flags & 4u);
+  if (rank != 0) {
+    // The siblings are done with the selection; while the leader finishes it they compute the part of the
+    // residual branch that needs no selection, o_bar = phi(q) S_bar, one slice of the state's rows each.
+    if (rla)
+      for (int s = rank - 1; s < kStateSplits; s += CS - 1)
+        state_role<D, GP, 256>(p, u, s, q_raw, q_is_bf16, reinterpret_cast<float*>(smem_raw));
+    return;
+  }
+
+  // ------------------------------------------------------------------ phase C (leader) ----------------------
+  const uint32_t* cand_key = reinterpret_cast<const uint32_t*>(smem_raw + SM::kCandKey);
+  const int* cand_idx = reinterpret_cast<const int*>(smem_raw + SM::kCandIdx);
+  const int* cand_cnt = reinterpret_cast<const int*>(smem_raw + SM::kCandCnt);
+  uint32_t* flat_key = reinterpret_cast<uint32_t*>(smem_raw + SM::kFlatKey);
+  int* flat_idx = reinterpret_cast<int*>(smem_raw + SM::kFlatIdx);
+  int* sel_tmp = reinterpret_cast<int*>(smem_raw + SM::kSelTmp);
+  int total = 0;
+  for (int r = 0; r < CS; ++r) {
+    const int cnt = cand_cnt[r];
+    for (int s = tid; s < cnt; s += kCsThreads) {
+      flat_key[total + s] = cand_key[r * kMaxTopK + s];
+      flat_idx[total + s] = cand_idx[r * kMaxTopK + s];
+    }
+    total += cnt;
+  }
+  __syncthreads();
+  select_topk(
+      flat_key, total, k_eff, [&](int c) { return flat_idx[c]; }, [&](int slot, uint32_t, int idx) { sel_tmp[slot] = idx; },
+      scratch);
+  int* sel_u = p.sel + (size_t)u * p.top_k;
+  int* sel_o = sel_user ? sel_user + (size_t)u * p.top_k : nullptr;
+  for (int s = tid; s < p.top_k; s += kCsThreads) {
+    if (s < k_eff) {
+      const int ia = sel_tmp[s];
+      int pos = 0;
+      for (int j = 0; j < k_eff; ++j) pos += sel_tmp[j] < ia;
+      sel_u[pos] = ia;
+      if (sel_o) sel_o[pos] = ia;
+    } else {
+      sel_u[s] = -1;
+      if (sel_o) sel_o[s] = -1;
+    }
+  }
+  if (tid == 0) p.n_sel[u] = k_eff;
+  SPLA_MARK(p, u, rank, 7);
+  if (rla && CS == 1)
+    for (int s = 0; s < kStateSplits; ++s) {
+      __syncthreads();
+      state_role<D, GP, 256>(p, u, s, q_raw, q_is_bf16, reinterpret_cast<float*>(smem_raw));
+    }
+}
+
+template <int D, int GP>
+static cudaError_t launch_one(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream) {
+  using SM = Smem<D, GP>;
+  const int U = p.batch * p.Hkv;
+  size_t smem = (size_t)SM::kEll + (size_t)p.G * p.chunk * sizeof(float);
+  auto kern = score_cluster_kernel<D, GP>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  if (p.cs > 8) {
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (e != cudaSuccess) return e;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(p.cs, U, 1);
+  cfg.blockDim = dim3(kCsThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = p.cs;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, p, q, q_is_bf16, sel_user);
+}
+
+template <int D>
+static cudaError_t launch_d(const Params& p, int GP, const void* q, int qb, int* sel_user, cudaStream_t s) {
+  switch (GP) {
+    case 1: return launch_one<D, 1>(p, q, qb, sel_user, s);
+    case 2: return launch_one<D, 2>(p, q, qb, sel_user, s);
+    case 4: return launch_one<D, 4>(p, q, qb, sel_user, s);
+    default: return launch_one<D, 8>(p, q, qb, sel_user, s);
+  }
+}
+
+// Decides whether the cluster kernel can serve a launch and with which cluster size / records per CTA.
+// Returns false when the general kernel has to be used (very long sequences, groups above 8).
+bool plan_score_cluster(int units, long long max_seq_blocks, int G, int d, int sm_count, int* cs_out, int* chunk_out) {
+  if (G > 8) return false;
+  if (max_seq_blocks < 1) max_seq_blocks = 1;
+  int cs = 1;
+  while (cs < kMaxCluster && max_seq_blocks > 576LL * cs) cs *= 2;            // keep the local ranking short
+  while (cs < kMaxCluster && (long long)units * cs * 2 <= 2LL * sm_count) cs *= 2;   // fill the machine once
+  const long long chunk = (max_seq_blocks + cs - 1) / cs;
+  const int chunk32 = (int)((chunk + 31) / 32 * 32);
+  if (chunk32 > 1024) return false;
+  const size_t ring = (size_t)kStages * kStageRec * 2 * d * 4;
+  if (ring + 4096 + (size_t)G * chunk32 * 4 > 200 * 1024) return false;
+  *cs_out = cs;
+  *chunk_out = chunk32;
+  return true;
+}
+
+cudaError_t launch_score_cluster(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream) {
+  const int GP = padded_group(p.G);
+  return p.d == 128 ? launch_d<128>(p, GP, q, q_is_bf16, sel_user, stream)
+                    : launch_d<64>(p, GP, q, q_is_bf16, sel_user, stream);
+}
+
+}  // namespace spla

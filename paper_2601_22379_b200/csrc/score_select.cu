@@ -12,6 +12,7 @@
 // (atomic ticket, no waiting) reduces the per-chunk normalisers, forms the aggregated score, and picks the
 // top-k by an 8-bit radix select on the score bits followed by an index-ordered compaction.
 #include "spla_internal.h"
+#include "state_role.cuh"
 
 namespace spla {
 
@@ -68,55 +69,7 @@ __global__ void __launch_bounds__(kScoreThreads, 2) score_select_kernel(const Pa
 
   // ------------------------------------------------------------------ o_bar role ----------------------
   if (c >= p.n_chunks_cap) {
-    const int s = c - p.n_chunks_cap;                      // which slice of the state's rows
-    float* phiq = reinterpret_cast<float*>(smem_raw);      // [GP][D]
-    float* red = phiq + GP * D;                            // [kScoreThreads / D][GP][D]
-    const float a2 = p.phi_scale * kLog2e;
-    constexpr int RG = kScoreThreads / D;                  // row groups working side by side
-    constexpr int ROWS = D / kStateSplits / RG;            // rows per thread
-    const int rg = tid / D, j = tid % D;
-    const float* S = p.state + (size_t)u * D * D + (size_t)(s * (D / kStateSplits) + rg) * D + j;
-    float sv[ROWS];
-#pragma unroll
-    for (int r = 0; r < ROWS; ++r) sv[r] = __ldcs(S + (size_t)r * RG * D);     // all loads in flight before use
-    for (int g = warp; g < G; g += NWARP) {
-      float x[VEC];
-      const size_t qoff = ((size_t)b * p.Hq + (size_t)h * G + g) * D + lane * VEC;
-      if (q_is_bf16) load_vec<VEC>(reinterpret_cast<const __nv_bfloat16*>(q_raw) + qoff, x);
-      else load_vec<VEC>(reinterpret_cast<const float*>(q_raw) + qoff, x);
-      float mx = -INFINITY;
-#pragma unroll
-      for (int v = 0; v < VEC; ++v) { x[v] *= a2; mx = fmaxf(mx, x[v]); }
-      mx = warp_max(mx);
-      float sum = 0.f;
-#pragma unroll
-      for (int v = 0; v < VEC; ++v) { x[v] = exp2f(x[v] - mx); sum += x[v]; }
-      sum = warp_sum(sum);
-      const float inv = 1.f / sum;
-#pragma unroll
-      for (int v = 0; v < VEC; ++v) phiq[g * D + lane * VEC + v] = x[v] * inv;
-    }
-    __syncthreads();
-    float acc[GP];
-#pragma unroll
-    for (int g = 0; g < GP; ++g) acc[g] = 0.f;
-#pragma unroll
-    for (int r = 0; r < ROWS; ++r) {
-      const int row = s * (D / kStateSplits) + rg + r * RG;
-#pragma unroll
-      for (int g = 0; g < GP; ++g)
-        if (g < G) acc[g] = fmaf(phiq[g * D + row], sv[r], acc[g]);
-    }
-#pragma unroll
-    for (int g = 0; g < GP; ++g) red[(rg * GP + g) * D + j] = acc[g];
-    __syncthreads();
-    for (int idx = tid; idx < G * D; idx += kScoreThreads) {
-      const int g = idx / D, jj = idx % D;
-      float t = 0.f;
-#pragma unroll
-      for (int r2 = 0; r2 < RG; ++r2) t += red[(r2 * GP + g) * D + jj];
-      p.obar_part[(((size_t)u * kStateSplits + s) * G + g) * D + jj] = t;
-    }
+    state_role<D, GP, kScoreThreads>(p, u, c - p.n_chunks_cap, q_raw, q_is_bf16, reinterpret_cast<float*>(smem_raw));
     return;
   }
 

@@ -193,8 +193,20 @@ extern "C" int spla_append_tokens(spla_cache_t* c, const void* k_new, const void
 static void plan_score_grid(const spla_cache* c, Params* p) {
   int64_t blocks = (c->len_bound + c->cfg.block_size - 1) / c->cfg.block_size;
   if (blocks < 1) blocks = 1;
+  p->cs = 0;
+  int cs = 0, chunk = 0;
+  if (!getenv("SPLA_NO_CLUSTER") && plan_score_cluster(p->batch * p->Hkv, blocks, p->G, p->d, c->sm_count, &cs, &chunk)) {
+    p->cs = cs;
+    p->chunk = chunk;
+    p->n_chunks_cap = cs;
+    return;
+  }
   p->chunk = score_chunk_for((long long)p->batch * p->Hkv, blocks, c->sm_count);
   p->n_chunks_cap = (int)((blocks + p->chunk - 1) / p->chunk);
+}
+
+static cudaError_t launch_score(const Params& p, const void* q, int qb, int* sel_user, cudaStream_t s) {
+  return p.cs > 0 ? launch_score_cluster(p, q, qb, sel_user, s) : launch_score_select(p, q, qb, sel_user, s);
 }
 
 // Selected blocks per CTA of the tensor-core attend kernel: more blocks per CTA means fewer split-K partials
@@ -217,7 +229,7 @@ extern "C" int spla_decode(spla_cache_t* c, const void* q, const float* rms_weig
   p.bpc = attend_bpc(c);
   const int qb = c->cfg.q_dtype == SPLA_BF16;
   cudaStream_t s = (cudaStream_t)stream;
-  cudaError_t e = launch_score_select(p, q, qb, sel_idx, s);
+  cudaError_t e = launch_score(p, q, qb, sel_idx, s);
   if (e != cudaSuccess) return cuda_fail(e, "spla_decode/score_select");
   e = launch_attend_merge(p, q, qb, rms_weight, nullptr, out, dbg_o_sparse, dbg_o_rla, s);
   if (e != cudaSuccess) return cuda_fail(e, "spla_decode/attend_merge");
@@ -241,7 +253,7 @@ extern "C" int spla_decode_profile(spla_cache_t* c, const void* q, const float* 
   const int qb = c->cfg.q_dtype == SPLA_BF16;
   cudaStream_t s = (cudaStream_t)stream;
   e = cudaEventRecord(c->ev[0], s);
-  if (e == cudaSuccess) e = launch_score_select(p, q, qb, nullptr, s);
+  if (e == cudaSuccess) e = launch_score(p, q, qb, nullptr, s);
   if (e == cudaSuccess) e = cudaEventRecord(c->ev[1], s);
   if (e == cudaSuccess) e = launch_attend_merge(p, q, qb, rms_weight, nullptr, out, nullptr, nullptr, s);
   if (e == cudaSuccess) e = cudaEventRecord(c->ev[2], s);
@@ -260,6 +272,7 @@ extern "C" int spla_decode_selected(spla_cache_t* c, const void* q, const float*
   Params p = c->p;
   p.n_chunks_cap = 0;                      // only the o_bar CTAs of the first kernel run
   p.chunk = kScoreChunkMin;
+  p.cs = 0;
   p.bpc = attend_bpc(c);
   const int qb = c->cfg.q_dtype == SPLA_BF16;
   cudaStream_t s = (cudaStream_t)stream;

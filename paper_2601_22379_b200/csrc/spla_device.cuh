@@ -27,6 +27,7 @@ struct Params {
   float sm_scale, phi_scale, rms_eps;
   int n_chunks_cap;                     // score-kernel chunks launched per unit
   int chunk;                            // block records per score CTA
+  int cs;                               // score kernel, cluster edition: CTAs per unit (0 = general kernel)
   int bpc;                              // selected blocks per CTA of the tensor-core attend kernel (1, 2 or 4)
   // caller buffers
   void* k_cache;

@@ -16,6 +16,9 @@ inline int padded_group(int G) {
 // score_select.cu
 int score_chunk_for(long long units, long long max_seq_blocks, int sm_count);
 cudaError_t launch_score_select(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream);
+// score_cluster.cu (G <= 8, at most 16 x 1024 blocks per sequence)
+bool plan_score_cluster(int units, long long max_seq_blocks, int G, int d, int sm_count, int* cs_out, int* chunk_out);
+cudaError_t launch_score_cluster(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream);
 // attend_merge.cu
 cudaError_t launch_attend_merge(const Params& p, const void* q, int q_is_bf16, const float* rms_weight,
                                 const int* sel_in, float* out, float* dbg_o_sparse, float* dbg_o_rla,

@@ -1,0 +1,70 @@
+// o_bar = phi(q) S_bar for one slice of the state's rows (Section 3.2 of the paper, Eq. rla-impl-1): the part of
+// the residual branch that needs neither the selection nor any K/V tile.  Run by spare CTAs of the score kernels.
+#pragma once
+
+#include "spla_device.cuh"
+
+namespace spla {
+
+// NT threads take part (the CTA may be larger; the others only join the barriers).
+// smem: (GP * D + (NT / D) * GP * D) floats.
+template <int D, int GP, int NT>
+__device__ __forceinline__ void state_role(const Params& p, int u, int s, const void* __restrict__ q_raw, int q_is_bf16,
+                                           float* smem) {
+  constexpr int VEC = D / 32;
+  constexpr int RG = NT / D;                             // row groups working side by side
+  constexpr int ROWS = D / kStateSplits / RG;            // rows per thread
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int b = u / p.Hkv, h = u % p.Hkv, G = p.G;
+  const bool act = tid < NT;
+  float* phiq = smem;                                    // [GP][D]
+  float* red = phiq + GP * D;                            // [RG][GP][D]
+  const float a2 = p.phi_scale * kLog2e;
+  const int rg = tid / D, j = tid % D;
+  const float* S = p.state + (size_t)u * D * D + (size_t)(s * (D / kStateSplits) + rg) * D + j;
+  float sv[ROWS];
+#pragma unroll
+  for (int r = 0; r < ROWS; ++r) sv[r] = act ? __ldcs(S + (size_t)r * RG * D) : 0.f;   // all loads in flight before use
+  for (int g = warp; g < G; g += NT / 32) {
+    float x[VEC];
+    const size_t qoff = ((size_t)b * p.Hq + (size_t)h * G + g) * D + lane * VEC;
+    if (q_is_bf16) load_vec<VEC>(reinterpret_cast<const __nv_bfloat16*>(q_raw) + qoff, x);
+    else load_vec<VEC>(reinterpret_cast<const float*>(q_raw) + qoff, x);
+    float mx = -INFINITY;
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) { x[v] *= a2; mx = fmaxf(mx, x[v]); }
+    mx = warp_max(mx);
+    float sum = 0.f;
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) { x[v] = exp2f(x[v] - mx); sum += x[v]; }
+    sum = warp_sum(sum);
+    const float inv = 1.f / sum;
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) phiq[g * D + lane * VEC + v] = x[v] * inv;
+  }
+  __syncthreads();
+  if (act) {
+    float acc[GP];
+#pragma unroll
+    for (int g = 0; g < GP; ++g) acc[g] = 0.f;
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+      const int row = s * (D / kStateSplits) + rg + r * RG;
+#pragma unroll
+      for (int g = 0; g < GP; ++g)
+        if (g < G) acc[g] = fmaf(phiq[g * D + row], sv[r], acc[g]);
+    }
+#pragma unroll
+    for (int g = 0; g < GP; ++g) red[(rg * GP + g) * D + j] = acc[g];
+  }
+  __syncthreads();
+  for (int idx = tid; idx < G * D; idx += blockDim.x) {
+    const int g = idx / D, jj = idx % D;
+    float t = 0.f;
+#pragma unroll
+    for (int r2 = 0; r2 < RG; ++r2) t += red[(r2 * GP + g) * D + jj];
+    p.obar_part[(((size_t)u * kStateSplits + s) * G + g) * D + jj] = t;
+  }
+}
+
+}  // namespace spla
