@@ -12,11 +12,11 @@ namespace spla {
 __device__ __forceinline__ bool arrive_last(int* ticket, int expected, int* flag_smem) {
   __syncthreads();                                   // all partial-result stores precede thread 0's fence
   if (threadIdx.x == 0) {
-    __threadfence();
+    asm volatile("fence.acq_rel.gpu;" ::: "memory");   // release the CTA's stores (cumulative over the barrier above)
     const int t = atomicAdd(ticket, 1);
     const int last = (t == expected - 1);
     if (last) *ticket = 0;
-    __threadfence();
+    asm volatile("fence.acq_rel.gpu;" ::: "memory");   // acquire the other CTAs' stores
     *flag_smem = last;
   }
   __syncthreads();
@@ -44,6 +44,27 @@ __device__ __forceinline__ void merge_unit(const Params& p, int u, int n_items, 
   const bool rla = !(p.flags & 4u) && p.n_sel[u] < nblk_u;
   float* wt_s = smem;                                // [n_items][G]: exp2(m_it - M) / L
 
+  // The first batch of partial results is requested before the weights are formed: the two are independent
+  // and each costs one L2 round trip.
+  const int hg = tid / C4, c4 = tid % C4;
+  const float* parts = p.att_acc + (size_t)u * p.top_k * 2 * G * D;
+  float4 a[IU], t[IU];
+  auto fetch = [&](int g, int it0) {
+#pragma unroll
+    for (int j = 0; j < IU; ++j) {
+      const int it = it0 + j;
+      if (it < n_items) {
+        const float* pp = parts + (size_t)it * 2 * G * D;
+        a[j] = __ldcg(reinterpret_cast<const float4*>(pp + (size_t)g * D) + c4);
+        t[j] = rla ? __ldcg(reinterpret_cast<const float4*>(pp + (size_t)(G + g) * D) + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+      } else {
+        a[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        t[j] = a[j];
+      }
+    }
+  };
+  if (hg < G) fetch(hg, 0);
+
   // softmax weights of the items: one warp per head, lanes over items
   const float* ml_u = p.att_ml + (size_t)u * p.top_k * G * 2;
   for (int g = warp; g < G; g += kAttendThreads / 32) {
@@ -66,8 +87,6 @@ __device__ __forceinline__ void merge_unit(const Params& p, int u, int n_items, 
   }
   __syncthreads();
 
-  const int hg = tid / C4, c4 = tid % C4;
-  const float* parts = p.att_acc + (size_t)u * p.top_k * 2 * G * D;
   for (int g0 = 0; g0 < G; g0 += HG) {
     const int g = g0 + hg;
     const bool live = g < G;
@@ -81,19 +100,7 @@ __device__ __forceinline__ void merge_unit(const Params& p, int u, int n_items, 
         }
       }
       for (int it0 = 0; it0 < n_items; it0 += IU) {
-        float4 a[IU], t[IU];
-#pragma unroll
-        for (int j = 0; j < IU; ++j) {
-          const int it = it0 + j;
-          if (it < n_items) {
-            const float* pp = parts + (size_t)it * 2 * G * D;
-            a[j] = __ldcg(reinterpret_cast<const float4*>(pp + (size_t)g * D) + c4);
-            t[j] = rla ? __ldcg(reinterpret_cast<const float4*>(pp + (size_t)(G + g) * D) + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
-          } else {
-            a[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-            t[j] = a[j];
-          }
-        }
+        if (g0 > 0 || it0 > 0) fetch(g, it0);
 #pragma unroll
         for (int j = 0; j < IU; ++j) {
           const int it = it0 + j;

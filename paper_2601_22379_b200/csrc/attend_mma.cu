@@ -72,7 +72,7 @@ constexpr int kPad = 8;   // floats of padding per row of the cross-warp reducti
 }  // namespace
 
 template <int D>
-__global__ void __launch_bounds__(kAttendThreads) attend_mma_kernel(const Params p, const __nv_bfloat16* __restrict__ q,
+__global__ void __launch_bounds__(kAttendThreads, 3) attend_mma_kernel(const Params p, const __nv_bfloat16* __restrict__ q,
                                                                     const float* __restrict__ rms_weight,
                                                                     float* __restrict__ out, float* __restrict__ dbg_sparse,
                                                                     float* __restrict__ dbg_rla) {
@@ -91,47 +91,11 @@ __global__ void __launch_bounds__(kAttendThreads) attend_mma_kernel(const Params
   const int G = p.G, B = p.B, bpc = p.bpc;
   const bool rla = !(p.flags & 4u);
 
-  const int nsel = p.n_sel[u];
-  const int n_items = (nsel + bpc - 1) / bpc;
-  if (item >= n_items) {
-    if (nsel == 0 && item == 0) write_zero_unit<D>(p, u, out, dbg_sparse, dbg_rla);
-    return;
-  }
-  SPLA_MARK(p, u, 32 + item, 0);
-  const int L = p.seq_lens[b];
-  const int j0 = item * bpc;
-  const int nb = min(bpc, nsel - j0);
-  const int tile_bytes = B * ROWB;
-  unsigned char* lse_base = smem_raw + (size_t)bpc * 2 * tile_bytes;
-
-  // ---- stage the tiles: 16-byte async copies, chunk index XOR (row & 7), rows past the sequence end zero-filled
-  int n_tok[4];
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    n_tok[j] = 0;
-    if (j < nb) {
-      const int blk = p.sel[(size_t)u * p.top_k + j0 + j];
-      n_tok[j] = min(B, L - blk * B);
-      const size_t tile = (size_t)u * p.max_blocks + blk;
-      const __nv_bfloat16* ksrc = reinterpret_cast<const __nv_bfloat16*>(p.k_cache) + tile * B * D;
-      const __nv_bfloat16* vsrc = reinterpret_cast<const __nv_bfloat16*>(p.v_cache) + tile * B * D;
-      const uint32_t kdst = smem_u32(smem_raw + (size_t)j * 2 * tile_bytes);
-      const uint32_t vdst = kdst + tile_bytes;
-      for (int idx = tid; idx < B * CPR; idx += kAttendThreads) {
-        const int row = idx / CPR, ch = idx % CPR;
-        const uint32_t off = row * ROWB + ((ch ^ (row & 7)) << 4);
-        const int sz = row < n_tok[j] ? 16 : 0;
-        cp_async16(kdst + off, ksrc + (size_t)row * D + ch * 8, sz);
-        cp_async16(vdst + off, vsrc + (size_t)row * D + ch * 8, sz);
-      }
-      if (tid < B / 4) cp_async16(smem_u32(lse_base + (size_t)j * B * 4) + tid * 16, p.tok_lse + tile * B + tid * 4, 16);
-    }
-    cp_async_commit();
-  }
-
-  // ---- query fragments (rows = heads of the group), held in registers for the whole CTA -----------------
+  pdl_launch_dependents();
+  // ---- query fragments first: they depend on nothing the preceding kernel writes, so under programmatic
+  // dependent launch this part overlaps that kernel's tail.  Rows = heads of the group, held in registers.
   // qa: rows 0..7 of the first product (raw q; the softmax scale is applied to the fp32 logits);
-  // fa: rows 8..15 of the second product, phi(q) = softmax(phi_scale * q) rounded to bf16.
+  // fa: rows 8..15 of the second product, phi(q) = softmax(phi_scale * q) in fp16.
   uint32_t qa[KS][2], fa[KS][2];
   {
     const bool hv = g < G;
@@ -140,10 +104,12 @@ __global__ void __launch_bounds__(kAttendThreads) attend_mma_kernel(const Params
     float mx = -INFINITY;
 #pragma unroll
     for (int kk = 0; kk < KS; ++kk) {
-      qa[kk][0] = hv ? qrow[8 * kk + t] : 0u;
-      qa[kk][1] = hv ? qrow[8 * kk + 4 + t] : 0u;
-      mx = fmaxf(mx, fmaxf(fmaxf(bf16_lo(qa[kk][0]), bf16_hi(qa[kk][0])), fmaxf(bf16_lo(qa[kk][1]), bf16_hi(qa[kk][1]))));
+      qa[kk][0] = hv ? __ldg(qrow + 8 * kk + t) : 0u;
+      qa[kk][1] = hv ? __ldg(qrow + 8 * kk + 4 + t) : 0u;
     }
+#pragma unroll
+    for (int kk = 0; kk < KS; ++kk)
+      mx = fmaxf(mx, fmaxf(fmaxf(bf16_lo(qa[kk][0]), bf16_hi(qa[kk][0])), fmaxf(bf16_lo(qa[kk][1]), bf16_hi(qa[kk][1]))));
     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
     float e[KS][4], sum = 0.f;
@@ -161,6 +127,50 @@ __global__ void __launch_bounds__(kAttendThreads) attend_mma_kernel(const Params
       fa[kk][0] = pack_f16(e[kk][0] * inv, e[kk][1] * inv);
       fa[kk][1] = pack_f16(e[kk][2] * inv, e[kk][3] * inv);
     }
+  }
+
+  pdl_wait();                                   // the selection of this step is complete and visible from here on
+
+  // one round trip: the count, the (speculatively addressed) block indices of this CTA, the sequence length
+  const int j0 = item * bpc;
+  const int nsel = __ldcg(p.n_sel + u);
+  const int L = __ldcg(p.seq_lens + b);
+  int blk_j[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) blk_j[j] = __ldcg(p.sel + (size_t)u * p.top_k + min(j0 + j, p.top_k - 1));
+  const int n_items = (nsel + bpc - 1) / bpc;
+  if (item >= n_items) {
+    if (nsel == 0 && item == 0) write_zero_unit<D>(p, u, out, dbg_sparse, dbg_rla);
+    return;
+  }
+  SPLA_MARK(p, u, 32 + item, 0);
+  const int nb = min(bpc, nsel - j0);
+  const int tile_bytes = B * ROWB;
+  unsigned char* lse_base = smem_raw + (size_t)bpc * 2 * tile_bytes;
+
+  // ---- stage the tiles: 16-byte async copies, chunk index XOR (row & 7), rows past the sequence end zero-filled
+  int n_tok[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    n_tok[j] = 0;
+    if (j < nb) {
+      const int blk = blk_j[j];
+      n_tok[j] = min(B, L - blk * B);
+      const size_t tile = (size_t)u * p.max_blocks + blk;
+      const __nv_bfloat16* ksrc = reinterpret_cast<const __nv_bfloat16*>(p.k_cache) + tile * B * D;
+      const __nv_bfloat16* vsrc = reinterpret_cast<const __nv_bfloat16*>(p.v_cache) + tile * B * D;
+      const uint32_t kdst = smem_u32(smem_raw + (size_t)j * 2 * tile_bytes);
+      const uint32_t vdst = kdst + tile_bytes;
+      for (int idx = tid; idx < B * CPR; idx += kAttendThreads) {
+        const int row = idx / CPR, ch = idx % CPR;
+        const uint32_t off = row * ROWB + ((ch ^ (row & 7)) << 4);
+        const int sz = row < n_tok[j] ? 16 : 0;
+        cp_async16(kdst + off, ksrc + (size_t)row * D + ch * 8, sz);
+        cp_async16(vdst + off, vsrc + (size_t)row * D + ch * 8, sz);
+      }
+      if (tid < B / 4) cp_async16(smem_u32(lse_base + (size_t)j * B * 4) + tid * 16, p.tok_lse + tile * B + tid * 4, 16);
+    }
+    cp_async_commit();
   }
 
   SPLA_MARK(p, u, 32 + item, 1);
@@ -319,8 +329,8 @@ static cudaError_t launch_mma(const Params& p, const void* q, const float* w, fl
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid((p.top_k + p.bpc - 1) / p.bpc, p.batch * p.Hkv);
-  kern<<<grid, kAttendThreads, smem, stream>>>(p, reinterpret_cast<const __nv_bfloat16*>(q), w, out, ds, dr);
-  return cudaGetLastError();
+  return launch_ex(kern, grid, dim3(kAttendThreads), smem, stream, 0, true, p, reinterpret_cast<const __nv_bfloat16*>(q), w, out,
+                   ds, dr);
 }
 
 cudaError_t launch_attend_mma(const Params& p, const void* q, const float* rms_weight, float* out, float* dbg_o_sparse,

@@ -133,6 +133,9 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   float* ell_s = reinterpret_cast<float*>(smem_raw + SM::kEll);          // [G][chunk]
   __shared__ int err_s;
 
+  pdl_wait();                                   // everything the preceding kernels wrote (statistics, lengths, q) is visible
+  pdl_launch_dependents();                      // only now may the next kernel begin its prologue: it reads q before its own wait
+
   // ---- queries first: the streaming below saturates the memory system, and a small load issued into that
   // traffic takes several microseconds.  Lane layout: `hl` of W lanes covers d = c * 4 W + 4 hl .. + 3.
   const int hl = lane % W, grp = lane / W;
@@ -411,19 +414,7 @@ static cudaError_t launch_one(const Params& p, const void* q, int q_is_bf16, int
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) return e;
   }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(p.cs, U, 1);
-  cfg.blockDim = dim3(kCsThreads, 1, 1);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = p.cs;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, p, q, q_is_bf16, sel_user);
+  return launch_ex(kern, dim3(p.cs, U, 1), dim3(kCsThreads, 1, 1), smem, stream, p.cs, true, p, q, q_is_bf16, sel_user);
 }
 
 template <int D>

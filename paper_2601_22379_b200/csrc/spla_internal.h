@@ -13,6 +13,36 @@ inline int padded_group(int G) {
   return gp;
 }
 
+// Launch with optional thread-block-cluster shape and programmatic dependent launch: with `pdl` the grid may
+// start while the preceding kernel of the stream drains; it must execute griddepcontrol.wait before it touches
+// anything that kernel produces (every kernel launched this way does so in its prologue).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_ex(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, int cluster_x,
+                             bool pdl, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  if (cluster_x > 0) {
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = cluster_x;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  if (pdl) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // score_select.cu
 int score_chunk_for(long long units, long long max_seq_blocks, int sm_count);
 cudaError_t launch_score_select(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream);
