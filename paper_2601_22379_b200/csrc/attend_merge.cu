@@ -252,16 +252,16 @@ static cudaError_t launch_g(const Params& p, int GP, const void* q, int qb, cons
   }
 }
 
-cudaError_t launch_attend_merge(const Params& p, const void* q, int q_is_bf16, const float* rms_weight,
-                                const int* sel_in, float* out, float* dbg_o_sparse, float* dbg_o_rla,
-                                cudaStream_t stream) {
+cudaError_t launch_attend_merge(const Params& p, const AttendMaps* maps, const void* q, int q_is_bf16,
+                                const float* rms_weight, const int* sel_in, float* out, float* dbg_o_sparse,
+                                float* dbg_o_rla, cudaStream_t stream) {
   if (sel_in) {
     adopt_selection_kernel<<<p.batch * p.Hkv, 64, 0, stream>>>(p, sel_in);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
-  if (p.kv_bf16 && q_is_bf16 && p.G <= 8)
-    return launch_attend_mma(p, q, rms_weight, out, dbg_o_sparse, dbg_o_rla, stream);
+  if (p.kv_bf16 && q_is_bf16 && p.G <= 8 && maps && maps->valid && p.acs > 0)
+    return launch_attend_mma(p, *maps, q, rms_weight, out, dbg_o_sparse, dbg_o_rla, stream);
   const int GP = padded_group(p.G);
   if (p.kv_bf16) {
     return p.d == 128 ? launch_g<__nv_bfloat16, 128>(p, GP, q, q_is_bf16, rms_weight, out, dbg_o_sparse, dbg_o_rla, stream)

@@ -1,34 +1,49 @@
 // Sparse attention + fused residual-linear term for bf16 K/V on tensor cores (GQA groups of up to 8 heads).
 //
-// For one (unit, group of selected blocks) the CTA stages the K and V tiles with 16-byte asynchronous copies
-// into an XOR-swizzled shared-memory layout, and each warp walks 16-token slices.  Per slice the query group
-// is the M side of two thin products that share one accumulator tile,
-//     rows 0..7  :  S   = Q K^T           (exact branch,  Section 2.2, Eq. gqa-sparse)
-//     rows 8..15 :  A   = phi(Q) phi(K)^T (linear branch, Section 3.2, Eq. rla-impl-2)
-// where phi(K) is formed element-wise from the very K fragments just used (one ex2 per element, with the
-// cached per-token log-sum-exp), so the selected linear term reads nothing extra.  After the online softmax
-// on rows 0..7 the tile [P ; A] is the left operand of one product with the V tile, which accumulates the
-// softmax numerator (rows 0..7) and o_tilde (rows 8..15) together.  The last CTA of the unit merges.
+// The CTAs that serve one (sequence, KV head) unit form a thread-block cluster; CTA r of the cluster walks the
+// selected blocks r, r + CS, r + 2 CS, ... through a two-slot shared-memory ring that TMA fills (tiled tensor
+// copies with the 128-byte swizzle, so the ldmatrix reads below are bank-conflict free).  Each warp takes
+// 16-token slices.  Per slice the query group is the M side of two thin products that share one accumulator,
+//     rows 0..7  :  S = Q K^T            (exact branch,  Section 2.2 of the paper, Eq. gqa-sparse)
+//     rows 8..15 :  A = phi(Q) phi(K)^T  (linear branch, Section 3.2, Eq. rla-impl-2)
+// where phi(K) is formed element-wise from the very K fragments just used (one ex2 per element, with the cached
+// per-token log-sum-exp), so the selected linear term reads nothing extra.  After the online softmax on rows
+// 0..7 the tile [P ; A] is the left operand of one product with the V tile, which accumulates the softmax
+// numerator and o_tilde together.  The linear coefficients keep ~16 bits: bf16 head plus bf16 remainder (for
+// groups of up to 4 heads the remainder rides in the rows that would otherwise be padding).
+//
+// Merge (Eq. rla-impl-3, Section 3.3): after a hardware cluster barrier CTA g of the cluster pulls head g's
+// partial results from its siblings over distributed shared memory, subtracts o_tilde from o_bar, applies the
+// RMSNorm and writes the output.  The only waits are two cluster barriers and bounded mbarrier polls.
+#include <cuda.h>
 #include <cuda_fp16.h>
 
-#include "attend_common.cuh"
 #include "spla_internal.h"
 
 namespace spla {
 
 namespace {
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+constexpr int kSlots = 2;
+
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_pending(int n) {   // at most n groups still in flight
-  switch (n) {
-    case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
-    case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
-    case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
-    default: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
-  }
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float ld_dsmem_f32(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+  return v;
+}
+// Tiled TMA load of one box (never multicast): coordinates {x = element column, y = row}.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+               "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+               : "memory");
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -71,25 +86,30 @@ constexpr int kPad = 8;   // floats of padding per row of the cross-warp reducti
 
 }  // namespace
 
-template <int D>
-__global__ void __launch_bounds__(kAttendThreads, 3) attend_mma_kernel(const Params p, const __nv_bfloat16* __restrict__ q,
-                                                                    const float* __restrict__ rms_weight,
-                                                                    float* __restrict__ out, float* __restrict__ dbg_sparse,
-                                                                    float* __restrict__ dbg_rla) {
+// PACK: the group has at most 4 heads, so accumulator rows 4..7 and 12..15 are padding; rows 12..15 then carry
+// the bf16 remainder of the linear coefficients and no extra products are needed for it.
+template <int D, bool PACK>
+__global__ void __launch_bounds__(kAttendThreads, 3)
+    attend_mma_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                      const __nv_bfloat16* __restrict__ q, const float* __restrict__ rms_weight, float* __restrict__ out,
+                      float* __restrict__ dbg_sparse, float* __restrict__ dbg_rla) {
   constexpr int KS = D / 16;        // k-steps of the two QK-type products
   constexpr int NT = D / 8;         // n-tiles of the PV-type product
-  constexpr int CPR = D / 8;        // 16-byte chunks per K/V row
-  constexpr int ROWB = D * 2;       // bytes per K/V row
+  constexpr int NH = D / 64;        // 64-column halves of a tile (one TMA box each)
   constexpr int NWARP = kAttendThreads / 32;
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  __shared__ int flag_s;
+  __shared__ __align__(8) uint64_t full[kSlots];
+  __shared__ float red_s[NWARP];
+  __shared__ int sel_s[kMaxTopK];
+  __shared__ int err_s;
 
-  const int u = blockIdx.y, item = blockIdx.x;
+  const int u = blockIdx.y;
+  const int rank = blockIdx.x, CS = gridDim.x;
   const int b = u / p.Hkv, h = u % p.Hkv;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
-  const int G = p.G, B = p.B, bpc = p.bpc;
-  const bool rla = !(p.flags & 4u);
+  const int G = p.G, B = p.B;
+  const bool rla_on = !(p.flags & 4u);
 
   pdl_launch_dependents();
   // ---- query fragments first: they depend on nothing the preceding kernel writes, so under programmatic
@@ -121,59 +141,45 @@ __global__ void __launch_bounds__(kAttendThreads, 3) attend_mma_kernel(const Par
     }
     sum += __shfl_xor_sync(0xffffffffu, sum, 1);
     sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-    const float inv = (hv && rla) ? 1.f / sum : 0.f;
+    const float inv = (hv && rla_on) ? 1.f / sum : 0.f;
 #pragma unroll
     for (int kk = 0; kk < KS; ++kk) {
       fa[kk][0] = pack_f16(e[kk][0] * inv, e[kk][1] * inv);
       fa[kk][1] = pack_f16(e[kk][2] * inv, e[kk][3] * inv);
     }
   }
+  if (tid == 0) {
+    for (int s = 0; s < kSlots; ++s) mbar_init(&full[s], 1);
+    err_s = 0;
+  }
 
   pdl_wait();                                   // the selection of this step is complete and visible from here on
 
-  // one round trip: the count, the (speculatively addressed) block indices of this CTA, the sequence length
-  const int j0 = item * bpc;
   const int nsel = __ldcg(p.n_sel + u);
   const int L = __ldcg(p.seq_lens + b);
-  int blk_j[4];
-#pragma unroll
-  for (int j = 0; j < 4; ++j) blk_j[j] = __ldcg(p.sel + (size_t)u * p.top_k + min(j0 + j, p.top_k - 1));
-  const int n_items = (nsel + bpc - 1) / bpc;
-  if (item >= n_items) {
-    if (nsel == 0 && item == 0) write_zero_unit<D>(p, u, out, dbg_sparse, dbg_rla);
-    return;
-  }
-  SPLA_MARK(p, u, 32 + item, 0);
-  const int nb = min(bpc, nsel - j0);
-  const int tile_bytes = B * ROWB;
-  unsigned char* lse_base = smem_raw + (size_t)bpc * 2 * tile_bytes;
+  for (int i = tid; i < p.top_k; i += kAttendThreads) sel_s[i] = __ldcg(p.sel + (size_t)u * p.top_k + i);
+  __syncthreads();                              // selection list and barrier initialisation visible to the CTA
+  SPLA_MARK(p, u, 32 + rank, 0);
 
-  // ---- stage the tiles: 16-byte async copies, chunk index XOR (row & 7), rows past the sequence end zero-filled
-  int n_tok[4];
+  const int nb = nsel > rank ? (nsel - rank + CS - 1) / CS : 0;     // my blocks: j = rank + i * CS
+  const int tile_bytes = B * D * 2;
+  const int slot_bytes = (2 * tile_bytes + B * 4 + 1023) & ~1023;   // K tile, V tile, per-token lse; the swizzle needs 1 KB alignment
+  auto issue = [&](int i) {                                          // thread 0 only
+    const int slot = i & 1;
+    const int blk = sel_s[rank + i * CS];
+    const uint32_t base = smem_u32(smem_raw + (size_t)slot * slot_bytes);
+    const int row0 = (int)(((size_t)u * p.max_blocks + blk) * B);
+    mbar_expect_tx(&full[slot], (uint32_t)(2 * tile_bytes + B * 4));
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    n_tok[j] = 0;
-    if (j < nb) {
-      const int blk = blk_j[j];
-      n_tok[j] = min(B, L - blk * B);
-      const size_t tile = (size_t)u * p.max_blocks + blk;
-      const __nv_bfloat16* ksrc = reinterpret_cast<const __nv_bfloat16*>(p.k_cache) + tile * B * D;
-      const __nv_bfloat16* vsrc = reinterpret_cast<const __nv_bfloat16*>(p.v_cache) + tile * B * D;
-      const uint32_t kdst = smem_u32(smem_raw + (size_t)j * 2 * tile_bytes);
-      const uint32_t vdst = kdst + tile_bytes;
-      for (int idx = tid; idx < B * CPR; idx += kAttendThreads) {
-        const int row = idx / CPR, ch = idx % CPR;
-        const uint32_t off = row * ROWB + ((ch ^ (row & 7)) << 4);
-        const int sz = row < n_tok[j] ? 16 : 0;
-        cp_async16(kdst + off, ksrc + (size_t)row * D + ch * 8, sz);
-        cp_async16(vdst + off, vsrc + (size_t)row * D + ch * 8, sz);
-      }
-      if (tid < B / 4) cp_async16(smem_u32(lse_base + (size_t)j * B * 4) + tid * 16, p.tok_lse + tile * B + tid * 4, 16);
+    for (int hh = 0; hh < NH; ++hh) {
+      tma_load_2d(base + hh * (B * 128), &map_k, hh * 64, row0, &full[slot]);
+      tma_load_2d(base + tile_bytes + hh * (B * 128), &map_v, hh * 64, row0, &full[slot]);
     }
-    cp_async_commit();
-  }
+    bulk_g2s(smem_raw + (size_t)slot * slot_bytes + 2 * tile_bytes, p.tok_lse + (size_t)row0, (uint32_t)(B * 4), &full[slot]);
+  };
+  if (tid == 0)
+    for (int i = 0; i < min(kSlots, nb); ++i) issue(i);
 
-  SPLA_MARK(p, u, 32 + item, 1);
   // ---- per-warp running state over its slices -----------------------------------------------------------
   float m_run = -INFINITY, l_run = 0.f;      // row g of the exact branch (l: this lane's share)
   float o[NT][4];
@@ -183,16 +189,29 @@ __global__ void __launch_bounds__(kAttendThreads, 3) attend_mma_kernel(const Par
   const float a2 = p.phi_scale * kLog2e;
   const int spb = B / 16;                    // slices per block
   const int mi = lane >> 3, r8 = lane & 7;   // ldmatrix: which 8x8 matrix this lane addresses, and which row
+  const int half_bytes = B * 128;
 
 #pragma unroll 1
-  for (int j = 0; j < nb; ++j) {
-    cp_async_wait_pending(4 - 1 - j);        // four groups were committed; block j is group j
-    __syncthreads();
-    if (j == 0) SPLA_MARK(p, u, 32 + item, 2);
-    const uint32_t ks = smem_u32(smem_raw + (size_t)j * 2 * tile_bytes);
+  for (int i = 0; i < nb; ++i) {
+    const int slot = i & 1;
+    if (!mbar_wait(&full[slot], (i >> 1) & 1)) { if (lane == 0) atomicExch(&err_s, 1); break; }
+    if (i == 0) SPLA_MARK(p, u, 32 + rank, 2);
+    unsigned char* sb = smem_raw + (size_t)slot * slot_bytes;
+    const uint32_t ks = smem_u32(sb);
     const uint32_t vs = ks + tile_bytes;
-    const float* lse_s = reinterpret_cast<const float*>(lse_base + (size_t)j * B * 4);
-    const int ntok = n_tok[j];
+    const float* lse_s = reinterpret_cast<const float*>(sb + 2 * tile_bytes);
+    const int blk = sel_s[rank + i * CS];
+    const int ntok = min(B, L - blk * B);
+    if (ntok < B) {
+      // the open block of the sequence: rows past its end hold whatever the cache memory holds; the value rows
+      // must be zero so that (probability 0) x (garbage) cannot produce a NaN
+      for (int idx = tid; idx < (B - ntok) * (D / 8); idx += kAttendThreads) {
+        const int row = ntok + idx / (D / 8), ch = idx % (D / 8);
+        *reinterpret_cast<uint4*>(sb + tile_bytes + (ch >> 3) * half_bytes + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) =
+            make_uint4(0u, 0u, 0u, 0u);
+      }
+      __syncthreads();
+    }
 #pragma unroll 1
     for (int sl = warp; sl < spb; sl += NWARP) {
       const int tok0 = sl * 16;
@@ -201,18 +220,19 @@ __global__ void __launch_bounds__(kAttendThreads, 3) attend_mma_kernel(const Par
       float sacc[2][4];
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt) { sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f; }
-      const uint32_t krow = ks + (tok0 + (mi >> 1) * 8 + r8) * ROWB;
+      const uint32_t krow = ks + (tok0 + (mi >> 1) * 8 + r8) * 128;
 #pragma unroll
       for (int kk = 0; kk < KS; ++kk) {
         uint32_t kb[4];
-        ldmatrix_x4(kb, krow + (((2 * kk + (mi & 1)) ^ r8) << 4));
+        const int ch = 2 * kk + (mi & 1);
+        ldmatrix_x4(kb, krow + (ch >> 3) * half_bytes + (((ch & 7) ^ r8) << 4));
         mma_bf16(sacc[0], qa[kk][0], 0u, qa[kk][1], 0u, kb[0], kb[1]);
         mma_bf16(sacc[1], qa[kk][0], 0u, qa[kk][1], 0u, kb[2], kb[3]);
         uint32_t pb[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float ls = i < 2 ? lse2_0 : lse2_1;
-          pb[i] = pack_f16(ex2(fmaf(bf16_lo(kb[i]), a2, -ls)), ex2(fmaf(bf16_hi(kb[i]), a2, -ls)));
+        for (int x = 0; x < 4; ++x) {
+          const float ls = x < 2 ? lse2_0 : lse2_1;
+          pb[x] = pack_f16(ex2(fmaf(bf16_lo(kb[x]), a2, -ls)), ex2(fmaf(bf16_hi(kb[x]), a2, -ls)));
         }
         mma_f16(sacc[0], 0u, fa[kk][0], 0u, fa[kk][1], pb[0], pb[1]);
         mma_f16(sacc[1], 0u, fa[kk][0], 0u, fa[kk][1], pb[2], pb[3]);
@@ -244,42 +264,56 @@ __global__ void __launch_bounds__(kAttendThreads, 3) attend_mma_kernel(const Par
       l_run = fmaf(l_run, corr, psum);
       // [P ; A] as the left operand of the product with V (bf16, like V).  The linear coefficients are split
       // into a bf16 head and a bf16 remainder so that o_tilde keeps ~16 bits of them.
-      const uint32_t pa0 = pack_bf16(sacc[0][0], sacc[0][1]), pa1 = pack_bf16(sacc[0][2], sacc[0][3]);
-      const uint32_t pa2 = pack_bf16(sacc[1][0], sacc[1][1]), pa3 = pack_bf16(sacc[1][2], sacc[1][3]);
+      const uint32_t pa0 = pack_bf16(sacc[0][0], sacc[0][1]), pa2 = pack_bf16(sacc[1][0], sacc[1][1]);
+      uint32_t pa1 = pack_bf16(sacc[0][2], sacc[0][3]), pa3 = pack_bf16(sacc[1][2], sacc[1][3]);
       const uint32_t ra1 = pack_bf16(sacc[0][2] - bf16_lo(pa1), sacc[0][3] - bf16_hi(pa1));
       const uint32_t ra3 = pack_bf16(sacc[1][2] - bf16_lo(pa3), sacc[1][3] - bf16_hi(pa3));
-      const uint32_t vrow = vs + (tok0 + (mi & 1) * 8 + r8) * ROWB;
+      if constexpr (PACK) {                            // rows 12..15 <- remainders of heads 0..3 (lanes 16 below)
+        const uint32_t u1 = __shfl_up_sync(0xffffffffu, ra1, 16), u3 = __shfl_up_sync(0xffffffffu, ra3, 16);
+        if (g >= 4) { pa1 = u1; pa3 = u3; }
+      }
+      const uint32_t vrow = vs + (tok0 + (mi & 1) * 8 + r8) * 128;
 #pragma unroll
       for (int np = 0; np < NT / 2; ++np) {
         uint32_t vb[4];
-        ldmatrix_x4_trans(vb, vrow + (((2 * np + (mi >> 1)) ^ r8) << 4));
+        const int ch = 2 * np + (mi >> 1);
+        ldmatrix_x4_trans(vb, vrow + (ch >> 3) * half_bytes + (((ch & 7) ^ r8) << 4));
         o[2 * np][0] *= corr; o[2 * np][1] *= corr;
         o[2 * np + 1][0] *= corr; o[2 * np + 1][1] *= corr;
         mma_bf16(o[2 * np], pa0, pa1, pa2, pa3, vb[0], vb[1]);
         mma_bf16(o[2 * np + 1], pa0, pa1, pa2, pa3, vb[2], vb[3]);
-        if (rla) {
-          mma_bf16(o[2 * np], 0u, ra1, 0u, ra3, vb[0], vb[1]);
-          mma_bf16(o[2 * np + 1], 0u, ra1, 0u, ra3, vb[2], vb[3]);
+        if constexpr (!PACK) {
+          if (rla_on) {
+            mma_bf16(o[2 * np], 0u, ra1, 0u, ra3, vb[0], vb[1]);
+            mma_bf16(o[2 * np + 1], 0u, ra1, 0u, ra3, vb[2], vb[3]);
+          }
         }
       }
     }
+    __syncthreads();                                   // every warp is done with this slot
+    if (tid == 0 && i + kSlots < nb) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy reads before the async-proxy refill
+      issue(i + kSlots);
+    }
   }
-  cp_async_wait_pending(0);
+  if (tid == 0 && err_s) atomicExch(p.status, -3);
 
-  SPLA_MARK(p, u, 32 + item, 3);
+  SPLA_MARK(p, u, 32 + rank, 3);
   // ---- fold the four warps together ------------------------------------------------------------------------
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-  __syncthreads();                                   // the tiles are dead: their space becomes the reduction buffer
+  __syncthreads();                                   // the ring is dead: its space becomes the reduction buffer
   float* red_o = reinterpret_cast<float*>(smem_raw);                    // [NWARP][16][D + kPad]
   float* red_m = red_o + NWARP * 16 * (D + kPad);                       // [NWARP][8]
   float* red_l = red_m + NWARP * 8;                                     // [NWARP][8]
+  float* mine = red_l + NWARP * 8;                                      // [2][8][D]   this CTA's partial result
+  float* mine_ml = mine + 2 * 8 * D;                                    // [8][2]      (max, sum) of the exact branch
   if (t == 0) red_m[warp * 8 + g] = m_run;
   __syncthreads();
   float M = red_m[g];
 #pragma unroll
   for (int w = 1; w < NWARP; ++w) M = fmaxf(M, red_m[w * 8 + g]);
-  const float f = ex2(m_run - M);                    // 0 for a warp that saw no token
+  const float f = M > -INFINITY ? ex2(m_run - M) : 0.f;                 // 0 for a warp (or a CTA) that saw no token
   if (t == 0) red_l[warp * 8 + g] = l_run * f;
   {
     float* ro = red_o + (size_t)warp * 16 * (D + kPad);
@@ -290,53 +324,112 @@ __global__ void __launch_bounds__(kAttendThreads, 3) attend_mma_kernel(const Par
     }
   }
   __syncthreads();
-  float* part = p.att_acc + ((size_t)u * p.top_k + item) * 2 * G * D;
-  for (int idx = tid; idx < 2 * G * D; idx += kAttendThreads) {
-    const int row = idx / D, col = idx % D;            // row < G: exact branch of head row; else linear branch
-    const int rr = row < G ? row : 8 + (row - G);
+  for (int idx = tid; idx < 2 * 8 * D; idx += kAttendThreads) {
+    const int br = idx / (8 * D), hd = (idx / D) % 8, col = idx % D;    // branch, head, column
     float s = 0.f;
+    if (hd < G) {
+      const int rr = br * 8 + hd;
 #pragma unroll
-    for (int w = 0; w < NWARP; ++w) s += red_o[((size_t)w * 16 + rr) * (D + kPad) + col];
-    part[idx] = s;
+      for (int w = 0; w < NWARP; ++w) {
+        s += red_o[((size_t)w * 16 + rr) * (D + kPad) + col];
+        if (PACK && br == 1) s += red_o[((size_t)w * 16 + rr + 4) * (D + kPad) + col];
+      }
+    }
+    mine[idx] = s;
   }
-  if (tid < G) {
+  if (tid < 8) {
     float Mg = red_m[tid], Lg = 0.f;
 #pragma unroll
     for (int w = 1; w < NWARP; ++w) Mg = fmaxf(Mg, red_m[w * 8 + tid]);
 #pragma unroll
     for (int w = 0; w < NWARP; ++w) Lg += red_l[w * 8 + tid];
-    float* ml = p.att_ml + (((size_t)u * p.top_k + item) * G + tid) * 2;
-    ml[0] = Mg;
-    ml[1] = Lg;
+    mine_ml[tid * 2] = Mg;
+    mine_ml[tid * 2 + 1] = Lg;
   }
+  SPLA_MARK(p, u, 32 + rank, 4);
 
-  SPLA_MARK(p, u, 32 + item, 4);
-  if (!arrive_last(&p.attend_ticket[u], n_items, &flag_s)) return;
-  SPLA_MARK(p, u, 32 + item, 5);
-  merge_unit<D>(p, u, n_items, rms_weight, out, dbg_sparse, dbg_rla, reinterpret_cast<float*>(smem_raw));
-  SPLA_MARK(p, u, 32 + item, 6);
+  cluster_sync_all();                                // ---- every CTA's partial result is in its shared memory
+  SPLA_MARK(p, u, 32 + rank, 5);
+
+  // ---- merge: CTA r of the cluster owns heads r, r + CS, ...; one thread per output column ---------------
+  const int nblk_u = (L + B - 1) / B;
+  const bool rla = rla_on && nsel < nblk_u;          // everything selected: the residual is exactly zero
+  for (int hd = rank; hd < G; hd += CS) {
+    const int col = tid;
+    float o_sp = 0.f, o_til = 0.f, o_bar = 0.f;
+    if (nsel > 0) {
+      float Mx = -INFINITY;
+      for (int r = 0; r < CS; ++r) Mx = fmaxf(Mx, ld_dsmem_f32(map_to_rank(smem_u32(mine_ml + hd * 2), (uint32_t)r)));
+      float Ls = 0.f;
+      for (int r = 0; r < CS; ++r) {
+        const uint32_t rm = map_to_rank(smem_u32(mine_ml + hd * 2), (uint32_t)r);
+        const float w = ex2(ld_dsmem_f32(rm) - Mx);
+        Ls = fmaf(w, ld_dsmem_f32(rm + 4), Ls);
+        if (col < D) {
+          o_sp = fmaf(w, ld_dsmem_f32(map_to_rank(smem_u32(mine + hd * D + col), (uint32_t)r)), o_sp);
+          if (rla) o_til += ld_dsmem_f32(map_to_rank(smem_u32(mine + (8 + hd) * D + col), (uint32_t)r));
+        }
+      }
+      o_sp /= Ls;
+      if (rla && col < D) {
+#pragma unroll
+        for (int s = 0; s < kStateSplits; ++s)
+          o_bar += __ldcg(p.obar_part + (((size_t)u * kStateSplits + s) * G + hd) * D + col);
+      }
+    }
+    const float r_ = (rla && col < D) ? o_bar - o_til : 0.f;
+    float sq = warp_sum(r_ * r_);
+    __syncthreads();
+    if (lane == 0) red_s[warp] = sq;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < NWARP; ++w) tot += red_s[w];
+    if (col < D) {
+      const size_t oidx = ((size_t)b * p.Hq + (size_t)h * G + hd) * D + col;
+      float res = o_sp;
+      if (rla) res += rms_weight[((size_t)h * G + hd) * D + col] * r_ * rsqrtf(tot / D + p.rms_eps);
+      out[oidx] = res;
+      if (dbg_sparse) dbg_sparse[oidx] = o_sp;
+      if (dbg_rla) dbg_rla[oidx] = r_;
+    }
+  }
+  SPLA_MARK(p, u, 32 + rank, 6);
+  cluster_sync_all();                                // ---- nobody leaves while a sibling may still read its memory
+}
+
+size_t attend_mma_smem_bytes(int B, int D) {
+  const size_t ring = (size_t)kSlots * ((2 * (size_t)B * D * 2 + (size_t)B * 4 + 1023) / 1024 * 1024);
+  const size_t fold = (size_t)((kAttendThreads / 32) * (16 * (D + kPad) + 16) + 2 * 8 * D + 16) * sizeof(float);
+  return ring > fold ? ring : fold;
 }
 
 template <int D>
-static cudaError_t launch_mma(const Params& p, const void* q, const float* w, float* out, float* ds, float* dr,
-                              cudaStream_t stream) {
-  const size_t tiles = (size_t)p.bpc * (2 * (size_t)p.B * D * 2 + (size_t)p.B * 4);
-  const size_t red = (size_t)(kAttendThreads / 32) * (16 * (D + kPad) + 16) * sizeof(float);
-  size_t smem = tiles > red ? tiles : red;
-  const size_t merge = (size_t)kMaxTopK * kMaxGroup * sizeof(float);
-  if (merge > smem) smem = merge;
-  auto kern = attend_mma_kernel<D>;
+static cudaError_t launch_mma(const Params& p, const AttendMaps& maps, const void* q, const float* w, float* out, float* ds,
+                              float* dr, cudaStream_t stream) {
+  const size_t smem = attend_mma_smem_bytes(p.B, D);
+  const dim3 grid(p.acs, p.batch * p.Hkv);
+  const CUtensorMap& mk = *reinterpret_cast<const CUtensorMap*>(maps.k);
+  const CUtensorMap& mv = *reinterpret_cast<const CUtensorMap*>(maps.v);
+  const __nv_bfloat16* qb = reinterpret_cast<const __nv_bfloat16*>(q);
+  if (p.G <= 4) {
+    auto kern = attend_mma_kernel<D, true>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess && p.acs > 8) e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (e != cudaSuccess) return e;
+    return launch_ex(kern, grid, dim3(kAttendThreads), smem, stream, p.acs, true, p, mk, mv, qb, w, out, ds, dr);
+  }
+  auto kern = attend_mma_kernel<D, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e == cudaSuccess && p.acs > 8) e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
   if (e != cudaSuccess) return e;
-  dim3 grid((p.top_k + p.bpc - 1) / p.bpc, p.batch * p.Hkv);
-  return launch_ex(kern, grid, dim3(kAttendThreads), smem, stream, 0, true, p, reinterpret_cast<const __nv_bfloat16*>(q), w, out,
-                   ds, dr);
+  return launch_ex(kern, grid, dim3(kAttendThreads), smem, stream, p.acs, true, p, mk, mv, qb, w, out, ds, dr);
 }
 
-cudaError_t launch_attend_mma(const Params& p, const void* q, const float* rms_weight, float* out, float* dbg_o_sparse,
-                              float* dbg_o_rla, cudaStream_t stream) {
-  return p.d == 128 ? launch_mma<128>(p, q, rms_weight, out, dbg_o_sparse, dbg_o_rla, stream)
-                    : launch_mma<64>(p, q, rms_weight, out, dbg_o_sparse, dbg_o_rla, stream);
+cudaError_t launch_attend_mma(const Params& p, const AttendMaps& maps, const void* q, const float* rms_weight, float* out,
+                              float* dbg_o_sparse, float* dbg_o_rla, cudaStream_t stream) {
+  return p.d == 128 ? launch_mma<128>(p, maps, q, rms_weight, out, dbg_o_sparse, dbg_o_rla, stream)
+                    : launch_mma<64>(p, maps, q, rms_weight, out, dbg_o_sparse, dbg_o_rla, stream);
 }
 
 }  // namespace spla

@@ -5,6 +5,8 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <cuda.h>
+
 #include "../../include/spla.h"
 #include "spla_internal.h"
 
@@ -18,6 +20,7 @@ struct spla_cache {
   cudaEvent_t ev[3];   // created on first use by spla_decode_profile
   bool have_ev;
   int sm_count;
+  AttendMaps maps;
 };
 
 static thread_local char g_cuda_err[256] = "";
@@ -28,6 +31,28 @@ static int cuda_fail(cudaError_t e, const char* where) {
 }
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// TMA tensor map over a K or V cache seen as a 2-D bf16 matrix [batch * H_kv * max_blocks * B rows][d columns]:
+// boxes of B rows x 64 columns (128 bytes, the widest the 128-byte swizzle allows).
+static bool make_kv_map(void* out128, void* base, int d, int B, unsigned long long rows) {
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static EncodeFn encode = nullptr;
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult st;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &st) != cudaSuccess || !fn) return false;
+    encode = (EncodeFn)fn;
+  }
+  const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)d * 2};
+  const cuuint32_t box[2] = {64u, (cuuint32_t)B};
+  const cuuint32_t estr[2] = {1u, 1u};
+  return encode(reinterpret_cast<CUtensorMap*>(out128), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 
 static int validate_config(const spla_config_t* c) {
   if (!c) return SPLA_ERR_INVALID_ARG;
@@ -151,7 +176,13 @@ extern "C" int spla_init_cache(const spla_config_t* config, const spla_buffers_t
 #ifdef SPLA_TRACE
   p.trace = getenv("SPLA_TRACE_PTR") ? (unsigned long long*)strtoull(getenv("SPLA_TRACE_PTR"), nullptr, 0) : nullptr;
 #endif
-  p.bpc = 1;
+  p.acs = 0;
+
+  c->maps.valid = false;
+  if (p.kv_bf16) {
+    const unsigned long long rows = (unsigned long long)p.batch * p.Hkv * p.max_blocks * p.B;
+    c->maps.valid = make_kv_map(c->maps.k, b->k_cache, p.d, p.B, rows) && make_kv_map(c->maps.v, b->v_cache, p.d, p.B, rows);
+  }
 
   cudaStream_t s = (cudaStream_t)stream;
   cudaError_t e = cudaMemsetAsync(b->workspace, 0, w.total, s);
@@ -209,6 +240,21 @@ static cudaError_t launch_score(const Params& p, const void* q, int qb, int* sel
   return p.cs > 0 ? launch_score_cluster(p, q, qb, sel_user, s) : launch_score_select(p, q, qb, sel_user, s);
 }
 
+// Cluster size of the tensor-core attend kernel: the largest power of two (at most 16 and at most top_k) for
+// which all CTAs are resident at once; each CTA of a cluster then walks top_k / size selected blocks.
+static int attend_cluster_size(const spla_cache* c) {
+  const size_t smem = attend_mma_smem_bytes(c->p.B, c->p.d) + 2048;
+  long long per_sm = (227 * 1024) / (long long)smem;
+  if (per_sm > 3) per_sm = 3;
+  if (per_sm < 1) return 0;                       // the tiles do not fit: use the general kernel
+  const long long slots = per_sm * c->sm_count;
+  const long long U = (long long)c->p.batch * c->p.Hkv;
+  int cs = 1;
+  while (cs * 2 <= 16 && cs * 2 <= c->p.top_k && U * cs * 2 <= slots) cs *= 2;
+  return cs;
+}
+
+
 // Selected blocks per CTA of the tensor-core attend kernel: more blocks per CTA means fewer split-K partials
 // to merge, as long as the grid still fills the machine.
 static int attend_bpc(const spla_cache* c) {
@@ -226,12 +272,12 @@ extern "C" int spla_decode(spla_cache_t* c, const void* q, const float* rms_weig
   if (!aligned(q, 16) || !aligned(out, 16)) return SPLA_ERR_INVALID_ARG;
   Params p = c->p;
   plan_score_grid(c, &p);
-  p.bpc = attend_bpc(c);
+  p.acs = attend_cluster_size(c);
   const int qb = c->cfg.q_dtype == SPLA_BF16;
   cudaStream_t s = (cudaStream_t)stream;
   cudaError_t e = launch_score(p, q, qb, sel_idx, s);
   if (e != cudaSuccess) return cuda_fail(e, "spla_decode/score_select");
-  e = launch_attend_merge(p, q, qb, rms_weight, nullptr, out, dbg_o_sparse, dbg_o_rla, s);
+  e = launch_attend_merge(p, &c->maps, q, qb, rms_weight, nullptr, out, dbg_o_sparse, dbg_o_rla, s);
   if (e != cudaSuccess) return cuda_fail(e, "spla_decode/attend_merge");
   return SPLA_OK;
 }
@@ -249,13 +295,13 @@ extern "C" int spla_decode_profile(spla_cache_t* c, const void* q, const float* 
   }
   Params p = c->p;
   plan_score_grid(c, &p);
-  p.bpc = attend_bpc(c);
+  p.acs = attend_cluster_size(c);
   const int qb = c->cfg.q_dtype == SPLA_BF16;
   cudaStream_t s = (cudaStream_t)stream;
   e = cudaEventRecord(c->ev[0], s);
   if (e == cudaSuccess) e = launch_score(p, q, qb, nullptr, s);
   if (e == cudaSuccess) e = cudaEventRecord(c->ev[1], s);
-  if (e == cudaSuccess) e = launch_attend_merge(p, q, qb, rms_weight, nullptr, out, nullptr, nullptr, s);
+  if (e == cudaSuccess) e = launch_attend_merge(p, &c->maps, q, qb, rms_weight, nullptr, out, nullptr, nullptr, s);
   if (e == cudaSuccess) e = cudaEventRecord(c->ev[2], s);
   if (e == cudaSuccess) e = cudaEventSynchronize(c->ev[2]);
   if (e == cudaSuccess) e = cudaEventElapsedTime(&stage_ms[0], c->ev[0], c->ev[1]);
@@ -273,13 +319,13 @@ extern "C" int spla_decode_selected(spla_cache_t* c, const void* q, const float*
   p.n_chunks_cap = 0;                      // only the o_bar CTAs of the first kernel run
   p.chunk = kScoreChunkMin;
   p.cs = 0;
-  p.bpc = attend_bpc(c);
+  p.acs = attend_cluster_size(c);
   const int qb = c->cfg.q_dtype == SPLA_BF16;
   cudaStream_t s = (cudaStream_t)stream;
   cudaError_t e = cudaSuccess;
   if (!(c->cfg.flags & SPLA_NO_RLA)) e = launch_score_select(p, q, qb, nullptr, s);
   if (e != cudaSuccess) return cuda_fail(e, "spla_decode_selected/o_bar");
-  e = launch_attend_merge(p, q, qb, rms_weight, sel_in, out, dbg_o_sparse, dbg_o_rla, s);
+  e = launch_attend_merge(p, &c->maps, q, qb, rms_weight, sel_in, out, dbg_o_sparse, dbg_o_rla, s);
   if (e != cudaSuccess) return cuda_fail(e, "spla_decode_selected/attend_merge");
   return SPLA_OK;
 }

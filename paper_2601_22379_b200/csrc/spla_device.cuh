@@ -28,7 +28,7 @@ struct Params {
   int n_chunks_cap;                     // score-kernel chunks launched per unit
   int chunk;                            // block records per score CTA
   int cs;                               // score kernel, cluster edition: CTAs per unit (0 = general kernel)
-  int bpc;                              // selected blocks per CTA of the tensor-core attend kernel (1, 2 or 4)
+  int acs;                              // tensor-core attend kernel: CTAs (cluster size) per unit
   // caller buffers
   void* k_cache;
   void* v_cache;

@@ -49,13 +49,19 @@ cudaError_t launch_score_select(const Params& p, const void* q, int q_is_bf16, i
 // score_cluster.cu (G <= 8, at most 16 x 1024 blocks per sequence)
 bool plan_score_cluster(int units, long long max_seq_blocks, int G, int d, int sm_count, int* cs_out, int* chunk_out);
 cudaError_t launch_score_cluster(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream);
+struct AttendMaps {                      // TMA tensor maps (CUtensorMap) of the K and V caches, opaque to the host code
+  alignas(64) unsigned char k[128];
+  alignas(64) unsigned char v[128];
+  bool valid;
+};
 // attend_merge.cu
-cudaError_t launch_attend_merge(const Params& p, const void* q, int q_is_bf16, const float* rms_weight,
-                                const int* sel_in, float* out, float* dbg_o_sparse, float* dbg_o_rla,
-                                cudaStream_t stream);
+cudaError_t launch_attend_merge(const Params& p, const AttendMaps* maps, const void* q, int q_is_bf16,
+                                const float* rms_weight, const int* sel_in, float* out, float* dbg_o_sparse,
+                                float* dbg_o_rla, cudaStream_t stream);
 // attend_mma.cu (bf16 K/V and q, G <= 8)
-cudaError_t launch_attend_mma(const Params& p, const void* q, const float* rms_weight, float* out, float* dbg_o_sparse,
-                              float* dbg_o_rla, cudaStream_t stream);
+size_t attend_mma_smem_bytes(int B, int D);
+cudaError_t launch_attend_mma(const Params& p, const AttendMaps& maps, const void* q, const float* rms_weight, float* out,
+                              float* dbg_o_sparse, float* dbg_o_rla, cudaStream_t stream);
 // append.cu
 cudaError_t launch_append(const Params& p, const void* k_new, const void* v_new, const int* n_new, int max_new,
                           cudaStream_t stream);
