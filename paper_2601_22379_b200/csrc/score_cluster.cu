@@ -2,7 +2,7 @@
 // cluster, so the selection no longer runs as a serial tail in one CTA behind a global-memory hand-off.
 //
 //   phase A  every CTA streams its share of the unit's statistics records through a ring of shared-memory
-//            stages filled by bulk asynchronous copies (a producer warp, full/empty mbarriers) and keeps the
+//            stages filled by bulk asynchronous copies (full/empty mbarriers; one thread feeds the ring) and keeps the
 //            Taylor log masses ell^m_i (Section 3.1 of the paper, Eq. taylor-2nd, diagonal covariance) and its
 //            per-head (max, sum exp) in shared memory;
 //   sync 1   hardware cluster barrier;
@@ -23,8 +23,8 @@ namespace spla {
 
 namespace {
 
-constexpr int kCsConsumers = 8;                          // consumer warps
-constexpr int kCsThreads = (kCsConsumers + 1) * 32;      // + one producer warp
+constexpr int kCsConsumers = 8;                          // warps; all consume, lane 0 of warp 0 also feeds the ring
+constexpr int kCsThreads = kCsConsumers * 32;
 constexpr int kStageRec = 32;                            // statistics records per ring stage
 constexpr int kStages = 3;
 constexpr int kMaxCluster = 16;
@@ -140,7 +140,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   // traffic takes several microseconds.  Lane layout: `hl` of W lanes covers d = c * 4 W + 4 hl .. + 3.
   const int hl = lane % W, grp = lane / W;
   float qm[GP][VECW], qv[GP][VECW];
-  if (warp < kCsConsumers) {
+  {
 #pragma unroll
     for (int g = 0; g < GP; ++g) {
       if (g < G) {
@@ -182,20 +182,16 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
 
   const float* stats_u = p.stats + (size_t)u * p.max_blocks * 2 * D;
 
-  if (warp == kCsConsumers) {
-    // ---------------------------------------------------------------- producer warp ------------------------
-    if (lane == 0) {
-      for (int r = 0; r < n_rounds; ++r) {
-        const int s = r % kStages;
-        if (r >= kStages && !mbar_wait(&empty[s], ((r / kStages) - 1) & 1)) { atomicExch(&err_s, 1); break; }
-        const int nrec = min(kStageRec, n_my - r * kStageRec);
-        const uint32_t bytes = (uint32_t)nrec * SM::kRecBytes;
-        mbar_expect_tx(&full[s], bytes);
-        bulk_g2s(smem_raw + (size_t)s * SM::kStageBytes, stats_u + (size_t)(rec_begin + r * kStageRec) * 2 * D, bytes, &full[s]);
-      }
-    }
-  } else {
-    // ---------------------------------------------------------------- consumer warps -----------------------
+  auto issue = [&](int r) {                      // thread 0 only: one bulk copy fills stage r % kStages
+    const int s = r % kStages;
+    const int nrec = min(kStageRec, n_my - r * kStageRec);
+    const uint32_t bytes = (uint32_t)nrec * SM::kRecBytes;
+    mbar_expect_tx(&full[s], bytes);
+    bulk_g2s(smem_raw + (size_t)s * SM::kStageBytes, stats_u + (size_t)(rec_begin + r * kStageRec) * 2 * D, bytes, &full[s]);
+  };
+  if (tid == 0)
+    for (int r = 0; r < min(kStages, n_rounds); ++r) issue(r);
+  {
     // After the group reduction the first W/2 lanes of a group hold the mean dots and the others the variance
     // dots, value index (hl % (W/2)) / LPV, each on LPV lanes.  Copy lane `sub` keeps the result of pass `sub`,
     // so the log / exp work of FB passes runs side by side.
@@ -233,6 +229,11 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[s]);                            // the stage is in registers: hand it back
+      if (tid == 0 && r + kStages < n_rounds) {                         // refill it once every warp has done the same
+        if (mbar_wait(&empty[s], (r / kStages) & 1)) issue(r + kStages);
+        else atomicExch(&err_s, 1);
+      }
+      __syncwarp();
       if (l0 < n_my) {
 #pragma unroll
         for (int p0 = 0; p0 < PASSES; p0 += FB) {
