@@ -111,6 +111,7 @@ __global__ void __launch_bounds__(kAttendThreads, 3)
   const int G = p.G, B = p.B;
   const bool rla_on = !(p.flags & 4u);
 
+  SPLA_MARK(p, u, 32 + rank, 1);
   pdl_launch_dependents();
   // ---- query fragments first: they depend on nothing the preceding kernel writes, so under programmatic
   // dependent launch this part overlaps that kernel's tail.  Rows = heads of the group, held in registers.
@@ -217,9 +218,14 @@ __global__ void __launch_bounds__(kAttendThreads, 3)
       const int tok0 = sl * 16;
       if (tok0 >= ntok) break;
       const float lse2_0 = lse_s[tok0 + g] * kLog2e, lse2_1 = lse_s[tok0 + 8 + g] * kLog2e;
-      float sacc[2][4];
+      // two accumulator tiles per n-tile (one per product) so that the dependent chain of each is half as long;
+      // rows 0..7 of the first and rows 8..15 of the second are the meaningful halves
+      float sacc[2][4], aacc[2][4];
 #pragma unroll
-      for (int nt = 0; nt < 2; ++nt) { sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f; }
+      for (int nt = 0; nt < 2; ++nt) {
+        sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f;
+        aacc[nt][0] = aacc[nt][1] = aacc[nt][2] = aacc[nt][3] = 0.f;
+      }
       const uint32_t krow = ks + (tok0 + (mi >> 1) * 8 + r8) * 128;
 #pragma unroll
       for (int kk = 0; kk < KS; ++kk) {
@@ -234,8 +240,8 @@ __global__ void __launch_bounds__(kAttendThreads, 3)
           const float ls = x < 2 ? lse2_0 : lse2_1;
           pb[x] = pack_f16(ex2(fmaf(bf16_lo(kb[x]), a2, -ls)), ex2(fmaf(bf16_hi(kb[x]), a2, -ls)));
         }
-        mma_f16(sacc[0], 0u, fa[kk][0], 0u, fa[kk][1], pb[0], pb[1]);
-        mma_f16(sacc[1], 0u, fa[kk][0], 0u, fa[kk][1], pb[2], pb[3]);
+        mma_f16(aacc[0], 0u, fa[kk][0], 0u, fa[kk][1], pb[0], pb[1]);
+        mma_f16(aacc[1], 0u, fa[kk][0], 0u, fa[kk][1], pb[2], pb[3]);
       }
       // online softmax on rows 0..7; rows 8..15 stay linear.  Tokens past the end of the sequence are masked.
       float mx = -INFINITY;
@@ -245,7 +251,7 @@ __global__ void __launch_bounds__(kAttendThreads, 3)
         for (int c = 0; c < 2; ++c) {
           const bool valid = tok0 + nt * 8 + 2 * t + c < ntok;
           sacc[nt][c] = valid ? sacc[nt][c] * sc2 : -INFINITY;
-          sacc[nt][2 + c] = valid ? sacc[nt][2 + c] : 0.f;
+          sacc[nt][2 + c] = valid ? aacc[nt][2 + c] : 0.f;
           mx = fmaxf(mx, sacc[nt][c]);
         }
       }

@@ -297,28 +297,45 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
 
   // ------------------------------------------------------------------ phase B -------------------------------
   SPLA_MARK(p, u, rank, 3);
-  if (tid < CS * G) {
-    const int r = tid / G, g = tid % G;
-    const uint32_t remote = map_to_rank(smem_u32(part_s + g * 2), (uint32_t)r);
-    all_part[(r * GP + g) * 2] = ld_dsmem_f32(remote);
-    all_part[(r * GP + g) * 2 + 1] = ld_dsmem_f32(remote + 4);
+  // Log-sum-exp of every head over the whole cluster, by each warp on its own (no block barrier): lane p
+  // fetches the (max, sum) pair of CTA p / GP and head p % GP over distributed shared memory, then the lanes
+  // of one head are folded with shuffles.
+  float lse_r[GP];
+  {
+    float m = -INFINITY, sm = 0.f;
+    for (int pr = lane; pr < CS * GP; pr += 32) {
+      const int r = pr / GP, g = pr % GP;
+      if (g < G) {
+        const uint32_t remote = map_to_rank(smem_u32(part_s + g * 2), (uint32_t)r);
+        lse_merge(m, sm, ld_dsmem_f32(remote), ld_dsmem_f32(remote + 4));
+      }
+    }
+#pragma unroll
+    for (int o = GP; o < 32; o <<= 1) {
+      const float m2 = __shfl_xor_sync(0xffffffffu, m, o), s2 = __shfl_xor_sync(0xffffffffu, sm, o);
+      lse_merge(m, sm, m2, s2);
+    }
+    const float lse = m + __logf(sm);
+#pragma unroll
+    for (int g = 0; g < GP; ++g) lse_r[g] = __shfl_sync(0xffffffffu, lse, g);
   }
-  __syncthreads();
-  if (tid < G) {
-    float m = -INFINITY, s = 0.f;
-    for (int r = 0; r < CS; ++r) lse_merge(m, s, all_part[(r * GP + tid) * 2], all_part[(r * GP + tid) * 2 + 1]);
-    lse_s[tid] = m + __logf(s);
-  }
-  __syncthreads();
 
   uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw + SM::kKeys);
   TopkScratch* scratch = reinterpret_cast<TopkScratch*>(smem_raw + SM::kScratch);
   const int k_eff = min(p.top_k, nblk);
+  const uint32_t cand_key0 = map_to_rank(smem_u32(smem_raw + SM::kCandKey), 0u) + (uint32_t)rank * kMaxTopK * 4;
+  const uint32_t cand_idx0 = map_to_rank(smem_u32(smem_raw + SM::kCandIdx), 0u) + (uint32_t)rank * kMaxTopK * 4;
+  auto push = [&](int slot, uint32_t key, int idx) {                  // into the leader's candidate table
+    st_dsmem_u32(cand_key0 + (uint32_t)slot * 4, key);
+    st_dsmem_u32(cand_idx0 + (uint32_t)slot * 4, (uint32_t)idx);
+  };
+  if (tid == 0) { scratch->lo = 0xffffffffu; scratch->hi = 0u; scratch->n_forced = 0; scratch->n_emit = 0; }
+  __syncthreads();
   {
-    float lse_r[GP];
-#pragma unroll
-    for (int g = 0; g < GP; ++g) lse_r[g] = g < G ? lse_s[g] : 0.f;
+    // aggregated score of this CTA's blocks; the statistics the selection needs are gathered on the way
     float* scores_u = p.scores + (size_t)u * p.max_blocks;
+    uint32_t mn = 0xffffffffu, mx = 0u;
+    int nf = 0;
     for (int li = tid; li < n_my; li += kCsThreads) {
       float sc = 0.f;
 #pragma unroll
@@ -327,7 +344,23 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
       const int i = rec_begin + li;
       scores_u[i] = sc;
       const bool forced = (i < p.n_sink) || (i >= nblk - p.n_local);
-      keys[li] = forced ? 0xffffffffu : __float_as_uint(sc);
+      const uint32_t key = forced ? 0xffffffffu : __float_as_uint(sc);
+      keys[li] = key;
+      if (forced) {
+        ++nf;
+        push(atomicAdd(&scratch->n_emit, 1), key, i);
+      } else {
+        mn = min(mn, key);
+        mx = max(mx, key);
+      }
+    }
+    mn = __reduce_min_sync(0xffffffffu, mn);
+    mx = __reduce_max_sync(0xffffffffu, mx);
+    nf = __reduce_add_sync(0xffffffffu, nf);
+    if (lane == 0) {
+      atomicMin(&scratch->lo, mn);
+      atomicMax(&scratch->hi, mx);
+      if (nf) atomicAdd(&scratch->n_forced, nf);
     }
   }
   __syncthreads();
@@ -335,15 +368,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
 
   // this CTA's best min(k_eff, n_my) blocks go to the leader's candidate table
   {
-    const uint32_t cand_key0 = map_to_rank(smem_u32(smem_raw + SM::kCandKey), 0u) + (uint32_t)rank * kMaxTopK * 4;
-    const uint32_t cand_idx0 = map_to_rank(smem_u32(smem_raw + SM::kCandIdx), 0u) + (uint32_t)rank * kMaxTopK * 4;
-    const int cnt = select_topk(
-        keys, n_my, k_eff, [&](int li) { return rec_begin + li; },
-        [&](int slot, uint32_t key, int idx) {
-          st_dsmem_u32(cand_key0 + (uint32_t)slot * 4, key);
-          st_dsmem_u32(cand_idx0 + (uint32_t)slot * 4, (uint32_t)idx);
-        },
-        scratch);
+    const int cnt = select_topk(keys, n_my, k_eff, [&](int li) { return rec_begin + li; }, push, scratch);
     if (tid == 0) st_dsmem_u32(map_to_rank(smem_u32(smem_raw + SM::kCandCnt), 0u) + (uint32_t)rank * 4, (uint32_t)cnt);
   }
   SPLA_MARK(p, u, rank, 5);
@@ -356,7 +381,8 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
     // residual branch that needs no selection, o_bar = phi(q) S_bar, one slice of the state's rows each.
     if (rla)
       for (int s = rank - 1; s < kStateSplits; s += CS - 1)
-        state_role<D, GP, 256>(p, u, s, q_raw, q_is_bf16, reinterpret_cast<float*>(smem_raw));
+        state_role<D, GP, kCsThreads>(p, u, s, q_raw, q_is_bf16, reinterpret_cast<float*>(smem_raw));
+    SPLA_MARK(p, u, rank, 7);
     return;
   }
 
@@ -368,24 +394,31 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   int* flat_idx = reinterpret_cast<int*>(smem_raw + SM::kFlatIdx);
   int* sel_tmp = reinterpret_cast<int*>(smem_raw + SM::kSelTmp);
   int total = 0;
-  for (int r = 0; r < CS; ++r) {
-    const int cnt = cand_cnt[r];
-    for (int s = tid; s < cnt; s += kCsThreads) {
-      flat_key[total + s] = cand_key[r * kMaxTopK + s];
-      flat_idx[total + s] = cand_idx[r * kMaxTopK + s];
+  for (int c = tid; c < CS * kMaxTopK; c += kCsThreads) {              // compact the table: slot s of CTA r
+    const int r = c / kMaxTopK, sl = c % kMaxTopK;
+    int base = 0;
+    for (int r2 = 0; r2 < r; ++r2) base += cand_cnt[r2];
+    if (sl < cand_cnt[r]) {
+      flat_key[base + sl] = cand_key[c];
+      flat_idx[base + sl] = cand_idx[c];
     }
-    total += cnt;
   }
+  for (int r = 0; r < CS; ++r) total += cand_cnt[r];
+  SPLA_MARK(p, u, 31, 0);
+  auto keep = [&](int slot, uint32_t, int idx) { sel_tmp[slot] = idx; };
+  auto flat_of = [&](int c) { return flat_idx[c]; };
   __syncthreads();
-  select_topk(
-      flat_key, total, k_eff, [&](int c) { return flat_idx[c]; }, [&](int slot, uint32_t, int idx) { sel_tmp[slot] = idx; },
-      scratch);
+  topk_prepare(flat_key, total, flat_of, keep, scratch);
+  SPLA_MARK(p, u, 31, 1);
+  select_topk(flat_key, total, k_eff, flat_of, keep, scratch);
+  SPLA_MARK(p, u, 31, 2);
   int* sel_u = p.sel + (size_t)u * p.top_k;
   int* sel_o = sel_user ? sel_user + (size_t)u * p.top_k : nullptr;
   for (int s = tid; s < p.top_k; s += kCsThreads) {
     if (s < k_eff) {
       const int ia = sel_tmp[s];
       int pos = 0;
+#pragma unroll 8
       for (int j = 0; j < k_eff; ++j) pos += sel_tmp[j] < ia;
       sel_u[pos] = ia;
       if (sel_o) sel_o[pos] = ia;
@@ -394,12 +427,13 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
       if (sel_o) sel_o[s] = -1;
     }
   }
+  SPLA_MARK(p, u, 31, 3);
   if (tid == 0) p.n_sel[u] = k_eff;
   SPLA_MARK(p, u, rank, 7);
   if (rla && CS == 1)
     for (int s = 0; s < kStateSplits; ++s) {
       __syncthreads();
-      state_role<D, GP, 256>(p, u, s, q_raw, q_is_bf16, reinterpret_cast<float*>(smem_raw));
+      state_role<D, GP, kCsThreads>(p, u, s, q_raw, q_is_bf16, reinterpret_cast<float*>(smem_raw));
     }
 }
 
