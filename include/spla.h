@@ -142,6 +142,14 @@ int spla_decode(spla_cache_t *cache, const void *q, const float *rms_weight, flo
                 float *dbg_o_sparse, float *dbg_o_rla, void *stream);
 
 /*
+ * Steps 1-2 of spla_decode only: scores the blocks (Section 3.1, Eq. taylor-2nd; Section 2.2, grouped BlockScore)
+ * and selects top_k of them (Section 2.1, Select).  sel_idx: DEVICE int32 [batch][H_kv][top_k], ascending, padded
+ * with -1.  The scores stay available to spla_copy_scores.  Together with spla_decode_selected this splits a
+ * decode step in two, e.g. to reuse one selection for several queries.
+ */
+int spla_select(spla_cache_t *cache, const void *q, int32_t *sel_idx, void *stream);
+
+/*
  * Same as spla_decode with the selection given instead of computed (steps 3-5 only): sel_in DEVICE int32
  * [batch][H_kv][top_k], ascending valid block indices padded with -1.  For testing against an oracle when a
  * tie makes several index sets correct, and for callers that select elsewhere.

@@ -19,7 +19,7 @@ SPLA_ADOPT_CONTENTS, SPLA_FIRST_ORDER, SPLA_NO_RLA = 1, 2, 4
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libspla.so")
 
 EXPORTS = ["spla_query_sizes", "spla_init_cache", "spla_append_tokens", "spla_decode", "spla_decode_selected",
-           "spla_decode_profile", "spla_select_blocks_noalloc",
+           "spla_decode_profile", "spla_select_blocks_noalloc", "spla_select",
            "spla_copy_scores", "spla_sync_status", "spla_set_length_bound", "spla_destroy_cache",
            "spla_status_string", "spla_last_cuda_error"]
 
@@ -62,6 +62,7 @@ def load(path: str | None = None) -> C.CDLL:
     lib.spla_append_tokens.argtypes = [vp, vp, vp, vp, i32, vp]
     lib.spla_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.spla_decode_selected.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.spla_select.argtypes = [vp, vp, vp, vp]
     lib.spla_decode_profile.argtypes = [vp, vp, vp, vp, C.POINTER(C.c_float), vp]
     lib.spla_select_blocks_noalloc.argtypes = [C.POINTER(SplaConfig), vp, vp, vp, vp, vp, vp]
     lib.spla_copy_scores.argtypes = [vp, vp, vp]
@@ -207,6 +208,15 @@ class SplaCache:
             _check(self.lib.spla_decode(self.handle, q.data_ptr(), _ptr(rms_weight), out.data_ptr(), _ptr(sel_idx),
                                         _ptr(dbg_o_sparse), _ptr(dbg_o_rla), _stream()), "spla_decode")
         return out
+
+    def select(self, q: torch.Tensor, sel_idx: torch.Tensor | None = None) -> torch.Tensor:
+        """Block scores + top-k only; returns sel_idx [batch, H_kv, top_k] int32."""
+        assert q.is_cuda and q.is_contiguous() and q.dtype == self.q_torch_dtype
+        if sel_idx is None:
+            sel_idx = self.new_sel_buffer()
+        with torch.cuda.device(self.device):
+            _check(self.lib.spla_select(self.handle, q.data_ptr(), sel_idx.data_ptr(), _stream()), "spla_select")
+        return sel_idx
 
     def decode_selected(self, q, rms_weight, sel_in: torch.Tensor, out=None, dbg_o_sparse=None, dbg_o_rla=None):
         cfg = self.cfg

@@ -2,7 +2,9 @@
 // Eq. taylor-2nd: block key mean and diagonal population covariance) and advance the global linear-attention
 // state S_bar += phi(k_t)^T v_t in fp32 (Section 3.2, Eq. rla-impl-1, "Numerical Stability").
 //
-// Four small kernels in stream order, all reading the OLD sequence lengths until the last one bumps them:
+// Appends of up to 32 tokens per sequence (the decode loop) run as ONE fused kernel, see append_fused_kernel.
+// Bulk appends (prefill) run as four kernels in stream order, all reading the OLD sequence lengths until the
+// last one bumps them:
 //   copy   : k_new, v_new -> cache; per-token logsumexp of phi_scale * k into tok_lse
 //   stats  : mean / variance of every touched block recomputed from the cached keys (two exact passes, so the
 //            result does not depend on how the tokens were split across append calls)
@@ -64,29 +66,65 @@ __global__ void __launch_bounds__(kCopyThreads) append_copy_kernel(const Params 
   if (lane == 0) p.tok_lse[pos] = mx + logf(s);
 }
 
+// Mean and population variance of one block, two exact passes, by kStatThreads threads (groups of D threads take
+// every TG-th token; the partial sums are combined in a fixed order, so every append path gives the same bits).
+// Token t of the block comes from the cache if its position is below `L_cached`, else from the new tokens.
+constexpr int kStatThreads = 256;
 template <typename T, int D>
-__global__ void __launch_bounds__(D) append_stats_kernel(const Params p, const int* __restrict__ n_new, int max_new) {
+__device__ __forceinline__ void block_stats_role(const Params& p, int u, int blk, int L_cached, int L_total, const T* kn,
+                                                 bool act, float (*red_s)[D], float* mean_s) {
+  constexpr int TG = kStatThreads / D;
+  const int tid = threadIdx.x;
+  const int t0 = blk * p.B;
+  const int cnt = act ? min(p.B, L_total - t0) : 0;
+  const int tg = tid / D, c = tid % D;
+  const T* kc = reinterpret_cast<const T*>(p.k_cache) + ((size_t)u * p.max_blocks * p.B + t0) * D + c;
+  auto key_at = [&](int t) {
+    const int pos = t0 + t;
+    return pos < L_cached ? to_float(kc[(size_t)t * D]) : to_float(kn[(size_t)(pos - L_cached) * D + c]);
+  };
+  float sum = 0.f;
+  for (int t = tg; t < cnt; t += TG) sum += key_at(t);
+  red_s[tg][c] = sum;
+  __syncthreads();
+  if (tg == 0) {
+    float tot = 0.f;
+#pragma unroll
+    for (int g2 = 0; g2 < TG; ++g2) tot += red_s[g2][c];
+    mean_s[c] = cnt > 0 ? tot / (float)cnt : 0.f;
+  }
+  __syncthreads();
+  const float mean = mean_s[c];
+  float ss = 0.f;
+  for (int t = tg; t < cnt; t += TG) {
+    const float dv = key_at(t) - mean;
+    ss = fmaf(dv, dv, ss);
+  }
+  __syncthreads();
+  red_s[tg][c] = ss;
+  __syncthreads();
+  if (tg == 0 && act) {
+    float tot = 0.f;
+#pragma unroll
+    for (int g2 = 0; g2 < TG; ++g2) tot += red_s[g2][c];
+    float* rec = p.stats + ((size_t)u * p.max_blocks + blk) * 2 * D;
+    rec[c] = mean;
+    rec[D + c] = tot / (float)cnt;
+  }
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kStatThreads) append_stats_kernel(const Params p, const int* __restrict__ n_new, int max_new) {
+  __shared__ float red_s[kStatThreads / D][D];
+  __shared__ float mean_s[D];
   const int u = blockIdx.y, b = u / p.Hkv;
   const int L = p.seq_lens[b];
   const int n = tokens_to_add(p, n_new, max_new, b, L);
-  if (n <= 0) return;
   const int blk = L / p.B + blockIdx.x;                    // x-th touched block
-  const int t0 = blk * p.B;
-  if (t0 >= L + n) return;
-  const int cnt = min(p.B, L + n - t0);
-  const int c = threadIdx.x;
-  const T* kb = reinterpret_cast<const T*>(p.k_cache) + ((size_t)u * p.max_blocks * p.B + t0) * D + c;
-  float sum = 0.f;
-  for (int t = 0; t < cnt; ++t) sum += to_float(kb[(size_t)t * D]);
-  const float mean = sum / (float)cnt;
-  float ss = 0.f;
-  for (int t = 0; t < cnt; ++t) {
-    const float dv = to_float(kb[(size_t)t * D]) - mean;
-    ss = fmaf(dv, dv, ss);
-  }
-  float* rec = p.stats + ((size_t)u * p.max_blocks + blk) * 2 * D;
-  rec[c] = mean;
-  rec[D + c] = ss / (float)cnt;
+  const bool act = n > 0 && blk * p.B < L + n;             // CTA-uniform
+  if (!act) return;
+  // the copy kernel has already stored the new tokens: everything is read from the cache
+  block_stats_role<T, D>(p, u, blk, L + n, L + n, static_cast<const T*>(nullptr), true, red_s, mean_s);
 }
 
 template <typename T, int D>
@@ -136,15 +174,145 @@ __global__ void append_lengths_kernel(const Params p, const int* __restrict__ n_
   if (n > 0) p.seq_lens[b] = L + n;
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Decode-step appends (a few tokens per sequence): everything above in ONE launch.  CTAs take one of three roles
+// by blockIdx.x; no role needs another's output, because the new tokens are read from k_new / v_new directly
+// (statistics of the open block: cached keys below the old length, new keys above it; state: the per-token
+// log-sum-exp is recomputed from the new keys).  Every CTA reads the old lengths; the last CTA to finish
+// (atomic ticket, nobody waits) advances them.
+constexpr int kFusedThreads = 256;
+constexpr int kFusedMaxNew = 32;
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kFusedThreads) append_fused_kernel(const Params p, const T* __restrict__ k_new,
+                                                                     const T* __restrict__ v_new,
+                                                                     const int* __restrict__ n_new, int max_new, int n_copy,
+                                                                     int n_stats) {
+  constexpr int VEC = D / 32;
+  constexpr int TG = kFusedThreads / D;            // thread groups of D threads
+  __shared__ float red_s[TG][D];
+  __shared__ float mean_s[D];
+  __shared__ float phi_s[kFusedMaxNew][kStateRows];
+  __shared__ float lse_s[kFusedMaxNew];
+  __shared__ int last_s;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int u = blockIdx.y, b = u / p.Hkv;
+  int role = blockIdx.x;
+
+  pdl_wait();                                      // the preceding decode still reads the cache and the lengths
+  pdl_launch_dependents();
+  const int L = p.seq_lens[b];
+  const int n = tokens_to_add(p, n_new, max_new, b, L);
+  const T* kn = k_new + (size_t)u * max_new * D;
+  const T* vn = v_new + (size_t)u * max_new * D;
+  const size_t unit_tok0 = (size_t)u * p.max_blocks * p.B;
+
+  if (role < n_copy) {
+    // ---- copy role: one warp per token; also the per-token log-sum-exp the decode reads ------------------
+    if (n < 0 && role == 0 && tid == 0) atomicExch(p.status, -2);
+    const int i = role * (kFusedThreads / 32) + warp;
+    if (n > 0 && i < n) {
+      const size_t pos = unit_tok0 + (size_t)(L + i);
+      float k[VEC];
+      load_vec<VEC>(kn + (size_t)i * D + lane * VEC, k);
+      copy_bytes<VEC * sizeof(T)>(reinterpret_cast<T*>(p.k_cache) + pos * D + lane * VEC, kn + (size_t)i * D + lane * VEC);
+      copy_bytes<VEC * sizeof(T)>(reinterpret_cast<T*>(p.v_cache) + pos * D + lane * VEC, vn + (size_t)i * D + lane * VEC);
+      float mx = -INFINITY;
+#pragma unroll
+      for (int v = 0; v < VEC; ++v) { k[v] *= p.phi_scale; mx = fmaxf(mx, k[v]); }
+      mx = warp_max(mx);
+      float sm = 0.f;
+#pragma unroll
+      for (int v = 0; v < VEC; ++v) sm += expf(k[v] - mx);
+      sm = warp_sum(sm);
+      if (lane == 0) p.tok_lse[pos] = mx + logf(sm);
+    }
+  } else if ((role -= n_copy) < n_stats) {
+    // ---- statistics role: one touched block; cached keys below the old length, new keys above it -----------
+    const int blk = L / p.B + role;
+    block_stats_role<T, D>(p, u, blk, L, L + max(n, 0), kn, n > 0 && blk * p.B < L + n, red_s, mean_s);
+  } else if (!(p.flags & 4u)) {
+    // ---- state role: S_bar[row0 .. row0 + 15][:] += sum_t phi(k_t)[row] v_t ------------------------------------
+    role -= n_stats;
+    const int row0 = role * kStateRows;
+    const int nn = max(n, 0);
+    const float a2 = p.phi_scale * kLog2e;
+    // log-sum-exp of every new token: 8 threads per token
+    {
+      const int t = tid >> 3, part = tid & 7;
+      float mx = -INFINITY, sm = 0.f;
+      if (t < nn) {
+        for (int c = part; c < D; c += 8) mx = fmaxf(mx, to_float(kn[(size_t)t * D + c]) * a2);
+      }
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+      if (t < nn) {
+        for (int c = part; c < D; c += 8) sm += exp2f(to_float(kn[(size_t)t * D + c]) * a2 - mx);
+      }
+      sm += __shfl_xor_sync(0xffffffffu, sm, 1);
+      sm += __shfl_xor_sync(0xffffffffu, sm, 2);
+      sm += __shfl_xor_sync(0xffffffffu, sm, 4);
+      if (t < nn && part == 0) lse_s[t] = mx + log2f(sm);        // base-2 domain
+    }
+    __syncthreads();
+    for (int idx = tid; idx < kFusedMaxNew * kStateRows; idx += kFusedThreads) {
+      const int t = idx / kStateRows, r = idx % kStateRows;
+      phi_s[t][r] = t < nn ? exp2f(to_float(kn[(size_t)t * D + row0 + r]) * a2 - lse_s[t]) : 0.f;
+    }
+    __syncthreads();
+    constexpr int RPT = kStateRows / TG;                         // rows per thread
+    const int tg = tid / D, j = tid % D;
+    float acc[RPT];
+#pragma unroll
+    for (int r = 0; r < RPT; ++r) acc[r] = 0.f;
+    for (int t = 0; t < nn; ++t) {
+      const float v = to_float(vn[(size_t)t * D + j]);
+#pragma unroll
+      for (int r = 0; r < RPT; ++r) acc[r] = fmaf(phi_s[t][tg * RPT + r], v, acc[r]);
+    }
+    if (nn > 0) {
+      float* S = p.state + (size_t)u * D * D + (size_t)(row0 + tg * RPT) * D + j;
+#pragma unroll
+      for (int r = 0; r < RPT; ++r) S[(size_t)r * D] += acc[r];
+    }
+  }
+
+  // ---- the last CTA of the whole launch advances the lengths ---------------------------------------------------
+  __syncthreads();
+  if (tid == 0) {
+    asm volatile("fence.acq_rel.gpu;" ::: "memory");
+    const int t = atomicAdd(p.append_ticket, 1);
+    last_s = (t == (int)(gridDim.x * gridDim.y) - 1);
+    if (last_s) *p.append_ticket = 0;
+    asm volatile("fence.acq_rel.gpu;" ::: "memory");
+  }
+  __syncthreads();
+  if (last_s) {
+    for (int bb = tid; bb < p.batch; bb += kFusedThreads) {
+      const int Lb = p.seq_lens[bb];
+      const int nb = tokens_to_add(p, n_new, max_new, bb, Lb);
+      if (nb > 0) p.seq_lens[bb] = Lb + nb;
+    }
+  }
+}
+
 template <typename T, int D>
 static cudaError_t launch_typed(const Params& p, const void* k_new, const void* v_new, const int* n_new, int max_new,
                                 cudaStream_t stream) {
   const int U = p.batch * p.Hkv;
   const T* kn = reinterpret_cast<const T*>(k_new);
   const T* vn = reinterpret_cast<const T*>(v_new);
+  if (max_new <= kFusedMaxNew) {
+    const int n_copy = (max_new + kFusedThreads / 32 - 1) / (kFusedThreads / 32);
+    const int n_stats = (max_new + p.B - 1) / p.B + 1;
+    const int n_state = (p.flags & 4u) ? 0 : D / kStateRows;
+    return launch_ex(append_fused_kernel<T, D>, dim3(n_copy + n_stats + n_state, U), dim3(kFusedThreads), 0, stream, 0, true,
+                     p, kn, vn, n_new, max_new, n_copy, n_stats);
+  }
   const int per_cta = kCopyThreads / 32;
   append_copy_kernel<T, D><<<dim3((max_new + per_cta - 1) / per_cta, U), kCopyThreads, 0, stream>>>(p, kn, vn, n_new, max_new);
-  append_stats_kernel<T, D><<<dim3((max_new + p.B - 1) / p.B + 1, U), D, 0, stream>>>(p, n_new, max_new);
+  append_stats_kernel<T, D><<<dim3((max_new + p.B - 1) / p.B + 1, U), kStatThreads, 0, stream>>>(p, n_new, max_new);
   if (!(p.flags & 4u))
     append_state_kernel<T, D><<<dim3(D / kStateRows, U), D, 0, stream>>>(p, kn, vn, n_new, max_new);
   append_lengths_kernel<<<(p.batch + 127) / 128, 128, 0, stream>>>(p, n_new, max_new);

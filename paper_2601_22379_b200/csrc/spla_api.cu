@@ -78,7 +78,7 @@ static int validate_config(const spla_config_t* c) {
 }
 
 struct WorkspaceLayout {
-  size_t ell, chunk_part, scores, obar_part, sel, n_sel, att_acc, att_ml, score_ticket, attend_ticket, status, total;
+  size_t ell, chunk_part, scores, obar_part, sel, n_sel, att_acc, att_ml, score_ticket, attend_ticket, append_ticket, status, total;
   int max_chunks;
 };
 
@@ -99,6 +99,7 @@ static WorkspaceLayout workspace_layout(const spla_config_t* c) {
   w.att_ml = take(U * c->top_k * G * 2 * 4);
   w.score_ticket = take(U * 4);
   w.attend_ticket = take(U * 4);
+  w.append_ticket = take(256);
   w.status = take(256);
   w.total = off;
   return w;
@@ -171,6 +172,7 @@ extern "C" int spla_init_cache(const spla_config_t* config, const spla_buffers_t
   p.obar_part = (float*)(ws + w.obar_part); p.sel = (int*)(ws + w.sel); p.n_sel = (int*)(ws + w.n_sel);
   p.att_acc = (float*)(ws + w.att_acc); p.att_ml = (float*)(ws + w.att_ml);
   p.score_ticket = (int*)(ws + w.score_ticket); p.attend_ticket = (int*)(ws + w.attend_ticket);
+  p.append_ticket = (int*)(ws + w.append_ticket);
   p.status = (int*)(ws + w.status);
   p.max_chunks = w.max_chunks;
 #ifdef SPLA_TRACE
@@ -315,6 +317,15 @@ extern "C" int spla_decode_profile(spla_cache_t* c, const void* q, const float* 
   if (e == cudaSuccess) e = cudaEventElapsedTime(&stage_ms[1], c->ev[1], c->ev[2]);
   if (e != cudaSuccess) return cuda_fail(e, "spla_decode_profile");
   return SPLA_OK;
+}
+
+extern "C" int spla_select(spla_cache_t* c, const void* q, int32_t* sel_idx, void* stream) {
+  if (!c || !q || !sel_idx) return SPLA_ERR_INVALID_ARG;
+  if (!aligned(q, 16)) return SPLA_ERR_INVALID_ARG;
+  Params p = c->p;
+  plan_score_grid(c, &p);
+  cudaError_t e = launch_score(p, q, c->cfg.q_dtype == SPLA_BF16, sel_idx, (cudaStream_t)stream);
+  return e == cudaSuccess ? SPLA_OK : cuda_fail(e, "spla_select");
 }
 
 extern "C" int spla_decode_selected(spla_cache_t* c, const void* q, const float* rms_weight, const int32_t* sel_in,

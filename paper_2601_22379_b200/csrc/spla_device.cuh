@@ -47,6 +47,7 @@ struct Params {
   float* att_ml;       // [U][top_k][G][2]        per selected block: (max, sum) in log2 domain
   int* score_ticket;   // [U]
   int* attend_ticket;  // [U]
+  int* append_ticket;  // [1]
   int* status;         // [1]
   int max_chunks;
 #ifdef SPLA_TRACE

@@ -76,6 +76,21 @@ def test_append_statistics_and_state_match_oracle(name, ctx):
     assert torch.equal(cache2.bufs.stats[:, :, :nblk], cache.bufs.stats[:, :, :nblk])
     assert torch.equal(cache2.bufs.tok_lse[:, :, :ctx], cache.bufs.tok_lse[:, :, :ctx])
     assert parity.rel_l2(cache2.bufs.rla_state.cpu().numpy(), cache.bufs.rla_state.cpu().numpy()) < 2e-6
+    # ... and so does the fused decode-step kernel (one, three and seventeen tokens per call)
+    cache3 = binding.SplaCache(runner.config_for(w), DEV)
+    pos, sizes = 0, [1, 3, 17, 1, 1, 32, 5]
+    i = 0
+    while pos < ctx:
+        m = min(sizes[i % len(sizes)], ctx - pos)
+        cache3.append_tokens(K[:, :, pos:pos + m].contiguous(), V[:, :, pos:pos + m].contiguous())
+        pos += m
+        i += 1
+    torch.cuda.synchronize()
+    assert cache3.sync_status() == 0 and cache3.bufs.seq_lens.cpu().tolist() == [ctx, ctx]
+    assert torch.equal(cache3.bufs.stats[:, :, :nblk], cache.bufs.stats[:, :, :nblk])
+    assert torch.equal(cache3.bufs.tok_lse[:, :, :ctx], cache.bufs.tok_lse[:, :, :ctx])
+    assert torch.equal(cache3.bufs.k_cache.reshape(2, w.n_kv_heads, -1, w.head_dim)[:, :, :ctx], K)
+    assert parity.rel_l2(cache3.bufs.rla_state.cpu().numpy(), cache.bufs.rla_state.cpu().numpy()) < 2e-6
 
 
 def test_ragged_append_with_device_lengths():
@@ -326,6 +341,20 @@ def test_decode_selected_uses_the_given_blocks():
             parity.check_outputs("o_sparse", osp[b, sl], res["o_sparse"], "bf16")
             parity.check_outputs("o_rla", orla[b, sl], res["o_rla"], "bf16")
             parity.check_outputs("out", out[b, sl], res["out"], "bf16")
+
+
+def test_select_then_decode_selected_equals_decode():
+    w = synth.BY_NAME["gqa_32k"].scaled(batch=2, context=64 * 50 + 9, n_needles=3)
+    cache, K, V, lens = runner.build_cache(w, DEV)
+    gamma = synth.gamma(w).to(DEV)
+    q = synth.step_queries(w, 0, DEV)
+    sel_a = cache.new_sel_buffer()
+    out_a = cache.decode(q, gamma, sel_idx=sel_a).clone()
+    sel_b = cache.select(q)
+    out_b = cache.decode_selected(q, gamma, sel_b)
+    torch.cuda.synchronize()
+    assert torch.equal(sel_a, sel_b)
+    np.testing.assert_allclose(out_b.cpu().numpy(), out_a.cpu().numpy(), rtol=1e-6, atol=1e-6)
 
 
 def test_scores_are_normalised_and_match_oracle():
