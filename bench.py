@@ -304,15 +304,42 @@ def run_ours(args, w):
     torch.cuda.synchronize()
     dec_ms = d0.elapsed_time(d1) / (n_dec_rep * GRAPH_STEPS)
 
-    # ---- per-kernel durations of the decode, CUDA events between the two kernels -----------------------------
-    n_prof = max(8, min(steps, 128))
-    sc_ms, at_ms = [], []
+    # ---- duration of the dominant kernel (block score + selection): a CUDA graph of back-to-back launches of that
+    # kernel alone, rotating over the caches (cold L2), timed with CUDA events on the launching stream -------------
+    sel_bufs = [c.new_sel_buffer() for c in caches]
+    with torch.cuda.stream(stream):
+        for i in range(R):
+            caches[i].select(qs[i], sel_bufs[i])                      # warm-up, also loads the kernel
+        graph_sel = None
+        if steps >= GRAPH_STEPS:
+            graph_sel = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph_sel, stream=stream):
+                for i in range(GRAPH_STEPS):
+                    caches[i % R].select(qs[i % n_in], sel_bufs[i % R])
+            graph_sel.replay()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_sel_rep = max(1, min(steps // GRAPH_STEPS, 64))
+        s0.record(stream)
+        for r in range(n_sel_rep):
+            if graph_sel is not None:
+                graph_sel.replay()
+            else:
+                for i in range(GRAPH_STEPS):
+                    caches[i % R].select(qs[i % n_in], sel_bufs[i % R])
+        s1.record(stream)
+    torch.cuda.synchronize()
+    sc = s0.elapsed_time(s1) / (n_sel_rep * GRAPH_STEPS)
+
+    # isolated kernel durations with events between the two kernels of one decode (each includes ~6 us of event
+    # and launch latency, measured on an empty kernel; reported for reference only)
+    n_prof = max(8, min(steps, 64))
+    sc_iso, at_iso = [], []
     with torch.cuda.stream(stream):
         for i in range(n_prof):
             a, b = caches[i % R].decode_profile(qs[i % n_in], gamma, outs[i % R])
-            sc_ms.append(a)
-            at_ms.append(b)
-    sc, at = statistics.mean(sc_ms), statistics.mean(at_ms)
+            sc_iso.append(a)
+            at_iso.append(b)
+    at = statistics.mean(at_iso)
 
     # ---- end to end through the public call with host buffers --------------------------------------------------
     hq = [q.cpu().pin_memory() for q in qs[:8]]
@@ -358,12 +385,12 @@ def run_ours(args, w):
         "clocks": clocks,
         "e2e": {"value": w.batch * w.n_q_heads * world / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
-        "gpu_launches": 6 * steps,
-        "roofline": {"bound": "hbm", "kernel": "score_select_kernel", "achieved": achieved, "peak": peak,
+        "gpu_launches": 3 * steps,
+        "roofline": {"bound": "hbm", "kernel": "score_cluster_kernel (block score + top-k)", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "bytes_per_launch": score_bytes, "ms_per_launch": sc, "traffic": args.traffic},
-        "kernels": {"score_select_ms": sc, "attend_merge_ms": at,
-                    "attend_merge_GBps": by["selected_kv"] / (at * 1e-3) / 1e9,
+        "kernels": {"score_select_ms": sc, "score_select_isolated_ms": statistics.mean(sc_iso),
+                    "attend_merge_isolated_ms": at, "decode_minus_score_ms": dec_ms - sc,
                     "decode_only_ms": dec_ms, "decode_only_GBps": by["total"] / (dec_ms * 1e-3) / 1e9,
                     "decode_only_frac_of_peak": by["total"] / (dec_ms * 1e-3) / 1e9 / peak,
                     "decode_only_frac_of_8TBps": by["total"] / (dec_ms * 1e-3) / 8e12,

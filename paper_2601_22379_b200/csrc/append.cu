@@ -79,11 +79,15 @@ __device__ __forceinline__ void block_stats_role(const Params& p, int u, int blk
   const int cnt = act ? min(p.B, L_total - t0) : 0;
   const int tg = tid / D, c = tid % D;
   const T* kc = reinterpret_cast<const T*>(p.k_cache) + ((size_t)u * p.max_blocks * p.B + t0) * D + c;
+  // One address per token (cached or new) and one load from it: no branch around the loads, so that the
+  // unrolled loop keeps several of them in flight.
   auto key_at = [&](int t) {
     const int pos = t0 + t;
-    return pos < L_cached ? to_float(kc[(size_t)t * D]) : to_float(kn[(size_t)(pos - L_cached) * D + c]);
+    const T* src = pos < L_cached ? kc + (size_t)t * D : kn + (size_t)(pos - L_cached) * D + c;
+    return to_float(*src);
   };
   float sum = 0.f;
+#pragma unroll 8
   for (int t = tg; t < cnt; t += TG) sum += key_at(t);
   red_s[tg][c] = sum;
   __syncthreads();
@@ -96,6 +100,7 @@ __device__ __forceinline__ void block_stats_role(const Params& p, int u, int blk
   __syncthreads();
   const float mean = mean_s[c];
   float ss = 0.f;
+#pragma unroll 8
   for (int t = tg; t < cnt; t += TG) {
     const float dv = key_at(t) - mean;
     ss = fmaf(dv, dv, ss);
@@ -237,18 +242,32 @@ __global__ void __launch_bounds__(kFusedThreads) append_fused_kernel(const Param
     const int row0 = role * kStateRows;
     const int nn = max(n, 0);
     const float a2 = p.phi_scale * kLog2e;
-    // log-sum-exp of every new token: 8 threads per token
+    // log-sum-exp of every new token: 8 threads per token, D / 8 consecutive channels each, loaded up front
     {
+      constexpr int CPT = D / 8;                                 // channels per thread
       const int t = tid >> 3, part = tid & 7;
-      float mx = -INFINITY, sm = 0.f;
+      float x[CPT];
       if (t < nn) {
-        for (int c = part; c < D; c += 8) mx = fmaxf(mx, to_float(kn[(size_t)t * D + c]) * a2);
+#pragma unroll
+        for (int c4 = 0; c4 < CPT / 4; ++c4) {
+          float y[4];
+          load_vec<4>(kn + (size_t)t * D + part * CPT + c4 * 4, y);
+#pragma unroll
+          for (int v = 0; v < 4; ++v) x[c4 * 4 + v] = y[v] * a2;
+        }
+      } else {
+#pragma unroll
+        for (int v = 0; v < CPT; ++v) x[v] = -INFINITY;
       }
+      float mx = -INFINITY, sm = 0.f;
+#pragma unroll
+      for (int v = 0; v < CPT; ++v) mx = fmaxf(mx, x[v]);
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
       if (t < nn) {
-        for (int c = part; c < D; c += 8) sm += exp2f(to_float(kn[(size_t)t * D + c]) * a2 - mx);
+#pragma unroll
+        for (int v = 0; v < CPT; ++v) sm += exp2f(x[v] - mx);
       }
       sm += __shfl_xor_sync(0xffffffffu, sm, 1);
       sm += __shfl_xor_sync(0xffffffffu, sm, 2);
@@ -307,6 +326,8 @@ static cudaError_t launch_typed(const Params& p, const void* k_new, const void* 
     const int n_copy = (max_new + kFusedThreads / 32 - 1) / (kFusedThreads / 32);
     const int n_stats = (max_new + p.B - 1) / p.B + 1;
     const int n_state = (p.flags & 4u) ? 0 : D / kStateRows;
+    // Same shared-memory carve-out as the decode kernels around it: a change of carve-out drains the SMs.
+    cudaFuncSetAttribute(append_fused_kernel<T, D>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     return launch_ex(append_fused_kernel<T, D>, dim3(n_copy + n_stats + n_state, U), dim3(kFusedThreads), 0, stream, 0, true,
                      p, kn, vn, n_new, max_new, n_copy, n_stats);
   }

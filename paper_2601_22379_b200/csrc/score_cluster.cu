@@ -133,6 +133,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   float* ell_s = reinterpret_cast<float*>(smem_raw + SM::kEll);          // [G][chunk]
   __shared__ int err_s;
 
+  SPLA_MARK(p, blockIdx.y, 30, 0);
   pdl_wait();                                   // everything the preceding kernels wrote (statistics, lengths, q) is visible
   pdl_launch_dependents();                      // only now may the next kernel begin its prologue: it reads q before its own wait
 
@@ -404,14 +405,12 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
     }
   }
   for (int r = 0; r < CS; ++r) total += cand_cnt[r];
-  SPLA_MARK(p, u, 31, 0);
   auto keep = [&](int slot, uint32_t, int idx) { sel_tmp[slot] = idx; };
   auto flat_of = [&](int c) { return flat_idx[c]; };
   __syncthreads();
   topk_prepare(flat_key, total, flat_of, keep, scratch);
-  SPLA_MARK(p, u, 31, 1);
   select_topk(flat_key, total, k_eff, flat_of, keep, scratch);
-  SPLA_MARK(p, u, 31, 2);
+
   int* sel_u = p.sel + (size_t)u * p.top_k;
   int* sel_o = sel_user ? sel_user + (size_t)u * p.top_k : nullptr;
   for (int s = tid; s < p.top_k; s += kCsThreads) {
@@ -427,7 +426,6 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
       if (sel_o) sel_o[s] = -1;
     }
   }
-  SPLA_MARK(p, u, 31, 3);
   if (tid == 0) p.n_sel[u] = k_eff;
   SPLA_MARK(p, u, rank, 7);
   if (rla && CS == 1)
