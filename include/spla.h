@@ -21,7 +21,7 @@
  * General rules
  *   - All device buffers are owned by the caller.  The library allocates no
  *     device memory, frees none, and never synchronises the device except in
- *     spla_sync_status.  Every call enqueues its work on the given stream
+ *     spla_sync_status and spla_decode_profile.  Every call enqueues its work on the given stream
  *     (a cudaStream_t passed as void*; NULL = the legacy default stream) and
  *     returns; results are ready when that stream reaches them.
  *   - Pointers marked DEVICE must be device memory of the current device,
@@ -63,6 +63,8 @@ typedef enum { SPLA_F32 = 0, SPLA_BF16 = 1 } spla_dtype_t;
 #define SPLA_ADOPT_CONTENTS 1u /* spla_init_cache keeps stats / rla_state / tok_lse / seq_lens as they are */
 #define SPLA_FIRST_ORDER 2u    /* block score without the covariance term (Eq. taylor-1st) */
 #define SPLA_NO_RLA 4u         /* out = o_sparse; the residual branch is skipped (the paper's SPA ablation) */
+#define SPLA_GENERAL_KERNELS 8u /* always use the general kernels (any group size up to 16, any length, fp32 or bf16)
+                                   instead of the cluster / tensor-core ones: for testing and comparison */
 
 typedef struct {
   int32_t batch;          /* sequences per call, >= 1 */

@@ -14,7 +14,7 @@ import torch
 
 SPLA_OK, SPLA_ERR_INVALID_ARG, SPLA_ERR_CAPACITY, SPLA_ERR_CUDA, SPLA_ERR_UNSUPPORTED = 0, -1, -2, -3, -4
 SPLA_F32, SPLA_BF16 = 0, 1
-SPLA_ADOPT_CONTENTS, SPLA_FIRST_ORDER, SPLA_NO_RLA = 1, 2, 4
+SPLA_ADOPT_CONTENTS, SPLA_FIRST_ORDER, SPLA_NO_RLA, SPLA_GENERAL_KERNELS = 1, 2, 4, 8
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libspla.so")
 

@@ -64,7 +64,7 @@ static int validate_config(const spla_config_t* c) {
   if ((c->kv_dtype != SPLA_F32 && c->kv_dtype != SPLA_BF16) || (c->q_dtype != SPLA_F32 && c->q_dtype != SPLA_BF16))
     return SPLA_ERR_INVALID_ARG;
   if (c->sm_scale < 0.f || c->phi_scale < 0.f || c->rms_eps < 0.f) return SPLA_ERR_INVALID_ARG;
-  if (c->flags & ~(SPLA_ADOPT_CONTENTS | SPLA_FIRST_ORDER | SPLA_NO_RLA)) return SPLA_ERR_INVALID_ARG;
+  if (c->flags & ~(SPLA_ADOPT_CONTENTS | SPLA_FIRST_ORDER | SPLA_NO_RLA | SPLA_GENERAL_KERNELS)) return SPLA_ERR_INVALID_ARG;
   const int G = c->n_q_heads / c->n_kv_heads;
   if (G > kMaxGroup) return SPLA_ERR_UNSUPPORTED;
   if (c->head_dim != 64 && c->head_dim != 128) return SPLA_ERR_UNSUPPORTED;
@@ -228,7 +228,7 @@ static void plan_score_grid(const spla_cache* c, Params* p) {
   if (blocks < 1) blocks = 1;
   p->cs = 0;
   int cs = 0, chunk = 0;
-  if (!getenv("SPLA_NO_CLUSTER") && plan_score_cluster(p->batch * p->Hkv, blocks, p->G, p->d, c->sm_count, &cs, &chunk)) {
+  if (!(c->cfg.flags & SPLA_GENERAL_KERNELS) && plan_score_cluster(p->batch * p->Hkv, blocks, p->G, p->d, c->sm_count, &cs, &chunk)) {
     p->cs = cs;
     p->chunk = chunk;
     p->n_chunks_cap = cs;
@@ -245,6 +245,7 @@ static cudaError_t launch_score(const Params& p, const void* q, int qb, int* sel
 // Cluster size of the tensor-core attend kernel: the largest power of two (at most 16 and at most top_k) for
 // which all CTAs are resident at once; each CTA of a cluster then walks top_k / size selected blocks.
 static int attend_cluster_size(const spla_cache* c) {
+  if (c->cfg.flags & SPLA_GENERAL_KERNELS) return 0;
   const size_t smem = attend_mma_smem_bytes(c->p.B, c->p.d) + 2048;
   long long per_sm = (227 * 1024) / (long long)smem;
   if (per_sm > 3) per_sm = 3;

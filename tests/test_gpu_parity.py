@@ -119,11 +119,12 @@ SMALL = [
 
 
 @pytest.mark.parametrize("name,over", SMALL)
-@pytest.mark.parametrize("forced", [(1, 4), (0, 0), (1, 1)])
-def test_decode_matches_oracle_small(name, over, forced):
+@pytest.mark.parametrize("forced,flags", [((1, 4), 0), ((0, 0), 0), ((1, 1), 0), ((1, 4), binding.SPLA_GENERAL_KERNELS)])
+def test_decode_matches_oracle_small(name, over, forced, flags):
+    """Default (cluster / tensor-core) kernels with three forced-block settings, and the general kernels."""
     w = synth.BY_NAME[name].scaled(**over)
     n_sink, n_local = forced
-    cache, K, V, lens = runner.build_cache(w, DEV, n_sink=n_sink, n_local=n_local)
+    cache, K, V, lens = runner.build_cache(w, DEV, n_sink=n_sink, n_local=n_local, flags=flags)
     gamma = synth.gamma(w).to(DEV)
     q = synth.step_queries(w, 0, DEV)
     lens_h = lens.cpu().numpy()
@@ -341,6 +342,36 @@ def test_decode_selected_uses_the_given_blocks():
             parity.check_outputs("o_sparse", osp[b, sl], res["o_sparse"], "bf16")
             parity.check_outputs("o_rla", orla[b, sl], res["o_rla"], "bf16")
             parity.check_outputs("out", out[b, sl], res["out"], "bf16")
+
+
+def test_graph_replay_of_append_and_decode_matches_eager_calls():
+    """The benchmark replays steps from a CUDA graph (with programmatic dependent launch between the kernels):
+    the replayed steps must give what the same calls give one by one."""
+    w = synth.BY_NAME["long_128k"].scaled(batch=2, context=64 * 200 + 30, n_steps=40)
+    gamma = synth.gamma(w).to(DEV)
+    steps = [(synth.step_kv(w, s, DEV), synth.step_queries(w, s, DEV)) for s in range(6)]
+    eager, K, V, lens = runner.build_cache(w, DEV)
+    ref = []
+    for (k1, v1), q in steps:
+        eager.append_tokens(k1, v1)
+        ref.append(eager.decode(q, gamma).clone())
+    cache, _, _, _ = runner.build_cache(w, DEV, prefill=(K, V, lens))
+    cache.set_length_bound(w.max_context - 8)               # replays append without the host seeing it
+    outs = [torch.empty_like(ref[0]) for _ in steps]
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        cache.decode(steps[0][1], gamma, out=outs[0])        # load the kernels before capturing
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for i, ((k1, v1), q) in enumerate(steps):
+                cache.append_tokens(k1, v1)
+                cache.decode(q, gamma, out=outs[i])
+        graph.replay()
+    torch.cuda.synchronize()
+    assert cache.sync_status() == 0
+    assert torch.equal(cache.bufs.seq_lens, eager.bufs.seq_lens)
+    for a, b in zip(outs, ref):
+        np.testing.assert_allclose(a.cpu().numpy(), b.cpu().numpy(), rtol=1e-5, atol=1e-6)
 
 
 def test_select_then_decode_selected_equals_decode():
