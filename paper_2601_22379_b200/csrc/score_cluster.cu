@@ -133,54 +133,46 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   float* ell_s = reinterpret_cast<float*>(smem_raw + SM::kEll);          // [G][chunk]
   __shared__ int err_s;
 
+  if (tid == 0) {                               // nothing here depends on the preceding kernel
+    for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kCsConsumers); }
+    err_s = 0;
+  }
   SPLA_MARK(p, blockIdx.y, 30, 0);
   pdl_wait();                                   // everything the preceding kernels wrote (statistics, lengths, q) is visible
   pdl_launch_dependents();                      // only now may the next kernel begin its prologue: it reads q before its own wait
 
-  // ---- queries first: the streaming below saturates the memory system, and a small load issued into that
-  // traffic takes several microseconds.  Lane layout: `hl` of W lanes covers d = c * 4 W + 4 hl .. + 3.
+  // ---- the query loads go out first and the ring is started as soon as the sequence length is known: a small
+  // load issued into the streaming traffic would take several microseconds.
+  // Lane layout: `hl` of W lanes covers d = c * 4 W + 4 hl .. + 3.
   const int hl = lane % W, grp = lane / W;
+  constexpr int CW = VECW >= 4 ? 4 : VECW;      // floats per vector load
+  constexpr int NC = VECW / CW;
   float qm[GP][VECW], qv[GP][VECW];
-  {
 #pragma unroll
-    for (int g = 0; g < GP; ++g) {
-      if (g < G) {
-        const size_t qrow = ((size_t)b * p.Hq + (size_t)h * G + g) * D;
+  for (int g = 0; g < GP; ++g) {
+    if (g < G) {
+      const size_t qrow = ((size_t)b * p.Hq + (size_t)h * G + g) * D;
 #pragma unroll
-        for (int c = 0; c < (VECW >= 4 ? VECW / 4 : 1); ++c) {
-          constexpr int CW = VECW >= 4 ? 4 : VECW;
-          float x[CW];
-          const size_t qoff = qrow + (size_t)c * W * 4 + hl * CW;
-          if (q_is_bf16) load_vec<CW>(reinterpret_cast<const __nv_bfloat16*>(q_raw) + qoff, x);
-          else load_vec<CW>(reinterpret_cast<const float*>(q_raw) + qoff, x);
+      for (int c = 0; c < NC; ++c) {
+        float x[CW];
+        const size_t qoff = qrow + (size_t)c * W * 4 + hl * CW;
+        if (q_is_bf16) load_vec<CW>(reinterpret_cast<const __nv_bfloat16*>(q_raw) + qoff, x);
+        else load_vec<CW>(reinterpret_cast<const float*>(q_raw) + qoff, x);
 #pragma unroll
-          for (int v = 0; v < CW; ++v) {
-            qm[g][c * CW + v] = x[v] * p.sm_scale;
-            qv[g][c * CW + v] = (p.flags & 2u) ? 0.f : 0.5f * qm[g][c * CW + v] * qm[g][c * CW + v];
-          }
-        }
-      } else {
-#pragma unroll
-        for (int v = 0; v < VECW; ++v) { qm[g][v] = 0.f; qv[g][v] = 0.f; }
+        for (int v = 0; v < CW; ++v) qm[g][c * CW + v] = x[v];
       }
+    } else {
+#pragma unroll
+      for (int v = 0; v < VECW; ++v) qm[g][v] = 0.f;
     }
   }
-  const int L = p.seq_lens[b];
+  const int L = __ldcg(p.seq_lens + b);
   const int nblk = (L + p.B - 1) / p.B;
   const int chunk = p.chunk;
   const int rec_begin = min(nblk, rank * chunk);
   const int rec_end = min(nblk, rec_begin + chunk);
   const int n_my = rec_end - rec_begin;
   const int n_rounds = (n_my + kStageRec - 1) / kStageRec;
-  SPLA_MARK(p, u, rank, 0);
-
-  if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kCsConsumers); }
-    err_s = 0;
-  }
-  __syncthreads();
-  SPLA_MARK(p, u, rank, 1);
-
   const float* stats_u = p.stats + (size_t)u * p.max_blocks * 2 * D;
 
   auto issue = [&](int r) {                      // thread 0 only: one bulk copy fills stage r % kStages
@@ -192,6 +184,18 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   };
   if (tid == 0)
     for (int r = 0; r < min(kStages, n_rounds); ++r) issue(r);
+  SPLA_MARK(p, u, rank, 0);
+#pragma unroll
+  for (int g = 0; g < GP; ++g) {
+#pragma unroll
+    for (int v = 0; v < VECW; ++v) {
+      qm[g][v] *= p.sm_scale;
+      qv[g][v] = (p.flags & 2u) ? 0.f : 0.5f * qm[g][v] * qm[g][v];
+    }
+  }
+  __syncthreads();                              // the barrier initialisation is visible to every consumer
+  SPLA_MARK(p, u, rank, 1);
+
   {
     // After the group reduction the first W/2 lanes of a group hold the mean dots and the others the variance
     // dots, value index (hl % (W/2)) / LPV, each on LPV lanes.  Copy lane `sub` keeps the result of pass `sub`,
@@ -215,8 +219,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
         const int rec = ps * NGRP + grp;
         if (l0 + rec < n_my) {
 #pragma unroll
-          for (int c = 0; c < (VECW >= 4 ? VECW / 4 : 1); ++c) {
-            constexpr int CW = VECW >= 4 ? 4 : VECW;
+          for (int c = 0; c < NC; ++c) {
             float a[CW], bb[CW];
             load_vec<CW>(st + (size_t)rec * 2 * D + c * W * 4 + hl * CW, a);
             load_vec<CW>(st + (size_t)rec * 2 * D + D + c * W * 4 + hl * CW, bb);
