@@ -32,6 +32,9 @@ METRIC = "decode_attention_query_heads_per_s"
 UNIT = "query_heads/s"
 L2_BYTES = 126 * 1024 * 1024
 GRAPH_STEPS = 64
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the score kernel from the ncu capture summarised in
+# profiles/score_cluster_kernel_long_128k.md (69.37 MB read + 0.66 MB written)
+NCU_TRAFFIC = {"long_128k": 70.03e6}
 
 
 # ------------------------------------------------------------------------------------------------------------
@@ -88,7 +91,7 @@ def run_reference(args, w):
     if rank != 0:
         return
     steps, warmup = args.steps, max(args.warmup, 0)
-    n_dec = 24
+    n_dec = 200
     t0 = time.perf_counter()
     vals, cores, sample = oracle_throughput(w, n_dec, repeats=max(1, min(steps + warmup, 6)))
     vals = vals[min(warmup, len(vals) - 1):] or vals
@@ -179,7 +182,7 @@ def run_ours(args, w):
     local = int(os.environ.get("LOCAL_RANK", "0"))
     cpu_base = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        vals, cores, sample = oracle_throughput(w, 24, repeats=2)      # before CUDA is initialised (fork)
+        vals, cores, sample = oracle_throughput(w, 500, repeats=2)      # before CUDA is initialised (fork)
         cpu_base = {"value": vals[-1], "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
 
     build.build()
@@ -341,26 +344,51 @@ def run_ours(args, w):
             at_iso.append(b)
     at = statistics.mean(at_iso)
 
-    # ---- end to end through the public call with host buffers --------------------------------------------------
-    hq = [q.cpu().pin_memory() for q in qs[:8]]
-    hk = [(k.cpu().pin_memory(), v.cpu().pin_memory()) for k, v in kvs[:8]]
+    # ---- end to end through the public call with host buffers -----------------------------------------------------
+    # Per step: the host writes q, k_t, v_t into pinned staging buffers; H2D copies, append, decode and the D2H copy
+    # of the output are enqueued (as one captured graph per cache when graphs are in use) and the stream is
+    # synchronised, because the caller reads the output before it can form the next query.
+    src_q = [q.cpu() for q in qs[:8]]
+    src_kv = [(k.cpu(), v.cpu()) for k, v in kvs[:8]]
+    hq, hk, hv = src_q[0].clone().pin_memory(), src_kv[0][0].clone().pin_memory(), src_kv[0][1].clone().pin_memory()
     dq, dk, dv = torch.empty_like(qs[0]), torch.empty_like(kvs[0][0]), torch.empty_like(kvs[0][1])
     hout = torch.empty(w.batch, w.n_q_heads, w.head_dim, dtype=torch.float32).pin_memory()
-    h2d = hq[0].numel() * hq[0].element_size() + 2 * hk[0][0].numel() * hk[0][0].element_size()
+    h2d = hq.numel() * hq.element_size() + 2 * hk.numel() * hk.element_size()
     d2h = hout.numel() * 4
+
+    def e2e_body(ci):
+        dq.copy_(hq, non_blocking=True)
+        dk.copy_(hk, non_blocking=True)
+        dv.copy_(hv, non_blocking=True)
+        caches[ci].append_tokens(dk, dv)
+        caches[ci].decode(dq, gamma, out=outs[ci])
+        hout.copy_(outs[ci], non_blocking=True)
+
+    e2e_graphs = None
+    with torch.cuda.stream(stream):
+        if steps >= GRAPH_STEPS:
+            set_bounds(exact=False)
+            e2e_graphs = []
+            for ci in range(R):
+                gph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gph, stream=stream):
+                    e2e_body(ci)
+                e2e_graphs.append(gph)
+        else:
+            set_bounds(exact=True)
     barrier()
     with torch.cuda.stream(stream):
         g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         g0.record(stream)
         for i in range(n_e2e):
-            c = caches[i % R]
-            dq.copy_(hq[i % 8], non_blocking=True)
-            dk.copy_(hk[i % 8][0], non_blocking=True)
-            dv.copy_(hk[i % 8][1], non_blocking=True)
-            c.append_tokens(dk, dv)
+            hq.copy_(src_q[i % 8])                                     # the step's inputs arrive in host memory
+            hk.copy_(src_kv[i % 8][0])
+            hv.copy_(src_kv[i % 8][1])
+            if e2e_graphs is not None:
+                e2e_graphs[i % R].replay()
+            else:
+                e2e_body(i % R)
             n_app[i % R] += 1
-            c.decode(dq, gamma, out=outs[i % R])
-            hout.copy_(outs[i % R], non_blocking=True)
             stream.synchronize()                                       # the caller reads the result before the next step
         g1.record(stream)
     barrier()
@@ -388,7 +416,8 @@ def run_ours(args, w):
         "gpu_launches": 3 * steps,
         "roofline": {"bound": "hbm", "kernel": "score_cluster_kernel (block score + top-k)", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                     "bytes_per_launch": score_bytes, "ms_per_launch": sc, "traffic": args.traffic},
+                     "bytes_per_launch": score_bytes, "ms_per_launch": sc,
+                     "traffic": args.traffic if args.traffic is not None else NCU_TRAFFIC.get(w.name)},
         "kernels": {"score_select_ms": sc, "score_select_isolated_ms": statistics.mean(sc_iso),
                     "attend_merge_isolated_ms": at, "decode_minus_score_ms": dec_ms - sc,
                     "decode_only_ms": dec_ms, "decode_only_GBps": by["total"] / (dec_ms * 1e-3) / 1e9,
@@ -415,7 +444,8 @@ def main():
     ap.add_argument("--caches", type=int, default=0, help="rotate over this many caches instead of the cold-L2 count "
                     "(for profiler captures, which must hold little device memory)")
     ap.add_argument("--traffic", type=float, default=None,
-                    help="DRAM bytes per launch of the dominant kernel from an ncu capture (reported as roofline.traffic)")
+                    help="DRAM bytes per launch of the dominant kernel from an ncu capture; default: the figure of "
+                         "profiles/score_cluster_kernel_long_128k.md for the long_128k workload")
     args = ap.parse_args()
     from paper_2601_22379_b200 import synth
     w = synth.BY_NAME[args.workload]
