@@ -26,6 +26,12 @@ notes of the repository):
     the G heads of the group (Section 2.2, grouped BlockScore equation);
   * the sink and local blocks the experiments force (Section 4, "Sparsity
     Specifications") count inside the top-k budget;
+  * strided selection (Section 3.1, "Strided Block Selection"): windows of C
+    tokens every s tokens, only those lying entirely inside one block
+    (starts 0, s, 2s, ... while start + C <= B); a window of a partial last
+    block counts the tokens it actually holds; a block's log mass is the
+    maximum of its windows' Taylor log masses, and the per-head
+    normalisation over blocks comes after this pooling;
   * ties are broken by (score descending, block index ascending);
   * RLA has no normaliser; RMS(.) is RMSNorm with a learnable scale gamma.
 
@@ -107,6 +113,41 @@ def block_covariance_full(K, B: int):
     return cov
 
 
+def window_starts(B: int, C: int, s: int):
+    """In-block start offsets of the strided windows that lie entirely inside a block."""
+    if not (0 < C <= B and s > 0):
+        raise ValueError("need 0 < C <= B and s > 0")
+    return list(range(0, B - C + 1, s))
+
+
+def window_statistics(K, B: int, C: int, s: int):
+    """Key mean and diagonal population variance of every strided window of every block
+    (Section 3.1, "Strided Block Selection": the Taylor statistics on sliding windows).
+
+    K: [L, d].  Returns mean [nblk, NW, d], var [nblk, NW, d], n [nblk, NW]; a window of
+    the partial last block holds n < C tokens, possibly none (then mean = var = 0).
+    """
+    K = np.asarray(K, dtype=F64)
+    L, d = K.shape
+    nblk, nb = block_lengths(L, B)
+    starts = window_starts(B, C, s)
+    NW = len(starts)
+    mean = np.zeros((nblk, NW, d), dtype=F64)
+    var = np.zeros((nblk, NW, d), dtype=F64)
+    n = np.zeros((nblk, NW), dtype=np.int64)
+    for i in range(nblk):
+        for w, t0 in enumerate(starts):
+            cnt = int(min(C, nb[i] - t0))
+            if cnt <= 0:
+                continue
+            kw = K[i * B + t0:i * B + t0 + cnt]
+            n[i, w] = cnt
+            mean[i, w] = kw.sum(axis=0) / cnt
+            dev = kw - mean[i, w]
+            var[i, w] = (dev * dev).sum(axis=0) / cnt
+    return mean, var, n
+
+
 # ---------------------------------------------------------------------------
 # Step 1: block score (Section 3.1)
 # ---------------------------------------------------------------------------
@@ -151,6 +192,32 @@ def block_scores(q_hat_group, mean, var, n, order: int = 2):
         w = np.exp(ell[m] - top)
         p[m] = w / np.sum(w)
     return ell, p, p.sum(axis=0)
+
+
+def pooled_block_scores(q_hat_group, wmean, wvar, wn, order: int = 2):
+    """BlockScore with strided windows: Taylor log mass per window, max-pooled over the
+    windows of a block, then normalised per head over the blocks and summed over the group
+    (Section 3.1, "Strided Block Selection"; Section 2.2 for the normalisation).
+
+    wmean, wvar [nblk, NW, d], wn [nblk, NW].  Returns ell_w [G, nblk, NW] (-inf for empty
+    windows), ell [G, nblk], p [G, nblk], score [nblk].
+    """
+    q_hat_group = np.asarray(q_hat_group, dtype=F64)
+    G = q_hat_group.shape[0]
+    nblk, NW = np.asarray(wn).shape
+    ell_w = np.full((G, nblk, NW), -np.inf, dtype=F64)
+    ell = np.zeros((G, nblk), dtype=F64)
+    p = np.zeros((G, nblk), dtype=F64)
+    for m in range(G):
+        for w in range(NW):
+            live = np.asarray(wn)[:, w] > 0
+            if live.any():
+                ell_w[m, live, w] = taylor_log_mass(q_hat_group[m], wmean[live, w], wvar[live, w], wn[live, w], order=order)
+        ell[m] = ell_w[m].max(axis=1)
+        top = np.max(ell[m])
+        e = np.exp(ell[m] - top)
+        p[m] = e / np.sum(e)
+    return ell_w, ell, p, p.sum(axis=0)
 
 
 # ---------------------------------------------------------------------------
@@ -234,7 +301,7 @@ def rla_by_subtraction(q_group, S_bar, K, V, toks, phi_scale: float = 1.0):
 # ---------------------------------------------------------------------------
 def decode_unit(q_group, K, V, gamma_group, *, block_size, top_k, n_sink=0, n_local=0,
                 sm_scale=None, phi_scale=1.0, rms_eps=1e-6, order=2, use_rla=True,
-                override_selection=None, S_bar=None, stats=None):
+                override_selection=None, S_bar=None, stats=None, window=None):
     """SPLA decode output for one (sequence, KV head) unit.
 
     q_group [G, d] raw queries of the group, K, V [L, d] the whole cache of
@@ -243,6 +310,8 @@ def decode_unit(q_group, K, V, gamma_group, *, block_size, top_k, n_sink=0, n_lo
     `override_selection` replaces steps 1-2 by a given index set (used when a
     correct implementation picked a different set inside the tie tolerance).
     `S_bar` / `stats` may be passed in pre-computed (incremental form).
+    `window` = (C, s) switches the score to strided windows with max-pooling;
+    `stats` then holds window statistics.
     Returns a dict with every intermediate the tests compare.
     """
     q_group = np.asarray(q_group, dtype=F64)
@@ -254,8 +323,13 @@ def decode_unit(q_group, K, V, gamma_group, *, block_size, top_k, n_sink=0, n_lo
         sm_scale = 1.0 / np.sqrt(d)
     q_hat = sm_scale * q_group
 
-    mean, var, n = block_statistics(K, B) if stats is None else stats
-    ell, p, score = block_scores(q_hat, mean, var, n, order=order)
+    ell_w = None
+    if window is None:
+        mean, var, n = block_statistics(K, B) if stats is None else stats
+        ell, p, score = block_scores(q_hat, mean, var, n, order=order)
+    else:
+        mean, var, n = window_statistics(K, B, window[0], window[1]) if stats is None else stats
+        ell_w, ell, p, score = pooled_block_scores(q_hat, mean, var, n, order=order)
     if override_selection is None:
         sel = select_blocks(score, top_k, n_sink, n_local)
     else:
@@ -274,7 +348,7 @@ def decode_unit(q_group, K, V, gamma_group, *, block_size, top_k, n_sink=0, n_lo
         o_bar = o_tilde = o_rla = np.zeros_like(o_sparse)
         out = o_sparse.copy()
     return dict(ell=ell, p=p, score=score, sel=sel, o_sparse=o_sparse, o_bar=o_bar,
-                o_tilde=o_tilde, o_rla=o_rla, out=out, mean=mean, var=var, n=n)
+                o_tilde=o_tilde, o_rla=o_rla, out=out, mean=mean, var=var, n=n, ell_w=ell_w)
 
 
 def decode(q, K, V, gamma, seq_lens, *, n_kv_heads, **cfg):
@@ -311,8 +385,14 @@ class UnitCache:
     definitional form.
     """
 
-    def __init__(self, d: int, block_size: int, phi_scale: float = 1.0):
+    def __init__(self, d: int, block_size: int, phi_scale: float = 1.0, window=None):
         self.d, self.B, self.phi_scale = d, block_size, phi_scale
+        self.window = window                      # (C, s) or None: strided windows kept beside the blocks
+        self.starts = window_starts(block_size, window[0], window[1]) if window else []
+        NW = len(self.starts)
+        self.wmean = np.zeros((0, NW, d), dtype=F64)
+        self.wm2 = np.zeros((0, NW, d), dtype=F64)
+        self.wn = np.zeros((0, NW), dtype=np.int64)
         self.K = np.zeros((0, d), dtype=F64)
         self.V = np.zeros((0, d), dtype=F64)
         self.mean = np.zeros((0, d), dtype=F64)
@@ -322,14 +402,17 @@ class UnitCache:
         self._chunks_k, self._chunks_v = [], []
 
     @classmethod
-    def from_prefill(cls, K, V, block_size: int, phi_scale: float = 1.0):
+    def from_prefill(cls, K, V, block_size: int, phi_scale: float = 1.0, window=None):
         """Cache holding an existing context: statistics and S_bar from their definitions."""
         K = np.asarray(K, dtype=F64)
         V = np.asarray(V, dtype=F64)
-        c = cls(K.shape[1], block_size, phi_scale)
+        c = cls(K.shape[1], block_size, phi_scale, window)
         c.K, c.V = K, V
         c.mean, var, c.n = block_statistics(K, block_size)
         c.m2 = var * c.n[:, None]
+        if window:
+            c.wmean, wvar, c.wn = window_statistics(K, block_size, window[0], window[1])
+            c.wm2 = wvar * c.wn[:, :, None]
         c.S_bar = rla_global_state(K, V, phi_scale)
         return c
 
@@ -345,6 +428,18 @@ class UnitCache:
                 self.mean = np.vstack([self.mean, np.zeros((1, self.d))])
                 self.m2 = np.vstack([self.m2, np.zeros((1, self.d))])
                 self.n = np.append(self.n, 0)
+                if self.window:
+                    NW = len(self.starts)
+                    self.wmean = np.concatenate([self.wmean, np.zeros((1, NW, self.d))])
+                    self.wm2 = np.concatenate([self.wm2, np.zeros((1, NW, self.d))])
+                    self.wn = np.concatenate([self.wn, np.zeros((1, NW), dtype=np.int64)])
+            t_in = int(self.n[-1])                # position of the new token inside its block
+            for w, t0 in enumerate(self.starts):
+                if t0 <= t_in < t0 + self.window[0]:
+                    self.wn[-1, w] += 1
+                    dw = k_t - self.wmean[-1, w]
+                    self.wmean[-1, w] += dw / self.wn[-1, w]
+                    self.wm2[-1, w] += dw * (k_t - self.wmean[-1, w])
             self.n[-1] += 1
             delta = k_t - self.mean[-1]
             self.mean[-1] += delta / self.n[-1]
@@ -360,9 +455,12 @@ class UnitCache:
             self._chunks_k, self._chunks_v = [], []
 
     def stats(self):
+        if self.window:
+            return self.wmean, self.wm2 / np.maximum(self.wn, 1)[:, :, None], self.wn
         return self.mean, self.m2 / self.n[:, None], self.n
 
     def decode(self, q_group, gamma_group, **cfg):
         self._materialise()
         return decode_unit(q_group, self.K, self.V, gamma_group, block_size=self.B,
-                           phi_scale=self.phi_scale, S_bar=self.S_bar, stats=self.stats(), **cfg)
+                           phi_scale=self.phi_scale, S_bar=self.S_bar, stats=self.stats(),
+                           window=self.window, **cfg)

@@ -376,3 +376,103 @@ def test_p9_incremental_cache_equals_from_scratch():
     np.testing.assert_allclose(a["out"], b["out"], rtol=1e-10, atol=1e-12)
     pre = O.UnitCache.from_prefill(K, V, B)
     np.testing.assert_allclose(pre.decode(q, gamma, **cfg)["out"], b["out"], rtol=1e-12, atol=1e-14)
+
+
+# ---------------------------------------------------------------------------
+# Strided windows (Section 3.1, "Strided Block Selection"): statistics on windows of C tokens
+# every s tokens, max-pooled per block
+# ---------------------------------------------------------------------------
+def test_window_layout_and_counts_small_table():
+    # B = 8, C = 4, s = 2: windows start at 0, 2, 4 inside a block.  13 tokens = one full block and one of 5:
+    # its windows [0,4), [2,6), [4,8) hold 4, 3 and 1 tokens (counted by hand).
+    assert O.window_starts(8, 4, 2) == [0, 2, 4]
+    assert O.window_starts(64, 32, 16) == [0, 16, 32]
+    assert len(O.window_starts(128, 32, 16)) == 7
+    K = RNG.standard_normal((13, 3))
+    mean, var, n = O.window_statistics(K, 8, 4, 2)
+    assert n.tolist() == [[4, 4, 4], [4, 3, 1]]
+    np.testing.assert_allclose(mean[1, 1], K[10:13].mean(axis=0), rtol=1e-14)
+    np.testing.assert_allclose(var[0, 2], K[4:8].var(axis=0), rtol=1e-13)     # numpy's population variance
+    np.testing.assert_allclose(var[1, 2], 0.0, atol=0)                        # one token: no spread
+
+
+def test_window_equal_to_block_reduces_to_block_mode():
+    d, B, L = 8, 16, 16 * 5 + 7
+    K, V = RNG.standard_normal((L, d)), RNG.standard_normal((L, d))
+    q, g = RNG.standard_normal((3, d)), 0.1 * RNG.standard_normal((3, d))
+    a = O.decode_unit(q, K, V, g, block_size=B, top_k=3, n_sink=1, n_local=1)
+    b = O.decode_unit(q, K, V, g, block_size=B, top_k=3, n_sink=1, n_local=1, window=(B, B))
+    np.testing.assert_array_equal(a["sel"], b["sel"])
+    np.testing.assert_allclose(a["score"], b["score"], rtol=1e-14)
+    np.testing.assert_allclose(a["out"], b["out"], rtol=1e-14)
+
+
+def test_window_constant_blocks_give_exact_largest_window_mass():
+    # every key of a block equal: each window's Taylor mass is exact, n_w exp(q k); the pooled value is the one
+    # of the fullest window, min(C, n_i) exp(q k_i), at both orders, partial last block included
+    d, B, C, s, L = 5, 16, 8, 4, 16 * 3 + 6
+    centres = RNG.standard_normal((4, d))
+    K = np.repeat(centres, B, axis=0)[:L]
+    q = RNG.standard_normal((1, d))
+    wm, wv, wn = O.window_statistics(K, B, C, s)
+    for order in (1, 2):
+        _, ell, p, score = O.pooled_block_scores(q, wm, wv, wn, order=order)
+        exact = np.log(np.minimum(C, [16, 16, 16, 6])) + centres @ q[0]
+        np.testing.assert_allclose(ell[0], exact, rtol=1e-13)
+        share = np.exp(exact - scipy.special.logsumexp(exact))
+        np.testing.assert_allclose(score, share, rtol=1e-12)
+
+
+def test_window_first_order_pooled_mass_never_exceeds_exact_block_mass():
+    # Jensen: n_w exp(q mean_w) <= sum over the window of exp(q k_t) <= the block's exact mass
+    d, B, C, s, L = 6, 32, 8, 4, 32 * 6 + 11
+    K = 1.5 * RNG.standard_normal((L, d))
+    q = RNG.standard_normal((2, d))
+    wm, wv, wn = O.window_statistics(K, B, C, s)
+    ell_w, ell, _, _ = O.pooled_block_scores(q, wm, wv, wn, order=1)
+    for m in range(2):
+        for i in range(ell.shape[1]):
+            exact = np.log(np.sum(np.exp(K[i * B:(i + 1) * B] @ q[m])))
+            assert ell[m, i] <= exact + 1e-12
+            assert ell[m, i] == ell_w[m, i].max()
+
+
+def test_window_pooling_finds_a_needle_that_fills_half_a_block():
+    # 32 of a block's 64 keys (one whole window) are shifted toward q: the window that holds exactly them sees the
+    # full shift, the block mean only half of it, so pooling ranks the block first where the block mean does not
+    d, B = 16, 64
+    K = 0.3 * RNG.standard_normal((B * 8, d))
+    V = RNG.standard_normal((B * 8, d))
+    q = RNG.standard_normal((1, d))
+    u = q[0] / np.linalg.norm(q[0])
+    K[3 * B + 16:3 * B + 48] += 2.0 * u          # half-block needle in block 3, window [16, 48)
+    K[5 * B:6 * B] += 1.3 * u                    # whole-block decoy in block 5
+    g = np.ones((1, d))
+    blk = O.decode_unit(q, K, V, g, block_size=B, top_k=1, sm_scale=1.0)
+    win = O.decode_unit(q, K, V, g, block_size=B, top_k=1, sm_scale=1.0, window=(32, 16))
+    assert blk["sel"][0] == 5 and win["sel"][0] == 3
+    assert int(np.argmax(win["ell_w"][0, 3])) == 1
+
+
+def test_window_scores_normalise_and_incremental_equals_definitional():
+    d, B, C, s = 8, 32, 16, 8
+    L0, L1 = 32 * 3 + 5, 32 * 5 + 19
+    K, V = RNG.standard_normal((L1, d)), RNG.standard_normal((L1, d))
+    q, g = RNG.standard_normal((4, d)), 0.1 * RNG.standard_normal((4, d))
+    ref = O.decode_unit(q, K, V, g, block_size=B, top_k=3, n_sink=1, n_local=1, window=(C, s))
+    np.testing.assert_allclose(ref["p"].sum(axis=1), 1.0, rtol=1e-14)
+    np.testing.assert_allclose(ref["score"].sum(), 4.0, rtol=1e-13)
+    c = O.UnitCache.from_prefill(K[:L0], V[:L0], B, window=(C, s))
+    for t in range(L0, L1):
+        c.append(K[t], V[t])
+    inc = c.decode(q, g, top_k=3, n_sink=1, n_local=1)
+    np.testing.assert_array_equal(inc["n"], ref["n"])
+    np.testing.assert_allclose(inc["mean"], ref["mean"], rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(inc["var"], ref["var"], rtol=1e-10, atol=1e-13)
+    np.testing.assert_allclose(inc["out"], ref["out"], rtol=1e-10, atol=1e-12)
+    # tokens permuted inside one stride segment leave every window untouched
+    Kp = K.copy()
+    Kp[8:16] = K[8:16][::-1]
+    wm, wv, _ = O.window_statistics(Kp, B, C, s)
+    np.testing.assert_allclose(wm, ref["mean"], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(wv, ref["var"], rtol=1e-11, atol=1e-14)
