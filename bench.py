@@ -41,6 +41,7 @@ NCU_TRAFFIC = {"long_128k": 70.03e6}
 # CPU baseline: the float64 oracle, as it stands, on the host cores (also the --impl reference arm)
 # ------------------------------------------------------------------------------------------------------------
 _ORACLE_UNITS = None
+WINDOW = None          # (C, s) when --window is given: strided selection windows instead of whole blocks
 
 
 def _oracle_worker(args):
@@ -50,7 +51,7 @@ def _oracle_worker(args):
     from oracle import spla_oracle as O
     K, V, qs, gam = _ORACLE_UNITS[idx]
     with threadpool_limits(limits=1):
-        cache = O.UnitCache.from_prefill(K, V, cfg["block_size"])
+        cache = O.UnitCache.from_prefill(K, V, cfg["block_size"], window=cfg["window"])
         t0 = time.perf_counter()
         for i in range(n_dec):
             cache.decode(qs[i % len(qs)], gam, top_k=cfg["top_k"], n_sink=cfg["n_sink"], n_local=cfg["n_local"])
@@ -72,7 +73,7 @@ def oracle_throughput(w, n_dec_per_unit: int, repeats: int = 1):
     _ORACLE_UNITS = [(K[h].double().numpy(), V[h].double().numpy(), [q[h * G:(h + 1) * G] for q in qs],
                       gam[h * G:(h + 1) * G]) for h in range(n_units)]
     del K, V
-    cfg = dict(block_size=w.block_size, top_k=w.top_k, n_sink=w.n_sink, n_local=w.n_local)
+    cfg = dict(block_size=w.block_size, top_k=w.top_k, n_sink=w.n_sink, n_local=w.n_local, window=WINDOW)
     values = []
     ctx = mp.get_context("fork")
     with ctx.Pool(n_units) as pool:
@@ -80,7 +81,7 @@ def oracle_throughput(w, n_dec_per_unit: int, repeats: int = 1):
             times = pool.map(_oracle_worker, [(i, n_dec_per_unit, cfg) for i in range(n_units)])
             values.append(n_units * n_dec_per_unit * G / max(times))
     _ORACLE_UNITS = None
-    sample = (f"{n_units} units (sequence 0, KV heads 0..{n_units - 1}) of {w.name}, {n_dec_per_unit} decode calls each, "
+    sample = (f"{n_units} units (sequence 0, KV heads 0..{n_units - 1}) of {workload_name(w)}, {n_dec_per_unit} decode calls each, "
               f"float64 numpy oracle with cached block statistics and state, one process per unit")
     return values, n_units, sample
 
@@ -105,16 +106,26 @@ def run_reference(args, w):
 
 
 # ------------------------------------------------------------------------------------------------------------
+def n_windows(w):
+    return (w.block_size - WINDOW[0]) // WINDOW[1] + 1 if WINDOW else 1
+
+
+def workload_name(w):
+    return w.name + (f"+windows(C={WINDOW[0]},s={WINDOW[1]})" if WINDOW else "")
+
+
 def base_line(args, w, value, ms_per_step):
     from paper_2601_22379_b200 import synth
-    by = synth.algorithmic_bytes_per_step(w)
+    by = synth.algorithmic_bytes_per_step(w, n_windows=n_windows(w))
     return {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16" if w.kv_dtype == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": w.name, "batch": w.batch, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads,
+        "config": {"workload": workload_name(w), "batch": w.batch, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads,
                    "head_dim": w.head_dim, "context": w.context, "block_size": w.block_size, "top_k": w.top_k,
                    "n_sink": w.n_sink, "n_local": w.n_local, "kv_dtype": w.kv_dtype,
+                   "selection": (f"strided windows C={WINDOW[0]} s={WINDOW[1]}, max-pooled per block" if WINDOW
+                                 else "whole-block statistics"),
                    "algorithmic_bytes_per_step": by["total"], "dense_kv_bytes_per_step": by["dense_kv"],
                    "parallelism": f"replicas x{args.gpus} (units are independent; no collective)"},
     }
@@ -192,7 +203,7 @@ def run_ours(args, w):
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
     steps, warmup = args.steps, max(args.warmup, 3)
-    by = synth.algorithmic_bytes_per_step(w)
+    by = synth.algorithmic_bytes_per_step(w, n_windows=n_windows(w))
     R = 2                                                             # caches to rotate over (cold-L2 protocol)
     while R * by["total"] < 3 * L2_BYTES and R < GRAPH_STEPS:
         R *= 2
@@ -204,7 +215,7 @@ def run_ours(args, w):
     prefill = runner.generate_prefill(wl, dev)
     caches = []
     for _ in range(R):
-        c, _, _, _ = runner.build_cache(wl, dev, prefill=prefill)
+        c, _, _, _ = runner.build_cache(wl, dev, prefill=prefill, window=WINDOW)
         caches.append(c)
     del prefill
     n_app = [0] * R                                                   # tokens appended per cache so far
@@ -417,7 +428,7 @@ def run_ours(args, w):
         "roofline": {"bound": "hbm", "kernel": "score_cluster_kernel (block score + top-k)", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "bytes_per_launch": score_bytes, "ms_per_launch": sc,
-                     "traffic": args.traffic if args.traffic is not None else NCU_TRAFFIC.get(w.name)},
+                     "traffic": args.traffic if args.traffic is not None else NCU_TRAFFIC.get(workload_name(w))},
         "kernels": {"score_select_ms": sc, "score_select_isolated_ms": statistics.mean(sc_iso),
                     "attend_merge_isolated_ms": at, "decode_minus_score_ms": dec_ms - sc,
                     "decode_only_ms": dec_ms, "decode_only_GBps": by["total"] / (dec_ms * 1e-3) / 1e9,
@@ -446,7 +457,12 @@ def main():
     ap.add_argument("--traffic", type=float, default=None,
                     help="DRAM bytes per launch of the dominant kernel from an ncu capture; default: the figure of "
                          "profiles/score_cluster_kernel_long_128k.md for the long_128k workload")
+    ap.add_argument("--window", default=None, metavar="C,s",
+                    help="strided selection windows (the paper's setting is 32,16) instead of whole-block statistics")
     args = ap.parse_args()
+    if args.window:
+        global WINDOW
+        WINDOW = tuple(int(x) for x in args.window.split(","))
     from paper_2601_22379_b200 import synth
     w = synth.BY_NAME[args.workload]
     if args.impl == "reference":

@@ -82,13 +82,19 @@ typedef struct {
   float phi_scale;        /* multiplies q and k inside the feature map phi = softmax; 0 -> 1 */
   float rms_eps;          /* epsilon of the RMSNorm; 0 -> 1e-6 */
   uint32_t flags;
+  int32_t window_size;    /* C: strided selection windows (Section 3.1, "Strided Block Selection"); 0 = whole blocks */
+  int32_t window_stride;  /* s: distance between window starts; 0 with window_size 0.  The paper uses C = 32, s = 16.
+                             Windows are the ones lying entirely inside a block: starts 0, s, 2s, ... while
+                             start + C <= B; at most 8 per block.  A block's log mass is the maximum over its
+                             windows, and the per-head normalisation over blocks comes after that pooling. */
 } spla_config_t;
 
 /* Device buffers of one cache, all caller-owned.  max_blocks = ceil(max_context / B). */
 typedef struct {
   void *k_cache;      /* DEVICE [batch][H_kv][max_blocks][B][d] kv_dtype; token t of a unit lives in block t / B */
   void *v_cache;      /* DEVICE same layout */
-  float *stats;       /* DEVICE [batch][H_kv][max_blocks][2][d] fp32: key mean, then population variance */
+  float *stats;       /* DEVICE [batch][H_kv][max_blocks][NW][2][d] fp32: key mean, then population variance, of each
+                         of the NW selection windows of a block (NW = 1: the whole block) */
   float *rla_state;   /* DEVICE [batch][H_kv][d][d] fp32 S_bar: row = feature of phi(k), column = value dim */
   float *tok_lse;     /* DEVICE [batch][H_kv][max_blocks * B] fp32: logsumexp_c(phi_scale * k_t[c]) per token */
   int32_t *seq_lens;  /* DEVICE [batch]: tokens cached per sequence */
@@ -184,7 +190,8 @@ int spla_sync_status(spla_cache_t *cache, void *stream);
  *   config:     HOST; batch, heads, head_dim, block_size, top_k, max_context, sink/local counts, q_dtype,
  *               sm_scale and SPLA_FIRST_ORDER are used.  The scratch needed, about
  *               batch * H_kv * max_blocks * (G + 1) * 4 bytes, must fit SPLA_NOALLOC_SCRATCH_BYTES, otherwise
- *               SPLA_ERR_UNSUPPORTED is returned and nothing is launched.
+ *               SPLA_ERR_UNSUPPORTED is returned and nothing is launched.  window_size must be 0 (whole-block
+ *               statistics), otherwise SPLA_ERR_UNSUPPORTED.
  *   stats:      DEVICE fp32 [batch][H_kv][max_blocks][2][d], as maintained by spla_append_tokens.
  *   seq_lens:   DEVICE int32 [batch].
  *   q:          DEVICE [batch][H_q][d] q_dtype.

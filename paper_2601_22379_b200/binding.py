@@ -29,7 +29,12 @@ class SplaConfig(C.Structure):
                 ("block_size", C.c_int32), ("top_k", C.c_int32), ("max_context", C.c_int32),
                 ("n_sink_blocks", C.c_int32), ("n_local_blocks", C.c_int32), ("kv_dtype", C.c_int32),
                 ("q_dtype", C.c_int32), ("sm_scale", C.c_float), ("phi_scale", C.c_float), ("rms_eps", C.c_float),
-                ("flags", C.c_uint32)]
+                ("flags", C.c_uint32), ("window_size", C.c_int32), ("window_stride", C.c_int32)]
+
+    @property
+    def n_windows(self) -> int:
+        """Selection windows per block (1 without strided windows)."""
+        return (self.block_size - self.window_size) // self.window_stride + 1 if self.window_size > 0 else 1
 
 
 class SplaBuffers(C.Structure):
@@ -104,10 +109,11 @@ def _stream() -> int:
 
 def make_config(*, batch, n_q_heads, n_kv_heads, head_dim, block_size, top_k, max_context, n_sink_blocks=1,
                 n_local_blocks=4, kv_dtype="bf16", q_dtype=None, sm_scale=0.0, phi_scale=0.0, rms_eps=0.0,
-                flags=0) -> SplaConfig:
+                flags=0, window_size=0, window_stride=0) -> SplaConfig:
     code = {"bf16": SPLA_BF16, "f32": SPLA_F32}
     return SplaConfig(batch, n_q_heads, n_kv_heads, head_dim, block_size, top_k, max_context, n_sink_blocks,
-                      n_local_blocks, code[kv_dtype], code[q_dtype or kv_dtype], sm_scale, phi_scale, rms_eps, flags)
+                      n_local_blocks, code[kv_dtype], code[q_dtype or kv_dtype], sm_scale, phi_scale, rms_eps, flags,
+                      window_size, window_stride)
 
 
 def query_sizes(cfg: SplaConfig) -> SplaSizes:
@@ -147,7 +153,8 @@ class SplaCache:
     """Owns the device buffers (as torch tensors) of one cache and forwards to the C ABI.
 
     Shapes follow include/spla.h: k_cache/v_cache [batch, H_kv, max_blocks, B, d], stats
-    [batch, H_kv, max_blocks, 2, d], rla_state [batch, H_kv, d, d], tok_lse [batch, H_kv, max_blocks * B].
+    [batch, H_kv, max_blocks, 2, d] (with strided windows [batch, H_kv, max_blocks, NW, 2, d]), rla_state
+    [batch, H_kv, d, d], tok_lse [batch, H_kv, max_blocks * B].
     """
 
     def __init__(self, cfg: SplaConfig, device="cuda:0"):
@@ -166,7 +173,8 @@ class SplaCache:
         self.bufs = _Bufs(
             k_cache=torch.empty(*shp, B, d, dtype=kv_t, device=dev),
             v_cache=torch.empty(*shp, B, d, dtype=kv_t, device=dev),
-            stats=torch.empty(*shp, 2, d, dtype=torch.float32, device=dev),
+            stats=torch.empty(*shp, *((cfg.n_windows,) if cfg.window_size > 0 else ()), 2, d, dtype=torch.float32,
+                              device=dev),
             rla_state=torch.empty(cfg.batch, cfg.n_kv_heads, d, d, dtype=torch.float32, device=dev),
             tok_lse=torch.empty(cfg.batch, cfg.n_kv_heads, self.max_blocks * B, dtype=torch.float32, device=dev),
             seq_lens=torch.empty(cfg.batch, dtype=torch.int32, device=dev),

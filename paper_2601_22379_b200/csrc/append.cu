@@ -66,17 +66,22 @@ __global__ void __launch_bounds__(kCopyThreads) append_copy_kernel(const Params 
   if (lane == 0) p.tok_lse[pos] = mx + logf(s);
 }
 
-// Mean and population variance of one block, two exact passes, by kStatThreads threads (groups of D threads take
-// every TG-th token; the partial sums are combined in a fixed order, so every append path gives the same bits).
-// Token t of the block comes from the cache if its position is below `L_cached`, else from the new tokens.
+// Mean and population variance of one selection window of one block (window w covers the block's tokens
+// [w * win_s, w * win_s + win_C); without strided windows that is the whole block), two exact passes, by
+// kStatThreads threads (groups of D threads take every TG-th token; the partial sums are combined in a fixed
+// order, so every append path gives the same bits).  Token t of the block comes from the cache if its position
+// is below `L_cached`, else from the new tokens.  A window that holds no token yet is left alone.
 constexpr int kStatThreads = 256;
 template <typename T, int D>
-__device__ __forceinline__ void block_stats_role(const Params& p, int u, int blk, int L_cached, int L_total, const T* kn,
+__device__ __forceinline__ void block_stats_role(const Params& p, int u, int blk, int w, int L_cached, int L_total, const T* kn,
                                                  bool act, float (*red_s)[D], float* mean_s) {
   constexpr int TG = kStatThreads / D;
   const int tid = threadIdx.x;
   const int t0 = blk * p.B;
-  const int cnt = act ? min(p.B, L_total - t0) : 0;
+  const int t_lo = w * p.win_s;
+  const int t_hi = act ? min(min(p.B, L_total - t0), t_lo + p.win_C) : 0;     // tokens [t_lo, t_hi) of the block
+  const int cnt = max(0, t_hi - t_lo);
+  act = act && cnt > 0;
   const int tg = tid / D, c = tid % D;
   const T* kc = reinterpret_cast<const T*>(p.k_cache) + ((size_t)u * p.max_blocks * p.B + t0) * D + c;
   // One address per token (cached or new) and one load from it: no branch around the loads, so that the
@@ -88,7 +93,7 @@ __device__ __forceinline__ void block_stats_role(const Params& p, int u, int blk
   };
   float sum = 0.f;
 #pragma unroll 8
-  for (int t = tg; t < cnt; t += TG) sum += key_at(t);
+  for (int t = t_lo + tg; t < t_hi; t += TG) sum += key_at(t);
   red_s[tg][c] = sum;
   __syncthreads();
   if (tg == 0) {
@@ -101,7 +106,7 @@ __device__ __forceinline__ void block_stats_role(const Params& p, int u, int blk
   const float mean = mean_s[c];
   float ss = 0.f;
 #pragma unroll 8
-  for (int t = tg; t < cnt; t += TG) {
+  for (int t = t_lo + tg; t < t_hi; t += TG) {
     const float dv = key_at(t) - mean;
     ss = fmaf(dv, dv, ss);
   }
@@ -112,7 +117,7 @@ __device__ __forceinline__ void block_stats_role(const Params& p, int u, int blk
     float tot = 0.f;
 #pragma unroll
     for (int g2 = 0; g2 < TG; ++g2) tot += red_s[g2][c];
-    float* rec = p.stats + ((size_t)u * p.max_blocks + blk) * 2 * D;
+    float* rec = p.stats + (((size_t)u * p.max_blocks + blk) * p.NW + w) * 2 * D;
     rec[c] = mean;
     rec[D + c] = tot / (float)cnt;
   }
@@ -125,11 +130,11 @@ __global__ void __launch_bounds__(kStatThreads) append_stats_kernel(const Params
   const int u = blockIdx.y, b = u / p.Hkv;
   const int L = p.seq_lens[b];
   const int n = tokens_to_add(p, n_new, max_new, b, L);
-  const int blk = L / p.B + blockIdx.x;                    // x-th touched block
+  const int blk = L / p.B + blockIdx.x / p.NW;             // a window of the x-th touched block
   const bool act = n > 0 && blk * p.B < L + n;             // CTA-uniform
   if (!act) return;
   // the copy kernel has already stored the new tokens: everything is read from the cache
-  block_stats_role<T, D>(p, u, blk, L + n, L + n, static_cast<const T*>(nullptr), true, red_s, mean_s);
+  block_stats_role<T, D>(p, u, blk, blockIdx.x % p.NW, L + n, L + n, static_cast<const T*>(nullptr), true, red_s, mean_s);
 }
 
 template <typename T, int D>
@@ -234,8 +239,8 @@ __global__ void __launch_bounds__(kFusedThreads) append_fused_kernel(const Param
     }
   } else if ((role -= n_copy) < n_stats) {
     // ---- statistics role: one touched block; cached keys below the old length, new keys above it -----------
-    const int blk = L / p.B + role;
-    block_stats_role<T, D>(p, u, blk, L, L + max(n, 0), kn, n > 0 && blk * p.B < L + n, red_s, mean_s);
+    const int blk = L / p.B + role / p.NW;
+    block_stats_role<T, D>(p, u, blk, role % p.NW, L, L + max(n, 0), kn, n > 0 && blk * p.B < L + n, red_s, mean_s);
   } else if (!(p.flags & 4u)) {
     // ---- state role: S_bar[row0 .. row0 + 15][:] += sum_t phi(k_t)[row] v_t ------------------------------------
     role -= n_stats;
@@ -324,7 +329,7 @@ static cudaError_t launch_typed(const Params& p, const void* k_new, const void* 
   const T* vn = reinterpret_cast<const T*>(v_new);
   if (max_new <= kFusedMaxNew) {
     const int n_copy = (max_new + kFusedThreads / 32 - 1) / (kFusedThreads / 32);
-    const int n_stats = (max_new + p.B - 1) / p.B + 1;
+    const int n_stats = ((max_new + p.B - 1) / p.B + 1) * p.NW;   // one CTA per window of every block that can be touched
     const int n_state = (p.flags & 4u) ? 0 : D / kStateRows;
     // Same shared-memory carve-out as the decode kernels around it: a change of carve-out drains the SMs.
     cudaFuncSetAttribute(append_fused_kernel<T, D>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
@@ -333,7 +338,7 @@ static cudaError_t launch_typed(const Params& p, const void* k_new, const void* 
   }
   const int per_cta = kCopyThreads / 32;
   append_copy_kernel<T, D><<<dim3((max_new + per_cta - 1) / per_cta, U), kCopyThreads, 0, stream>>>(p, kn, vn, n_new, max_new);
-  append_stats_kernel<T, D><<<dim3((max_new + p.B - 1) / p.B + 1, U), kStatThreads, 0, stream>>>(p, n_new, max_new);
+  append_stats_kernel<T, D><<<dim3(((max_new + p.B - 1) / p.B + 1) * p.NW, U), kStatThreads, 0, stream>>>(p, n_new, max_new);
   if (!(p.flags & 4u))
     append_state_kernel<T, D><<<dim3(D / kStateRows, U), D, 0, stream>>>(p, kn, vn, n_new, max_new);
   append_lengths_kernel<<<(p.batch + 127) / 128, 128, 0, stream>>>(p, n_new, max_new);

@@ -49,6 +49,14 @@ __device__ __forceinline__ void st_dsmem_u32(uint32_t addr, uint32_t v) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// Order-preserving map of a float onto an unsigned integer (larger float <=> larger key; every key is above 0).
+__device__ __forceinline__ uint32_t float_order_key(float x) {
+  const uint32_t b = __float_as_uint(x);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float float_from_order_key(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
 __device__ __forceinline__ void lse_merge(float& m, float& s, float m2, float s2) {
   const float nm = fmaxf(m, m2);
   if (nm > -INFINITY) s = s * __expf(m - nm) + s2 * __expf(m2 - nm);
@@ -130,7 +138,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   float* wred = reinterpret_cast<float*>(smem_raw + SM::kWred);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw + SM::kBars);
   uint64_t* empty = full + kStages;
-  float* ell_s = reinterpret_cast<float*>(smem_raw + SM::kEll);          // [G][chunk]
+  float* ell_s = reinterpret_cast<float*>(smem_raw + SM::kEll);          // [G][chunk] log mass per block
   __shared__ int err_s;
 
   if (tid == 0) {                               // nothing here depends on the preceding kernel
@@ -168,12 +176,15 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   }
   const int L = __ldcg(p.seq_lens + b);
   const int nblk = (L + p.B - 1) / p.B;
-  const int chunk = p.chunk;
-  const int rec_begin = min(nblk, rank * chunk);
-  const int rec_end = min(nblk, rec_begin + chunk);
-  const int n_my = rec_end - rec_begin;
+  const int chunk = p.chunk;                      // blocks per CTA
+  const int NW = p.NW;                            // selection windows per block; a "record" is one window
+  const int blk_begin = min(nblk, rank * chunk);
+  const int blk_end = min(nblk, blk_begin + chunk);
+  const int nb_my = blk_end - blk_begin;          // blocks of this CTA
+  const int rec_begin = blk_begin * NW;
+  const int n_my = nb_my * NW;                    // records of this CTA
   const int n_rounds = (n_my + kStageRec - 1) / kStageRec;
-  const float* stats_u = p.stats + (size_t)u * p.max_blocks * 2 * D;
+  const float* stats_u = p.stats + (size_t)u * p.max_blocks * NW * 2 * D;
 
   auto issue = [&](int r) {                      // thread 0 only: one bulk copy fills stage r % kStages
     const int s = r % kStages;
@@ -193,6 +204,8 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
       qv[g][v] = (p.flags & 2u) ? 0.f : 0.5f * qm[g][v] * qm[g][v];
     }
   }
+  if (NW > 1)                                   // pooled slots start below every key
+    for (int x = tid; x < G * chunk; x += kCsThreads) reinterpret_cast<uint32_t*>(ell_s)[x] = 0u;
   __syncthreads();                              // the barrier initialisation is visible to every consumer
   SPLA_MARK(p, u, rank, 1);
 
@@ -204,7 +217,9 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
     const int sub = hl % LPV;
     const bool fin_lane = hl < W / 2 && sub < FB && my_g < G;
     const float ln_full = logf((float)p.B);
-    const float ln_last = logf((float)max(1, L - (nblk - 1) * p.B));
+    const int n_last = L - (nblk - 1) * p.B;     // tokens of the last block
+    const float ln_last = logf((float)max(1, n_last));
+    const float ln_win = logf((float)p.win_C);
     float run_max = -INFINITY, run_sum = 0.f;
 
 #pragma unroll 1
@@ -262,16 +277,49 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
           }
           const int li = l0 + (p0 + sub) * NGRP + grp;
           if (fin_lane && li < n_my) {
-            const float ell = (rec_begin + li == nblk - 1 ? ln_last : ln_full) + dm_keep + __logf(1.f + dv_keep);
-            ell_s[my_g * chunk + li] = ell;
-            const float nm = fmaxf(run_max, ell);
-            run_sum = run_sum * __expf(run_max - nm) + __expf(ell - nm);
-            run_max = nm;
+            if (NW == 1) {
+              const float ell = (rec_begin + li == nblk - 1 ? ln_last : ln_full) + dm_keep + __logf(1.f + dv_keep);
+              ell_s[my_g * chunk + li] = ell;
+              const float nm = fmaxf(run_max, ell);
+              run_sum = run_sum * __expf(run_max - nm) + __expf(ell - nm);
+              run_max = nm;
+            } else {
+              // strided windows (Section 3.1, "Strided Block Selection"): log mass of window w of a block,
+              // max-pooled into the block's slot right away through an order-preserving integer key
+              const int lb = li / NW, w = li - lb * NW;
+              float ln_n = ln_win;
+              if (blk_begin + lb == nblk - 1) {
+                const int cnt = min(p.win_C, n_last - w * p.win_s);
+                ln_n = cnt > 0 ? logf((float)cnt) : -INFINITY;
+              }
+              atomicMax(reinterpret_cast<uint32_t*>(ell_s) + my_g * chunk + lb, float_order_key(ln_n + dm_keep + __logf(1.f + dv_keep)));
+            }
           }
         }
       }
     }
     SPLA_MARK(p, u, rank, 2);
+    if (NW > 1) {
+      // the pooled keys back to floats, and this CTA's (max, sum exp) per head from them; lane 0 of every warp
+      // then holds the warp's pair
+      __syncthreads();
+#pragma unroll
+      for (int g = 0; g < GP; ++g) {
+        float m = -INFINITY, sm = 0.f;
+        if (g < G)
+          for (int lb = tid; lb < nb_my; lb += kCsThreads) {
+            const float x = float_from_order_key(reinterpret_cast<const uint32_t*>(ell_s)[g * chunk + lb]);
+            ell_s[g * chunk + lb] = x;
+            lse_merge(m, sm, x, 1.f);
+          }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const float m2 = __shfl_xor_sync(0xffffffffu, m, o), s2 = __shfl_xor_sync(0xffffffffu, sm, o);
+          lse_merge(m, sm, m2, s2);
+        }
+        if (lane == 0) { wred[(warp * GP + g) * 2 + 0] = m; wred[(warp * GP + g) * 2 + 1] = sm; }
+      }
+    }
     // fold the finalising lanes of a head: copy lanes (xor < LPV), then the record groups of the warp (xor W)
 #pragma unroll
     for (int o = 1; o < FB; o <<= 1) {
@@ -282,7 +330,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
       const float m2 = __shfl_xor_sync(0xffffffffu, run_max, 16), s2 = __shfl_xor_sync(0xffffffffu, run_sum, 16);
       lse_merge(run_max, run_sum, m2, s2);
     }
-    if (fin_lane && sub == 0 && grp == 0) {
+    if (NW == 1 && fin_lane && sub == 0 && grp == 0) {
       wred[(warp * GP + my_g) * 2 + 0] = run_max;
       wred[(warp * GP + my_g) * 2 + 1] = run_sum;
     }
@@ -340,12 +388,12 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
     float* scores_u = p.scores + (size_t)u * p.max_blocks;
     uint32_t mn = 0xffffffffu, mx = 0u;
     int nf = 0;
-    for (int li = tid; li < n_my; li += kCsThreads) {
+    for (int li = tid; li < nb_my; li += kCsThreads) {
       float sc = 0.f;
 #pragma unroll
       for (int g = 0; g < GP; ++g)
         if (g < G) sc += __expf(ell_s[g * chunk + li] - lse_r[g]);
-      const int i = rec_begin + li;
+      const int i = blk_begin + li;
       scores_u[i] = sc;
       const bool forced = (i < p.n_sink) || (i >= nblk - p.n_local);
       const uint32_t key = forced ? 0xffffffffu : __float_as_uint(sc);
@@ -372,7 +420,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
 
   // this CTA's best min(k_eff, n_my) blocks go to the leader's candidate table
   {
-    const int cnt = select_topk(keys, n_my, k_eff, [&](int li) { return rec_begin + li; }, push, scratch);
+    const int cnt = select_topk(keys, nb_my, k_eff, [&](int li) { return blk_begin + li; }, push, scratch);
     if (tid == 0) st_dsmem_u32(map_to_rank(smem_u32(smem_raw + SM::kCandCnt), 0u) + (uint32_t)rank * 4, (uint32_t)cnt);
   }
   SPLA_MARK(p, u, rank, 5);
@@ -465,7 +513,7 @@ static cudaError_t launch_d(const Params& p, int GP, const void* q, int qb, int*
 
 // Decides whether the cluster kernel can serve a launch and with which cluster size / records per CTA.
 // Returns false when the general kernel has to be used (very long sequences, groups above 8).
-bool plan_score_cluster(int units, long long max_seq_blocks, int G, int d, int sm_count, int* cs_out, int* chunk_out) {
+bool plan_score_cluster(int units, long long max_seq_blocks, int NW, int G, int d, int sm_count, int* cs_out, int* chunk_out) {
   if (G > 8) return false;
   if (max_seq_blocks < 1) max_seq_blocks = 1;
   int cs = 1;

@@ -76,8 +76,10 @@ __global__ void __launch_bounds__(kScoreThreads, 2) score_select_kernel(const Pa
   // ------------------------------------------------------------------ score role ----------------------
   const int L = p.seq_lens[b];
   const int nblk = (L + p.B - 1) / p.B;
-  const int chunk = p.chunk;
-  const int n_chunks = max(1, (nblk + chunk - 1) / chunk);
+  const int NW = p.NW;                              // selection windows per block; a "record" is one window
+  const int nrec = nblk * NW;
+  const int chunk = p.chunk;                        // records per CTA
+  const int n_chunks = max(1, (nrec + chunk - 1) / chunk);
   if (c >= n_chunks) return;
   SPLA_MARK(p, u, c, 0);
 
@@ -101,8 +103,9 @@ __global__ void __launch_bounds__(kScoreThreads, 2) score_select_kernel(const Pa
     }
   }
 
-  const float* stats_u = p.stats + (size_t)u * p.max_blocks * 2 * D;
-  float* ell_u = p.ell + (size_t)u * G * p.max_blocks;
+  const size_t ell_stride = (size_t)p.max_blocks * NW;
+  const float* stats_u = p.stats + (size_t)u * ell_stride * 2 * D;
+  float* ell_u = p.ell + (size_t)u * G * ell_stride;
   // After the warp reduction lanes 0..15 hold the mean dots and lanes 16..31 the variance dots, value index
   // lane / LPV, each replicated on LPV lanes.  Copy lane `sub` finalises record `sub` of the batch, so the
   // log / exp work of FB records runs side by side instead of one record at a time.
@@ -110,7 +113,9 @@ __global__ void __launch_bounds__(kScoreThreads, 2) score_select_kernel(const Pa
   const int sub = lane % LPV;
   const bool fin_lane = lane < 16 && sub < FB && my_g < G;
   const float ln_full = logf((float)p.B);
-  const float ln_last = logf((float)max(1, L - (nblk - 1) * p.B));
+  const int n_last = L - (nblk - 1) * p.B;          // tokens of the last block
+  const float ln_last = logf((float)max(1, n_last));
+  const float ln_win = logf((float)p.win_C);
   float run_max = -INFINITY, run_sum = 0.f;
 
   const int rounds = chunk / kRound;
@@ -121,12 +126,12 @@ __global__ void __launch_bounds__(kScoreThreads, 2) score_select_kernel(const Pa
 #pragma unroll
     for (int r = 0; r < UNR; ++r) {
       const int i = base + round * kRound + r;
-      load_record<VEC>(stats_u + (size_t)i * 2 * D, D, lane, i < nblk, mean[buf][r], var[buf][r]);
+      load_record<VEC>(stats_u + (size_t)i * 2 * D, D, lane, i < nrec, mean[buf][r], var[buf][r]);
     }
   };
   auto compute_round = [&](int round, int buf) {
     const int i0 = base + round * kRound;
-    if (i0 >= nblk) return;                                // warp-uniform
+    if (i0 >= nrec) return;                                // warp-uniform
 #pragma unroll
     for (int r0 = 0; r0 < UNR; r0 += FB) {
       float dm_keep = 0.f, dv_keep = 0.f;
@@ -150,12 +155,24 @@ __global__ void __launch_bounds__(kScoreThreads, 2) score_select_kernel(const Pa
         if (sub == rr) { dm_keep = vals[0]; dv_keep = other; }
       }
       const int i = i0 + r0 + sub;
-      if (fin_lane && i < nblk) {
-        const float ell = (i == nblk - 1 ? ln_last : ln_full) + dm_keep + __logf(1.f + dv_keep);
-        ell_u[(size_t)my_g * p.max_blocks + i] = ell;
-        const float nm = fmaxf(run_max, ell);
-        run_sum = run_sum * __expf(run_max - nm) + __expf(ell - nm);
-        run_max = nm;
+      if (fin_lane && i < nrec) {
+        if (NW == 1) {
+          const float ell = (i == nblk - 1 ? ln_last : ln_full) + dm_keep + __logf(1.f + dv_keep);
+          ell_u[(size_t)my_g * ell_stride + i] = ell;
+          const float nm = fmaxf(run_max, ell);
+          run_sum = run_sum * __expf(run_max - nm) + __expf(ell - nm);
+          run_max = nm;
+        } else {
+          // strided windows (Section 3.1, "Strided Block Selection"): the log mass of window w of block blk; the
+          // pooling over a block's windows and the normalisers are left to the selecting CTA
+          const int blk = i / NW, w = i - blk * NW;
+          float ln_n = ln_win;
+          if (blk == nblk - 1) {
+            const int cnt = min(p.win_C, n_last - w * p.win_s);
+            ln_n = cnt > 0 ? logf((float)cnt) : -INFINITY;
+          }
+          ell_u[(size_t)my_g * ell_stride + i] = ln_n + dm_keep + __logf(1.f + dv_keep);
+        }
       }
     }
   };
@@ -223,12 +240,49 @@ __global__ void __launch_bounds__(kScoreThreads, 2) score_select_kernel(const Pa
     for (int j = 0; j < SB; ++j) {
       const int i = i0 + j * kScoreThreads + tid;
 #pragma unroll
-      for (int g = 0; g < GP; ++g) e[j][g] = (g < G && i < nblk) ? __ldcg(ell_u + (size_t)g * p.max_blocks + i) : -INFINITY;
+      for (int g = 0; g < GP; ++g) {
+        float x = -INFINITY;
+        if (g < G && i < nblk)
+          for (int w = 0; w < NW; ++w) x = fmaxf(x, __ldcg(ell_u + (size_t)g * ell_stride + (size_t)i * NW + w));   // max-pool
+        e[j][g] = x;
+      }
     }
   };
   load_batch(0);
 
-  for (int g = warp; g < G; g += NWARP) {
+  if (NW > 1) {
+    // windows: the normalisers are those of the pooled log masses, which only exist here
+    float* wred2 = reinterpret_cast<float*>(smem_raw);                // [NWARP][GP][2]; the keys are written later
+    float m[GP], sm[GP];
+#pragma unroll
+    for (int g = 0; g < GP; ++g) { m[g] = -INFINITY; sm[g] = 0.f; }
+    for (int i0 = 0; i0 < nblk; i0 += kScoreThreads * SB) {
+      if (i0 > 0) load_batch(i0);
+#pragma unroll
+      for (int j = 0; j < SB; ++j)
+#pragma unroll
+        for (int g = 0; g < GP; ++g) lse_merge(m[g], sm[g], e[j][g], e[j][g] > -INFINITY ? 1.f : 0.f);
+    }
+#pragma unroll
+    for (int g = 0; g < GP; ++g) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float m2 = __shfl_xor_sync(0xffffffffu, m[g], o), s2 = __shfl_xor_sync(0xffffffffu, sm[g], o);
+        lse_merge(m[g], sm[g], m2, s2);
+      }
+      if (lane == 0) { wred2[(warp * GP + g) * 2] = m[g]; wred2[(warp * GP + g) * 2 + 1] = sm[g]; }
+    }
+    __syncthreads();
+    if (tid < G) {
+      float mm = -INFINITY, ss = 0.f;
+#pragma unroll
+      for (int w = 0; w < NWARP; ++w) lse_merge(mm, ss, wred2[(w * GP + tid) * 2], wred2[(w * GP + tid) * 2 + 1]);
+      lse_s[tid] = mm + __logf(ss);
+    }
+    __syncthreads();
+    load_batch(0);
+  }
+  for (int g = warp; g < G && NW == 1; g += NWARP) {
     float m = -INFINITY, s = 0.f;
 #pragma unroll 4
     for (int cc = lane; cc < n_chunks; cc += 32) {

@@ -56,6 +56,7 @@ extern "C" int spla_select_blocks_noalloc(const spla_config_t* cfg, const float*
   spla_sizes_t sz;
   const int rc = spla_query_sizes(cfg, &sz);                 // validates the configuration (host only)
   if (rc != SPLA_OK) return rc;
+  if (cfg->window_size != 0) return SPLA_ERR_UNSUPPORTED;   // whole-block statistics only
   if (((uintptr_t)stats % 16) || ((uintptr_t)q % 16) || ((uintptr_t)seq_lens % 4) || ((uintptr_t)sel_idx % 4))
     return SPLA_ERR_INVALID_ARG;
 
@@ -86,6 +87,7 @@ extern "C" int spla_select_blocks_noalloc(const spla_config_t* cfg, const float*
   p.d = cfg->head_dim; p.B = cfg->block_size; p.top_k = cfg->top_k;
   p.max_context = cfg->max_context; p.max_blocks = (int)max_blocks; p.max_chunks = (int)max_chunks;
   p.n_sink = cfg->n_sink_blocks; p.n_local = cfg->n_local_blocks;
+  p.NW = 1; p.win_C = cfg->block_size; p.win_s = cfg->block_size;
   p.flags = (cfg->flags & SPLA_FIRST_ORDER) | SPLA_NO_RLA;      // score + select only: no o_bar CTAs
   p.kv_bf16 = cfg->kv_dtype == SPLA_BF16;
   p.sm_scale = cfg->sm_scale == 0.f ? 1.0f / sqrtf((float)cfg->head_dim) : cfg->sm_scale;

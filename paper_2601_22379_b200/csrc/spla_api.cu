@@ -54,6 +54,11 @@ static bool make_kv_map(void* out128, void* base, int d, int B, unsigned long lo
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Selection windows per block: the strided windows that lie entirely inside a block (1 without windows).
+static int windows_per_block(const spla_config_t* c) {
+  return c->window_size > 0 ? (c->block_size - c->window_size) / c->window_stride + 1 : 1;
+}
+
 static int validate_config(const spla_config_t* c) {
   if (!c) return SPLA_ERR_INVALID_ARG;
   if (c->batch < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->top_k < 1 || c->max_context < 1)
@@ -74,6 +79,10 @@ static int validate_config(const spla_config_t* c) {
   const int64_t max_blocks = ((int64_t)c->max_context + c->block_size - 1) / c->block_size;
   if (max_blocks > kMaxBlocks) return SPLA_ERR_UNSUPPORTED;
   if ((int64_t)c->batch * c->n_kv_heads > 65535) return SPLA_ERR_UNSUPPORTED;
+  if (c->window_size < 0 || c->window_stride < 0 || (c->window_size == 0) != (c->window_stride == 0))
+    return SPLA_ERR_INVALID_ARG;
+  if (c->window_size > c->block_size) return SPLA_ERR_INVALID_ARG;
+  if (windows_per_block(c) > kMaxWindows) return SPLA_ERR_UNSUPPORTED;
   return SPLA_OK;
 }
 
@@ -86,10 +95,11 @@ static WorkspaceLayout workspace_layout(const spla_config_t* c) {
   WorkspaceLayout w;
   const size_t U = (size_t)c->batch * c->n_kv_heads, G = c->n_q_heads / c->n_kv_heads, d = c->head_dim;
   const size_t max_blocks = ((size_t)c->max_context + c->block_size - 1) / c->block_size;
-  w.max_chunks = (int)((max_blocks + kScoreChunkMin - 1) / kScoreChunkMin);
+  const size_t NW = windows_per_block(c);
+  w.max_chunks = (int)((max_blocks * NW + kScoreChunkMin - 1) / kScoreChunkMin);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-  w.ell = take(U * G * max_blocks * 4);
+  w.ell = take(U * G * max_blocks * NW * 4);
   w.chunk_part = take(U * w.max_chunks * G * 2 * 4);
   w.scores = take(U * max_blocks * 4);
   w.obar_part = take(U * kStateSplits * G * d * 4);
@@ -114,7 +124,7 @@ extern "C" int spla_query_sizes(const spla_config_t* config, spla_sizes_t* sizes
   const size_t e = config->kv_dtype == SPLA_BF16 ? 2 : 4;
   sizes_out->k_cache = U * max_blocks * B * d * e;
   sizes_out->v_cache = sizes_out->k_cache;
-  sizes_out->stats = U * max_blocks * 2 * d * 4;
+  sizes_out->stats = U * max_blocks * windows_per_block(config) * 2 * d * 4;
   sizes_out->rla_state = U * d * d * 4;
   sizes_out->tok_lse = U * max_blocks * B * 4;
   sizes_out->seq_lens = (size_t)config->batch * 4;
@@ -162,6 +172,9 @@ extern "C" int spla_init_cache(const spla_config_t* config, const spla_buffers_t
   p.max_context = config->max_context;
   p.max_blocks = (config->max_context + config->block_size - 1) / config->block_size;
   p.n_sink = config->n_sink_blocks; p.n_local = config->n_local_blocks;
+  p.NW = windows_per_block(config);
+  p.win_C = config->window_size > 0 ? config->window_size : config->block_size;
+  p.win_s = config->window_size > 0 ? config->window_stride : config->block_size;
   p.flags = config->flags; p.kv_bf16 = config->kv_dtype == SPLA_BF16;
   p.sm_scale = c->cfg.sm_scale; p.phi_scale = c->cfg.phi_scale; p.rms_eps = c->cfg.rms_eps;
   p.k_cache = b->k_cache; p.v_cache = b->v_cache; p.stats = b->stats; p.state = b->rla_state;
@@ -228,14 +241,14 @@ static void plan_score_grid(const spla_cache* c, Params* p) {
   if (blocks < 1) blocks = 1;
   p->cs = 0;
   int cs = 0, chunk = 0;
-  if (!(c->cfg.flags & SPLA_GENERAL_KERNELS) && plan_score_cluster(p->batch * p->Hkv, blocks, p->G, p->d, c->sm_count, &cs, &chunk)) {
+  if (!(c->cfg.flags & SPLA_GENERAL_KERNELS) && plan_score_cluster(p->batch * p->Hkv, blocks, p->NW, p->G, p->d, c->sm_count, &cs, &chunk)) {
     p->cs = cs;
     p->chunk = chunk;
     p->n_chunks_cap = cs;
     return;
   }
-  p->chunk = score_chunk_for((long long)p->batch * p->Hkv, blocks, c->sm_count);
-  p->n_chunks_cap = (int)((blocks + p->chunk - 1) / p->chunk);
+  p->chunk = score_chunk_for((long long)p->batch * p->Hkv, blocks * p->NW, c->sm_count);   // in records (windows)
+  p->n_chunks_cap = (int)((blocks * p->NW + p->chunk - 1) / p->chunk);
 }
 
 static cudaError_t launch_score(const Params& p, const void* q, int qb, int* sel_user, cudaStream_t s) {

@@ -14,6 +14,7 @@ constexpr int kScoreChunkMax = 512;
 constexpr int kStateSplits = 4;         // CTAs per unit that compute o_bar = phi(q) S_bar
 constexpr int kAttendThreads = 128;     // sparse-attend kernel: 4 warps per selected block
 constexpr int kMaxGroup = 16;
+constexpr int kMaxWindows = 8;          // selection windows per block, at most
 constexpr int kMaxTopK = 64;
 constexpr int kMaxBlocks = 32768;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -25,6 +26,7 @@ struct Params {
   unsigned flags;
   int kv_bf16;                          // K/V cache element type: 1 = bf16, 0 = fp32
   float sm_scale, phi_scale, rms_eps;
+  int NW, win_C, win_s;                 // selection windows per block, their size and stride (1, B, B: whole blocks)
   int n_chunks_cap;                     // score-kernel chunks launched per unit
   int chunk;                            // block records per score CTA
   int cs;                               // score kernel, cluster edition: CTAs per unit (0 = general kernel)

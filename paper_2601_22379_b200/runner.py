@@ -10,13 +10,15 @@ import torch
 from . import binding, synth
 
 
-def config_for(w: synth.Workload, *, flags: int = 0, n_sink=None, n_local=None, extra_context: int = 0):
+def config_for(w: synth.Workload, *, flags: int = 0, n_sink=None, n_local=None, extra_context: int = 0,
+               window=None):
     return binding.make_config(
         batch=w.batch, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, head_dim=w.head_dim,
         block_size=w.block_size, top_k=w.top_k, max_context=w.max_context + extra_context,
         n_sink_blocks=w.n_sink if n_sink is None else n_sink,
         n_local_blocks=w.n_local if n_local is None else n_local,
-        kv_dtype=w.kv_dtype, flags=flags)
+        kv_dtype=w.kv_dtype, flags=flags, window_size=window[0] if window else 0,
+        window_stride=window[1] if window else 0)
 
 
 def generate_prefill(w: synth.Workload, device):
@@ -34,13 +36,13 @@ def generate_prefill(w: synth.Workload, device):
 
 
 def build_cache(w: synth.Workload, device="cuda:0", *, flags: int = 0, n_sink=None, n_local=None, chunk: int = 0,
-                prefill=None):
+                prefill=None, window=None):
     """Creates a cache for `w` and appends the whole prefilled context (optionally in `chunk`-token calls).
 
-    Returns (cache, K, V, lens) with K, V the generated inputs (kept so that a checker can hand the same bits
+    `window` = (C, s) turns on strided selection windows.  Returns (cache, K, V, lens) with K, V the generated inputs (kept so that a checker can hand the same bits
     to another implementation).
     """
-    cache = binding.SplaCache(config_for(w, flags=flags, n_sink=n_sink, n_local=n_local), device)
+    cache = binding.SplaCache(config_for(w, flags=flags, n_sink=n_sink, n_local=n_local, window=window), device)
     K, V, lens = prefill if prefill is not None else generate_prefill(w, device)
     Lmax = K.shape[2]
     ragged = bool((lens != Lmax).any().item())

@@ -193,11 +193,12 @@ def step_kv(w: Workload, step: int, device="cpu"):
     return k.to(w.torch_dtype).to(device), v.to(w.torch_dtype).to(device)
 
 
-def algorithmic_bytes_per_step(w: Workload, lens=None) -> dict:
+def algorithmic_bytes_per_step(w: Workload, lens=None, n_windows: int = 1) -> dict:
     """Bytes one decode step must move, per the method's own accounting.
 
     Block statistics of every block + K and V of the selected blocks + the
     global RLA state, summed over units; next to the dense-decode KV footprint.
+    With strided selection windows every block carries `n_windows` statistics records.
     """
     lens = seq_lens(w) if lens is None else np.asarray(lens)
     e = 2 if w.kv_dtype == "bf16" else 4
@@ -205,7 +206,7 @@ def algorithmic_bytes_per_step(w: Workload, lens=None) -> dict:
     stats = sel = state = dense = 0
     for L in lens:
         nblk = -(-int(L) // B)
-        stats += H * nblk * 2 * d * 4
+        stats += H * nblk * n_windows * 2 * d * 4
         sel += H * min(w.top_k, nblk) * B * d * 2 * e
         state += H * d * d * 4
         dense += H * int(L) * d * 2 * e

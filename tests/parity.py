@@ -67,12 +67,13 @@ def check_outputs(name, got, want, kv_dtype, scale_floor=0.0):
     return ma, rl
 
 
-def oracle_unit(w, q_bhd, K_unit, V_unit, gamma, h, *, n_sink, n_local, override=None, order=2, use_rla=True):
+def oracle_unit(w, q_bhd, K_unit, V_unit, gamma, h, *, n_sink, n_local, override=None, order=2, use_rla=True,
+                window=None):
     G = w.group
     return O.decode_unit(
         q_bhd[h * G:(h + 1) * G].double().cpu().numpy(), K_unit.double().cpu().numpy(), V_unit.double().cpu().numpy(),
         gamma[h * G:(h + 1) * G].double().cpu().numpy(), block_size=w.block_size, top_k=w.top_k, n_sink=n_sink,
-        n_local=n_local, override_selection=override, order=order, use_rla=use_rla)
+        n_local=n_local, override_selection=override, order=order, use_rla=use_rla, window=window)
 
 
 def compare_unit(w, res, out_gpu, osp_gpu, orla_gpu, sel_gpu, h, *, n_sink, n_local, rerun=None):

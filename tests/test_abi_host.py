@@ -46,6 +46,11 @@ def test_query_sizes_follow_the_documented_layouts(lib):
     f32 = binding.make_config(batch=1, n_q_heads=1, n_kv_heads=1, head_dim=64, block_size=64, top_k=8,
                               max_context=4112, kv_dtype="f32")
     assert binding.query_sizes(f32).k_cache == 65 * 64 * 64 * 4
+    # strided windows C = 32, s = 16 inside blocks of 64: three statistics records per block
+    win = binding.make_config(batch=4, n_q_heads=32, n_kv_heads=8, head_dim=128, block_size=64, top_k=32,
+                              max_context=131072 + 64, window_size=32, window_stride=16)
+    assert win.n_windows == 3 and binding.query_sizes(win).stats == 3 * sz.stats
+    assert binding.query_sizes(win).k_cache == sz.k_cache
 
 
 @pytest.mark.parametrize("kw,status", [
@@ -60,6 +65,11 @@ def test_query_sizes_follow_the_documented_layouts(lib):
     (dict(top_k=65, n_sink_blocks=0, n_local_blocks=0), binding.SPLA_ERR_UNSUPPORTED),
     (dict(n_q_heads=8 * 17), binding.SPLA_ERR_UNSUPPORTED),
     (dict(max_context=64 * 32768 + 1), binding.SPLA_ERR_UNSUPPORTED),
+    (dict(window_size=32), binding.SPLA_ERR_INVALID_ARG),                      # a window needs a stride
+    (dict(window_stride=16), binding.SPLA_ERR_INVALID_ARG),
+    (dict(window_size=128, window_stride=16), binding.SPLA_ERR_INVALID_ARG),   # wider than the block
+    (dict(window_size=-1, window_stride=16), binding.SPLA_ERR_INVALID_ARG),
+    (dict(window_size=8, window_stride=4), binding.SPLA_ERR_UNSUPPORTED),      # 15 windows per block: above 8
 ])
 def test_bad_configurations_are_rejected_on_the_host(lib, kw, status):
     base = dict(batch=2, n_q_heads=32, n_kv_heads=8, head_dim=128, block_size=64, top_k=32, max_context=4096)

@@ -22,7 +22,8 @@ def _decode_all(cache, w, q, gamma):
     return out.cpu().numpy(), osp.cpu().numpy(), orla.cpu().numpy(), sel.cpu().numpy()
 
 
-def _check_units(w, cache, q, gamma, K, V, lens, units, n_sink, n_local, extra=None, order=2, use_rla=True):
+def _check_units(w, cache, q, gamma, K, V, lens, units, n_sink, n_local, extra=None, order=2, use_rla=True,
+                 window=None):
     """extra: optional dict (b,h) -> (K_tail, V_tail) of appended tokens."""
     out, osp, orla, sel = _decode_all(cache, w, q, gamma)
     n_exact = 0
@@ -35,7 +36,7 @@ def _check_units(w, cache, q, gamma, K, V, lens, units, n_sink, n_local, extra=N
 
         def run(override=None):
             return parity.oracle_unit(w, q[b], Ku, Vu, gamma, h, n_sink=n_sink, n_local=n_local, override=override,
-                                      order=order, use_rla=use_rla)
+                                      order=order, use_rla=use_rla, window=window)
         res = run()
         n_exact += parity.compare_unit(w, res, out[b], osp[b], orla[b], sel[b, h], h, n_sink=n_sink, n_local=n_local,
                                        rerun=run)
@@ -195,8 +196,8 @@ def test_config2_gqa_32k_full_three_query_seeds():
                 assert set(nb[b, h].tolist()) <= set(sel[b, h].tolist())
 
 
-def _stepped_full(w, n_units, check_steps):
-    cache, K, V, lens = runner.build_cache(w, DEV)
+def _stepped_full(w, n_units, check_steps, window=None):
+    cache, K, V, lens = runner.build_cache(w, DEV, window=window)
     gamma = synth.gamma(w).to(DEV)
     gam = gamma.double().cpu().numpy()
     lens_h = lens.cpu().numpy()
@@ -206,7 +207,7 @@ def _stepped_full(w, n_units, check_steps):
     for (b, h) in units:
         L = int(lens_h[b])
         orc[(b, h)] = O.UnitCache.from_prefill(K[b, h, :L].double().cpu().numpy(), V[b, h, :L].double().cpu().numpy(),
-                                               w.block_size)
+                                               w.block_size, window=window)
     del K, V
     for step in range(w.n_steps):
         k1, v1 = synth.step_kv(w, step, DEV)
