@@ -17,6 +17,7 @@ namespace spla {
 constexpr int kCopyThreads = 256;
 constexpr int kStateRows = 16;     // rows of S_bar per CTA
 constexpr int kStateTokens = 32;   // tokens staged per inner step
+constexpr int kStateUmmaMinTokens = 256;   // appends at least this long take the tensor-core state kernel
 
 __device__ __forceinline__ int tokens_to_add(const Params& p, const int* n_new, int max_new, int b, int L) {
   int n = n_new ? n_new[b] : max_new;
@@ -323,7 +324,7 @@ __global__ void __launch_bounds__(kFusedThreads) append_fused_kernel(const Param
 
 template <typename T, int D>
 static cudaError_t launch_typed(const Params& p, const void* k_new, const void* v_new, const int* n_new, int max_new,
-                                cudaStream_t stream) {
+                                const AttendMaps* state_maps, cudaStream_t stream) {
   const int U = p.batch * p.Hkv;
   const T* kn = reinterpret_cast<const T*>(k_new);
   const T* vn = reinterpret_cast<const T*>(v_new);
@@ -339,19 +340,27 @@ static cudaError_t launch_typed(const Params& p, const void* k_new, const void* 
   const int per_cta = kCopyThreads / 32;
   append_copy_kernel<T, D><<<dim3((max_new + per_cta - 1) / per_cta, U), kCopyThreads, 0, stream>>>(p, kn, vn, n_new, max_new);
   append_stats_kernel<T, D><<<dim3(((max_new + p.B - 1) / p.B + 1) * p.NW, U), kStatThreads, 0, stream>>>(p, n_new, max_new);
-  if (!(p.flags & 4u))
-    append_state_kernel<T, D><<<dim3(D / kStateRows, U), D, 0, stream>>>(p, kn, vn, n_new, max_new);
+  if (!(p.flags & 4u)) {
+    // long appends of a bf16 cache with d = 128: the rank-n update is a dense contraction, done on the tensor cores
+    // from the tokens the copy kernel has just stored; everything else on the FMA pipe
+    if (sizeof(T) == 2 && D == 128 && state_maps && state_maps->valid && max_new >= kStateUmmaMinTokens) {
+      const cudaError_t e = launch_state_umma(p, state_maps, n_new, max_new, stream);
+      if (e != cudaSuccess) return e;
+    } else {
+      append_state_kernel<T, D><<<dim3(D / kStateRows, U), D, 0, stream>>>(p, kn, vn, n_new, max_new);
+    }
+  }
   append_lengths_kernel<<<(p.batch + 127) / 128, 128, 0, stream>>>(p, n_new, max_new);
   return cudaGetLastError();
 }
 
 cudaError_t launch_append(const Params& p, const void* k_new, const void* v_new, const int* n_new, int max_new,
-                          cudaStream_t stream) {
+                          const AttendMaps* state_maps, cudaStream_t stream) {
   if (p.kv_bf16)
-    return p.d == 128 ? launch_typed<__nv_bfloat16, 128>(p, k_new, v_new, n_new, max_new, stream)
-                      : launch_typed<__nv_bfloat16, 64>(p, k_new, v_new, n_new, max_new, stream);
-  return p.d == 128 ? launch_typed<float, 128>(p, k_new, v_new, n_new, max_new, stream)
-                    : launch_typed<float, 64>(p, k_new, v_new, n_new, max_new, stream);
+    return p.d == 128 ? launch_typed<__nv_bfloat16, 128>(p, k_new, v_new, n_new, max_new, state_maps, stream)
+                      : launch_typed<__nv_bfloat16, 64>(p, k_new, v_new, n_new, max_new, state_maps, stream);
+  return p.d == 128 ? launch_typed<float, 128>(p, k_new, v_new, n_new, max_new, state_maps, stream)
+                    : launch_typed<float, 64>(p, k_new, v_new, n_new, max_new, state_maps, stream);
 }
 
 }  // namespace spla

@@ -21,6 +21,7 @@ struct spla_cache {
   bool have_ev;
   int sm_count;
   AttendMaps maps;
+  AttendMaps state_maps;   // the same caches in boxes of 64 tokens, for the tensor-core state kernel
 };
 
 static thread_local char g_cuda_err[256] = "";
@@ -87,7 +88,7 @@ static int validate_config(const spla_config_t* c) {
 }
 
 struct WorkspaceLayout {
-  size_t ell, chunk_part, scores, obar_part, sel, n_sel, att_acc, att_ml, score_ticket, attend_ticket, append_ticket, status, total;
+  size_t ell, chunk_part, scores, obar_part, sel, n_sel, att_acc, att_ml, score_ticket, attend_ticket, append_ticket, state_part, state_ticket, status, total;
   int max_chunks;
 };
 
@@ -110,6 +111,8 @@ static WorkspaceLayout workspace_layout(const spla_config_t* c) {
   w.score_ticket = take(U * 4);
   w.attend_ticket = take(U * 4);
   w.append_ticket = take(256);
+  w.state_part = take(state_umma_part_bytes((int)U, (int)d));
+  w.state_ticket = take(U * 4);
   w.status = take(256);
   w.total = off;
   return w;
@@ -186,6 +189,7 @@ extern "C" int spla_init_cache(const spla_config_t* config, const spla_buffers_t
   p.att_acc = (float*)(ws + w.att_acc); p.att_ml = (float*)(ws + w.att_ml);
   p.score_ticket = (int*)(ws + w.score_ticket); p.attend_ticket = (int*)(ws + w.attend_ticket);
   p.append_ticket = (int*)(ws + w.append_ticket);
+  p.state_part = (float*)(ws + w.state_part); p.state_ticket = (int*)(ws + w.state_ticket);
   p.status = (int*)(ws + w.status);
   p.max_chunks = w.max_chunks;
 #ifdef SPLA_TRACE
@@ -194,9 +198,13 @@ extern "C" int spla_init_cache(const spla_config_t* config, const spla_buffers_t
   p.acs = 0;
 
   c->maps.valid = false;
+  c->state_maps.valid = false;
   if (p.kv_bf16) {
     const unsigned long long rows = (unsigned long long)p.batch * p.Hkv * p.max_blocks * p.B;
     c->maps.valid = make_kv_map(c->maps.k, b->k_cache, p.d, p.B, rows) && make_kv_map(c->maps.v, b->v_cache, p.d, p.B, rows);
+    c->state_maps.valid = p.d == 128 && rows >= 64 && rows < (1ull << 31) && !(config->flags & SPLA_GENERAL_KERNELS) &&
+                          make_kv_map(c->state_maps.k, b->k_cache, p.d, 64, rows) &&
+                          make_kv_map(c->state_maps.v, b->v_cache, p.d, 64, rows);
   }
 
   cudaStream_t s = (cudaStream_t)stream;
@@ -229,7 +237,7 @@ extern "C" int spla_append_tokens(spla_cache_t* c, const void* k_new, const void
   if (!c || !k_new || !v_new || max_new < 1) return SPLA_ERR_INVALID_ARG;
   if (!aligned(k_new, 16) || !aligned(v_new, 16)) return SPLA_ERR_INVALID_ARG;
   if (c->len_bound + max_new > c->cfg.max_context) return SPLA_ERR_CAPACITY;
-  cudaError_t e = launch_append(c->p, k_new, v_new, n_new, max_new, (cudaStream_t)stream);
+  cudaError_t e = launch_append(c->p, k_new, v_new, n_new, max_new, &c->state_maps, (cudaStream_t)stream);
   if (e != cudaSuccess) return cuda_fail(e, "spla_append_tokens");
   c->len_bound += max_new;
   return SPLA_OK;

@@ -50,6 +50,8 @@ struct Params {
   int* score_ticket;   // [U]
   int* attend_ticket;  // [U]
   int* append_ticket;  // [1]
+  float* state_part;   // [U][splits][d][d]  partial S_bar updates of the tensor-core state kernel
+  int* state_ticket;   // [U]
   int* status;         // [1]
   int max_chunks;
 #ifdef SPLA_TRACE

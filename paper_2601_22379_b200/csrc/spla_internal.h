@@ -54,6 +54,10 @@ struct AttendMaps {                      // TMA tensor maps (CUtensorMap) of the
   alignas(64) unsigned char v[128];
   bool valid;
 };
+// state_umma.cu (bulk S_bar update on tcgen05 tensor cores: bf16 cache, d = 128; maps with boxes of 64 tokens)
+int state_umma_splits(int units);
+size_t state_umma_part_bytes(int units, int d);
+cudaError_t launch_state_umma(const Params& p, const AttendMaps* maps, const int* n_new, int max_new, cudaStream_t stream);
 // attend_merge.cu
 cudaError_t launch_attend_merge(const Params& p, const AttendMaps* maps, const void* q, int q_is_bf16,
                                 const float* rms_weight, const int* sel_in, float* out, float* dbg_o_sparse,
@@ -63,7 +67,9 @@ size_t attend_mma_smem_bytes(int B, int D);
 cudaError_t launch_attend_mma(const Params& p, const AttendMaps& maps, const void* q, const float* rms_weight, float* out,
                               float* dbg_o_sparse, float* dbg_o_rla, cudaStream_t stream);
 // append.cu
+// `state_maps` (may be null): tensor maps with boxes of 64 tokens; when given, bulk appends of a bf16 cache with
+// d = 128 update S_bar on the tensor cores instead of the FMA kernel.
 cudaError_t launch_append(const Params& p, const void* k_new, const void* v_new, const int* n_new, int max_new,
-                          cudaStream_t stream);
+                          const AttendMaps* state_maps, cudaStream_t stream);
 
 }  // namespace spla

@@ -65,7 +65,8 @@ def test_append_statistics_and_state_match_oracle(name, ctx):
             st = cache.bufs.stats[b, h, :nblk].cpu().numpy()
             assert parity.rel_l2(st[:, 0], mean) < 2e-6 and parity.rel_l2(st[:, 1], var) < 2e-6
             S = cache.bufs.rla_state[b, h].cpu().numpy()
-            assert parity.rel_l2(S, O.rla_global_state(Kd, Vd)) < 2e-6
+            tensor_path = w.kv_dtype == "bf16" and w.head_dim == 128 and ctx >= 256
+            assert parity.rel_l2(S, O.rla_global_state(Kd, Vd)) < (parity.STATE_TOL_TENSOR if tensor_path else parity.STATE_TOL_FMA)
             lse = cache.bufs.tok_lse[b, h, :ctx].cpu().numpy()
             ref = np.log(np.sum(np.exp(Kd - Kd.max(axis=1, keepdims=True)), axis=1)) + Kd.max(axis=1)
             assert np.max(np.abs(lse - ref)) < 2e-5
@@ -76,7 +77,7 @@ def test_append_statistics_and_state_match_oracle(name, ctx):
     torch.cuda.synchronize()
     assert torch.equal(cache2.bufs.stats[:, :, :nblk], cache.bufs.stats[:, :, :nblk])
     assert torch.equal(cache2.bufs.tok_lse[:, :, :ctx], cache.bufs.tok_lse[:, :, :ctx])
-    assert parity.rel_l2(cache2.bufs.rla_state.cpu().numpy(), cache.bufs.rla_state.cpu().numpy()) < 2e-6
+    assert parity.rel_l2(cache2.bufs.rla_state.cpu().numpy(), cache.bufs.rla_state.cpu().numpy()) < parity.STATE_TOL_TENSOR
     # ... and so does the fused decode-step kernel (one, three and seventeen tokens per call)
     cache3 = binding.SplaCache(runner.config_for(w), DEV)
     pos, sizes = 0, [1, 3, 17, 1, 1, 32, 5]
@@ -91,7 +92,7 @@ def test_append_statistics_and_state_match_oracle(name, ctx):
     assert torch.equal(cache3.bufs.stats[:, :, :nblk], cache.bufs.stats[:, :, :nblk])
     assert torch.equal(cache3.bufs.tok_lse[:, :, :ctx], cache.bufs.tok_lse[:, :, :ctx])
     assert torch.equal(cache3.bufs.k_cache.reshape(2, w.n_kv_heads, -1, w.head_dim)[:, :, :ctx], K)
-    assert parity.rel_l2(cache3.bufs.rla_state.cpu().numpy(), cache.bufs.rla_state.cpu().numpy()) < 2e-6
+    assert parity.rel_l2(cache3.bufs.rla_state.cpu().numpy(), cache.bufs.rla_state.cpu().numpy()) < parity.STATE_TOL_TENSOR
 
 
 def test_ragged_append_with_device_lengths():
@@ -420,3 +421,38 @@ def test_capacity_overflow_is_reported_not_faulted():
     assert cache.sync_status() == binding.SPLA_ERR_CAPACITY
     assert cache.sync_status() == 0
     assert cache.bufs.seq_lens.cpu().tolist() == [259, 259] and torch.equal(before, cache.bufs.rla_state)
+
+
+# ---------------------------------------------------------------------------------------------------------
+# bulk state update on the tensor cores (bf16 cache, d = 128, appends of at least 256 tokens)
+# ---------------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name,over,chunk", [
+    ("gqa_32k", dict(batch=2, context=64 * 40 + 37, n_needles=0), 0),                    # 16 splits, ragged last tile
+    ("ragged_serving", dict(batch=9, context=5000, context_min=1, n_steps=4), 0),        # device lengths, 2 splits
+    ("ragged_serving", dict(batch=24, context=1200, context_min=200, n_steps=4), 0),     # one split: adds to S_bar itself
+    ("long_128k", dict(batch=1, context=64 * 300 + 1, n_needles=0), 4096 + 333),         # several tensor-core appends in a row
+    ("very_long_1m", dict(context=128 * 100 + 77, n_needles=0), 0),                      # B = 128
+])
+def test_tensor_core_state_update_matches_oracle_and_fma_kernel(name, over, chunk):
+    w = synth.BY_NAME[name].scaled(**over)
+    cache, K, V, lens = runner.build_cache(w, DEV, chunk=chunk)
+    fma, _, _, _ = runner.build_cache(w, DEV, prefill=(K, V, lens), flags=binding.SPLA_GENERAL_KERNELS, chunk=chunk)
+    torch.cuda.synchronize()
+    assert cache.sync_status() == 0 and fma.sync_status() == 0
+    assert torch.equal(cache.bufs.seq_lens, lens)
+    lens_h = lens.cpu().numpy()
+    for b in range(w.batch):
+        L = int(lens_h[b])
+        for h in (0, w.n_kv_heads - 1):
+            S = O.rla_global_state(K[b, h, :L].double().cpu().numpy(), V[b, h, :L].double().cpu().numpy())
+            got = cache.bufs.rla_state[b, h].cpu().numpy()
+            if L == 0:
+                assert not got.any()
+                continue
+            tol = parity.STATE_TOL_TENSOR if L >= 64 else 1e-5      # a handful of tokens: few terms, same per-term error
+            assert parity.rel_l2(got, S) < tol, (b, h, L)
+            assert parity.rel_l2(got, fma.bufs.rla_state[b, h].cpu().numpy()) < 2 * parity.STATE_TOL_TENSOR
+    # same inputs, same launch configuration: the update is reproducible bit for bit (partials are added in split order)
+    again, _, _, _ = runner.build_cache(w, DEV, prefill=(K, V, lens), chunk=chunk)
+    torch.cuda.synchronize()
+    assert torch.equal(again.bufs.rla_state, cache.bufs.rla_state)
