@@ -10,7 +10,7 @@
 //
 // Per CTA (one unit, one split of the unit's new tokens), 10 warps:
 //   warp 0     : producer - tiled TMA loads of K and V tiles (64 tokens) into a 4-stage ring;
-//   warps 2..9 : transform - phi(k) = exp(phi_scale k - lse_t) in place (lse_t from the per-token table the copy
+//   warps 2..9 : transform (two groups of four warps, alternating tiles) - phi(k) = exp(phi_scale k - lse_t) in place (lse_t from the per-token table the copy
 //                kernel has just filled), split into a bf16 head (written over K) and a bf16 remainder (second
 //                buffer), so that the product carries 16 significant bits of phi; rows past the last new token
 //                are zeroed in all three tiles;
@@ -107,6 +107,19 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
+#ifdef SPLA_TRACE
+#define SU_MARK(i, k)                                                                       \
+  do {                                                                                      \
+    if (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && (i) < 32) {                        \
+      unsigned long long t_;                                                                \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                \
+      p.trace[(size_t)(i) * 8 + (k)] = t_;                                                  \
+    }                                                                                       \
+  } while (0)
+#else
+#define SU_MARK(i, k) do { } while (0)
+#endif
+
 }  // namespace
 
 __global__ void __launch_bounds__(kSuThreads, 1)
@@ -138,7 +151,7 @@ __global__ void __launch_bounds__(kSuThreads, 1)
   const size_t unit_tok0 = (size_t)u * p.max_blocks * p.B;
 
   if (tid == 0) {
-    for (int s = 0; s < kSuStages; ++s) { mbar_init(&full[s], 1); mbar_init(&ready[s], kSuTransformWarps); mbar_init(&empty[s], 1); }
+    for (int s = 0; s < kSuStages; ++s) { mbar_init(&full[s], 1); mbar_init(&ready[s], kSuTransformWarps / 2); mbar_init(&empty[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], kSuTransformWarps); }
     abort_s = 0;
   }
@@ -162,6 +175,7 @@ __global__ void __launch_bounds__(kSuThreads, 1)
           if (i >= kSuStages && !mbar_wait(&empty[s], ((i / kSuStages) - 1) & 1)) { atomicExch(&abort_s, 1); break; }
           const uint32_t base = smem_u32(smem_raw + (size_t)s * kSuStageBytes);
           const int row = (int)(unit_tok0 + (size_t)L + (size_t)(t_begin + i) * kSuTile);
+          SU_MARK(i, 0);
           mbar_expect_tx(&full[s], 2 * kSuTileBytes);
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
@@ -182,6 +196,7 @@ __global__ void __launch_bounds__(kSuThreads, 1)
           const bool first = i % kSuGroup == 0, last = i % kSuGroup == kSuGroup - 1 || i == my_tiles - 1;
           if (first && g >= 2 && !mbar_wait(&acc_empty[ab], ((g >> 1) - 1) & 1)) { atomicExch(&abort_s, 1); break; }
           if (!mbar_wait(&ready[s], (i / kSuStages) & 1)) { atomicExch(&abort_s, 1); break; }
+          SU_MARK(i, 3);
           tc_fence_after();
           const uint32_t base = smem_u32(smem_raw + (size_t)s * kSuStageBytes);
 #pragma unroll
@@ -191,16 +206,19 @@ __global__ void __launch_bounds__(kSuThreads, 1)
               umma_bf16(tmem + ab * kSuD, umma_desc(base + part * kSuTileBytes + kk * 2048),
                         umma_desc(base + 2 * kSuTileBytes + kk * 2048), (!first || part > 0 || kk > 0) ? 1u : 0u);
           umma_commit(&empty[s]);                        // the stage may be refilled once these have read it
+          SU_MARK(i, 4);
           if (last) umma_commit(&acc_full[ab]);          // and the group's sum may be drained
         }
       }
     } else {
       // ---------------------------------------------------------------- transform --------------------------------
-      // Thread tt owns 64 bytes (four 16-byte chunks) of row r of half h of every tile.  The swizzle moves chunks
-      // only inside their 128-byte row, and phi is elementwise given the token's log-sum-exp, so the channel a
-      // chunk holds does not matter here.
-      const int tt = tid - 64;
-      const int h = tt >> 7, r = (tt & 127) >> 1, c0 = (tt & 1) * 4;
+      // Two groups of four warps take the tiles in turn, so that one group's waits (tile landed, proxy fence, drain)
+      // overlap the other's arithmetic.  Thread tg of a group owns the 16-byte chunks tg, tg + 128, ... of a tile
+      // (consecutive lanes on consecutive chunks: no bank conflicts), which lie in the rows tg / 8 + 16 k of both
+      // halves.  The swizzle moves chunks only inside their 128-byte row, and phi is elementwise given the
+      // token's log-sum-exp, so which channels a chunk holds does not matter here.
+      const int wg = (warp - 2) >> 2, tg = (tid - 64) & 127;
+      const int r0 = tg >> 3;
       const float a2 = p.phi_scale * kLog2e;
       const float* lse = p.tok_lse + unit_tok0 + L;
       bool ok = true;
@@ -228,33 +246,49 @@ __global__ void __launch_bounds__(kSuThreads, 1)
         __syncwarp();
         if (lane == 0) mbar_arrive1(&acc_empty[ab]);
       };
-      for (int i = 0; i < my_tiles && !*abort_flag; ++i) {
-        const int s = i % kSuStages;
-        const int pos = (t_begin + i) * kSuTile + r;     // token index among the new ones
-        const bool valid = pos < n;
-        const float nl2 = valid ? -__ldg(lse + pos) * kLog2e : 0.f;
-        if (!mbar_wait(&full[s], (i / kSuStages) & 1)) { ok = false; break; }
-        unsigned char* st = smem_raw + (size_t)s * kSuStageBytes + h * kSuHalfBytes + r * 128;
+      // the tokens' log-sum-exps are fetched one tile ahead: a global load in the loop would be its critical path
+      float lse_next[4];
+      auto load_lse = [&](int i) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          uint4* kp = reinterpret_cast<uint4*>(st + (c0 + j) * 16);
-          uint4* lp = reinterpret_cast<uint4*>(st + kSuTileBytes + (c0 + j) * 16);
+        for (int k = 0; k < 4; ++k) {
+          const int pos = (t_begin + i) * kSuTile + r0 + 16 * k;
+          lse_next[k] = (i < my_tiles && pos < n) ? __ldg(lse + pos) : 0.f;
+        }
+      };
+      load_lse(wg);
+      for (int i = wg; i < my_tiles && !*abort_flag; i += 2) {
+        const int s = i % kSuStages;
+        float nl2[4];
+        bool valid[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          nl2[k] = -lse_next[k] * kLog2e;
+          valid[k] = (t_begin + i) * kSuTile + r0 + 16 * k < n;   // token index among the new ones
+        }
+        load_lse(i + 2);
+        if (!mbar_wait(&full[s], (i / kSuStages) & 1)) { ok = false; break; }
+        if (tg == 0) SU_MARK(i, 1);
+        unsigned char* st = smem_raw + (size_t)s * kSuStageBytes + tg * 16;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          uint4* kp = reinterpret_cast<uint4*>(st + j * 2048);
+          uint4* lp = reinterpret_cast<uint4*>(st + kSuTileBytes + j * 2048);
           uint4 hi4 = make_uint4(0u, 0u, 0u, 0u), lo4 = hi4;
-          if (valid) {
+          if (valid[j & 3]) {
             const uint4 raw = *kp;
             const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
             uint32_t ho[4], lo[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              const float f0 = ex2(fmaf(__uint_as_float(w[e] << 16), a2, nl2));
-              const float f1 = ex2(fmaf(__uint_as_float(w[e] & 0xffff0000u), a2, nl2));
+              const float f0 = ex2(fmaf(__uint_as_float(w[e] << 16), a2, nl2[j & 3]));
+              const float f1 = ex2(fmaf(__uint_as_float(w[e] & 0xffff0000u), a2, nl2[j & 3]));
               ho[e] = pack_bf16(f0, f1);
               lo[e] = pack_bf16(f0 - __uint_as_float(ho[e] << 16), f1 - __uint_as_float(ho[e] & 0xffff0000u));
             }
             hi4 = make_uint4(ho[0], ho[1], ho[2], ho[3]);
             lo4 = make_uint4(lo[0], lo[1], lo[2], lo[3]);
           } else {
-            *reinterpret_cast<uint4*>(st + 2 * kSuTileBytes + (c0 + j) * 16) = hi4;   // V of a row that is not a new token
+            *reinterpret_cast<uint4*>(st + 2 * kSuTileBytes + j * 2048) = hi4;   // V of a row that is not a new token
           }
           *kp = hi4;
           *lp = lo4;
@@ -262,8 +296,10 @@ __global__ void __launch_bounds__(kSuThreads, 1)
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the tensor core's reads
         __syncwarp();
         if (lane == 0) mbar_arrive1(&ready[s]);
-        // one group behind the issuer: by now the previous group's instructions have long completed
-        if (i % kSuGroup == kSuGroup - 1 && i / kSuGroup >= 1 && ok) { drain(drained); ++drained; }
+        if (tg == 0) SU_MARK(i, 2);
+        // one accumulator group behind the issuer: by now those instructions have long completed
+        while (ok && drained < i / kSuGroup) { drain(drained); ++drained; }
+        if (tg == 0) SU_MARK(i, 5);
         if (!ok) break;
       }
       while (ok && !*abort_flag && drained < n_groups) { drain(drained); ++drained; }
