@@ -73,14 +73,14 @@ __global__ void __launch_bounds__(kCopyThreads) append_copy_kernel(const Params 
 // order, so every append path gives the same bits).  Token t of the block comes from the cache if its position
 // is below `L_cached`, else from the new tokens.  A window that holds no token yet is left alone.
 constexpr int kStatThreads = 256;
-template <typename T, int D>
+template <typename T, int D, bool WIN>
 __device__ __forceinline__ void block_stats_role(const Params& p, int u, int blk, int w, int L_cached, int L_total, const T* kn,
                                                  bool act, float (*red_s)[D], float* mean_s) {
   constexpr int TG = kStatThreads / D;
   const int tid = threadIdx.x;
   const int t0 = blk * p.B;
-  const int t_lo = w * p.win_s;
-  const int t_hi = act ? min(min(p.B, L_total - t0), t_lo + p.win_C) : 0;     // tokens [t_lo, t_hi) of the block
+  const int t_lo = WIN ? w * p.win_s : 0;
+  const int t_hi = act ? (WIN ? min(min(p.B, L_total - t0), t_lo + p.win_C) : min(p.B, L_total - t0)) : 0;   // tokens [t_lo, t_hi)
   const int cnt = max(0, t_hi - t_lo);
   act = act && cnt > 0;
   const int tg = tid / D, c = tid % D;
@@ -118,7 +118,7 @@ __device__ __forceinline__ void block_stats_role(const Params& p, int u, int blk
     float tot = 0.f;
 #pragma unroll
     for (int g2 = 0; g2 < TG; ++g2) tot += red_s[g2][c];
-    float* rec = p.stats + (((size_t)u * p.max_blocks + blk) * p.NW + w) * 2 * D;
+    float* rec = p.stats + (WIN ? ((size_t)u * p.max_blocks + blk) * p.NW + w : (size_t)u * p.max_blocks + blk) * 2 * D;
     rec[c] = mean;
     rec[D + c] = tot / (float)cnt;
   }
@@ -135,7 +135,7 @@ __global__ void __launch_bounds__(kStatThreads) append_stats_kernel(const Params
   const bool act = n > 0 && blk * p.B < L + n;             // CTA-uniform
   if (!act) return;
   // the copy kernel has already stored the new tokens: everything is read from the cache
-  block_stats_role<T, D>(p, u, blk, blockIdx.x % p.NW, L + n, L + n, static_cast<const T*>(nullptr), true, red_s, mean_s);
+  block_stats_role<T, D, true>(p, u, blk, blockIdx.x % p.NW, L + n, L + n, static_cast<const T*>(nullptr), true, red_s, mean_s);
 }
 
 template <typename T, int D>
@@ -194,8 +194,8 @@ __global__ void append_lengths_kernel(const Params p, const int* __restrict__ n_
 constexpr int kFusedThreads = 256;
 constexpr int kFusedMaxNew = 32;
 
-template <typename T, int D>
-__global__ void __launch_bounds__(kFusedThreads) append_fused_kernel(const Params p, const T* __restrict__ k_new,
+template <typename T, int D, bool WIN>
+__global__ void __launch_bounds__(kFusedThreads, 4) append_fused_kernel(const Params p, const T* __restrict__ k_new,
                                                                      const T* __restrict__ v_new,
                                                                      const int* __restrict__ n_new, int max_new, int n_copy,
                                                                      int n_stats) {
@@ -240,8 +240,8 @@ __global__ void __launch_bounds__(kFusedThreads) append_fused_kernel(const Param
     }
   } else if ((role -= n_copy) < n_stats) {
     // ---- statistics role: one touched block; cached keys below the old length, new keys above it -----------
-    const int blk = L / p.B + role / p.NW;
-    block_stats_role<T, D>(p, u, blk, role % p.NW, L, L + max(n, 0), kn, n > 0 && blk * p.B < L + n, red_s, mean_s);
+    const int blk = L / p.B + (WIN ? role / p.NW : role);
+    block_stats_role<T, D, WIN>(p, u, blk, WIN ? role % p.NW : 0, L, L + max(n, 0), kn, n > 0 && blk * p.B < L + n, red_s, mean_s);
   } else if (!(p.flags & 4u)) {
     // ---- state role: S_bar[row0 .. row0 + 15][:] += sum_t phi(k_t)[row] v_t ------------------------------------
     role -= n_stats;
@@ -333,8 +333,9 @@ static cudaError_t launch_typed(const Params& p, const void* k_new, const void* 
     const int n_stats = ((max_new + p.B - 1) / p.B + 1) * p.NW;   // one CTA per window of every block that can be touched
     const int n_state = (p.flags & 4u) ? 0 : D / kStateRows;
     // Same shared-memory carve-out as the decode kernels around it: a change of carve-out drains the SMs.
-    cudaFuncSetAttribute(append_fused_kernel<T, D>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    return launch_ex(append_fused_kernel<T, D>, dim3(n_copy + n_stats + n_state, U), dim3(kFusedThreads), 0, stream, 0, true,
+    auto kern = p.NW > 1 ? append_fused_kernel<T, D, true> : append_fused_kernel<T, D, false>;
+    cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    return launch_ex(kern, dim3(n_copy + n_stats + n_state, U), dim3(kFusedThreads), 0, stream, 0, true,
                      p, kn, vn, n_new, max_new, n_copy, n_stats);
   }
   const int per_cta = kCopyThreads / 32;

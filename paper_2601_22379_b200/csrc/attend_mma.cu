@@ -89,7 +89,7 @@ constexpr int kPad = 8;   // floats of padding per row of the cross-warp reducti
 // PACK: the group has at most 4 heads, so accumulator rows 4..7 and 12..15 are padding; rows 12..15 then carry
 // the bf16 remainder of the linear coefficients and no extra products are needed for it.
 template <int D, bool PACK>
-__global__ void __launch_bounds__(kAttendThreads, 3)
+__global__ void __launch_bounds__(kAttendThreads, 2)
     attend_mma_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                       const __nv_bfloat16* __restrict__ q, const float* __restrict__ rms_weight, float* __restrict__ out,
                       float* __restrict__ dbg_sparse, float* __restrict__ dbg_rla) {

@@ -111,7 +111,9 @@ struct Smem {
 
 }  // namespace
 
-template <int D, int GP>
+// WIN: strided selection windows (several statistics records per block, max-pooled); without them the kernel is
+// compiled with one record per block as a constant.
+template <int D, int GP, bool WIN>
 __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Params p, const void* __restrict__ q_raw,
                                                                       int q_is_bf16, int* __restrict__ sel_user) {
   using SM = Smem<D, GP>;
@@ -177,7 +179,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   const int L = __ldcg(p.seq_lens + b);
   const int nblk = (L + p.B - 1) / p.B;
   const int chunk = p.chunk;                      // blocks per CTA
-  const int NW = p.NW;                            // selection windows per block; a "record" is one window
+  const int NW = WIN ? p.NW : 1;                  // selection windows per block; a "record" is one window
   const int blk_begin = min(nblk, rank * chunk);
   const int blk_end = min(nblk, blk_begin + chunk);
   const int nb_my = blk_end - blk_begin;          // blocks of this CTA
@@ -204,7 +206,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
       qv[g][v] = (p.flags & 2u) ? 0.f : 0.5f * qm[g][v] * qm[g][v];
     }
   }
-  if (NW > 1)                                   // pooled slots start below every key
+  if (WIN)                                      // pooled slots start below every key
     for (int x = tid; x < G * chunk; x += kCsThreads) reinterpret_cast<uint32_t*>(ell_s)[x] = 0u;
   __syncthreads();                              // the barrier initialisation is visible to every consumer
   SPLA_MARK(p, u, rank, 1);
@@ -277,7 +279,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
           }
           const int li = l0 + (p0 + sub) * NGRP + grp;
           if (fin_lane && li < n_my) {
-            if (NW == 1) {
+            if (!WIN) {
               const float ell = (rec_begin + li == nblk - 1 ? ln_last : ln_full) + dm_keep + __logf(1.f + dv_keep);
               ell_s[my_g * chunk + li] = ell;
               const float nm = fmaxf(run_max, ell);
@@ -299,7 +301,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
       }
     }
     SPLA_MARK(p, u, rank, 2);
-    if (NW > 1) {
+    if (WIN) {
       // the pooled keys back to floats, and this CTA's (max, sum exp) per head from them; lane 0 of every warp
       // then holds the warp's pair
       __syncthreads();
@@ -330,7 +332,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
       const float m2 = __shfl_xor_sync(0xffffffffu, run_max, 16), s2 = __shfl_xor_sync(0xffffffffu, run_sum, 16);
       lse_merge(run_max, run_sum, m2, s2);
     }
-    if (NW == 1 && fin_lane && sub == 0 && grp == 0) {
+    if (!WIN && fin_lane && sub == 0 && grp == 0) {
       wred[(warp * GP + my_g) * 2 + 0] = run_max;
       wred[(warp * GP + my_g) * 2 + 1] = run_sum;
     }
@@ -486,12 +488,12 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
     }
 }
 
-template <int D, int GP>
-static cudaError_t launch_one(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream) {
+template <int D, int GP, bool WIN>
+static cudaError_t launch_win(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream) {
   using SM = Smem<D, GP>;
   const int U = p.batch * p.Hkv;
   size_t smem = (size_t)SM::kEll + (size_t)p.G * p.chunk * sizeof(float);
-  auto kern = score_cluster_kernel<D, GP>;
+  auto kern = score_cluster_kernel<D, GP, WIN>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   if (p.cs > 8) {
@@ -499,6 +501,12 @@ static cudaError_t launch_one(const Params& p, const void* q, int q_is_bf16, int
     if (e != cudaSuccess) return e;
   }
   return launch_ex(kern, dim3(p.cs, U, 1), dim3(kCsThreads, 1, 1), smem, stream, p.cs, true, p, q, q_is_bf16, sel_user);
+}
+
+template <int D, int GP>
+static cudaError_t launch_one(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream) {
+  return p.NW > 1 ? launch_win<D, GP, true>(p, q, q_is_bf16, sel_user, stream)
+                  : launch_win<D, GP, false>(p, q, q_is_bf16, sel_user, stream);
 }
 
 template <int D>

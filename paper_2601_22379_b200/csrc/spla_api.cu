@@ -269,7 +269,7 @@ static int attend_cluster_size(const spla_cache* c) {
   if (c->cfg.flags & SPLA_GENERAL_KERNELS) return 0;
   const size_t smem = attend_mma_smem_bytes(c->p.B, c->p.d) + 2048;
   long long per_sm = (227 * 1024) / (long long)smem;
-  if (per_sm > 3) per_sm = 3;
+  if (per_sm > 2) per_sm = 2;                     // the kernel is compiled for two CTAs per SM (no register spills)
   if (per_sm < 1) return 0;                       // the tiles do not fit: use the general kernel
   const long long slots = per_sm * c->sm_count;
   const long long U = (long long)c->p.batch * c->p.Hkv;
