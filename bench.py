@@ -356,24 +356,25 @@ def run_ours(args, w):
     at = statistics.mean(at_iso)
 
     # ---- end to end through the public call with host buffers -----------------------------------------------------
-    # Per step: the host writes q, k_t, v_t into pinned staging buffers; H2D copies, append, decode and the D2H copy
-    # of the output are enqueued (as one captured graph per cache when graphs are in use) and the stream is
-    # synchronised, because the caller reads the output before it can form the next query.
-    src_q = [q.cpu() for q in qs[:8]]
-    src_kv = [(k.cpu(), v.cpu()) for k, v in kvs[:8]]
-    hq, hk, hv = src_q[0].clone().pin_memory(), src_kv[0][0].clone().pin_memory(), src_kv[0][1].clone().pin_memory()
-    dq, dk, dv = torch.empty_like(qs[0]), torch.empty_like(kvs[0][0]), torch.empty_like(kvs[0][1])
+    # Per step: the host writes q, k_t, v_t into a pinned staging buffer; the H2D copy, append and decode are enqueued
+    # (as one captured graph per cache when graphs are in use), the output goes device -> host by the merge kernel's own
+    # stores into a pinned host buffer (no separate copy), and the stream is synchronised, because the caller reads
+    # the output before it can form the next query.
+    # q, k_t and v_t travel in one staging buffer: one host write and one H2D copy per step instead of three
+    nq, nk = qs[0].numel(), kvs[0][0].numel()
+    src = [torch.cat([qs[i].reshape(-1), kvs[i][0].reshape(-1), kvs[i][1].reshape(-1)]).cpu() for i in range(8)]
+    hstage = src[0].clone().pin_memory()
+    dstage = torch.empty_like(src[0], device=dev)
+    dq = dstage[:nq].view_as(qs[0])
+    dk, dv = dstage[nq:nq + nk].view_as(kvs[0][0]), dstage[nq + nk:].view_as(kvs[0][1])
     hout = torch.empty(w.batch, w.n_q_heads, w.head_dim, dtype=torch.float32).pin_memory()
-    h2d = hq.numel() * hq.element_size() + 2 * hk.numel() * hk.element_size()
+    h2d = hstage.numel() * hstage.element_size()
     d2h = hout.numel() * 4
 
     def e2e_body(ci):
-        dq.copy_(hq, non_blocking=True)
-        dk.copy_(hk, non_blocking=True)
-        dv.copy_(hv, non_blocking=True)
+        dstage.copy_(hstage, non_blocking=True)
         caches[ci].append_tokens(dk, dv)
-        caches[ci].decode(dq, gamma, out=outs[ci])
-        hout.copy_(outs[ci], non_blocking=True)
+        caches[ci].decode(dq, gamma, out=hout)      # the merge kernel stores the output straight into pinned host memory
 
     e2e_graphs = None
     with torch.cuda.stream(stream):
@@ -392,9 +393,7 @@ def run_ours(args, w):
         g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         g0.record(stream)
         for i in range(n_e2e):
-            hq.copy_(src_q[i % 8])                                     # the step's inputs arrive in host memory
-            hk.copy_(src_kv[i % 8][0])
-            hv.copy_(src_kv[i % 8][1])
+            hstage.copy_(src[i % 8])                                   # the step's inputs arrive in host memory
             if e2e_graphs is not None:
                 e2e_graphs[i % R].replay()
             else:

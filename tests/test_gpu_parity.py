@@ -456,3 +456,17 @@ def test_tensor_core_state_update_matches_oracle_and_fma_kernel(name, over, chun
     again, _, _, _ = runner.build_cache(w, DEV, prefill=(K, V, lens), chunk=chunk)
     torch.cuda.synchronize()
     assert torch.equal(again.bufs.rla_state, cache.bufs.rla_state)
+
+
+def test_decode_into_pinned_host_memory_equals_decode_into_device_memory():
+    """`out` may be page-locked host memory (what the benchmark's end-to-end leg passes): same bits as a device buffer."""
+    w = synth.BY_NAME["gqa_32k"].scaled(batch=2, context=64 * 30 + 9)
+    cache, K, V, lens = runner.build_cache(w, DEV)
+    gamma = synth.gamma(w).to(DEV)
+    q = synth.step_queries(w, 0, DEV)
+    dev_out = cache.decode(q, gamma)
+    host_out = torch.empty(w.batch, w.n_q_heads, w.head_dim, dtype=torch.float32).pin_memory()
+    cache.decode(q, gamma, out=host_out)
+    torch.cuda.synchronize()
+    assert cache.sync_status() == 0
+    assert torch.equal(host_out, dev_out.cpu())
