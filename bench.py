@@ -185,12 +185,9 @@ def measured_peaks():
 
 def run_ours(args, w):
     import torch
-    import torch.distributed as dist
-    from paper_2601_22379_b200 import build, runner, synth
+    from paper_2601_22379_b200 import build, replicas, runner, synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local = replicas.env_world()
     cpu_base = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         vals, cores, sample = oracle_throughput(w, 500, repeats=2)      # before CUDA is initialised (fork)
@@ -199,8 +196,7 @@ def run_ours(args, w):
     build.build()
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+    replicas.init("nccl", dev)
 
     steps, warmup = args.steps, max(args.warmup, 3)
     by = synth.algorithmic_bytes_per_step(w, n_windows=n_windows(w))
@@ -272,9 +268,7 @@ def run_ours(args, w):
     torch.cuda.synchronize()
 
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        replicas.barrier(dev)
 
     # ---- the timed region: exactly `steps` steps ----------------------------------------------------------
     sampler = ClockSampler(local)
@@ -404,12 +398,8 @@ def run_ours(args, w):
     barrier()
     e2e_ms = g0.elapsed_time(g1) / n_e2e
 
-    t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = float(t[0]), float(t[1])
-    qh_per_step = w.batch * w.n_q_heads * world
-    value = qh_per_step * steps / (total_ms * 1e-3)
+    total_ms, e2e_ms = replicas.max_over_ranks([total_ms, e2e_ms], dev)
+    value = replicas.whole_job_rate(w.batch * w.n_q_heads, steps, total_ms)
 
     peak, peak_kind = measured_peaks()
     score_bytes = by["stats"] + by["state"]
@@ -439,8 +429,7 @@ def run_ours(args, w):
         line["cpu_baseline"] = cpu_base
     if rank == 0:
         print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.shutdown()
 
 
 def main():

@@ -61,3 +61,23 @@ def test_p10_planted_needles_are_selected_by_the_oracle():
             r = O.decode_unit(q[0, h * G:(h + 1) * G], K[h].double().numpy(), V[h].double().numpy(), g[h * G:(h + 1) * G],
                               block_size=w.block_size, top_k=w.top_k, n_sink=w.n_sink, n_local=w.n_local)
             assert set(nb[0, h].tolist()) <= set(r["sel"].tolist()), (name, h)
+
+
+def test_benchmark_configurations_use_the_papers_sparsity_specifications():
+    """Golden: the hyper-parameters the paper states (tests/golden/sparsity_specifications.txt)."""
+    import pathlib
+    from oracle import spla_oracle as O
+    spec = {}
+    for line in (pathlib.Path(__file__).parent / "golden" / "sparsity_specifications.txt").read_text().splitlines():
+        line = line.split("#")[0].strip()
+        if line:
+            k, v = line.split("=")
+            spec[k.strip()] = int(v)
+    long_128k, very_long = synth.BY_NAME["long_128k"], synth.BY_NAME["very_long_1m"]
+    assert long_128k.top_k == very_long.top_k == spec["top_k"]
+    assert long_128k.block_size == spec["block_size_gpu"] and very_long.block_size == spec["block_size_tpu"]
+    for w in synth.CONFIGS:
+        assert (w.n_sink, w.n_local) == (spec["n_sink_blocks"], spec["n_local_blocks"])
+    C, s = spec["window_size"], spec["window_stride"]
+    assert O.window_starts(spec["block_size_gpu"], C, s) == [0, 16, 32]
+    assert O.window_starts(spec["block_size_tpu"], C, s) == [0, 16, 32, 48, 64, 80, 96]
