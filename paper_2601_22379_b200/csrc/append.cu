@@ -248,6 +248,14 @@ __global__ void __launch_bounds__(kFusedThreads, 4) append_fused_kernel(const Pa
     const int row0 = role * kStateRows;
     const int nn = max(n, 0);
     const float a2 = p.phi_scale * kLog2e;
+    // The rows of S_bar this thread will update are requested first: the load comes from DRAM and would
+    // otherwise sit at the end of the role's dependency chain.
+    constexpr int RPT = kStateRows / TG;                         // rows per thread
+    const int tg = tid / D, j = tid % D;
+    float* S = p.state + (size_t)u * D * D + (size_t)(row0 + tg * RPT) * D + j;
+    float s_old[RPT];
+#pragma unroll
+    for (int r = 0; r < RPT; ++r) s_old[r] = nn > 0 ? __ldcs(S + (size_t)r * D) : 0.f;
     // log-sum-exp of every new token: 8 threads per token, D / 8 consecutive channels each, loaded up front
     {
       constexpr int CPT = D / 8;                                 // channels per thread
@@ -286,8 +294,6 @@ __global__ void __launch_bounds__(kFusedThreads, 4) append_fused_kernel(const Pa
       phi_s[t][r] = t < nn ? exp2f(to_float(kn[(size_t)t * D + row0 + r]) * a2 - lse_s[t]) : 0.f;
     }
     __syncthreads();
-    constexpr int RPT = kStateRows / TG;                         // rows per thread
-    const int tg = tid / D, j = tid % D;
     float acc[RPT];
 #pragma unroll
     for (int r = 0; r < RPT; ++r) acc[r] = 0.f;
@@ -297,9 +303,8 @@ __global__ void __launch_bounds__(kFusedThreads, 4) append_fused_kernel(const Pa
       for (int r = 0; r < RPT; ++r) acc[r] = fmaf(phi_s[t][tg * RPT + r], v, acc[r]);
     }
     if (nn > 0) {
-      float* S = p.state + (size_t)u * D * D + (size_t)(row0 + tg * RPT) * D + j;
 #pragma unroll
-      for (int r = 0; r < RPT; ++r) S[(size_t)r * D] += acc[r];
+      for (int r = 0; r < RPT; ++r) S[(size_t)r * D] = s_old[r] + acc[r];
     }
   }
 
