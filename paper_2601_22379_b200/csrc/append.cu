@@ -189,8 +189,8 @@ __global__ void append_lengths_kernel(const Params p, const int* __restrict__ n_
 // Decode-step appends (a few tokens per sequence): everything above in ONE launch.  CTAs take one of three roles
 // by blockIdx.x; no role needs another's output, because the new tokens are read from k_new / v_new directly
 // (statistics of the open block: cached keys below the old length, new keys above it; state: the per-token
-// log-sum-exp is recomputed from the new keys).  Every CTA reads the old lengths; the last CTA to finish
-// (atomic ticket, nobody waits) advances them.
+// log-sum-exp is recomputed from the new keys).  Every CTA reads the old lengths; the last CTA to have read them
+// (atomic ticket at the start, nobody waits) advances them.
 constexpr int kFusedThreads = 256;
 constexpr int kFusedMaxNew = 32;
 
@@ -212,11 +212,32 @@ __global__ void __launch_bounds__(kFusedThreads, 4) append_fused_kernel(const Pa
 
   pdl_wait();                                      // the preceding decode still reads the cache and the lengths
   pdl_launch_dependents();
+  SPLA_MARK(p, u, blockIdx.x, 0);
   const int L = p.seq_lens[b];
   const int n = tokens_to_add(p, n_new, max_new, b, L);
   const T* kn = k_new + (size_t)u * max_new * D;
   const T* vn = v_new + (size_t)u * max_new * D;
   const size_t unit_tok0 = (size_t)u * p.max_blocks * p.B;
+
+  // ---- the lengths are advanced by whichever CTA is the last to have read them ----------------------------------
+  // Every CTA works from the length it read above.  Once all CTAs of the launch hold theirs (the barrier below
+  // consumes each thread's value, so no load of a length is still in flight), the last one to check in may store the
+  // new lengths while the others are still busy: nothing in this launch reads them again, and the next kernel
+  // starts after this grid has completed.  No fence and no wait at the end of the kernel.
+  if (__syncthreads_or(L < 0)) return;               // (lengths are never negative)
+  if (tid == 0) {
+    const int t = atomicAdd(p.append_ticket, 1);
+    last_s = (t == (int)(gridDim.x * gridDim.y) - 1);
+    if (last_s) *p.append_ticket = 0;
+  }
+  __syncthreads();
+  if (last_s) {
+    for (int bb = tid; bb < p.batch; bb += kFusedThreads) {
+      const int Lb = p.seq_lens[bb];
+      const int nb = tokens_to_add(p, n_new, max_new, bb, Lb);
+      if (nb > 0) p.seq_lens[bb] = Lb + nb;
+    }
+  }
 
   if (role < n_copy) {
     // ---- copy role: one warp per token; also the per-token log-sum-exp the decode reads ------------------
@@ -308,23 +329,7 @@ __global__ void __launch_bounds__(kFusedThreads, 4) append_fused_kernel(const Pa
     }
   }
 
-  // ---- the last CTA of the whole launch advances the lengths ---------------------------------------------------
-  __syncthreads();
-  if (tid == 0) {
-    asm volatile("fence.acq_rel.gpu;" ::: "memory");
-    const int t = atomicAdd(p.append_ticket, 1);
-    last_s = (t == (int)(gridDim.x * gridDim.y) - 1);
-    if (last_s) *p.append_ticket = 0;
-    asm volatile("fence.acq_rel.gpu;" ::: "memory");
-  }
-  __syncthreads();
-  if (last_s) {
-    for (int bb = tid; bb < p.batch; bb += kFusedThreads) {
-      const int Lb = p.seq_lens[bb];
-      const int nb = tokens_to_add(p, n_new, max_new, bb, Lb);
-      if (nb > 0) p.seq_lens[bb] = Lb + nb;
-    }
-  }
+  SPLA_MARK(p, u, blockIdx.x, 2);
 }
 
 template <typename T, int D>
