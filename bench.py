@@ -34,7 +34,7 @@ L2_BYTES = 126 * 1024 * 1024
 GRAPH_STEPS = 64
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the score kernel from the ncu capture summarised in
 # profiles/score_cluster_kernel_long_128k.md (69.37 MB read + 0.66 MB written)
-NCU_TRAFFIC = {"long_128k": 70.03e6}
+NCU_TRAFFIC = {"long_128k": 70.03e6, "long_128k+windows(C=32,s=16)": 208.8e6}
 
 
 # ------------------------------------------------------------------------------------------------------------
@@ -443,8 +443,8 @@ def main():
     ap.add_argument("--caches", type=int, default=0, help="rotate over this many caches instead of the cold-L2 count "
                     "(for profiler captures, which must hold little device memory)")
     ap.add_argument("--traffic", type=float, default=None,
-                    help="DRAM bytes per launch of the dominant kernel from an ncu capture; default: the figure of "
-                         "profiles/score_cluster_kernel_long_128k.md for the long_128k workload")
+                    help="DRAM bytes per launch of the dominant kernel from an ncu capture; default: the figures of "
+                         "profiles/score_cluster_kernel_long_128k*.md for the long_128k workload")
     ap.add_argument("--window", default=None, metavar="C,s",
                     help="strided selection windows (the paper's setting is 32,16) instead of whole-block statistics")
     args = ap.parse_args()
