@@ -185,7 +185,7 @@ def measured_peaks():
 
 def run_ours(args, w):
     import torch
-    from paper_2601_22379_b200 import build, replicas, runner, synth
+    from paper_2601_22379_b200 import binding, build, replicas, runner, synth
 
     world, rank, local = replicas.env_world()
     cpu_base = None
@@ -402,6 +402,19 @@ def run_ours(args, w):
     value = replicas.whole_job_rate(w.batch * w.n_q_heads, steps, total_ms)
 
     peak, peak_kind = measured_peaks()
+    # a plain read-only stream over a buffer four times the L2, as a second reference beside the copy peak
+    probe = torch.empty(4 * L2_BYTES, dtype=torch.uint8, device=dev)
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            binding.probe_read(probe)
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        p0.record(stream)
+        for _ in range(10):
+            binding.probe_read(probe)
+        p1.record(stream)
+    torch.cuda.synchronize()
+    read_peak = 10 * probe.numel() / (p0.elapsed_time(p1) * 1e-3) / 1e9
+    del probe
     score_bytes = by["stats"] + by["state"]
     achieved = score_bytes / (sc * 1e-3) / 1e9
     line = base_line(args, w, value, ms_per_step=total_ms / steps)
@@ -416,6 +429,7 @@ def run_ours(args, w):
         "gpu_launches": 3 * steps,
         "roofline": {"bound": "hbm", "kernel": "score_cluster_kernel (block score + top-k)", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                     "read_stream_GBps": read_peak, "frac_of_read_stream": achieved / read_peak,
                      "bytes_per_launch": score_bytes, "ms_per_launch": sc,
                      "traffic": args.traffic if args.traffic is not None else NCU_TRAFFIC.get(workload_name(w))},
         "kernels": {"score_select_ms": sc, "score_select_isolated_ms": statistics.mean(sc_iso),

@@ -208,6 +208,14 @@ int spla_sync_status(spla_cache_t *cache, void *stream);
 int spla_select_blocks_noalloc(const spla_config_t *config, const float *stats, const int32_t *seq_lens,
                                const void *q, int32_t *sel_idx, float *scores_out, void *stream);
 
+/*
+ * Measurement aid with no counterpart in the paper: one read-only pass over `bytes` bytes at `buf` (DEVICE,
+ * 16-byte aligned; the contents do not matter and are not changed) by a plain streaming kernel, enqueued on
+ * `stream`.  A caller times it with events to learn what a pure read stream reaches on its GPU; the benchmark
+ * reports that figure beside the copy bandwidth.  Allocates nothing.
+ */
+int spla_probe_read(const void *buf, size_t bytes, void *stream);
+
 /* Tells the library an upper bound of the current sequence lengths after adopting contents (HOST value). */
 int spla_set_length_bound(spla_cache_t *cache, int32_t max_seq_len);
 

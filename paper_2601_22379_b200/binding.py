@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libspla.so"
 
 EXPORTS = ["spla_query_sizes", "spla_init_cache", "spla_append_tokens", "spla_decode", "spla_decode_selected",
            "spla_decode_profile", "spla_select_blocks_noalloc", "spla_select",
-           "spla_copy_scores", "spla_sync_status", "spla_set_length_bound", "spla_destroy_cache",
+           "spla_copy_scores", "spla_probe_read", "spla_sync_status", "spla_set_length_bound", "spla_destroy_cache",
            "spla_status_string", "spla_last_cuda_error"]
 
 
@@ -71,6 +71,7 @@ def load(path: str | None = None) -> C.CDLL:
     lib.spla_decode_profile.argtypes = [vp, vp, vp, vp, C.POINTER(C.c_float), vp]
     lib.spla_select_blocks_noalloc.argtypes = [C.POINTER(SplaConfig), vp, vp, vp, vp, vp, vp]
     lib.spla_copy_scores.argtypes = [vp, vp, vp]
+    lib.spla_probe_read.argtypes = [vp, C.c_size_t, vp]
     lib.spla_sync_status.argtypes = [vp, vp]
     lib.spla_set_length_bound.argtypes = [vp, i32]
     lib.spla_destroy_cache.argtypes = [vp]
@@ -147,6 +148,13 @@ def select_blocks_noalloc(cfg: SplaConfig, stats: torch.Tensor, seq_lens: torch.
     with torch.cuda.device(stats.device):
         return load().spla_select_blocks_noalloc(C.byref(cfg), stats.data_ptr(), seq_lens.data_ptr(), q.data_ptr(),
                                                  sel_idx.data_ptr(), _ptr(scores_out), _stream())
+
+
+def probe_read(buf: torch.Tensor):
+    """One read-only streaming pass over a device tensor (measurement aid)."""
+    assert buf.is_cuda and buf.is_contiguous()
+    with torch.cuda.device(buf.device):
+        _check(load().spla_probe_read(buf.data_ptr(), buf.numel() * buf.element_size(), _stream()), "spla_probe_read")
 
 
 class SplaCache:
