@@ -264,14 +264,15 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
             float vals[NV];
 #pragma unroll
             for (int g = 0; g < GP; ++g) {
-              float dm = 0.f, dv = 0.f;
+              // packed fp32 FMAs (two products per instruction): even and odd channels accumulate side by side
+              float2 am = make_float2(0.f, 0.f), av = make_float2(0.f, 0.f);
 #pragma unroll
-              for (int v = 0; v < VECW; ++v) {
-                dm = fmaf(qm[g][v], mean[p0 + pp][v], dm);
-                dv = fmaf(qv[g][v], var[p0 + pp][v], dv);
+              for (int v = 0; v < VECW; v += 2) {
+                am = __ffma2_rn(make_float2(qm[g][v], qm[g][v + 1]), make_float2(mean[p0 + pp][v], mean[p0 + pp][v + 1]), am);
+                av = __ffma2_rn(make_float2(qv[g][v], qv[g][v + 1]), make_float2(var[p0 + pp][v], var[p0 + pp][v + 1]), av);
               }
-              vals[g] = dm;
-              vals[GP + g] = dv;
+              vals[g] = am.x + am.y;
+              vals[GP + g] = av.x + av.y;
             }
             group_reduce_multi<NV, W>(vals, lane);
             const float other = __shfl_xor_sync(0xffffffffu, vals[0], W / 2);   // variance dot of the same head
