@@ -222,6 +222,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
     const int n_last = L - (nblk - 1) * p.B;     // tokens of the last block
     const float ln_last = logf((float)max(1, n_last));
     const float ln_win = logf((float)p.win_C);
+    const unsigned nw_magic = 0xffffffffu / (unsigned)NW + 1u;   // floor(x / NW) = umulhi(x, magic) for x < 2^16, NW <= 8
     float run_max = -INFINITY, run_sum = 0.f;
 
 #pragma unroll 1
@@ -289,7 +290,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
             } else {
               // strided windows (Section 3.1, "Strided Block Selection"): log mass of window w of a block,
               // max-pooled into the block's slot right away through an order-preserving integer key
-              const int lb = li / NW, w = li - lb * NW;
+              const int lb = (int)__umulhi((unsigned)li, nw_magic), w = li - lb * NW;   // li / NW without a division
               float ln_n = ln_win;
               if (blk_begin + lb == nblk - 1) {
                 const int cnt = min(p.win_C, n_last - w * p.win_s);
