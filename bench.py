@@ -234,9 +234,8 @@ def run_ours(args, w):
         counter["i"] += 1
         c = caches[i % R]
         k1, v1 = kvs[i % n_in]
-        c.append_tokens(k1, v1)
+        c.append_decode(k1, v1, qs[i % n_in], gamma, out=outs[i % R])    # the step: append, then decode, one call
         n_app[i % R] += 1
-        c.decode(qs[i % n_in], gamma, out=outs[i % R])
 
     def decode_only(i):
         caches[i % R].decode(qs[i % n_in], gamma, out=outs[i % R])
@@ -367,8 +366,7 @@ def run_ours(args, w):
 
     def e2e_body(ci):
         dstage.copy_(hstage, non_blocking=True)
-        caches[ci].append_tokens(dk, dv)
-        caches[ci].decode(dq, gamma, out=hout)      # the merge kernel stores the output straight into pinned host memory
+        caches[ci].append_decode(dk, dv, dq, gamma, out=hout)   # the merge kernel stores the output straight into pinned host memory
 
     e2e_graphs = None
     with torch.cuda.stream(stream):

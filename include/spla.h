@@ -150,6 +150,17 @@ int spla_decode(spla_cache_t *cache, const void *q, const float *rms_weight, flo
                 float *dbg_o_sparse, float *dbg_o_rla, void *stream);
 
 /*
+ * One whole step of the order of use the file comment gives: spla_append_tokens(k_new, v_new, n_new, max_new)
+ * followed by spla_decode(q, ...), with the same arguments, the same results and the same error behaviour.  Made as
+ * one call, the library knows that the score kernel follows this step's append directly, and lets it stream the
+ * statistics of the blocks that were already complete while the append is still running.  q (like k_new, v_new)
+ * must be ready in stream order when the call is made.
+ */
+int spla_append_decode(spla_cache_t *cache, const void *k_new, const void *v_new, const int32_t *n_new, int32_t max_new,
+                       const void *q, const float *rms_weight, float *out, int32_t *sel_idx, float *dbg_o_sparse,
+                       float *dbg_o_rla, void *stream);
+
+/*
  * Steps 1-2 of spla_decode only: scores the blocks (Section 3.1, Eq. taylor-2nd; Section 2.2, grouped BlockScore)
  * and selects top_k of them (Section 2.1, Select).  sel_idx: DEVICE int32 [batch][H_kv][top_k], ascending, padded
  * with -1.  The scores stay available to spla_copy_scores.  Together with spla_decode_selected this splits a

@@ -19,7 +19,7 @@ SPLA_ADOPT_CONTENTS, SPLA_FIRST_ORDER, SPLA_NO_RLA, SPLA_GENERAL_KERNELS = 1, 2,
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libspla.so")
 
 EXPORTS = ["spla_query_sizes", "spla_init_cache", "spla_append_tokens", "spla_decode", "spla_decode_selected",
-           "spla_decode_profile", "spla_select_blocks_noalloc", "spla_select",
+           "spla_decode_profile", "spla_select_blocks_noalloc", "spla_select", "spla_append_decode",
            "spla_copy_scores", "spla_probe_read", "spla_sync_status", "spla_set_length_bound", "spla_destroy_cache",
            "spla_status_string", "spla_last_cuda_error"]
 
@@ -68,6 +68,7 @@ def load(path: str | None = None) -> C.CDLL:
     lib.spla_decode.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.spla_decode_selected.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.spla_select.argtypes = [vp, vp, vp, vp]
+    lib.spla_append_decode.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.spla_decode_profile.argtypes = [vp, vp, vp, vp, C.POINTER(C.c_float), vp]
     lib.spla_select_blocks_noalloc.argtypes = [C.POINTER(SplaConfig), vp, vp, vp, vp, vp, vp]
     lib.spla_copy_scores.argtypes = [vp, vp, vp]
@@ -223,6 +224,26 @@ class SplaCache:
         with torch.cuda.device(self.device):
             _check(self.lib.spla_decode(self.handle, q.data_ptr(), _ptr(rms_weight), out.data_ptr(), _ptr(sel_idx),
                                         _ptr(dbg_o_sparse), _ptr(dbg_o_rla), _stream()), "spla_decode")
+        return out
+
+    def append_decode(self, k_new: torch.Tensor, v_new: torch.Tensor, q: torch.Tensor, rms_weight, out=None,
+                      n_new: torch.Tensor | None = None, sel_idx=None, dbg_o_sparse=None, dbg_o_rla=None) -> torch.Tensor:
+        """One step: `append_tokens(k_new, v_new, n_new)` then `decode(q, ...)`, as one call."""
+        cfg = self.cfg
+        assert k_new.is_cuda and k_new.is_contiguous() and v_new.is_contiguous() and k_new.shape == v_new.shape
+        assert k_new.dtype == self.kv_torch_dtype and v_new.dtype == self.kv_torch_dtype
+        assert tuple(k_new.shape[:2]) == (cfg.batch, cfg.n_kv_heads) and k_new.shape[3] == cfg.head_dim
+        assert q.is_cuda and q.is_contiguous() and q.dtype == self.q_torch_dtype
+        assert tuple(q.shape) == (cfg.batch, cfg.n_q_heads, cfg.head_dim)
+        if n_new is not None:
+            assert n_new.dtype == torch.int32 and n_new.is_cuda and n_new.numel() == cfg.batch
+        if out is None:
+            out = torch.empty(cfg.batch, cfg.n_q_heads, cfg.head_dim, dtype=torch.float32, device=self.device)
+        with torch.cuda.device(self.device):
+            _check(self.lib.spla_append_decode(self.handle, k_new.data_ptr(), v_new.data_ptr(), _ptr(n_new),
+                                               k_new.shape[2], q.data_ptr(), _ptr(rms_weight), out.data_ptr(),
+                                               _ptr(sel_idx), _ptr(dbg_o_sparse), _ptr(dbg_o_rla), _stream()),
+                   "spla_append_decode")
         return out
 
     def select(self, q: torch.Tensor, sel_idx: torch.Tensor | None = None) -> torch.Tensor:

@@ -113,9 +113,14 @@ struct Smem {
 
 // WIN: strided selection windows (several statistics records per block, max-pooled); without them the kernel is
 // compiled with one record per block as a constant.
-template <int D, int GP, bool WIN>
+// EARLY: the kernel follows the append of the same step in the stream and does not wait for it before streaming:
+// the blocks that were complete before that append (at most `pending_new` tokens per sequence) cannot change any
+// more, so their statistics are streamed while the append still runs; only then does the kernel wait for the
+// append, read the final length and take the few remaining blocks (those the append wrote to) from global memory.
+template <int D, int GP, bool WIN, bool EARLY>
 __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Params p, const void* __restrict__ q_raw,
-                                                                      int q_is_bf16, int* __restrict__ sel_user) {
+                                                                      int q_is_bf16, int* __restrict__ sel_user,
+                                                                      int pending_new) {
   using SM = Smem<D, GP>;
   constexpr int W = GP <= 4 ? 16 : 32;          // lanes that share one record
   constexpr int NGRP = 32 / W;                  // records a warp works on side by side
@@ -148,8 +153,10 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
     err_s = 0;
   }
   SPLA_MARK(p, blockIdx.y, 30, 0);
-  pdl_wait();                                   // everything the preceding kernels wrote (statistics, lengths, q) is visible
-  pdl_launch_dependents();                      // only now may the next kernel begin its prologue: it reads q before its own wait
+  if (!EARLY) {
+    pdl_wait();                                 // everything the preceding kernels wrote (statistics, lengths, q) is visible
+    pdl_launch_dependents();                    // only now may the next kernel begin its prologue: it reads q before its own wait
+  }
 
   // ---- the query loads go out first and the ring is started as soon as the sequence length is known: a small
   // load issued into the streaming traffic would take several microseconds.
@@ -176,21 +183,34 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
       for (int v = 0; v < VECW; ++v) qm[g][v] = 0.f;
     }
   }
-  const int L = __ldcg(p.seq_lens + b);
-  const int nblk = (L + p.B - 1) / p.B;
+  // EARLY: this length may be the one before or after the running append; minus `pending_new` it bounds from below
+  // the tokens that were there before it
+  int L0;
+  if (EARLY) {                                    // one read for the whole CTA: the value may change under our feet
+    __shared__ int l0_s;
+    if (tid == 0) l0_s = __ldcg(p.seq_lens + b);
+    __syncthreads();
+    L0 = l0_s;
+  } else {
+    L0 = __ldcg(p.seq_lens + b);
+  }
+  int L = L0;
+  int nblk = (L + p.B - 1) / p.B;
   const int chunk = p.chunk;                      // blocks per CTA
   const int NW = WIN ? p.NW : 1;                  // selection windows per block; a "record" is one window
-  const int blk_begin = min(nblk, rank * chunk);
-  const int blk_end = min(nblk, blk_begin + chunk);
-  const int nb_my = blk_end - blk_begin;          // blocks of this CTA
-  const int rec_begin = blk_begin * NW;
-  const int n_my = nb_my * NW;                    // records of this CTA
-  const int n_rounds = (n_my + kStageRec - 1) / kStageRec;
+  const int cta_blk0 = rank * chunk;              // first block of this CTA's share
+  const int nblk_stream = EARLY ? max(0, L0 - pending_new) / p.B : nblk;    // blocks whose records the ring may fetch
+  const int n_stream = max(0, min(cta_blk0 + chunk, nblk_stream) - cta_blk0) * NW;
+  int blk_begin = min(nblk, cta_blk0);
+  int nb_my = min(nblk, blk_begin + chunk) - blk_begin;   // blocks of this CTA (EARLY: refreshed after the wait)
+  int n_my = nb_my * NW;                          // records of this CTA
+  const int rec_begin = cta_blk0 * NW;            // (a CTA that has records starts at its share's first block)
+  const int n_rounds = (n_stream + kStageRec - 1) / kStageRec;
   const float* stats_u = p.stats + (size_t)u * p.max_blocks * NW * 2 * D;
 
   auto issue = [&](int r) {                      // thread 0 only: one bulk copy fills stage r % kStages
     const int s = r % kStages;
-    const int nrec = min(kStageRec, n_my - r * kStageRec);
+    const int nrec = min(kStageRec, n_stream - r * kStageRec);
     const uint32_t bytes = (uint32_t)nrec * SM::kRecBytes;
     mbar_expect_tx(&full[s], bytes);
     bulk_g2s(smem_raw + (size_t)s * SM::kStageBytes, stats_u + (size_t)(rec_begin + r * kStageRec) * 2 * D, bytes, &full[s]);
@@ -219,44 +239,17 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
     const int sub = hl % LPV;
     const bool fin_lane = hl < W / 2 && sub < FB && my_g < G;
     const float ln_full = logf((float)p.B);
-    const int n_last = L - (nblk - 1) * p.B;     // tokens of the last block
-    const float ln_last = logf((float)max(1, n_last));
+    // EARLY: while streaming, every block is a full one; the last block of the sequence comes after the wait
+    int nblk_fin = EARLY ? 0x7fffffff : nblk;
+    int n_last = L - (nblk - 1) * p.B;           // tokens of the last block
+    float ln_last = logf((float)max(1, n_last));
     const float ln_win = logf((float)p.win_C);
     const unsigned nw_magic = 0xffffffffu / (unsigned)NW + 1u;   // floor(x / NW) = umulhi(x, magic) for x < 2^16, NW <= 8
     float run_max = -INFINITY, run_sum = 0.f;
 
-#pragma unroll 1
-    for (int r = 0; r < n_rounds; ++r) {
-      const int s = r % kStages;
-      if (!mbar_wait(&full[s], (r / kStages) & 1)) { if (lane == 0) atomicExch(&err_s, 1); break; }
-      const int l0 = r * kStageRec + warp * UNR;                       // first record of this warp, CTA-local
-      const float* st = reinterpret_cast<const float*>(smem_raw + (size_t)s * SM::kStageBytes) + (size_t)(warp * UNR) * 2 * D;
-      float mean[PASSES][VECW], var[PASSES][VECW];
-#pragma unroll
-      for (int ps = 0; ps < PASSES; ++ps) {
-        const int rec = ps * NGRP + grp;
-        if (l0 + rec < n_my) {
-#pragma unroll
-          for (int c = 0; c < NC; ++c) {
-            float a[CW], bb[CW];
-            load_vec<CW>(st + (size_t)rec * 2 * D + c * W * 4 + hl * CW, a);
-            load_vec<CW>(st + (size_t)rec * 2 * D + D + c * W * 4 + hl * CW, bb);
-#pragma unroll
-            for (int v = 0; v < CW; ++v) { mean[ps][c * CW + v] = a[v]; var[ps][c * CW + v] = bb[v]; }
-          }
-        } else {
-#pragma unroll
-          for (int v = 0; v < VECW; ++v) { mean[ps][v] = 0.f; var[ps][v] = 0.f; }
-        }
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&empty[s]);                            // the stage is in registers: hand it back
-      if (tid == 0 && r + kStages < n_rounds) {                         // refill it once every warp has done the same
-        if (mbar_wait(&empty[s], (r / kStages) & 1)) issue(r + kStages);
-        else atomicExch(&err_s, 1);
-      }
-      __syncwarp();
-      if (l0 < n_my) {
+    // dots of the records a warp holds in registers -> log masses (and, with whole blocks, the running normaliser);
+    // `limit` is the number of local records that exist for this call
+    auto finish_passes = [&](int l0, int limit, float (&mean)[PASSES][VECW], float (&var)[PASSES][VECW]) {
 #pragma unroll
         for (int p0 = 0; p0 < PASSES; p0 += FB) {
           float dm_keep = 0.f, dv_keep = 0.f;
@@ -280,9 +273,9 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
             if (sub == pp) { dm_keep = vals[0]; dv_keep = other; }
           }
           const int li = l0 + (p0 + sub) * NGRP + grp;
-          if (fin_lane && li < n_my) {
+          if (fin_lane && li < limit) {
             if (!WIN) {
-              const float ell = (rec_begin + li == nblk - 1 ? ln_last : ln_full) + dm_keep + __logf(1.f + dv_keep);
+              const float ell = (rec_begin + li == nblk_fin - 1 ? ln_last : ln_full) + dm_keep + __logf(1.f + dv_keep);
               ell_s[my_g * chunk + li] = ell;
               const float nm = fmaxf(run_max, ell);
               run_sum = run_sum * __expf(run_max - nm) + __expf(ell - nm);
@@ -292,13 +285,90 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
               // max-pooled into the block's slot right away through an order-preserving integer key
               const int lb = (int)__umulhi((unsigned)li, nw_magic), w = li - lb * NW;   // li / NW without a division
               float ln_n = ln_win;
-              if (blk_begin + lb == nblk - 1) {
+              if (cta_blk0 + lb == nblk_fin - 1) {
                 const int cnt = min(p.win_C, n_last - w * p.win_s);
                 ln_n = cnt > 0 ? logf((float)cnt) : -INFINITY;
               }
               atomicMax(reinterpret_cast<uint32_t*>(ell_s) + my_g * chunk + lb, float_order_key(ln_n + dm_keep + __logf(1.f + dv_keep)));
             }
           }
+        }
+    };
+#pragma unroll 1
+    for (int r = 0; r < n_rounds; ++r) {
+      const int s = r % kStages;
+      if (!mbar_wait(&full[s], (r / kStages) & 1)) { if (lane == 0) atomicExch(&err_s, 1); break; }
+      const int l0 = r * kStageRec + warp * UNR;                       // first record of this warp, CTA-local
+      const float* st = reinterpret_cast<const float*>(smem_raw + (size_t)s * SM::kStageBytes) + (size_t)(warp * UNR) * 2 * D;
+      float mean[PASSES][VECW], var[PASSES][VECW];
+#pragma unroll
+      for (int ps = 0; ps < PASSES; ++ps) {
+        const int rec = ps * NGRP + grp;
+        if (l0 + rec < n_stream) {
+#pragma unroll
+          for (int c = 0; c < NC; ++c) {
+            float a[CW], bb[CW];
+            load_vec<CW>(st + (size_t)rec * 2 * D + c * W * 4 + hl * CW, a);
+            load_vec<CW>(st + (size_t)rec * 2 * D + D + c * W * 4 + hl * CW, bb);
+#pragma unroll
+            for (int v = 0; v < CW; ++v) { mean[ps][c * CW + v] = a[v]; var[ps][c * CW + v] = bb[v]; }
+          }
+        } else {
+#pragma unroll
+          for (int v = 0; v < VECW; ++v) { mean[ps][v] = 0.f; var[ps][v] = 0.f; }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty[s]);                            // the stage is in registers: hand it back
+      if (tid == 0 && r + kStages < n_rounds) {                         // refill it once every warp has done the same
+        if (mbar_wait(&empty[s], (r / kStages) & 1)) issue(r + kStages);
+        else atomicExch(&err_s, 1);
+      }
+      __syncwarp();
+      if (l0 < n_stream) finish_passes(l0, n_stream, mean, var);
+    }
+    if constexpr (EARLY) {
+      // now the append must be complete: final length, and the blocks it wrote to (the last ones of the sequence, a
+      // handful of records) through plain loads into stage 0, one more round
+      pdl_wait();
+      pdl_launch_dependents();
+      L = __ldcg(p.seq_lens + b);
+      nblk = (L + p.B - 1) / p.B;
+      blk_begin = min(nblk, cta_blk0);
+      nb_my = min(nblk, blk_begin + chunk) - blk_begin;
+      n_my = nb_my * NW;
+      nblk_fin = nblk;
+      n_last = L - (nblk - 1) * p.B;
+      ln_last = logf((float)max(1, n_last));
+      const int n_late = n_my - n_stream;
+      if (n_late > 0) {                            // CTA-uniform
+        __syncthreads();                           // every warp is done with the ring
+        float4* dst = reinterpret_cast<float4*>(smem_raw);
+        const float4* src = reinterpret_cast<const float4*>(stats_u + (size_t)(rec_begin + n_stream) * 2 * D);
+        for (int x = tid; x < n_late * (SM::kRecBytes / 16); x += kCsThreads) dst[x] = __ldcg(src + x);
+        __syncthreads();
+        for (int base = 0; base < n_late; base += kStageRec) {
+          const int l0 = n_stream + base + warp * UNR;
+          const float* st = reinterpret_cast<const float*>(smem_raw) + (size_t)(base + warp * UNR) * 2 * D;
+          float mean[PASSES][VECW], var[PASSES][VECW];
+#pragma unroll
+          for (int ps = 0; ps < PASSES; ++ps) {
+            const int rec = ps * NGRP + grp;
+            if (l0 + rec < n_my) {
+#pragma unroll
+              for (int c = 0; c < NC; ++c) {
+                float a[CW], bb[CW];
+                load_vec<CW>(st + (size_t)rec * 2 * D + c * W * 4 + hl * CW, a);
+                load_vec<CW>(st + (size_t)rec * 2 * D + D + c * W * 4 + hl * CW, bb);
+#pragma unroll
+                for (int v = 0; v < CW; ++v) { mean[ps][c * CW + v] = a[v]; var[ps][c * CW + v] = bb[v]; }
+              }
+            } else {
+#pragma unroll
+              for (int v = 0; v < VECW; ++v) { mean[ps][v] = 0.f; var[ps][v] = 0.f; }
+            }
+          }
+          if (l0 < n_my) finish_passes(l0, n_my, mean, var);
         }
       }
     }
@@ -490,34 +560,37 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
     }
 }
 
-template <int D, int GP, bool WIN>
-static cudaError_t launch_win(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream) {
+template <int D, int GP, bool WIN, bool EARLY>
+static cudaError_t launch_win(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new, cudaStream_t stream) {
   using SM = Smem<D, GP>;
   const int U = p.batch * p.Hkv;
   size_t smem = (size_t)SM::kEll + (size_t)p.G * p.chunk * sizeof(float);
-  auto kern = score_cluster_kernel<D, GP, WIN>;
+  auto kern = score_cluster_kernel<D, GP, WIN, EARLY>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   if (p.cs > 8) {
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) return e;
   }
-  return launch_ex(kern, dim3(p.cs, U, 1), dim3(kCsThreads, 1, 1), smem, stream, p.cs, true, p, q, q_is_bf16, sel_user);
+  return launch_ex(kern, dim3(p.cs, U, 1), dim3(kCsThreads, 1, 1), smem, stream, p.cs, true, p, q, q_is_bf16, sel_user, pending_new);
 }
 
 template <int D, int GP>
-static cudaError_t launch_one(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream) {
-  return p.NW > 1 ? launch_win<D, GP, true>(p, q, q_is_bf16, sel_user, stream)
-                  : launch_win<D, GP, false>(p, q, q_is_bf16, sel_user, stream);
+static cudaError_t launch_one(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new, cudaStream_t stream) {
+  if (pending_new > 0)
+    return p.NW > 1 ? launch_win<D, GP, true, true>(p, q, q_is_bf16, sel_user, pending_new, stream)
+                    : launch_win<D, GP, false, true>(p, q, q_is_bf16, sel_user, pending_new, stream);
+  return p.NW > 1 ? launch_win<D, GP, true, false>(p, q, q_is_bf16, sel_user, 0, stream)
+                  : launch_win<D, GP, false, false>(p, q, q_is_bf16, sel_user, 0, stream);
 }
 
 template <int D>
-static cudaError_t launch_d(const Params& p, int GP, const void* q, int qb, int* sel_user, cudaStream_t s) {
+static cudaError_t launch_d(const Params& p, int GP, const void* q, int qb, int* sel_user, int pending_new, cudaStream_t s) {
   switch (GP) {
-    case 1: return launch_one<D, 1>(p, q, qb, sel_user, s);
-    case 2: return launch_one<D, 2>(p, q, qb, sel_user, s);
-    case 4: return launch_one<D, 4>(p, q, qb, sel_user, s);
-    default: return launch_one<D, 8>(p, q, qb, sel_user, s);
+    case 1: return launch_one<D, 1>(p, q, qb, sel_user, pending_new, s);
+    case 2: return launch_one<D, 2>(p, q, qb, sel_user, pending_new, s);
+    case 4: return launch_one<D, 4>(p, q, qb, sel_user, pending_new, s);
+    default: return launch_one<D, 8>(p, q, qb, sel_user, pending_new, s);
   }
 }
 
@@ -539,10 +612,13 @@ bool plan_score_cluster(int units, long long max_seq_blocks, int NW, int G, int 
   return true;
 }
 
-cudaError_t launch_score_cluster(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream) {
+// pending_new > 0: the kernel directly follows, in the stream, an append of at most that many tokens per sequence
+// and may stream the older blocks' statistics before that append has completed.
+cudaError_t launch_score_cluster(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new,
+                                 cudaStream_t stream) {
   const int GP = padded_group(p.G);
-  return p.d == 128 ? launch_d<128>(p, GP, q, q_is_bf16, sel_user, stream)
-                    : launch_d<64>(p, GP, q, q_is_bf16, sel_user, stream);
+  return p.d == 128 ? launch_d<128>(p, GP, q, q_is_bf16, sel_user, pending_new, stream)
+                    : launch_d<64>(p, GP, q, q_is_bf16, sel_user, pending_new, stream);
 }
 
 }  // namespace spla

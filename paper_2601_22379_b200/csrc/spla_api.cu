@@ -259,8 +259,8 @@ static void plan_score_grid(const spla_cache* c, Params* p) {
   p->n_chunks_cap = (int)((blocks * p->NW + p->chunk - 1) / p->chunk);
 }
 
-static cudaError_t launch_score(const Params& p, const void* q, int qb, int* sel_user, cudaStream_t s) {
-  return p.cs > 0 ? launch_score_cluster(p, q, qb, sel_user, s) : launch_score_select(p, q, qb, sel_user, s);
+static cudaError_t launch_score(const Params& p, const void* q, int qb, int* sel_user, cudaStream_t s, int pending_new = 0) {
+  return p.cs > 0 ? launch_score_cluster(p, q, qb, sel_user, pending_new, s) : launch_score_select(p, q, qb, sel_user, s);
 }
 
 // Cluster size of the tensor-core attend kernel: the largest power of two (at most 16 and at most top_k) for
@@ -303,6 +303,32 @@ extern "C" int spla_decode(spla_cache_t* c, const void* q, const float* rms_weig
   if (e != cudaSuccess) return cuda_fail(e, "spla_decode/score_select");
   e = launch_attend_merge(p, &c->maps, q, qb, rms_weight, nullptr, out, dbg_o_sparse, dbg_o_rla, s);
   if (e != cudaSuccess) return cuda_fail(e, "spla_decode/attend_merge");
+  return SPLA_OK;
+}
+
+// One decode step, append then decode, as one call.  Because the score kernel then directly follows this step's
+// append kernel in the stream, it is told so and streams the statistics of the blocks that were complete before
+// the append while the append is still running; it waits for the append only before it reads the final lengths
+// and the few blocks the append wrote to.  Same results as the two calls made one after the other.
+extern "C" int spla_append_decode(spla_cache_t* c, const void* k_new, const void* v_new, const int32_t* n_new,
+                                  int32_t max_new, const void* q, const float* rms_weight, float* out,
+                                  int32_t* sel_idx, float* dbg_o_sparse, float* dbg_o_rla, void* stream) {
+  if (!c || !q || !out) return SPLA_ERR_INVALID_ARG;
+  if (!rms_weight && !(c->cfg.flags & SPLA_NO_RLA)) return SPLA_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(out, 16)) return SPLA_ERR_INVALID_ARG;
+  const int rc = spla_append_tokens(c, k_new, v_new, n_new, max_new, stream);
+  if (rc != SPLA_OK) return rc;
+  Params p = c->p;
+  plan_score_grid(c, &p);
+  p.acs = attend_cluster_size(c);
+  const int qb = c->cfg.q_dtype == SPLA_BF16;
+  cudaStream_t s = (cudaStream_t)stream;
+  // only the fused decode-step append kernel opens the dependent launch early enough for this to matter
+  const int pending = (max_new <= 32) ? max_new : 0;
+  cudaError_t e = launch_score(p, q, qb, sel_idx, s, pending);
+  if (e != cudaSuccess) return cuda_fail(e, "spla_append_decode/score_select");
+  e = launch_attend_merge(p, &c->maps, q, qb, rms_weight, nullptr, out, dbg_o_sparse, dbg_o_rla, s);
+  if (e != cudaSuccess) return cuda_fail(e, "spla_append_decode/attend_merge");
   return SPLA_OK;
 }
 

@@ -48,7 +48,8 @@ int score_chunk_for(long long units, long long max_seq_blocks, int sm_count);
 cudaError_t launch_score_select(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream);
 // score_cluster.cu (G <= 8, at most 16 x 1024 blocks per sequence)
 bool plan_score_cluster(int units, long long max_seq_blocks, int NW, int G, int d, int sm_count, int* cs_out, int* chunk_out);
-cudaError_t launch_score_cluster(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream);
+cudaError_t launch_score_cluster(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new,
+                                 cudaStream_t stream);
 struct AttendMaps {                      // TMA tensor maps (CUtensorMap) of the K and V caches, opaque to the host code
   alignas(64) unsigned char k[128];
   alignas(64) unsigned char v[128];
