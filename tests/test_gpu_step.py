@@ -126,3 +126,35 @@ def test_one_call_step_capacity_is_checked_on_the_host():
     with pytest.raises(binding.SplaError) as e:
         cache.append_decode(k1, v1, q, gamma)
     assert e.value.status == binding.SPLA_ERR_CAPACITY
+
+
+def test_many_one_call_steps_on_one_cache_in_one_graph():
+    """150 steps on the same cache captured in one graph (every score kernel starts while the append in front of it
+    is running, across two block boundaries), against the same steps made as separate calls: bit for bit."""
+    n = 150
+    w = synth.BY_NAME["gqa_32k"].scaled(batch=2, context=64 * 20 + 50, n_needles=0, n_steps=n)
+    a, K, V, lens = runner.build_cache(w, DEV)
+    b, _, _, _ = runner.build_cache(w, DEV, prefill=(K, V, lens))
+    gamma = synth.gamma(w).to(DEV)
+    kvs = [synth.step_kv(w, s, DEV) for s in range(8)]
+    qs = [synth.step_queries(w, s, DEV) for s in range(8)]
+    cfg = a.cfg
+    outs_a = torch.empty(n, cfg.batch, cfg.n_q_heads, cfg.head_dim, dtype=torch.float32, device=DEV)
+    outs_b = torch.empty_like(outs_a)
+    sel_a = torch.empty(n, cfg.batch, cfg.n_kv_heads, cfg.top_k, dtype=torch.int32, device=DEV)
+    sel_b = torch.empty_like(sel_a)
+    for s in range(n):
+        a.append_tokens(*kvs[s % 8])
+        a.decode(qs[s % 8], gamma, out=outs_a[s], sel_idx=sel_a[s])
+    g = torch.cuda.CUDAGraph()
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        with torch.cuda.graph(g, stream=st):
+            for s in range(n):
+                b.append_decode(*kvs[s % 8], qs[s % 8], gamma, out=outs_b[s], sel_idx=sel_b[s])
+        g.replay()
+    torch.cuda.synchronize()
+    assert a.sync_status() == 0 and b.sync_status() == 0
+    assert torch.equal(sel_a, sel_b)
+    assert torch.equal(outs_a, outs_b)
+    _same_cache(a, b)
