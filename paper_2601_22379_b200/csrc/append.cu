@@ -3,18 +3,18 @@
 // state S_bar += phi(k_t)^T v_t in fp32 (Section 3.2, Eq. rla-impl-1, "Numerical Stability").
 //
 // Appends of up to 32 tokens per sequence (the decode loop) run as ONE fused kernel, see append_fused_kernel.
-// Bulk appends (prefill) run as four kernels in stream order, all reading the OLD sequence lengths until the
+// Bulk appends (prefill) run as three kernels in stream order, all reading the OLD sequence lengths until the
 // last one bumps them:
-//   copy   : k_new, v_new -> cache; per-token logsumexp of phi_scale * k into tok_lse
-//   stats  : mean / variance of every touched block recomputed from the cached keys (two exact passes, so the
-//            result does not depend on how the tokens were split across append calls)
-//   state  : rank-n update of S_bar, rows tiled over CTAs, phi(k) staged through shared memory
+//   block  : one CTA per touched block: its keys (cached ones below the old length, new ones above) are staged in
+//            shared memory once; from there the new tokens go to the cache (k_new, v_new -> cache), their
+//            logsumexp of phi_scale * k to tok_lse, and the block's mean / variance records are recomputed (two
+//            exact passes, so the result does not depend on how the tokens were split across append calls)
+//   state  : rank-n update of S_bar (tensor cores for long bf16 appends, else rows tiled over CTAs on the FMA pipe)
 //   lengths: seq_lens += n_new
 #include "spla_internal.h"
 
 namespace spla {
 
-constexpr int kCopyThreads = 256;
 constexpr int kStateRows = 16;     // rows of S_bar per CTA
 constexpr int kStateTokens = 32;   // tokens staged per inner step
 constexpr int kStateUmmaMinTokens = 256;   // appends at least this long take the tensor-core state kernel
@@ -33,49 +33,15 @@ __device__ __forceinline__ void copy_bytes(void* dst, const void* src) {
   else *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<const uint32_t*>(src);
 }
 
-template <typename T, int D>
-__global__ void __launch_bounds__(kCopyThreads) append_copy_kernel(const Params p, const T* __restrict__ k_new,
-                                                                   const T* __restrict__ v_new,
-                                                                   const int* __restrict__ n_new, int max_new) {
-  constexpr int VEC = D / 32;
-  const int u = blockIdx.y, b = u / p.Hkv;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int L = p.seq_lens[b];
-  const int n = tokens_to_add(p, n_new, max_new, b, L);
-  if (n < 0) {
-    if (blockIdx.x == 0 && threadIdx.x == 0) atomicExch(p.status, -2);
-    return;
-  }
-  const int i = blockIdx.x * (kCopyThreads / 32) + warp;
-  if (i >= n) return;
-  const size_t src = ((size_t)u * max_new + i) * D + lane * VEC;
-  const size_t pos = (size_t)u * p.max_blocks * p.B + (size_t)(L + i);
-  T* kd = reinterpret_cast<T*>(p.k_cache) + pos * D + lane * VEC;
-  T* vd = reinterpret_cast<T*>(p.v_cache) + pos * D + lane * VEC;
-  float k[VEC];
-  load_vec<VEC>(k_new + src, k);
-  copy_bytes<VEC * sizeof(T)>(kd, k_new + src);
-  copy_bytes<VEC * sizeof(T)>(vd, v_new + src);
-  float mx = -INFINITY;
-#pragma unroll
-  for (int v = 0; v < VEC; ++v) { k[v] *= p.phi_scale; mx = fmaxf(mx, k[v]); }
-  mx = warp_max(mx);
-  float s = 0.f;
-#pragma unroll
-  for (int v = 0; v < VEC; ++v) s += expf(k[v] - mx);
-  s = warp_sum(s);
-  if (lane == 0) p.tok_lse[pos] = mx + logf(s);
-}
-
 // Mean and population variance of one selection window of one block (window w covers the block's tokens
 // [w * win_s, w * win_s + win_C); without strided windows that is the whole block), two exact passes, by
 // kStatThreads threads (groups of D threads take every TG-th token; the partial sums are combined in a fixed
-// order, so every append path gives the same bits).  Token t of the block comes from the cache if its position
-// is below `L_cached`, else from the new tokens.  A window that holds no token yet is left alone.
+// order, so every append path gives the same bits).  `key_at(t)` returns channel (tid % D) of the block's token t.
+// A window that holds no token yet is left alone.
 constexpr int kStatThreads = 256;
-template <typename T, int D, bool WIN>
-__device__ __forceinline__ void block_stats_role(const Params& p, int u, int blk, int w, int L_cached, int L_total, const T* kn,
-                                                 bool act, float (*red_s)[D], float* mean_s) {
+template <int D, bool WIN, typename KeyAt>
+__device__ __forceinline__ void block_stats_core(const Params& p, int u, int blk, int w, int L_total, bool act,
+                                                 float (*red_s)[D], float* mean_s, KeyAt key_at) {
   constexpr int TG = kStatThreads / D;
   const int tid = threadIdx.x;
   const int t0 = blk * p.B;
@@ -84,14 +50,6 @@ __device__ __forceinline__ void block_stats_role(const Params& p, int u, int blk
   const int cnt = max(0, t_hi - t_lo);
   act = act && cnt > 0;
   const int tg = tid / D, c = tid % D;
-  const T* kc = reinterpret_cast<const T*>(p.k_cache) + ((size_t)u * p.max_blocks * p.B + t0) * D + c;
-  // One address per token (cached or new) and one load from it: no branch around the loads, so that the
-  // unrolled loop keeps several of them in flight.
-  auto key_at = [&](int t) {
-    const int pos = t0 + t;
-    const T* src = pos < L_cached ? kc + (size_t)t * D : kn + (size_t)(pos - L_cached) * D + c;
-    return to_float(*src);
-  };
   float sum = 0.f;
 #pragma unroll 8
   for (int t = t_lo + tg; t < t_hi; t += TG) sum += key_at(t);
@@ -124,18 +82,103 @@ __device__ __forceinline__ void block_stats_role(const Params& p, int u, int blk
   }
 }
 
+// The same from global memory: token t of the block comes from the cache if its position is below `L_cached`,
+// else from the new tokens `kn`.
+template <typename T, int D, bool WIN>
+__device__ __forceinline__ void block_stats_role(const Params& p, int u, int blk, int w, int L_cached, int L_total, const T* kn,
+                                                 bool act, float (*red_s)[D], float* mean_s) {
+  const int t0 = blk * p.B;
+  const int c = threadIdx.x % D;
+  const T* kc = reinterpret_cast<const T*>(p.k_cache) + ((size_t)u * p.max_blocks * p.B + t0) * D + c;
+  // One address per token (cached or new) and one load from it: no branch around the loads, so that the
+  // unrolled loop keeps several of them in flight.
+  block_stats_core<D, WIN>(p, u, blk, w, L_total, act, red_s, mean_s, [&](int t) {
+    const int pos = t0 + t;
+    const T* src = pos < L_cached ? kc + (size_t)t * D : kn + (size_t)(pos - L_cached) * D + c;
+    return to_float(*src);
+  });
+}
+
+// Bulk append, one CTA per touched block (blockIdx.x-th block at or after the one the old length falls in).  The
+// block's keys are staged once in shared memory, 16 bytes per thread and load, several loads in flight: cached
+// keys below the old length, new keys above it; the new keys and values go on to the cache from the same
+// registers.  Then, from shared memory: the per-token logsumexp of the new tokens (one warp per token) and the
+// statistics records of all the block's windows.
+constexpr int kBlockLoads = 4;                       // 16-byte loads of K (and of V) in flight per thread
 template <typename T, int D>
-__global__ void __launch_bounds__(kStatThreads) append_stats_kernel(const Params p, const int* __restrict__ n_new, int max_new) {
+__global__ void __launch_bounds__(kStatThreads) append_block_kernel(const Params p, const T* __restrict__ k_new,
+                                                                    const T* __restrict__ v_new,
+                                                                    const int* __restrict__ n_new, int max_new) {
+  extern __shared__ __align__(16) unsigned char tile_raw[];
   __shared__ float red_s[kStatThreads / D][D];
   __shared__ float mean_s[D];
+  constexpr int VEC = D / 32;
+  constexpr int CH = D * (int)sizeof(T) / 16;        // 16-byte chunks per token
+  T* tile = reinterpret_cast<T*>(tile_raw);          // [B][D]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int u = blockIdx.y, b = u / p.Hkv;
   const int L = p.seq_lens[b];
   const int n = tokens_to_add(p, n_new, max_new, b, L);
-  const int blk = L / p.B + blockIdx.x / p.NW;             // a window of the x-th touched block
-  const bool act = n > 0 && blk * p.B < L + n;             // CTA-uniform
-  if (!act) return;
-  // the copy kernel has already stored the new tokens: everything is read from the cache
-  block_stats_role<T, D, true>(p, u, blk, blockIdx.x % p.NW, L + n, L + n, static_cast<const T*>(nullptr), true, red_s, mean_s);
+  if (n < 0) {
+    if (blockIdx.x == 0 && tid == 0) atomicExch(p.status, -2);
+    return;
+  }
+  const int blk = L / p.B + blockIdx.x;
+  const int t0 = blk * p.B;
+  if (n == 0 || t0 >= L + n) return;                 // CTA-uniform
+  const int cnt = min(p.B, L + n - t0);              // tokens the block holds after the append
+  const int t_new = max(0, L - t0);                  // its first new token
+
+  const size_t blk_tok0 = (size_t)u * p.max_blocks * p.B + t0;
+  uint4* kc = reinterpret_cast<uint4*>(reinterpret_cast<T*>(p.k_cache) + blk_tok0 * D);
+  uint4* vc = reinterpret_cast<uint4*>(reinterpret_cast<T*>(p.v_cache) + blk_tok0 * D);
+  // new token i of the unit sits at chunk (t0 - L + t) * CH + ch of kn / vn
+  const uint4* kn = reinterpret_cast<const uint4*>(k_new + (size_t)u * max_new * D) + (ptrdiff_t)(t0 - L) * CH;
+  const uint4* vn = reinterpret_cast<const uint4*>(v_new + (size_t)u * max_new * D) + (ptrdiff_t)(t0 - L) * CH;
+  uint4* tile4 = reinterpret_cast<uint4*>(tile_raw);
+  const int total = cnt * CH, first_new = t_new * CH;
+  for (int base = 0; base < total; base += kBlockLoads * kStatThreads) {
+    uint4 kk[kBlockLoads], vv[kBlockLoads];
+#pragma unroll
+    for (int j = 0; j < kBlockLoads; ++j) {
+      const int idx = base + j * kStatThreads + tid;
+      if (idx < total) {
+        if (idx >= first_new) { kk[j] = __ldcs(kn + idx); vv[j] = __ldcs(vn + idx); }
+        else kk[j] = kc[idx];
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < kBlockLoads; ++j) {
+      const int idx = base + j * kStatThreads + tid;
+      if (idx < total) {
+        tile4[idx] = kk[j];
+        if (idx >= first_new) { kc[idx] = kk[j]; vc[idx] = vv[j]; }
+      }
+    }
+  }
+  __syncthreads();
+
+  // per-token logsumexp of phi_scale * k, the value the decode and the state update read
+  for (int t = t_new + warp; t < cnt; t += kStatThreads / 32) {
+    float k[VEC];
+    load_vec<VEC>(tile + (size_t)t * D + lane * VEC, k);
+    float mx = -INFINITY;
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) { k[v] *= p.phi_scale; mx = fmaxf(mx, k[v]); }
+    mx = warp_max(mx);
+    float s = 0.f;
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) s += expf(k[v] - mx);
+    s = warp_sum(s);
+    if (lane == 0) p.tok_lse[blk_tok0 + t] = mx + logf(s);
+  }
+
+  const int c = tid % D;
+  for (int w = 0; w < p.NW; ++w) {
+    block_stats_core<D, true>(p, u, blk, w, L + n, true, red_s, mean_s,
+                              [&](int t) { return to_float(tile[(size_t)t * D + c]); });
+    __syncthreads();                                 // the next window reuses the reduction buffers
+  }
 }
 
 template <typename T, int D>
@@ -348,9 +391,12 @@ static cudaError_t launch_typed(const Params& p, const void* k_new, const void* 
     return launch_ex(kern, dim3(n_copy + n_stats + n_state, U), dim3(kFusedThreads), 0, stream, 0, true,
                      p, kn, vn, n_new, max_new, n_copy, n_stats);
   }
-  const int per_cta = kCopyThreads / 32;
-  append_copy_kernel<T, D><<<dim3((max_new + per_cta - 1) / per_cta, U), kCopyThreads, 0, stream>>>(p, kn, vn, n_new, max_new);
-  append_stats_kernel<T, D><<<dim3(((max_new + p.B - 1) / p.B + 1) * p.NW, U), kStatThreads, 0, stream>>>(p, n_new, max_new);
+  {
+    const size_t tile_bytes = (size_t)p.B * D * sizeof(T);
+    auto kern = append_block_kernel<T, D>;
+    if (tile_bytes > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tile_bytes);
+    kern<<<dim3((max_new + p.B - 1) / p.B + 1, U), kStatThreads, tile_bytes, stream>>>(p, kn, vn, n_new, max_new);
+  }
   if (!(p.flags & 4u)) {
     // long appends of a bf16 cache with d = 128: the rank-n update is a dense contraction, done on the tensor cores
     // from the tokens the copy kernel has just stored; everything else on the FMA pipe
