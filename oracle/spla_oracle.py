@@ -33,6 +33,10 @@ notes of the repository):
     maximum of its windows' Taylor log masses, and the per-head
     normalisation over blocks comes after this pooling;
   * ties are broken by (score descending, block index ascending);
+  * 16-bit statistics (an option; the paper does not say in which precision
+    the block summaries are kept): mean and variance are computed in full
+    precision, rounded once to bfloat16 (round to nearest, ties to even)
+    and the Taylor score uses the rounded values; ln n_i stays exact;
   * RLA has no normaliser; RMS(.) is RMSNorm with a learnable scale gamma.
 
 Parity unpinned: the paper prints no worked numeric example, so the *final
@@ -52,6 +56,19 @@ F64 = np.float64
 # ---------------------------------------------------------------------------
 # Elementary pieces
 # ---------------------------------------------------------------------------
+def round_bf16(x):
+    """The bfloat16 value nearest to x (ties to even), returned as float64.
+
+    bfloat16 keeps the sign, the 8 exponent bits and the upper 7 fraction bits
+    of a float32: round the float32 nearest to x to a multiple of 2^16 in its
+    bit pattern.  Finite inputs of normal float32 range are expected.
+    """
+    bits = np.asarray(x, dtype=F64).astype(np.float32).view(np.uint32).astype(np.uint64)
+    keep_odd = (bits >> np.uint64(16)) & np.uint64(1)
+    bits = (bits + np.uint64(0x7FFF) + keep_odd) & np.uint64(0xFFFF0000)
+    return bits.astype(np.uint32).view(np.float32).astype(F64)
+
+
 def phi(x, phi_scale: float = 1.0):
     """Feature map of the linear branch: softmax over the feature dimension.
 
@@ -301,7 +318,7 @@ def rla_by_subtraction(q_group, S_bar, K, V, toks, phi_scale: float = 1.0):
 # ---------------------------------------------------------------------------
 def decode_unit(q_group, K, V, gamma_group, *, block_size, top_k, n_sink=0, n_local=0,
                 sm_scale=None, phi_scale=1.0, rms_eps=1e-6, order=2, use_rla=True,
-                override_selection=None, S_bar=None, stats=None, window=None):
+                override_selection=None, S_bar=None, stats=None, window=None, stats_bf16=False):
     """SPLA decode output for one (sequence, KV head) unit.
 
     q_group [G, d] raw queries of the group, K, V [L, d] the whole cache of
@@ -312,6 +329,7 @@ def decode_unit(q_group, K, V, gamma_group, *, block_size, top_k, n_sink=0, n_lo
     `S_bar` / `stats` may be passed in pre-computed (incremental form).
     `window` = (C, s) switches the score to strided windows with max-pooling;
     `stats` then holds window statistics.
+    `stats_bf16` rounds the means and variances to bfloat16 before the score.
     Returns a dict with every intermediate the tests compare.
     """
     q_group = np.asarray(q_group, dtype=F64)
@@ -326,9 +344,13 @@ def decode_unit(q_group, K, V, gamma_group, *, block_size, top_k, n_sink=0, n_lo
     ell_w = None
     if window is None:
         mean, var, n = block_statistics(K, B) if stats is None else stats
-        ell, p, score = block_scores(q_hat, mean, var, n, order=order)
     else:
         mean, var, n = window_statistics(K, B, window[0], window[1]) if stats is None else stats
+    if stats_bf16:
+        mean, var = round_bf16(mean), round_bf16(var)
+    if window is None:
+        ell, p, score = block_scores(q_hat, mean, var, n, order=order)
+    else:
         ell_w, ell, p, score = pooled_block_scores(q_hat, mean, var, n, order=order)
     if override_selection is None:
         sel = select_blocks(score, top_k, n_sink, n_local)

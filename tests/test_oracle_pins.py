@@ -476,3 +476,75 @@ def test_window_scores_normalise_and_incremental_equals_definitional():
     wm, wv, _ = O.window_statistics(Kp, B, C, s)
     np.testing.assert_allclose(wm, ref["mean"], rtol=1e-12, atol=1e-14)
     np.testing.assert_allclose(wv, ref["var"], rtol=1e-11, atol=1e-14)
+
+
+# ---------------------------------------------------------------------------
+# Q  16-bit statistics (a reading: the paper leaves the precision of the block summaries open)
+# ---------------------------------------------------------------------------
+def test_bf16_rounding_matches_the_library_cast_and_ties_go_to_even():
+    x = np.concatenate([RNG.standard_normal(20000) * np.exp(RNG.uniform(-20, 20, 20000)), [0.0, -0.0, 1.0, -1.0, 3.0e38]])
+    want = torch.from_numpy(x).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(O.round_bf16(x), want)
+    # bfloat16 has 8 significant bits: the spacing in [1, 2) is 2^-7, so 1 + 2^-8 is a tie
+    u = 2.0 ** -7
+    assert O.round_bf16(1 + u / 2) == 1.0                 # tie -> even mantissa (1.0)
+    assert O.round_bf16(1 + 3 * u / 2) == 1 + 2 * u       # tie -> even mantissa (1 + 2u)
+    assert O.round_bf16(1 + u / 2 + 1e-6) == 1 + u        # just above the tie (by more than a float32 step)
+    assert O.round_bf16(-(1 + 3 * u / 2)) == -(1 + 2 * u)
+    assert np.max(np.abs(O.round_bf16(x[:20000]) - x[:20000]) / np.abs(x[:20000])) <= 2.0 ** -8 * (1 + 1e-6)
+
+
+def test_bf16_statistics_change_the_log_mass_by_at_most_the_rounding_bound():
+    """|ell_16 - ell| <= 2^-8 (sum_c |q_c||mean_c| + 1/2 sum_c q_c^2 var_c): every statistic moves by at most half a
+    unit in the last place, i.e. 2^-8 relative (8 significant bits), and log(1 + x) is 1-Lipschitz for x >= 0."""
+    d, B, G, L = 32, 16, 4, 16 * 37 + 5
+    K = RNG.standard_normal((L, d)) * np.exp(RNG.uniform(-1, 1, d))
+    V = RNG.standard_normal((L, d))
+    q = RNG.standard_normal((G, d)) * 3
+    gamma = np.ones((G, d))
+    cfg = dict(block_size=B, top_k=6, n_sink=1, n_local=1)
+    a = O.decode_unit(q, K, V, gamma, **cfg)
+    b = O.decode_unit(q, K, V, gamma, stats_bf16=True, **cfg)
+    q_hat = q / np.sqrt(d)
+    bound = 2.0 ** -8 * (1 + 1e-6) * (np.abs(q_hat) @ np.abs(a["mean"]).T + 0.5 * (q_hat ** 2) @ a["var"].T)
+    diff = np.abs(b["ell"] - a["ell"])
+    assert np.all(diff <= bound + 1e-15)
+    assert np.max(diff) > 1e-6                                   # and the option is not a no-op
+    assert np.array_equal(b["mean"], O.round_bf16(a["mean"])) and np.array_equal(b["var"], O.round_bf16(a["var"]))
+    # the rest of the path is untouched by the option: same selection -> same outputs
+    c = O.decode_unit(q, K, V, gamma, stats_bf16=True, override_selection=a["sel"], **cfg)
+    assert np.array_equal(c["out"], a["out"])
+
+
+def test_bf16_statistics_are_exact_when_the_statistics_are_representable():
+    """Blocks of identical keys with bfloat16-representable entries: mean = key, variance = 0, nothing is rounded,
+    so the option must not change a single bit; same for windows."""
+    d, B, G = 16, 8, 2
+    nblk = 9
+    base = O.round_bf16(RNG.standard_normal((nblk, d)))
+    K = np.repeat(base, B, axis=0)[: nblk * B - 3]
+    V = RNG.standard_normal(K.shape)
+    q = RNG.standard_normal((G, d))
+    gamma = np.ones((G, d))
+    for window in (None, (4, 2)):
+        cfg = dict(block_size=B, top_k=4, n_sink=1, n_local=1, window=window)
+        a = O.decode_unit(q, K, V, gamma, **cfg)
+        b = O.decode_unit(q, K, V, gamma, stats_bf16=True, **cfg)
+        assert np.array_equal(a["score"], b["score"]) and np.array_equal(a["out"], b["out"])
+
+
+def test_bf16_statistics_incremental_cache_equals_definitional_form():
+    d, B, G = 16, 8, 2
+    K = RNG.standard_normal((8 * 11 + 3, d))
+    V = RNG.standard_normal(K.shape)
+    q = RNG.standard_normal((G, d))
+    gamma = RNG.uniform(0.5, 1.5, (G, d))
+    for window in (None, (4, 4)):
+        cache = O.UnitCache.from_prefill(K[:40], V[:40], B, window=window)
+        cache.append(K[40:], V[40:])
+        cfg = dict(top_k=5, n_sink=1, n_local=1, stats_bf16=True)
+        a = cache.decode(q, gamma, **cfg)
+        b = O.decode_unit(q, K, V, gamma, block_size=B, window=window, **cfg)
+        assert np.array_equal(a["sel"], b["sel"])
+        np.testing.assert_allclose(a["score"], b["score"], rtol=1e-2, atol=0)   # rounding may flip where Welford and two-pass differ in the last bit
+        np.testing.assert_allclose(a["out"], b["out"], rtol=1e-9, atol=1e-12)
