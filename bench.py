@@ -42,6 +42,7 @@ NCU_TRAFFIC = {"long_128k": 70.03e6, "long_128k+windows(C=32,s=16)": 208.8e6}
 # ------------------------------------------------------------------------------------------------------------
 _ORACLE_UNITS = None
 WINDOW = None          # (C, s) when --window is given: strided selection windows instead of whole blocks
+STATS_BF16 = False     # --stats-bf16: the block statistics are stored (and streamed) as bfloat16
 
 
 def _oracle_worker(args):
@@ -54,7 +55,8 @@ def _oracle_worker(args):
         cache = O.UnitCache.from_prefill(K, V, cfg["block_size"], window=cfg["window"])
         t0 = time.perf_counter()
         for i in range(n_dec):
-            cache.decode(qs[i % len(qs)], gam, top_k=cfg["top_k"], n_sink=cfg["n_sink"], n_local=cfg["n_local"])
+            cache.decode(qs[i % len(qs)], gam, top_k=cfg["top_k"], n_sink=cfg["n_sink"], n_local=cfg["n_local"],
+                         stats_bf16=cfg["stats_bf16"])
         return time.perf_counter() - t0
 
 
@@ -73,7 +75,8 @@ def oracle_throughput(w, n_dec_per_unit: int, repeats: int = 1):
     _ORACLE_UNITS = [(K[h].double().numpy(), V[h].double().numpy(), [q[h * G:(h + 1) * G] for q in qs],
                       gam[h * G:(h + 1) * G]) for h in range(n_units)]
     del K, V
-    cfg = dict(block_size=w.block_size, top_k=w.top_k, n_sink=w.n_sink, n_local=w.n_local, window=WINDOW)
+    cfg = dict(block_size=w.block_size, top_k=w.top_k, n_sink=w.n_sink, n_local=w.n_local, window=WINDOW,
+               stats_bf16=STATS_BF16)
     values = []
     ctx = mp.get_context("fork")
     with ctx.Pool(n_units) as pool:
@@ -111,12 +114,16 @@ def n_windows(w):
 
 
 def workload_name(w):
-    return w.name + (f"+windows(C={WINDOW[0]},s={WINDOW[1]})" if WINDOW else "")
+    return w.name + (f"+windows(C={WINDOW[0]},s={WINDOW[1]})" if WINDOW else "") + ("+stats_bf16" if STATS_BF16 else "")
+
+
+def stat_bytes():
+    return 2 if STATS_BF16 else 4
 
 
 def base_line(args, w, value, ms_per_step):
     from paper_2601_22379_b200 import synth
-    by = synth.algorithmic_bytes_per_step(w, n_windows=n_windows(w))
+    by = synth.algorithmic_bytes_per_step(w, n_windows=n_windows(w), stat_bytes=stat_bytes())
     return {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -125,7 +132,7 @@ def base_line(args, w, value, ms_per_step):
                    "head_dim": w.head_dim, "context": w.context, "block_size": w.block_size, "top_k": w.top_k,
                    "n_sink": w.n_sink, "n_local": w.n_local, "kv_dtype": w.kv_dtype,
                    "selection": (f"strided windows C={WINDOW[0]} s={WINDOW[1]}, max-pooled per block" if WINDOW
-                                 else "whole-block statistics"),
+                                 else "whole-block statistics") + (", statistics stored as bfloat16" if STATS_BF16 else ""),
                    "algorithmic_bytes_per_step": by["total"], "dense_kv_bytes_per_step": by["dense_kv"],
                    "parallelism": f"replicas x{args.gpus} (units are independent; no collective)"},
     }
@@ -199,7 +206,7 @@ def run_ours(args, w):
     replicas.init("nccl", dev)
 
     steps, warmup = args.steps, max(args.warmup, 3)
-    by = synth.algorithmic_bytes_per_step(w, n_windows=n_windows(w))
+    by = synth.algorithmic_bytes_per_step(w, n_windows=n_windows(w), stat_bytes=stat_bytes())
     R = 2                                                             # caches to rotate over (cold-L2 protocol)
     while R * by["total"] < 3 * L2_BYTES and R < GRAPH_STEPS:
         R *= 2
@@ -211,7 +218,8 @@ def run_ours(args, w):
     prefill = runner.generate_prefill(wl, dev)
     caches = []
     for _ in range(R):
-        c, _, _, _ = runner.build_cache(wl, dev, prefill=prefill, window=WINDOW)
+        c, _, _, _ = runner.build_cache(wl, dev, prefill=prefill, window=WINDOW,
+                                        flags=binding.SPLA_STATS_BF16 if STATS_BF16 else 0)
         caches.append(c)
     del prefill
     n_app = [0] * R                                                   # tokens appended per cache so far
@@ -459,10 +467,13 @@ def main():
                          "profiles/score_cluster_kernel_long_128k*.md for the long_128k workload")
     ap.add_argument("--window", default=None, metavar="C,s",
                     help="strided selection windows (the paper's setting is 32,16) instead of whole-block statistics")
+    ap.add_argument("--stats-bf16", action="store_true",
+                    help="store the block statistics as bfloat16 (half the bytes for the score kernel to stream)")
     args = ap.parse_args()
+    global WINDOW, STATS_BF16
     if args.window:
-        global WINDOW
         WINDOW = tuple(int(x) for x in args.window.split(","))
+    STATS_BF16 = args.stats_bf16
     from paper_2601_22379_b200 import synth
     w = synth.BY_NAME[args.workload]
     if args.impl == "reference":

@@ -65,6 +65,10 @@ typedef enum { SPLA_F32 = 0, SPLA_BF16 = 1 } spla_dtype_t;
 #define SPLA_NO_RLA 4u         /* out = o_sparse; the residual branch is skipped (the paper's SPA ablation) */
 #define SPLA_GENERAL_KERNELS 8u /* always use the general kernels (any group size up to 16, any length, fp32 or bf16)
                                    instead of the cluster / tensor-core ones: for testing and comparison */
+#define SPLA_STATS_BF16 16u    /* the block statistics are stored as bfloat16: they are computed in fp32 as always and
+                                   rounded once (to nearest even) when written; the Taylor score of Section 3.1 reads
+                                   the rounded values (ln n_i stays exact).  Halves the bytes the score streams; the
+                                   paper does not say in which precision its block summaries are kept. */
 
 typedef struct {
   int32_t batch;          /* sequences per call, >= 1 */
@@ -93,8 +97,8 @@ typedef struct {
 typedef struct {
   void *k_cache;      /* DEVICE [batch][H_kv][max_blocks][B][d] kv_dtype; token t of a unit lives in block t / B */
   void *v_cache;      /* DEVICE same layout */
-  float *stats;       /* DEVICE [batch][H_kv][max_blocks][NW][2][d] fp32: key mean, then population variance, of each
-                         of the NW selection windows of a block (NW = 1: the whole block) */
+  void *stats;        /* DEVICE [batch][H_kv][max_blocks][NW][2][d] fp32 (bfloat16 with SPLA_STATS_BF16): key mean, then
+                         population variance, of each of the NW selection windows of a block (NW = 1: the whole block) */
   float *rla_state;   /* DEVICE [batch][H_kv][d][d] fp32 S_bar: row = feature of phi(k), column = value dim */
   float *tok_lse;     /* DEVICE [batch][H_kv][max_blocks * B] fp32: logsumexp_c(phi_scale * k_t[c]) per token */
   int32_t *seq_lens;  /* DEVICE [batch]: tokens cached per sequence */
@@ -202,7 +206,7 @@ int spla_sync_status(spla_cache_t *cache, void *stream);
  *               sm_scale and SPLA_FIRST_ORDER are used.  The scratch needed, about
  *               batch * H_kv * max_blocks * (G + 1) * 4 bytes, must fit SPLA_NOALLOC_SCRATCH_BYTES, otherwise
  *               SPLA_ERR_UNSUPPORTED is returned and nothing is launched.  window_size must be 0 (whole-block
- *               statistics), otherwise SPLA_ERR_UNSUPPORTED.
+ *               statistics) and SPLA_STATS_BF16 unset (fp32 records), otherwise SPLA_ERR_UNSUPPORTED.
  *   stats:      DEVICE fp32 [batch][H_kv][max_blocks][2][d], as maintained by spla_append_tokens.
  *   seq_lens:   DEVICE int32 [batch].
  *   q:          DEVICE [batch][H_q][d] q_dtype.

@@ -14,7 +14,7 @@ import torch
 
 SPLA_OK, SPLA_ERR_INVALID_ARG, SPLA_ERR_CAPACITY, SPLA_ERR_CUDA, SPLA_ERR_UNSUPPORTED = 0, -1, -2, -3, -4
 SPLA_F32, SPLA_BF16 = 0, 1
-SPLA_ADOPT_CONTENTS, SPLA_FIRST_ORDER, SPLA_NO_RLA, SPLA_GENERAL_KERNELS = 1, 2, 4, 8
+SPLA_ADOPT_CONTENTS, SPLA_FIRST_ORDER, SPLA_NO_RLA, SPLA_GENERAL_KERNELS, SPLA_STATS_BF16 = 1, 2, 4, 8, 16
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libspla.so")
 
@@ -162,7 +162,8 @@ class SplaCache:
     """Owns the device buffers (as torch tensors) of one cache and forwards to the C ABI.
 
     Shapes follow include/spla.h: k_cache/v_cache [batch, H_kv, max_blocks, B, d], stats
-    [batch, H_kv, max_blocks, 2, d] (with strided windows [batch, H_kv, max_blocks, NW, 2, d]), rla_state
+    [batch, H_kv, max_blocks, 2, d] (with strided windows [batch, H_kv, max_blocks, NW, 2, d]; fp32, or bfloat16
+    with SPLA_STATS_BF16), rla_state
     [batch, H_kv, d, d], tok_lse [batch, H_kv, max_blocks * B].
     """
 
@@ -182,8 +183,8 @@ class SplaCache:
         self.bufs = _Bufs(
             k_cache=torch.empty(*shp, B, d, dtype=kv_t, device=dev),
             v_cache=torch.empty(*shp, B, d, dtype=kv_t, device=dev),
-            stats=torch.empty(*shp, *((cfg.n_windows,) if cfg.window_size > 0 else ()), 2, d, dtype=torch.float32,
-                              device=dev),
+            stats=torch.empty(*shp, *((cfg.n_windows,) if cfg.window_size > 0 else ()), 2, d, device=dev,
+                              dtype=torch.bfloat16 if cfg.flags & SPLA_STATS_BF16 else torch.float32),
             rla_state=torch.empty(cfg.batch, cfg.n_kv_heads, d, d, dtype=torch.float32, device=dev),
             tok_lse=torch.empty(cfg.batch, cfg.n_kv_heads, self.max_blocks * B, dtype=torch.float32, device=dev),
             seq_lens=torch.empty(cfg.batch, dtype=torch.int32, device=dev),
@@ -191,7 +192,7 @@ class SplaCache:
         )
         b = self.bufs
         assert b.k_cache.numel() * b.k_cache.element_size() == sz.k_cache
-        assert b.stats.numel() * 4 == sz.stats and b.tok_lse.numel() * 4 == sz.tok_lse
+        assert b.stats.numel() * b.stats.element_size() == sz.stats and b.tok_lse.numel() * 4 == sz.tok_lse
         cb = SplaBuffers(b.k_cache.data_ptr(), b.v_cache.data_ptr(), b.stats.data_ptr(), b.rla_state.data_ptr(),
                          b.tok_lse.data_ptr(), b.seq_lens.data_ptr(), b.workspace.data_ptr(), sz.workspace)
         self.handle = C.c_void_p()

@@ -76,9 +76,16 @@ __device__ __forceinline__ void block_stats_core(const Params& p, int u, int blk
     float tot = 0.f;
 #pragma unroll
     for (int g2 = 0; g2 < TG; ++g2) tot += red_s[g2][c];
-    float* rec = p.stats + (WIN ? ((size_t)u * p.max_blocks + blk) * p.NW + w : (size_t)u * p.max_blocks + blk) * 2 * D;
-    rec[c] = mean;
-    rec[D + c] = tot / (float)cnt;
+    const size_t rec_off = (WIN ? ((size_t)u * p.max_blocks + blk) * p.NW + w : (size_t)u * p.max_blocks + blk) * 2 * D;
+    if (p.flags & kStatsBf16) {                      // 16-bit records: rounded once, here
+      __nv_bfloat16* rec = reinterpret_cast<__nv_bfloat16*>(p.stats) + rec_off;
+      rec[c] = __float2bfloat16_rn(mean);
+      rec[D + c] = __float2bfloat16_rn(tot / (float)cnt);
+    } else {
+      float* rec = p.stats + rec_off;
+      rec[c] = mean;
+      rec[D + c] = tot / (float)cnt;
+    }
   }
 }
 

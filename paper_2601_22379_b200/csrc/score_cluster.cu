@@ -84,11 +84,10 @@ __device__ __forceinline__ void group_reduce_multi(float (&v)[N], int lane) {
 }
 
 // Layout of the dynamic shared memory (identical in every CTA, which distributed shared memory relies on).
-template <int D, int GP>
+template <int D, int GP, typename ST>
 struct Smem {
-  static constexpr int kRecBytes = 2 * D * 4;
+  static constexpr int kRecBytes = 2 * D * (int)sizeof(ST);        // ST: element type of the statistics records
   static constexpr int kStageBytes = kStageRec * kRecBytes;
-  static constexpr int kRingBytes = kStages * kStageBytes;
   // after streaming the ring is dead and holds the selection's work arrays:
   static constexpr int kKeys = 0;                                   // uint32 [1024]        this CTA's block keys
   static constexpr int kCandKey = kKeys + 1024 * 4;                 // uint32 [16][64]      (the leader's copy is the live one)
@@ -98,8 +97,9 @@ struct Smem {
   static constexpr int kFlatIdx = kFlatKey + kMaxCluster * kMaxTopK * 4;
   static constexpr int kSelTmp = kFlatIdx + kMaxCluster * kMaxTopK * 4;    // int [64]
   static constexpr int kScratch = (kSelTmp + kMaxTopK * 4 + 15) / 16 * 16; // TopkScratch
-  static constexpr int kWorkEnd = kScratch + (int)sizeof(TopkScratch);
-  static_assert(kWorkEnd <= kRingBytes, "selection work arrays must fit in the dead ring");
+  static constexpr int kWorkEnd = (kScratch + (int)sizeof(TopkScratch) + 1023) / 1024 * 1024;
+  // the ring, padded where the work arrays need more than its stages
+  static constexpr int kRingBytes = kStages * kStageBytes > kWorkEnd ? kStages * kStageBytes : kWorkEnd;
   // fixed region after the ring:
   static constexpr int kPart = kRingBytes;                          // float [GP][2]  this CTA's (max, sum)
   static constexpr int kAllPart = kPart + GP * 2 * 4;               // float [16][GP][2]
@@ -117,11 +117,12 @@ struct Smem {
 // the blocks that were complete before that append (at most `pending_new` tokens per sequence) cannot change any
 // more, so their statistics are streamed while the append still runs; only then does the kernel wait for the
 // append, read the final length and take the few remaining blocks (those the append wrote to) from global memory.
-template <int D, int GP, bool WIN, bool EARLY>
+// ST: element type of the statistics records (float, or __nv_bfloat16 with half the bytes to stream).
+template <int D, int GP, bool WIN, bool EARLY, typename ST>
 __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Params p, const void* __restrict__ q_raw,
                                                                       int q_is_bf16, int* __restrict__ sel_user,
                                                                       int pending_new) {
-  using SM = Smem<D, GP>;
+  using SM = Smem<D, GP, ST>;
   constexpr int W = GP <= 4 ? 16 : 32;          // lanes that share one record
   constexpr int NGRP = 32 / W;                  // records a warp works on side by side
   constexpr int PASSES = UNR / NGRP;
@@ -206,7 +207,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   int n_my = nb_my * NW;                          // records of this CTA
   const int rec_begin = cta_blk0 * NW;            // (a CTA that has records starts at its share's first block)
   const int n_rounds = (n_stream + kStageRec - 1) / kStageRec;
-  const float* stats_u = p.stats + (size_t)u * p.max_blocks * NW * 2 * D;
+  const ST* stats_u = reinterpret_cast<const ST*>(p.stats) + (size_t)u * p.max_blocks * NW * 2 * D;
 
   auto issue = [&](int r) {                      // thread 0 only: one bulk copy fills stage r % kStages
     const int s = r % kStages;
@@ -299,7 +300,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
       const int s = r % kStages;
       if (!mbar_wait(&full[s], (r / kStages) & 1)) { if (lane == 0) atomicExch(&err_s, 1); break; }
       const int l0 = r * kStageRec + warp * UNR;                       // first record of this warp, CTA-local
-      const float* st = reinterpret_cast<const float*>(smem_raw + (size_t)s * SM::kStageBytes) + (size_t)(warp * UNR) * 2 * D;
+      const ST* st = reinterpret_cast<const ST*>(smem_raw + (size_t)s * SM::kStageBytes) + (size_t)(warp * UNR) * 2 * D;
       float mean[PASSES][VECW], var[PASSES][VECW];
 #pragma unroll
       for (int ps = 0; ps < PASSES; ++ps) {
@@ -349,7 +350,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
         __syncthreads();
         for (int base = 0; base < n_late; base += kStageRec) {
           const int l0 = n_stream + base + warp * UNR;
-          const float* st = reinterpret_cast<const float*>(smem_raw) + (size_t)(base + warp * UNR) * 2 * D;
+          const ST* st = reinterpret_cast<const ST*>(smem_raw) + (size_t)(base + warp * UNR) * 2 * D;
           float mean[PASSES][VECW], var[PASSES][VECW];
 #pragma unroll
           for (int ps = 0; ps < PASSES; ++ps) {
@@ -560,12 +561,12 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
     }
 }
 
-template <int D, int GP, bool WIN, bool EARLY>
+template <int D, int GP, bool WIN, bool EARLY, typename ST>
 static cudaError_t launch_win(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new, cudaStream_t stream) {
-  using SM = Smem<D, GP>;
+  using SM = Smem<D, GP, ST>;
   const int U = p.batch * p.Hkv;
   size_t smem = (size_t)SM::kEll + (size_t)p.G * p.chunk * sizeof(float);
-  auto kern = score_cluster_kernel<D, GP, WIN, EARLY>;
+  auto kern = score_cluster_kernel<D, GP, WIN, EARLY, ST>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   if (p.cs > 8) {
@@ -575,13 +576,19 @@ static cudaError_t launch_win(const Params& p, const void* q, int q_is_bf16, int
   return launch_ex(kern, dim3(p.cs, U, 1), dim3(kCsThreads, 1, 1), smem, stream, p.cs, true, p, q, q_is_bf16, sel_user, pending_new);
 }
 
+template <int D, int GP, typename ST>
+static cudaError_t launch_st(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new, cudaStream_t stream) {
+  if (pending_new > 0)
+    return p.NW > 1 ? launch_win<D, GP, true, true, ST>(p, q, q_is_bf16, sel_user, pending_new, stream)
+                    : launch_win<D, GP, false, true, ST>(p, q, q_is_bf16, sel_user, pending_new, stream);
+  return p.NW > 1 ? launch_win<D, GP, true, false, ST>(p, q, q_is_bf16, sel_user, 0, stream)
+                  : launch_win<D, GP, false, false, ST>(p, q, q_is_bf16, sel_user, 0, stream);
+}
+
 template <int D, int GP>
 static cudaError_t launch_one(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new, cudaStream_t stream) {
-  if (pending_new > 0)
-    return p.NW > 1 ? launch_win<D, GP, true, true>(p, q, q_is_bf16, sel_user, pending_new, stream)
-                    : launch_win<D, GP, false, true>(p, q, q_is_bf16, sel_user, pending_new, stream);
-  return p.NW > 1 ? launch_win<D, GP, true, false>(p, q, q_is_bf16, sel_user, 0, stream)
-                  : launch_win<D, GP, false, false>(p, q, q_is_bf16, sel_user, 0, stream);
+  return (p.flags & kStatsBf16) ? launch_st<D, GP, __nv_bfloat16>(p, q, q_is_bf16, sel_user, pending_new, stream)
+                                : launch_st<D, GP, float>(p, q, q_is_bf16, sel_user, pending_new, stream);
 }
 
 template <int D>

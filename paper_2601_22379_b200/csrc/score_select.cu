@@ -21,10 +21,16 @@ namespace {
 constexpr int UNR = 4;                                  // records per warp per round
 constexpr int kRound = (kScoreThreads / 32) * UNR;      // records per CTA per round (32)
 
+// One statistics record (mean, then variance; fp32 or bfloat16 elements) spread over a warp, VEC channels per lane.
 template <int VEC>
-__device__ __forceinline__ void load_record(const float* rec, int D, int lane, bool valid, float (&mean)[VEC],
-                                            float (&var)[VEC]) {
-  if (valid) {
+__device__ __forceinline__ void load_record(const float* stats, size_t rec_elem, bool rec_bf16, int D, int lane, bool valid,
+                                            float (&mean)[VEC], float (&var)[VEC]) {
+  if (valid && rec_bf16) {
+    const __nv_bfloat16* rec = reinterpret_cast<const __nv_bfloat16*>(stats) + rec_elem;
+    load_vec<VEC>(rec + lane * VEC, mean);
+    load_vec<VEC>(rec + D + lane * VEC, var);
+  } else if (valid) {
+    const float* rec = stats + rec_elem;
     if constexpr (VEC == 4) {
       const float4 a = __ldcs(reinterpret_cast<const float4*>(rec + lane * 4));
       const float4 b = __ldcs(reinterpret_cast<const float4*>(rec + D + lane * 4));
@@ -104,7 +110,8 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
   }
 
   const size_t ell_stride = (size_t)p.max_blocks * NW;
-  const float* stats_u = p.stats + (size_t)u * ell_stride * 2 * D;
+  const size_t stats_u = (size_t)u * ell_stride * 2 * D;      // first element of the unit's records
+  const bool rec_bf16 = (p.flags & kStatsBf16) != 0;
   float* ell_u = p.ell + (size_t)u * G * ell_stride;
   // After the warp reduction lanes 0..15 hold the mean dots and lanes 16..31 the variance dots, value index
   // lane / LPV, each replicated on LPV lanes.  Copy lane `sub` finalises record `sub` of the batch, so the
@@ -126,7 +133,7 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
 #pragma unroll
     for (int r = 0; r < UNR; ++r) {
       const int i = base + round * kRound + r;
-      load_record<VEC>(stats_u + (size_t)i * 2 * D, D, lane, i < nrec, mean[buf][r], var[buf][r]);
+      load_record<VEC>(p.stats, stats_u + (size_t)i * 2 * D, rec_bf16, D, lane, i < nrec, mean[buf][r], var[buf][r]);
     }
   };
   auto compute_round = [&](int round, int buf) {

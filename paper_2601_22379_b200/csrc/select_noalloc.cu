@@ -56,7 +56,7 @@ extern "C" int spla_select_blocks_noalloc(const spla_config_t* cfg, const float*
   spla_sizes_t sz;
   const int rc = spla_query_sizes(cfg, &sz);                 // validates the configuration (host only)
   if (rc != SPLA_OK) return rc;
-  if (cfg->window_size != 0) return SPLA_ERR_UNSUPPORTED;   // whole-block statistics only
+  if (cfg->window_size != 0 || (cfg->flags & SPLA_STATS_BF16)) return SPLA_ERR_UNSUPPORTED;   // whole-block fp32 statistics only
   if (((uintptr_t)stats % 16) || ((uintptr_t)q % 16) || ((uintptr_t)seq_lens % 4) || ((uintptr_t)sel_idx % 4))
     return SPLA_ERR_INVALID_ARG;
 

@@ -70,7 +70,7 @@ static int validate_config(const spla_config_t* c) {
   if ((c->kv_dtype != SPLA_F32 && c->kv_dtype != SPLA_BF16) || (c->q_dtype != SPLA_F32 && c->q_dtype != SPLA_BF16))
     return SPLA_ERR_INVALID_ARG;
   if (c->sm_scale < 0.f || c->phi_scale < 0.f || c->rms_eps < 0.f) return SPLA_ERR_INVALID_ARG;
-  if (c->flags & ~(SPLA_ADOPT_CONTENTS | SPLA_FIRST_ORDER | SPLA_NO_RLA | SPLA_GENERAL_KERNELS)) return SPLA_ERR_INVALID_ARG;
+  if (c->flags & ~(SPLA_ADOPT_CONTENTS | SPLA_FIRST_ORDER | SPLA_NO_RLA | SPLA_GENERAL_KERNELS | SPLA_STATS_BF16)) return SPLA_ERR_INVALID_ARG;
   const int G = c->n_q_heads / c->n_kv_heads;
   if (G > kMaxGroup) return SPLA_ERR_UNSUPPORTED;
   if (c->head_dim != 64 && c->head_dim != 128) return SPLA_ERR_UNSUPPORTED;
@@ -127,7 +127,7 @@ extern "C" int spla_query_sizes(const spla_config_t* config, spla_sizes_t* sizes
   const size_t e = config->kv_dtype == SPLA_BF16 ? 2 : 4;
   sizes_out->k_cache = U * max_blocks * B * d * e;
   sizes_out->v_cache = sizes_out->k_cache;
-  sizes_out->stats = U * max_blocks * windows_per_block(config) * 2 * d * 4;
+  sizes_out->stats = U * max_blocks * windows_per_block(config) * 2 * d * ((config->flags & SPLA_STATS_BF16) ? 2 : 4);
   sizes_out->rla_state = U * d * d * 4;
   sizes_out->tok_lse = U * max_blocks * B * 4;
   sizes_out->seq_lens = (size_t)config->batch * 4;
@@ -180,7 +180,7 @@ extern "C" int spla_init_cache(const spla_config_t* config, const spla_buffers_t
   p.win_s = config->window_size > 0 ? config->window_stride : config->block_size;
   p.flags = config->flags; p.kv_bf16 = config->kv_dtype == SPLA_BF16;
   p.sm_scale = c->cfg.sm_scale; p.phi_scale = c->cfg.phi_scale; p.rms_eps = c->cfg.rms_eps;
-  p.k_cache = b->k_cache; p.v_cache = b->v_cache; p.stats = b->stats; p.state = b->rla_state;
+  p.k_cache = b->k_cache; p.v_cache = b->v_cache; p.stats = reinterpret_cast<float*>(b->stats); p.state = b->rla_state;
   p.tok_lse = b->tok_lse; p.seq_lens = b->seq_lens;
   const WorkspaceLayout w = workspace_layout(config);
   char* ws = reinterpret_cast<char*>(b->workspace);

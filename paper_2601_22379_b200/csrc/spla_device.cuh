@@ -16,6 +16,7 @@ constexpr int kAttendThreads = 128;     // sparse-attend kernel: 4 warps per sel
 constexpr int kMaxGroup = 16;
 constexpr int kMaxWindows = 8;          // selection windows per block, at most
 constexpr int kMaxTopK = 64;
+constexpr unsigned kStatsBf16 = 16u;     // Params::flags bit: statistics records are bfloat16 (SPLA_STATS_BF16)
 constexpr int kMaxBlocks = 32768;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -34,7 +35,7 @@ struct Params {
   // caller buffers
   void* k_cache;
   void* v_cache;
-  float* stats;
+  float* stats;                         // fp32 records, or bfloat16 ones behind the same pointer (flags & kStatsBf16)
   float* state;
   float* tok_lse;
   int* seq_lens;

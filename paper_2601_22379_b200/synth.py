@@ -193,12 +193,13 @@ def step_kv(w: Workload, step: int, device="cpu"):
     return k.to(w.torch_dtype).to(device), v.to(w.torch_dtype).to(device)
 
 
-def algorithmic_bytes_per_step(w: Workload, lens=None, n_windows: int = 1) -> dict:
+def algorithmic_bytes_per_step(w: Workload, lens=None, n_windows: int = 1, stat_bytes: int = 4) -> dict:
     """Bytes one decode step must move, per the method's own accounting.
 
     Block statistics of every block + K and V of the selected blocks + the
     global RLA state, summed over units; next to the dense-decode KV footprint.
-    With strided selection windows every block carries `n_windows` statistics records.
+    With strided selection windows every block carries `n_windows` statistics records; `stat_bytes` is the size of
+    one statistics element (4: fp32, 2: the bfloat16 option).
     """
     lens = seq_lens(w) if lens is None else np.asarray(lens)
     e = 2 if w.kv_dtype == "bf16" else 4
@@ -206,7 +207,7 @@ def algorithmic_bytes_per_step(w: Workload, lens=None, n_windows: int = 1) -> di
     stats = sel = state = dense = 0
     for L in lens:
         nblk = -(-int(L) // B)
-        stats += H * nblk * n_windows * 2 * d * 4
+        stats += H * nblk * n_windows * 2 * d * stat_bytes
         sel += H * min(w.top_k, nblk) * B * d * 2 * e
         state += H * d * d * 4
         dense += H * int(L) * d * 2 * e

@@ -20,6 +20,11 @@ import torch
 from oracle import spla_oracle as O
 
 TIE_BAND = 1e-4
+# bfloat16 statistics: the library rounds an fp32 statistic, the oracle an fp64 one; where the two straddle a rounding
+# boundary the stored values differ by one unit in the last place (2^-7 relative), which moves that block's log mass
+# by up to 2^-7 |q_c mean_c| (or 2^-8 q_c^2 var_c): a few 1e-3 at most for the workloads here, and only for the
+# handful of records where it happens.
+TIE_BAND_STATS_BF16 = 5e-3
 STATE_TOL_FMA = 2e-6          # S_bar kept by the fp32 FMA kernels
 STATE_TOL_TENSOR = 4e-6       # S_bar after a bulk append on the tensor cores (bf16 cache, d = 128, >= 256 tokens)
 
@@ -34,7 +39,7 @@ def max_abs(a, b):
     return float(np.max(np.abs(np.asarray(a, dtype=np.float64) - np.asarray(b, dtype=np.float64)))) if np.size(a) else 0.0
 
 
-def check_selection(sel_gpu, oracle_res, top_k, n_sink, n_local):
+def check_selection(sel_gpu, oracle_res, top_k, n_sink, n_local, tie_band=TIE_BAND):
     """Returns True if identical, False if different but inside the tie band; raises otherwise."""
     sel_gpu = np.asarray(sel_gpu, dtype=np.int64)
     sel_ref = np.asarray(oracle_res["sel"], dtype=np.int64)
@@ -52,7 +57,7 @@ def check_selection(sel_gpu, oracle_res, top_k, n_sink, n_local):
     free_ref = sorted((i for i in r if i not in forced), key=lambda i: (-score[i], i))
     s_k = score[free_ref[-1]]
     for i in set(g) ^ set(r):
-        assert abs(score[i] - s_k) <= TIE_BAND * s_k, (
+        assert abs(score[i] - s_k) <= tie_band * s_k, (
             f"block {i} (oracle score {score[i]:.9g}) differs outside the tie band around {s_k:.9g}")
     return False
 
@@ -73,18 +78,19 @@ def check_outputs(name, got, want, kv_dtype, scale_floor=0.0):
 
 
 def oracle_unit(w, q_bhd, K_unit, V_unit, gamma, h, *, n_sink, n_local, override=None, order=2, use_rla=True,
-                window=None):
+                window=None, stats_bf16=False):
     G = w.group
     return O.decode_unit(
         q_bhd[h * G:(h + 1) * G].double().cpu().numpy(), K_unit.double().cpu().numpy(), V_unit.double().cpu().numpy(),
         gamma[h * G:(h + 1) * G].double().cpu().numpy(), block_size=w.block_size, top_k=w.top_k, n_sink=n_sink,
-        n_local=n_local, override_selection=override, order=order, use_rla=use_rla, window=window)
+        n_local=n_local, override_selection=override, order=order, use_rla=use_rla, window=window,
+        stats_bf16=stats_bf16)
 
 
-def compare_unit(w, res, out_gpu, osp_gpu, orla_gpu, sel_gpu, h, *, n_sink, n_local, rerun=None):
+def compare_unit(w, res, out_gpu, osp_gpu, orla_gpu, sel_gpu, h, *, n_sink, n_local, rerun=None, tie_band=TIE_BAND):
     """Compares one unit.  `rerun(override)` recomputes the oracle with the library's selection when needed."""
     G = w.group
-    same = check_selection(sel_gpu, res, w.top_k, n_sink, n_local)
+    same = check_selection(sel_gpu, res, w.top_k, n_sink, n_local, tie_band)
     if not same:
         res = rerun([int(i) for i in sel_gpu if i >= 0])
     sl = slice(h * G, (h + 1) * G)

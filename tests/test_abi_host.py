@@ -51,6 +51,11 @@ def test_query_sizes_follow_the_documented_layouts(lib):
                               max_context=131072 + 64, window_size=32, window_stride=16)
     assert win.n_windows == 3 and binding.query_sizes(win).stats == 3 * sz.stats
     assert binding.query_sizes(win).k_cache == sz.k_cache
+    # 16-bit statistics: half the bytes, everything else unchanged
+    half = binding.make_config(batch=4, n_q_heads=32, n_kv_heads=8, head_dim=128, block_size=64, top_k=32,
+                               max_context=131072 + 64, flags=binding.SPLA_STATS_BF16)
+    hs = binding.query_sizes(half)
+    assert hs.stats * 2 == sz.stats and hs.k_cache == sz.k_cache and hs.workspace == sz.workspace
 
 
 @pytest.mark.parametrize("kw,status", [
@@ -58,7 +63,7 @@ def test_query_sizes_follow_the_documented_layouts(lib):
     (dict(batch=0), binding.SPLA_ERR_INVALID_ARG),
     (dict(n_sink_blocks=20, n_local_blocks=20), binding.SPLA_ERR_INVALID_ARG),
     (dict(flags=64), binding.SPLA_ERR_INVALID_ARG),
-    (dict(flags=16), binding.SPLA_ERR_INVALID_ARG),
+    (dict(flags=32), binding.SPLA_ERR_INVALID_ARG),
     (dict(sm_scale=-1.0), binding.SPLA_ERR_INVALID_ARG),
     (dict(head_dim=96), binding.SPLA_ERR_UNSUPPORTED),
     (dict(block_size=48), binding.SPLA_ERR_UNSUPPORTED),

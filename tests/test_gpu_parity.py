@@ -24,6 +24,8 @@ def _decode_all(cache, w, q, gamma):
 
 def _check_units(w, cache, q, gamma, K, V, lens, units, n_sink, n_local, extra=None, order=2, use_rla=True,
                  window=None):
+    stats_bf16 = bool(cache.cfg.flags & binding.SPLA_STATS_BF16)
+    tie_band = parity.TIE_BAND_STATS_BF16 if stats_bf16 else parity.TIE_BAND
     """extra: optional dict (b,h) -> (K_tail, V_tail) of appended tokens."""
     out, osp, orla, sel = _decode_all(cache, w, q, gamma)
     n_exact = 0
@@ -36,10 +38,10 @@ def _check_units(w, cache, q, gamma, K, V, lens, units, n_sink, n_local, extra=N
 
         def run(override=None):
             return parity.oracle_unit(w, q[b], Ku, Vu, gamma, h, n_sink=n_sink, n_local=n_local, override=override,
-                                      order=order, use_rla=use_rla, window=window)
+                                      order=order, use_rla=use_rla, window=window, stats_bf16=stats_bf16)
         res = run()
         n_exact += parity.compare_unit(w, res, out[b], osp[b], orla[b], sel[b, h], h, n_sink=n_sink, n_local=n_local,
-                                       rerun=run)
+                                       rerun=run, tie_band=tie_band)
     return n_exact
 
 
@@ -197,8 +199,10 @@ def test_config2_gqa_32k_full_three_query_seeds():
                 assert set(nb[b, h].tolist()) <= set(sel[b, h].tolist())
 
 
-def _stepped_full(w, n_units, check_steps, window=None):
-    cache, K, V, lens = runner.build_cache(w, DEV, window=window)
+def _stepped_full(w, n_units, check_steps, window=None, flags=0):
+    cache, K, V, lens = runner.build_cache(w, DEV, window=window, flags=flags)
+    stats_bf16 = bool(flags & binding.SPLA_STATS_BF16)
+    tie_band = parity.TIE_BAND_STATS_BF16 if stats_bf16 else parity.TIE_BAND
     gamma = synth.gamma(w).to(DEV)
     gam = gamma.double().cpu().numpy()
     lens_h = lens.cpu().numpy()
@@ -223,9 +227,9 @@ def _stepped_full(w, n_units, check_steps, window=None):
         for (b, h), oc in orc.items():
             def run(override=None):
                 return oc.decode(qh[b, h * G:(h + 1) * G], gam[h * G:(h + 1) * G], top_k=w.top_k, n_sink=w.n_sink,
-                                 n_local=w.n_local, override_selection=override)
+                                 n_local=w.n_local, override_selection=override, stats_bf16=stats_bf16)
             parity.compare_unit(w, run(), out[b], osp[b], orla[b], sel[b, h], h, n_sink=w.n_sink, n_local=w.n_local,
-                                rerun=run)
+                                rerun=run, tie_band=tie_band)
     torch.cuda.synchronize()
     assert cache.sync_status() == 0
     assert torch.equal(cache.bufs.seq_lens.cpu(), torch.as_tensor(lens_h) + w.n_steps)
