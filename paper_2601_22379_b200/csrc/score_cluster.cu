@@ -29,6 +29,8 @@ constexpr int kStageRec = 32;                            // statistics records p
 constexpr int kStages = 3;
 constexpr int kMaxCluster = 16;
 constexpr int UNR = kStageRec / kCsConsumers;            // records per warp per stage (4)
+constexpr int kSlotRec = 16;                             // records per slot of the tensor-core streaming path
+static_assert(2 * kStages <= 8, "barrier area holds eight mbarriers");
 
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -63,6 +65,19 @@ __device__ __forceinline__ void lse_merge(float& m, float& s, float m2, float s2
   m = nm;
 }
 
+// Warp-level tensor-core product D += A B with fp32 accumulators.  Fragment layout (PTX ISA, mma.m16n8k16;
+// g = lane / 4, t = lane % 4): A rows g and g + 8, B column g, D rows g and g + 8 at columns 2t, 2t + 1.
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
 // Sums N per-lane values over aligned groups of W lanes (W = 16 or 32, N <= W a power of two) by halving:
 // afterwards v[0] of lane l holds the group total of the value with index (l % W) / (W / N).
 template <int N, int W>
@@ -88,6 +103,11 @@ template <int D, int GP, typename ST>
 struct Smem {
   static constexpr int kRecBytes = 2 * D * (int)sizeof(ST);        // ST: element type of the statistics records
   static constexpr int kStageBytes = kStageRec * kRecBytes;
+  // tensor-core streaming (groups of up to four heads): the ring is cut into slots of 16 records, one MMA tile each
+  static constexpr bool kMma = GP <= 4 && sizeof(ST) == 2;         // 16-bit records, groups of up to four heads
+  static constexpr int kSlotBytes = kSlotRec * kRecBytes;
+  static constexpr int kSlots = kCsConsumers;                      // one ring position per warp
+  static constexpr int kStreamBytes = kMma ? kSlots * kSlotBytes : kStages * kStageBytes;
   // after streaming the ring is dead and holds the selection's work arrays:
   static constexpr int kKeys = 0;                                   // uint32 [1024]        this CTA's block keys
   static constexpr int kCandKey = kKeys + 1024 * 4;                 // uint32 [16][64]      (the leader's copy is the live one)
@@ -99,14 +119,14 @@ struct Smem {
   static constexpr int kScratch = (kSelTmp + kMaxTopK * 4 + 15) / 16 * 16; // TopkScratch
   static constexpr int kWorkEnd = (kScratch + (int)sizeof(TopkScratch) + 1023) / 1024 * 1024;
   // the ring, padded where the work arrays need more than its stages
-  static constexpr int kRingBytes = kStages * kStageBytes > kWorkEnd ? kStages * kStageBytes : kWorkEnd;
+  static constexpr int kRingBytes = kStreamBytes > kWorkEnd ? kStreamBytes : kWorkEnd;
   // fixed region after the ring:
   static constexpr int kPart = kRingBytes;                          // float [GP][2]  this CTA's (max, sum)
   static constexpr int kAllPart = kPart + GP * 2 * 4;               // float [16][GP][2]
   static constexpr int kLse = kAllPart + kMaxCluster * GP * 2 * 4;  // float [GP]
   static constexpr int kWred = kLse + GP * 4;                       // float [8][GP][2]
-  static constexpr int kBars = (kWred + kCsConsumers * GP * 2 * 4 + 7) / 8 * 8;   // uint64 [2 * kStages]
-  static constexpr int kEll = (kBars + 2 * kStages * 8 + 15) / 16 * 16;            // float [G][chunk]
+  static constexpr int kBars = (kWred + kCsConsumers * GP * 2 * 4 + 7) / 8 * 8;   // uint64 [8]: full / empty, or one per slot
+  static constexpr int kEll = (kBars + 8 * 8 + 15) / 16 * 16;                      // float [G][chunk]
 };
 
 }  // namespace
@@ -149,8 +169,14 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   float* ell_s = reinterpret_cast<float*>(smem_raw + SM::kEll);          // [G][chunk] log mass per block
   __shared__ int err_s;
 
+  const int chunk = p.chunk;                      // blocks per CTA
+  const int NW = WIN ? p.NW : 1;                  // selection windows per block; a "record" is one window
+  const int cta_blk0 = rank * chunk;              // first block of this CTA's share
+  const int rec_begin = cta_blk0 * NW;            // (a CTA that has records starts at its share's first block)
+  const ST* stats_u = reinterpret_cast<const ST*>(p.stats) + (size_t)u * p.max_blocks * NW * 2 * D;
   if (tid == 0) {                               // nothing here depends on the preceding kernel
-    for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kCsConsumers); }
+    if constexpr (SM::kMma) { for (int s = 0; s < SM::kSlots; ++s) mbar_init(&full[s], 1); }
+    else { for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kCsConsumers); } }
     err_s = 0;
   }
   SPLA_MARK(p, blockIdx.y, 30, 0);
@@ -165,9 +191,54 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   const int hl = lane % W, grp = lane / W;
   constexpr int CW = VECW >= 4 ? 4 : VECW;      // floats per vector load
   constexpr int NC = VECW / CW;
+  // Tensor-core streaming (16-bit records, groups of up to four heads): a slot of 16 records is the A operand of
+  // mma.m16n8k16 (16 x d, row-major, as stored), the B operand's eight columns are the group's scaled queries, each
+  // split in two bf16 parts, bf16(q) and bf16(q - bf16(q)) (column n: head n / 2, part n % 2), whose products are
+  // added after the MMA: the query enters with 16 significant bits, the statistics exactly, the sums are fp32.
+  // Thread (g8, t4) owns 16 consecutive bytes of every 64 of a record half (mean or variance), which it fetches with
+  // one 128-bit load per row; the k index inside an MMA is a permutation of the channels, the same for A and B.
+  constexpr bool MMA = SM::kMma;
+  constexpr int NJ = D * (int)sizeof(ST) / 64;   // 16-byte chunks per thread and record half
+  const int g8 = lane >> 2, t4 = lane & 3;
+  uint32_t bq[MMA ? NJ : 1][4], bv[MMA ? NJ : 1][4];
+  if constexpr (MMA) {
+    const int head = g8 >> 1, part = g8 & 1;
+#pragma unroll
+    for (int j = 0; j < NJ; ++j) {
+      float x[8];                                // channels 32 j + 8 t4 .. + 7
+      if (head < G) {
+        const size_t qoff = ((size_t)b * p.Hq + (size_t)h * G + head) * D + (size_t)j * 32 + t4 * 8;
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          float y[4];
+          if (q_is_bf16) load_vec<4>(reinterpret_cast<const __nv_bfloat16*>(q_raw) + qoff + c * 4, y);
+          else load_vec<4>(reinterpret_cast<const float*>(q_raw) + qoff + c * 4, y);
+#pragma unroll
+          for (int v = 0; v < 4; ++v) x[c * 4 + v] = y[v];
+        }
+      } else {
+#pragma unroll
+        for (int v = 0; v < 8; ++v) x[v] = 0.f;
+      }
+      float qa[8], qb2[8];                       // this thread's part of q_hat and of q_hat^2 / 2
+#pragma unroll
+      for (int v = 0; v < 8; ++v) {
+        const float qh = x[v] * p.sm_scale;
+        const float qq = (p.flags & 2u) ? 0.f : 0.5f * qh * qh;
+        const float h1 = __bfloat162float(__float2bfloat16_rn(qh)), h2 = __bfloat162float(__float2bfloat16_rn(qq));
+        qa[v] = part ? qh - h1 : h1;
+        qb2[v] = part ? qq - h2 : h2;
+      }
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        bq[j][v] = pack_bf16(qa[2 * v], qa[2 * v + 1]);
+        bv[j][v] = pack_bf16(qb2[2 * v], qb2[2 * v + 1]);
+      }
+    }
+  }
   float qm[GP][VECW], qv[GP][VECW];
 #pragma unroll
-  for (int g = 0; g < GP; ++g) {
+  for (int g = 0; g < GP && !MMA; ++g) {
     if (g < G) {
       const size_t qrow = ((size_t)b * p.Hq + (size_t)h * G + g) * D;
 #pragma unroll
@@ -197,17 +268,12 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   }
   int L = L0;
   int nblk = (L + p.B - 1) / p.B;
-  const int chunk = p.chunk;                      // blocks per CTA
-  const int NW = WIN ? p.NW : 1;                  // selection windows per block; a "record" is one window
-  const int cta_blk0 = rank * chunk;              // first block of this CTA's share
   const int nblk_stream = EARLY ? max(0, L0 - pending_new) / p.B : nblk;    // blocks whose records the ring may fetch
   const int n_stream = max(0, min(cta_blk0 + chunk, nblk_stream) - cta_blk0) * NW;
   int blk_begin = min(nblk, cta_blk0);
   int nb_my = min(nblk, blk_begin + chunk) - blk_begin;   // blocks of this CTA (EARLY: refreshed after the wait)
   int n_my = nb_my * NW;                          // records of this CTA
-  const int rec_begin = cta_blk0 * NW;            // (a CTA that has records starts at its share's first block)
   const int n_rounds = (n_stream + kStageRec - 1) / kStageRec;
-  const ST* stats_u = reinterpret_cast<const ST*>(p.stats) + (size_t)u * p.max_blocks * NW * 2 * D;
 
   auto issue = [&](int r) {                      // thread 0 only: one bulk copy fills stage r % kStages
     const int s = r % kStages;
@@ -216,11 +282,23 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
     mbar_expect_tx(&full[s], bytes);
     bulk_g2s(smem_raw + (size_t)s * SM::kStageBytes, stats_u + (size_t)(rec_begin + r * kStageRec) * 2 * D, bytes, &full[s]);
   };
-  if (tid == 0)
-    for (int r = 0; r < min(kStages, n_rounds); ++r) issue(r);
+  // tensor-core path: slot r (16 records) goes to ring position r % kSlots and is consumed by the warp of that
+  // number, which then refills its position itself with slot r + kSlots (so every warp sees the phases of its
+  // barrier in order)
+  const int n_slots = (n_stream + kSlotRec - 1) / kSlotRec;
+  auto issue_slot = [&](int r) {                // one thread
+    const int pos = r % SM::kSlots;
+    const uint32_t bytes = (uint32_t)min(kSlotRec, n_stream - r * kSlotRec) * SM::kRecBytes;
+    mbar_expect_tx(&full[pos], bytes);
+    bulk_g2s(smem_raw + (size_t)pos * SM::kSlotBytes, stats_u + (size_t)(rec_begin + r * kSlotRec) * 2 * D, bytes, &full[pos]);
+  };
+  if (tid == 0) {
+    if constexpr (MMA) { for (int r = 0; r < min(SM::kSlots, n_slots); ++r) issue_slot(r); }
+    else { for (int r = 0; r < min(kStages, n_rounds); ++r) issue(r); }
+  }
   SPLA_MARK(p, u, rank, 0);
 #pragma unroll
-  for (int g = 0; g < GP; ++g) {
+  for (int g = 0; g < GP && !MMA; ++g) {
 #pragma unroll
     for (int v = 0; v < VECW; ++v) {
       qm[g][v] *= p.sm_scale;
@@ -247,6 +325,60 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
     const float ln_win = logf((float)p.win_C);
     const unsigned nw_magic = 0xffffffffu / (unsigned)NW + 1u;   // floor(x / NW) = umulhi(x, magic) for x < 2^16, NW <= 8
     float run_max = -INFINITY, run_sum = 0.f;
+
+    // Tensor-core path: one slot of 16 records -> dots of head t4 with records g8 and g8 + 8 of the slot -> log
+    // masses.  `li0` is the CTA-local index of the slot's first record, `limit` the number of local records that
+    // exist for this call.  Rows past the limit hold stale bytes; every row is independent and theirs are dropped.
+    auto consume_slot = [&](const unsigned char* slot, int li0, int limit) {
+      float cm[4] = {0.f, 0.f, 0.f, 0.f}, cv[4] = {0.f, 0.f, 0.f, 0.f};
+      const unsigned char* r0 = slot + (size_t)g8 * SM::kRecBytes + t4 * 16;
+      const unsigned char* r1 = r0 + 8 * SM::kRecBytes;
+      constexpr int HALF = SM::kRecBytes / 2;                      // the variance follows the mean
+#pragma unroll
+      for (int j = 0; j < (MMA ? NJ : 0); ++j) {
+        const uint4 m0 = *reinterpret_cast<const uint4*>(r0 + j * 64), m1 = *reinterpret_cast<const uint4*>(r1 + j * 64);
+        const uint4 v0 = *reinterpret_cast<const uint4*>(r0 + HALF + j * 64), v1 = *reinterpret_cast<const uint4*>(r1 + HALF + j * 64);
+        mma_bf16(cm, m0.x, m1.x, m0.y, m1.y, bq[j][0], bq[j][1]);
+        mma_bf16(cv, v0.x, v1.x, v0.y, v1.y, bv[j][0], bv[j][1]);
+        mma_bf16(cm, m0.z, m1.z, m0.w, m1.w, bq[j][2], bq[j][3]);
+        mma_bf16(cv, v0.z, v1.z, v0.w, v1.w, bv[j][2], bv[j][3]);
+      }
+      // columns 2 t4 and 2 t4 + 1 are the two query parts of head t4
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        const float dm = cm[2 * hf] + cm[2 * hf + 1], dv = cv[2 * hf] + cv[2 * hf + 1];
+        const int li = li0 + g8 + 8 * hf;
+        if (t4 < G && li < limit) {
+          if (!WIN) {
+            const float ell = (rec_begin + li == nblk_fin - 1 ? ln_last : ln_full) + dm + __logf(1.f + dv);
+            ell_s[t4 * chunk + li] = ell;
+            const float nm = fmaxf(run_max, ell);
+            run_sum = run_sum * __expf(run_max - nm) + __expf(ell - nm);
+            run_max = nm;
+          } else {
+            // strided windows (Section 3.1, "Strided Block Selection"): log mass of window w of a block,
+            // max-pooled into the block's slot right away through an order-preserving integer key
+            const int lb = (int)__umulhi((unsigned)li, nw_magic), w = li - lb * NW;   // li / NW without a division
+            float ln_n = ln_win;
+            if (cta_blk0 + lb == nblk_fin - 1) {
+              const int cnt = min(p.win_C, n_last - w * p.win_s);
+              ln_n = cnt > 0 ? logf((float)cnt) : -INFINITY;
+            }
+            atomicMax(reinterpret_cast<uint32_t*>(ell_s) + t4 * chunk + lb, float_order_key(ln_n + dm + __logf(1.f + dv)));
+          }
+        }
+      }
+    };
+    if constexpr (MMA) {
+#pragma unroll 1
+      for (int r = warp; r < n_slots; r += SM::kSlots) {          // warp w owns ring position w
+        const int pos = r % SM::kSlots;
+        if (!mbar_wait(&full[pos], (r / SM::kSlots) & 1)) { if (lane == 0) atomicExch(&err_s, 1); break; }
+        consume_slot(smem_raw + (size_t)pos * SM::kSlotBytes, r * kSlotRec, n_stream);
+        __syncwarp();                                              // every lane has its operands: the slot is free
+        if (lane == 0 && r + SM::kSlots < n_slots) issue_slot(r + SM::kSlots);
+      }
+    }
 
     // dots of the records a warp holds in registers -> log masses (and, with whole blocks, the running normaliser);
     // `limit` is the number of local records that exist for this call
@@ -296,7 +428,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
         }
     };
 #pragma unroll 1
-    for (int r = 0; r < n_rounds; ++r) {
+    for (int r = 0; r < (MMA ? 0 : n_rounds); ++r) {
       const int s = r % kStages;
       if (!mbar_wait(&full[s], (r / kStages) & 1)) { if (lane == 0) atomicExch(&err_s, 1); break; }
       const int l0 = r * kStageRec + warp * UNR;                       // first record of this warp, CTA-local
@@ -348,7 +480,10 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
         const float4* src = reinterpret_cast<const float4*>(stats_u + (size_t)(rec_begin + n_stream) * 2 * D);
         for (int x = tid; x < n_late * (SM::kRecBytes / 16); x += kCsThreads) dst[x] = __ldcg(src + x);
         __syncthreads();
-        for (int base = 0; base < n_late; base += kStageRec) {
+        if constexpr (MMA)
+          for (int base = warp * kSlotRec; base < n_late; base += kCsConsumers * kSlotRec)
+            consume_slot(smem_raw + (size_t)base * SM::kRecBytes, n_stream + base, n_my);
+        for (int base = 0; base < (MMA ? 0 : n_late); base += kStageRec) {
           const int l0 = n_stream + base + warp * UNR;
           const ST* st = reinterpret_cast<const ST*>(smem_raw) + (size_t)(base + warp * UNR) * 2 * D;
           float mean[PASSES][VECW], var[PASSES][VECW];
@@ -395,17 +530,29 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
         if (lane == 0) { wred[(warp * GP + g) * 2 + 0] = m; wred[(warp * GP + g) * 2 + 1] = sm; }
       }
     }
+    if constexpr (MMA) {
+      // lanes with the same t4 hold partial normalisers of head t4: fold over g8
+#pragma unroll
+      for (int o = 4; o < 32; o <<= 1) {
+        const float m2 = __shfl_xor_sync(0xffffffffu, run_max, o), s2 = __shfl_xor_sync(0xffffffffu, run_sum, o);
+        lse_merge(run_max, run_sum, m2, s2);
+      }
+      if (!WIN && lane < G) {
+        wred[(warp * GP + lane) * 2 + 0] = run_max;
+        wred[(warp * GP + lane) * 2 + 1] = run_sum;
+      }
+    }
     // fold the finalising lanes of a head: copy lanes (xor < LPV), then the record groups of the warp (xor W)
 #pragma unroll
-    for (int o = 1; o < FB; o <<= 1) {
+    for (int o = 1; o < (MMA ? 0 : FB); o <<= 1) {
       const float m2 = __shfl_xor_sync(0xffffffffu, run_max, o), s2 = __shfl_xor_sync(0xffffffffu, run_sum, o);
       lse_merge(run_max, run_sum, m2, s2);
     }
-    if constexpr (NGRP == 2) {
+    if constexpr (NGRP == 2 && !MMA) {
       const float m2 = __shfl_xor_sync(0xffffffffu, run_max, 16), s2 = __shfl_xor_sync(0xffffffffu, run_sum, 16);
       lse_merge(run_max, run_sum, m2, s2);
     }
-    if (!WIN && fin_lane && sub == 0 && grp == 0) {
+    if (!MMA && !WIN && fin_lane && sub == 0 && grp == 0) {
       wred[(warp * GP + my_g) * 2 + 0] = run_max;
       wred[(warp * GP + my_g) * 2 + 1] = run_sum;
     }
