@@ -667,22 +667,76 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   uint32_t* flat_key = reinterpret_cast<uint32_t*>(smem_raw + SM::kFlatKey);
   int* flat_idx = reinterpret_cast<int*>(smem_raw + SM::kFlatIdx);
   int* sel_tmp = reinterpret_cast<int*>(smem_raw + SM::kSelTmp);
-  int total = 0;
-  for (int c = tid; c < CS * kMaxTopK; c += kCsThreads) {              // compact the table: slot s of CTA r
-    const int r = c / kMaxTopK, sl = c % kMaxTopK;
+  // Lower bounds of the k_eff-th best key, so that most of the table drops out before any ranking: with n_full
+  // CTAs that sent a full list of k_eff candidates, the q-th best key of each of them, q = ceil(k_eff / n_full), has
+  // at least k_eff candidates at or above the smallest of these q-th best keys.
+  uint32_t* list_min = reinterpret_cast<uint32_t*>(scratch->hist);      // [kMaxCluster] per-list bound, then the survivor counter
+  int* n_surv = scratch->hist + kMaxCluster;
+  int n_full = 0;
+  for (int r = 0; r < CS; ++r) n_full += cand_cnt[r] == k_eff;
+  const int quota = n_full > 0 ? (k_eff + n_full - 1) / n_full : 0;
+  for (int r = warp; r < CS; r += kCsConsumers) {
+    const int cnt = cand_cnt[r];
+    uint32_t v0 = lane < cnt ? cand_key[r * kMaxTopK + lane] : 0u;
+    uint32_t v1 = lane + 32 < cnt ? cand_key[r * kMaxTopK + lane + 32] : 0u;
+    uint32_t m = 0xffffffffu;                                           // "no bound from this list" for the minimum below
+    if (cnt == k_eff && quota <= 8) {
+      for (int round = 0; round < quota; ++round) {                     // knock the largest out, quota times
+        m = __reduce_max_sync(0xffffffffu, max(v0, v1));
+        const uint32_t in0 = __ballot_sync(0xffffffffu, v0 == m);
+        const uint32_t in1 = __ballot_sync(0xffffffffu, v1 == m);
+        if (in0) { if (lane == __ffs(in0) - 1) v0 = 0u; }
+        else if (lane == __ffs(in1) - 1) v1 = 0u;
+      }
+    }
+    if (lane == 0) list_min[r] = m;
+  }
+  if (tid == 0) *n_surv = 0;
+  __syncthreads();
+  uint32_t bound = 0xffffffffu;
+  for (int r = 0; r < CS; ++r) bound = min(bound, list_min[r]);
+  if (bound == 0xffffffffu) bound = 0u;                                 // no full list, or too large a quota: keep all
+  for (int c0 = 0; c0 < CS * kMaxTopK; c0 += kCsThreads) {             // the survivors, in no particular order
+    const int c = c0 + tid, r = c / kMaxTopK, sl = c % kMaxTopK;
+    const bool live = c < CS * kMaxTopK && sl < cand_cnt[r] && cand_key[c] >= bound;
+    const uint32_t vote = __ballot_sync(0xffffffffu, live);
     int base = 0;
-    for (int r2 = 0; r2 < r; ++r2) base += cand_cnt[r2];
-    if (sl < cand_cnt[r]) {
-      flat_key[base + sl] = cand_key[c];
-      flat_idx[base + sl] = cand_idx[c];
+    if (lane == 0 && vote) base = atomicAdd(n_surv, __popc(vote));
+    base = __shfl_sync(0xffffffffu, base, 0);
+    if (live) {
+      const int dst = base + __popc(vote & ((1u << lane) - 1u));
+      flat_key[dst] = cand_key[c];
+      flat_idx[dst] = cand_idx[c];
     }
   }
-  for (int r = 0; r < CS; ++r) total += cand_cnt[r];
+  __syncthreads();
+  const int total = *n_surv;
   auto keep = [&](int slot, uint32_t, int idx) { sel_tmp[slot] = idx; };
   auto flat_of = [&](int c) { return flat_idx[c]; };
-  __syncthreads();
-  topk_prepare(flat_key, total, flat_of, keep, scratch);
-  select_topk(flat_key, total, k_eff, flat_of, keep, scratch);
+  SPLA_MARK(p, u, 31, 0);
+  if (total <= 2 * kCsThreads) {
+    // few survivors (the usual case): every thread ranks its candidates against all others by counting, reading the
+    // table with broadcast 128-bit loads; no shared-memory atomics, one barrier
+    if (tid < 4) { flat_key[total + tid] = 0u; flat_idx[total + tid] = 0x7fffffff; }   // padding that precedes nothing
+    __syncthreads();
+    for (int c = tid; c < total; c += kCsThreads) {
+      const uint32_t a = flat_key[c];
+      const int ia = flat_idx[c];
+      int rk = 0;
+      for (int j = 0; j < total; j += 4) {
+        const uint4 kk = *reinterpret_cast<const uint4*>(flat_key + j);
+        const int4 ii = *reinterpret_cast<const int4*>(flat_idx + j);
+        rk += pair_before(kk.x, ii.x, a, ia) + pair_before(kk.y, ii.y, a, ia) + pair_before(kk.z, ii.z, a, ia) +
+              pair_before(kk.w, ii.w, a, ia);
+      }
+      if (rk < k_eff) sel_tmp[rk] = ia;
+    }
+    __syncthreads();
+  } else {
+    topk_prepare(flat_key, total, flat_of, keep, scratch);
+    select_topk(flat_key, total, k_eff, flat_of, keep, scratch);
+  }
+  SPLA_MARK(p, u, 31, 2);
 
   int* sel_u = p.sel + (size_t)u * p.top_k;
   int* sel_o = sel_user ? sel_user + (size_t)u * p.top_k : nullptr;
