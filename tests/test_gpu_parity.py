@@ -474,3 +474,30 @@ def test_decode_into_pinned_host_memory_equals_decode_into_device_memory():
     torch.cuda.synchronize()
     assert cache.sync_status() == 0
     assert torch.equal(host_out, dev_out.cpu())
+
+
+@pytest.mark.parametrize("ctx,top_k,flags", [
+    (64 * 700 + 10, 16, 0),                                # cluster kernel, few candidates: ranked by counting
+    (64 * 2500, 64, 0),                                    # 16 CTAs x 64 candidates, all equal: the histogram path
+    (64 * 700 + 10, 16, binding.SPLA_STATS_BF16),          # tensor-core score path
+    (64 * 300, 16, binding.SPLA_GENERAL_KERNELS),
+])
+def test_equal_scores_select_the_lowest_block_indices(ctx, top_k, flags):
+    """Every block holds the same keys, so all full blocks score exactly the same: the selection is decided by the
+    tie rule alone (score descending, then block index ascending) after the forced sink and local blocks."""
+    w = synth.BY_NAME["gqa_32k"].scaled(batch=1, context=ctx, n_needles=0, top_k=top_k)
+    K, V, lens = runner.generate_prefill(w, DEV)
+    K = K[:, :, :w.block_size].repeat(1, 1, -(-ctx // w.block_size), 1)[:, :, :ctx].contiguous()
+    cache, _, _, _ = runner.build_cache(w, DEV, prefill=(K, V, lens), flags=flags)
+    gamma = synth.gamma(w).to(DEV)
+    q = synth.step_queries(w, 0, DEV)
+    out, osp, orla, sel = _decode_all(cache, w, q, gamma)
+    nblk = -(-ctx // w.block_size)
+    n_free = top_k - w.n_sink - w.n_local
+    want = sorted(set(range(w.n_sink)) | set(range(nblk - w.n_local, nblk)) | set(range(w.n_sink, w.n_sink + n_free)))
+    for h in range(w.n_kv_heads):
+        assert sel[0, h].tolist() == want
+    res = parity.oracle_unit(w, q[0], K[0, 0], V[0, 0], gamma, 0, n_sink=w.n_sink, n_local=w.n_local,
+                             stats_bf16=bool(flags & binding.SPLA_STATS_BF16))
+    assert res["sel"].tolist() == want
+    parity.check_outputs("out", out[0, :w.group], res["out"], w.kv_dtype)
