@@ -34,7 +34,7 @@ L2_BYTES = 126 * 1024 * 1024
 GRAPH_STEPS = 64
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the score kernel from the ncu capture summarised in
 # profiles/score_cluster_kernel_long_128k.md (69.37 MB read + 0.66 MB written)
-NCU_TRAFFIC = {"long_128k": 70.03e6, "long_128k+windows(C=32,s=16)": 208.8e6}
+NCU_TRAFFIC = {"long_128k": 70.00e6, "long_128k+windows(C=32,s=16)": 208.8e6, "long_128k+stats_bf16": 35.79e6}
 
 
 # ------------------------------------------------------------------------------------------------------------

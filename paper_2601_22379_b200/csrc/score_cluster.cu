@@ -667,20 +667,27 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   uint32_t* flat_key = reinterpret_cast<uint32_t*>(smem_raw + SM::kFlatKey);
   int* flat_idx = reinterpret_cast<int*>(smem_raw + SM::kFlatIdx);
   int* sel_tmp = reinterpret_cast<int*>(smem_raw + SM::kSelTmp);
-  // Lower bounds of the k_eff-th best key, so that most of the table drops out before any ranking: with n_full
-  // CTAs that sent a full list of k_eff candidates, the q-th best key of each of them, q = ceil(k_eff / n_full), has
-  // at least k_eff candidates at or above the smallest of these q-th best keys.
-  uint32_t* list_min = reinterpret_cast<uint32_t*>(scratch->hist);      // [kMaxCluster] per-list bound, then the survivor counter
-  int* n_surv = scratch->hist + kMaxCluster;
+  // Two lower bounds of the k_eff-th best key, so that most of the table drops out before any ranking.  With n_full
+  // CTAs that sent a full list of k_eff candidates: (a) the smallest key of any one full list (that list alone holds
+  // k_eff keys from there upwards: good when one part of the sequence dominates); (b) the smallest, over the full
+  // lists, of each list's q-th best key, q = ceil(k_eff / n_full) (n_full q >= k_eff keys lie at or above it: good
+  // when the lists look alike).  The larger of the two is used.
+  uint32_t* list_min = reinterpret_cast<uint32_t*>(scratch->hist);      // [kMaxCluster] bound (a) per list
+  uint32_t* list_qth = list_min + kMaxCluster;                          // [kMaxCluster] q-th best per list
+  int* n_surv = scratch->hist + 2 * kMaxCluster;                        // survivor counter
   int n_full = 0;
   for (int r = 0; r < CS; ++r) n_full += cand_cnt[r] == k_eff;
   const int quota = n_full > 0 ? (k_eff + n_full - 1) / n_full : 0;
   for (int r = warp; r < CS; r += kCsConsumers) {
     const int cnt = cand_cnt[r];
-    uint32_t v0 = lane < cnt ? cand_key[r * kMaxTopK + lane] : 0u;
-    uint32_t v1 = lane + 32 < cnt ? cand_key[r * kMaxTopK + lane + 32] : 0u;
+    const bool is_full = cnt == k_eff;
+    uint32_t v0 = lane < cnt ? cand_key[r * kMaxTopK + lane] : (is_full ? 0xffffffffu : 0u);
+    uint32_t v1 = lane + 32 < cnt ? cand_key[r * kMaxTopK + lane + 32] : (is_full ? 0xffffffffu : 0u);
+    const uint32_t lmin = __reduce_min_sync(0xffffffffu, min(v0, v1));  // (the padding of a full list is neutral here)
+    if (lane >= cnt) v0 = 0u;
+    if (lane + 32 >= cnt) v1 = 0u;
     uint32_t m = 0xffffffffu;                                           // "no bound from this list" for the minimum below
-    if (cnt == k_eff && quota <= 8) {
+    if (is_full && quota <= 8) {
       for (int round = 0; round < quota; ++round) {                     // knock the largest out, quota times
         m = __reduce_max_sync(0xffffffffu, max(v0, v1));
         const uint32_t in0 = __ballot_sync(0xffffffffu, v0 == m);
@@ -689,13 +696,14 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
         else if (lane == __ffs(in1) - 1) v1 = 0u;
       }
     }
-    if (lane == 0) list_min[r] = m;
+    if (lane == 0) { list_min[r] = is_full ? lmin : 0u; list_qth[r] = m; }
   }
   if (tid == 0) *n_surv = 0;
   __syncthreads();
-  uint32_t bound = 0xffffffffu;
-  for (int r = 0; r < CS; ++r) bound = min(bound, list_min[r]);
-  if (bound == 0xffffffffu) bound = 0u;                                 // no full list, or too large a quota: keep all
+  uint32_t bound_a = 0u, bound_b = 0xffffffffu;
+  for (int r = 0; r < CS; ++r) { bound_a = max(bound_a, list_min[r]); bound_b = min(bound_b, list_qth[r]); }
+  if (bound_b == 0xffffffffu) bound_b = 0u;                             // no full list, or too large a quota
+  const uint32_t bound = max(bound_a, bound_b);
   for (int c0 = 0; c0 < CS * kMaxTopK; c0 += kCsThreads) {             // the survivors, in no particular order
     const int c = c0 + tid, r = c / kMaxTopK, sl = c % kMaxTopK;
     const bool live = c < CS * kMaxTopK && sl < cand_cnt[r] && cand_key[c] >= bound;
@@ -714,7 +722,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   auto keep = [&](int slot, uint32_t, int idx) { sel_tmp[slot] = idx; };
   auto flat_of = [&](int c) { return flat_idx[c]; };
   SPLA_MARK(p, u, 31, 0);
-  if (total <= 2 * kCsThreads) {
+  if (total <= kCsThreads) {
     // few survivors (the usual case): every thread ranks its candidates against all others by counting, reading the
     // table with broadcast 128-bit loads; no shared-memory atomics, one barrier
     if (tid < 4) { flat_key[total + tid] = 0u; flat_idx[total + tid] = 0x7fffffff; }   // padding that precedes nothing
