@@ -154,3 +154,60 @@ def test_noalloc_entry_rejects_bf16_statistics():
         ctypes.byref(cfg), cache.bufs.stats.data_ptr(), cache.bufs.seq_lens.data_ptr(), q.data_ptr(),
         cache.new_sel_buffer().data_ptr(), None, None)          # rejected on the host: nothing is launched
     assert rc == binding.SPLA_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("hq,hkv", [(1, 1), (2, 1), (3, 1), (5, 1), (8, 1), (16, 1), (6, 2)])
+def test_bf16_statistics_group_sizes(hq, hkv):
+    """Groups of 1-4 heads take the tensor-core score path (unused B columns are zero), 5-8 the FMA path of the
+    cluster kernel, 16 the general kernel."""
+    w = synth.BY_NAME["gqa_32k"].scaled(batch=1, n_q_heads=hq, n_kv_heads=hkv, context=64 * 40 + 3, n_needles=3)
+    cache, K, V, lens = runner.build_cache(w, DEV, flags=F16)
+    gamma = synth.gamma(w).to(DEV)
+    q = synth.step_queries(w, 0, DEV)
+    _check_units(w, cache, q, gamma, K, V, lens.cpu().numpy(), _all_units(w), w.n_sink, w.n_local)
+
+
+@pytest.mark.parametrize("B,d,dt", [(16, 64, "bf16"), (32, 128, "f32"), (128, 64, "f32"), (128, 128, "bf16"), (64, 64, "bf16")])
+@pytest.mark.parametrize("window", [None, "half"])
+def test_bf16_statistics_block_sizes_head_dims_dtypes(B, d, dt, window):
+    w = synth.BY_NAME["gqa_32k"].scaled(batch=1, n_q_heads=4, n_kv_heads=2, head_dim=d, block_size=B, kv_dtype=dt,
+                                       context=B * 33 + B // 2, n_needles=2, top_k=8, n_outlier_channels=2)
+    win = (B // 2, B // 4) if window else None
+    cache, K, V, lens = runner.build_cache(w, DEV, flags=F16, window=win)
+    gamma = synth.gamma(w).to(DEV)
+    q = synth.step_queries(w, 0, DEV)
+    _check_units(w, cache, q, gamma, K, V, lens.cpu().numpy(), _all_units(w), w.n_sink, w.n_local, window=win)
+
+
+def test_bf16_statistics_steps_across_block_boundaries_every_unit():
+    """Append one token then decode, 70 steps (more than a block), every unit checked at every eighth step: the
+    one-call step with the early-starting tensor-core score kernel."""
+    w = synth.BY_NAME["long_128k"].scaled(batch=2, context=64 * 30 + 40, n_steps=70)
+    cache, K, V, lens = runner.build_cache(w, DEV, flags=F16)
+    gamma = synth.gamma(w).to(DEV)
+    lens_h = lens.cpu().numpy()
+    extra = {u: (torch.zeros(0, w.head_dim, dtype=w.torch_dtype, device=DEV),) * 2 for u in _all_units(w)}
+    cfg = cache.cfg
+    for step in range(w.n_steps):
+        k1, v1 = synth.step_kv(w, step, DEV)
+        q = synth.step_queries(w, step, DEV)
+        for (b, h) in extra:
+            extra[(b, h)] = (torch.cat([extra[(b, h)][0], k1[b, h]]), torch.cat([extra[(b, h)][1], v1[b, h]]))
+        sel = cache.new_sel_buffer()
+        osp = torch.empty(cfg.batch, cfg.n_q_heads, cfg.head_dim, dtype=torch.float32, device=DEV)
+        orla = torch.empty_like(osp)
+        out = cache.append_decode(k1, v1, q, gamma, sel_idx=sel, dbg_o_sparse=osp, dbg_o_rla=orla)
+        torch.cuda.synchronize()
+        assert cache.sync_status() == 0
+        if step % 8 and step != w.n_steps - 1:
+            continue
+        for (b, h) in _all_units(w):
+            Ku = torch.cat([K[b, h, :int(lens_h[b])], extra[(b, h)][0]])
+            Vu = torch.cat([V[b, h, :int(lens_h[b])], extra[(b, h)][1]])
+
+            def run(override=None):
+                return parity.oracle_unit(w, q[b], Ku, Vu, gamma, h, n_sink=w.n_sink, n_local=w.n_local,
+                                          override=override, stats_bf16=True)
+            parity.compare_unit(w, run(), out[b].cpu().numpy(), osp[b].cpu().numpy(), orla[b].cpu().numpy(),
+                                sel[b, h].cpu().numpy(), h, n_sink=w.n_sink, n_local=w.n_local, rerun=run,
+                                tie_band=parity.TIE_BAND_STATS_BF16)
