@@ -145,6 +145,10 @@ __global__ void __launch_bounds__(kAttendThreads) attend_merge_kernel(const Para
   }
   __syncthreads();
 
+  // (kept in registers: with small tiles the fold buffer of pass 2 reaches over the statistics in shared memory)
+  float my_m = 0.f, my_l = 0.f;
+  if (tid < G) { my_m = m_s[tid]; my_l = l_s[tid]; }
+
   // ---- pass 2: both branches share the V tile ---------------------------------------------------------
   const int ts = tid / D, col = tid % D;
   float acc[NV];
@@ -197,8 +201,8 @@ __global__ void __launch_bounds__(kAttendThreads) attend_merge_kernel(const Para
   }
   if (tid < G) {
     float* ml = p.att_ml + (((size_t)u * p.top_k + item) * G + tid) * 2;
-    ml[0] = m_s[tid];
-    ml[1] = l_s[tid];
+    ml[0] = my_m;
+    ml[1] = my_l;
   }
   if (!arrive_last(&p.attend_ticket[u], nsel, &flag_s)) return;
 
