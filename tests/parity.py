@@ -67,7 +67,11 @@ def output_tolerances(kv_dtype: str):
 
 
 def check_outputs(name, got, want, kv_dtype, scale_floor=0.0):
-    tol = output_tolerances(kv_dtype)
+    tol = dict(output_tolerances(kv_dtype))
+    if kv_dtype != "bf16":
+        # fp32 inputs: the criterion is the relative L2 error (1e-5); the absolute bound is an extra guard and scales
+        # with the magnitude of the compared vector (the pre-norm residual is not bounded by the values' scale)
+        tol["max_abs"] *= max(1.0, float(np.max(np.abs(want))) if np.size(want) else 1.0)
     ma, rl = max_abs(got, want), rel_l2(got, want)
     if np.linalg.norm(want) <= scale_floor:          # a vanishing residual: absolute check only
         assert ma <= tol["max_abs"], f"{name}: max-abs {ma:.3e}"
