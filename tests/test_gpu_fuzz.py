@@ -1,6 +1,7 @@
 """Seeded random configurations of the whole path (shapes, lengths, forced blocks, windows, flags) against the oracle:
 a net under the hand-picked cases of the other files.  Every case is small enough for the oracle to check several
 units in well under a second."""
+import os
 import random
 
 import pytest
@@ -14,7 +15,7 @@ pytestmark = pytest.mark.gpu
 
 
 def _draw(case: int):
-    rnd = random.Random(22379 * 1000 + case)
+    rnd = random.Random(22379 * 1000 + case + int(os.environ.get("SPLA_FUZZ_OFFSET", "0")))   # other offsets: more cases by hand
     d = rnd.choice([64, 128])
     B = rnd.choice([16, 32, 64, 128])
     hkv = rnd.choice([1, 2, 3])
