@@ -279,16 +279,6 @@ static int attend_cluster_size(const spla_cache* c) {
 }
 
 
-// Selected blocks per CTA of the tensor-core attend kernel: more blocks per CTA means fewer split-K partials
-// to merge, as long as the grid still fills the machine.
-static int attend_bpc(const spla_cache* c) {
-  const long long items = (long long)c->p.batch * c->p.Hkv * c->p.top_k;
-  const size_t tile = (size_t)c->p.B * c->p.d * 2 * 2 + (size_t)c->p.B * 4;
-  int bpc = 1;
-  while (bpc < 4 && items / (bpc * 2) >= 3LL * c->sm_count && tile * bpc * 2 <= 100 * 1024) bpc *= 2;
-  return bpc;
-}
-
 extern "C" int spla_decode(spla_cache_t* c, const void* q, const float* rms_weight, float* out, int32_t* sel_idx,
                            float* dbg_o_sparse, float* dbg_o_rla, void* stream) {
   if (!c || !q || !out) return SPLA_ERR_INVALID_ARG;
