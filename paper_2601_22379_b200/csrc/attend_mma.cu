@@ -432,6 +432,22 @@ static cudaError_t launch_mma(const Params& p, const AttendMaps& maps, const voi
   return launch_ex(kern, grid, dim3(kAttendThreads), smem, stream, p.acs, true, p, mk, mv, qb, w, out, ds, dr);
 }
 
+template <int D>
+static int max_clusters_mma(const Params& p) {
+  const size_t smem = attend_mma_smem_bytes(p.B, D);
+  const dim3 grid(p.acs, p.batch * p.Hkv);
+  auto query = [&](auto kern) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess && p.acs > 8) e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (e != cudaSuccess) { cudaGetLastError(); return -1; }
+    return max_active_clusters(kern, grid, dim3(kAttendThreads), smem, p.acs);
+  };
+  return p.G <= 4 ? query(attend_mma_kernel<D, true>) : query(attend_mma_kernel<D, false>);
+}
+
+// Clusters of p.acs CTAs of the attend kernel the device holds at once; -1 if the query fails.
+int attend_mma_max_clusters(const Params& p) { return p.d == 128 ? max_clusters_mma<128>(p) : max_clusters_mma<64>(p); }
+
 cudaError_t launch_attend_mma(const Params& p, const AttendMaps& maps, const void* q, const float* rms_weight, float* out,
                               float* dbg_o_sparse, float* dbg_o_rla, cudaStream_t stream) {
   return p.d == 128 ? launch_mma<128>(p, maps, q, rms_weight, out, dbg_o_sparse, dbg_o_rla, stream)

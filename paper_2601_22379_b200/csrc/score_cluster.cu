@@ -770,8 +770,11 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
     }
 }
 
+// `occupancy` non-null: nothing is launched; it receives the number of clusters of this launch that the device holds
+// at once (-1 if the query fails).
 template <int D, int GP, bool WIN, bool EARLY, typename ST>
-static cudaError_t launch_win(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new, cudaStream_t stream) {
+static cudaError_t launch_win(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new, cudaStream_t stream,
+                              int* occupancy) {
   using SM = Smem<D, GP, ST>;
   const int U = p.batch * p.Hkv;
   size_t smem = (size_t)SM::kEll + (size_t)p.G * p.chunk * sizeof(float);
@@ -782,42 +785,53 @@ static cudaError_t launch_win(const Params& p, const void* q, int q_is_bf16, int
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) return e;
   }
+  if (occupancy) {
+    *occupancy = max_active_clusters(kern, dim3(p.cs, U, 1), dim3(kCsThreads, 1, 1), smem, p.cs);
+    return cudaSuccess;
+  }
   return launch_ex(kern, dim3(p.cs, U, 1), dim3(kCsThreads, 1, 1), smem, stream, p.cs, true, p, q, q_is_bf16, sel_user, pending_new);
 }
 
 template <int D, int GP, typename ST>
-static cudaError_t launch_st(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new, cudaStream_t stream) {
+static cudaError_t launch_st(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new, cudaStream_t stream,
+                             int* occ) {
   if (pending_new > 0)
-    return p.NW > 1 ? launch_win<D, GP, true, true, ST>(p, q, q_is_bf16, sel_user, pending_new, stream)
-                    : launch_win<D, GP, false, true, ST>(p, q, q_is_bf16, sel_user, pending_new, stream);
-  return p.NW > 1 ? launch_win<D, GP, true, false, ST>(p, q, q_is_bf16, sel_user, 0, stream)
-                  : launch_win<D, GP, false, false, ST>(p, q, q_is_bf16, sel_user, 0, stream);
+    return p.NW > 1 ? launch_win<D, GP, true, true, ST>(p, q, q_is_bf16, sel_user, pending_new, stream, occ)
+                    : launch_win<D, GP, false, true, ST>(p, q, q_is_bf16, sel_user, pending_new, stream, occ);
+  return p.NW > 1 ? launch_win<D, GP, true, false, ST>(p, q, q_is_bf16, sel_user, 0, stream, occ)
+                  : launch_win<D, GP, false, false, ST>(p, q, q_is_bf16, sel_user, 0, stream, occ);
 }
 
 template <int D, int GP>
-static cudaError_t launch_one(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new, cudaStream_t stream) {
-  return (p.flags & kStatsBf16) ? launch_st<D, GP, __nv_bfloat16>(p, q, q_is_bf16, sel_user, pending_new, stream)
-                                : launch_st<D, GP, float>(p, q, q_is_bf16, sel_user, pending_new, stream);
+static cudaError_t launch_one(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new, cudaStream_t stream,
+                              int* occ) {
+  return (p.flags & kStatsBf16) ? launch_st<D, GP, __nv_bfloat16>(p, q, q_is_bf16, sel_user, pending_new, stream, occ)
+                                : launch_st<D, GP, float>(p, q, q_is_bf16, sel_user, pending_new, stream, occ);
 }
 
 template <int D>
-static cudaError_t launch_d(const Params& p, int GP, const void* q, int qb, int* sel_user, int pending_new, cudaStream_t s) {
+static cudaError_t launch_d(const Params& p, int GP, const void* q, int qb, int* sel_user, int pending_new, cudaStream_t s,
+                            int* occ) {
   switch (GP) {
-    case 1: return launch_one<D, 1>(p, q, qb, sel_user, pending_new, s);
-    case 2: return launch_one<D, 2>(p, q, qb, sel_user, pending_new, s);
-    case 4: return launch_one<D, 4>(p, q, qb, sel_user, pending_new, s);
-    default: return launch_one<D, 8>(p, q, qb, sel_user, pending_new, s);
+    case 1: return launch_one<D, 1>(p, q, qb, sel_user, pending_new, s, occ);
+    case 2: return launch_one<D, 2>(p, q, qb, sel_user, pending_new, s, occ);
+    case 4: return launch_one<D, 4>(p, q, qb, sel_user, pending_new, s, occ);
+    default: return launch_one<D, 8>(p, q, qb, sel_user, pending_new, s, occ);
   }
 }
 
 // Decides whether the cluster kernel can serve a launch and with which cluster size / records per CTA.
 // Returns false when the general kernel has to be used (very long sequences, groups above 8).
-bool plan_score_cluster(int units, long long max_seq_blocks, int NW, int G, int d, int sm_count, int* cs_out, int* chunk_out) {
+// `cs_cap` bounds the cluster size from above where the block count leaves a choice (the caller lowers it when the
+// device cannot hold all clusters of the first choice at once).
+bool plan_score_cluster(int units, long long max_seq_blocks, int NW, int G, int d, int sm_count, int cs_cap, int* cs_out,
+                        int* chunk_out) {
   if (G > 8) return false;
   if (max_seq_blocks < 1) max_seq_blocks = 1;
+  if (cs_cap > kMaxCluster) cs_cap = kMaxCluster;
   int cs = 1;
   while (cs < kMaxCluster && max_seq_blocks > 576LL * cs) cs *= 2;            // keep the local ranking short
-  while (cs < kMaxCluster && (long long)units * cs * 2 <= 2LL * sm_count) cs *= 2;   // fill the machine once
+  while (cs < cs_cap && (long long)units * cs * 2 <= 2LL * sm_count) cs *= 2; // fill the machine once
   const long long chunk = (max_seq_blocks + cs - 1) / cs;
   const int chunk32 = (int)((chunk + 31) / 32 * 32);
   if (chunk32 > 1024) return false;
@@ -833,8 +847,17 @@ bool plan_score_cluster(int units, long long max_seq_blocks, int NW, int G, int 
 cudaError_t launch_score_cluster(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new,
                                  cudaStream_t stream) {
   const int GP = padded_group(p.G);
-  return p.d == 128 ? launch_d<128>(p, GP, q, q_is_bf16, sel_user, pending_new, stream)
-                    : launch_d<64>(p, GP, q, q_is_bf16, sel_user, pending_new, stream);
+  return p.d == 128 ? launch_d<128>(p, GP, q, q_is_bf16, sel_user, pending_new, stream, nullptr)
+                    : launch_d<64>(p, GP, q, q_is_bf16, sel_user, pending_new, stream, nullptr);
+}
+
+int score_cluster_max_clusters(const Params& p) {
+  const int GP = padded_group(p.G);
+  int n = -1;
+  const cudaError_t e = p.d == 128 ? launch_d<128>(p, GP, nullptr, 0, nullptr, 0, nullptr, &n)
+                                   : launch_d<64>(p, GP, nullptr, 0, nullptr, 0, nullptr, &n);
+  if (e != cudaSuccess) { cudaGetLastError(); return -1; }
+  return n;
 }
 
 }  // namespace spla

@@ -17,6 +17,9 @@ struct spla_cache {
   spla_buffers_t buf;
   Params p;
   int64_t len_bound;   // host-side upper bound of the longest sequence
+  // clusters the device holds at once, as last queried: score kernel for (cs, chunk), attend kernel per log2(acs)
+  int score_occ_cs = 0, score_occ_chunk = 0, score_occ_n = -1;
+  int attend_occ[5] = {-2, -2, -2, -2, -2};
   cudaEvent_t ev[3];   // created on first use by spla_decode_profile
   bool have_ev;
   int sm_count;
@@ -243,17 +246,40 @@ extern "C" int spla_append_tokens(spla_cache_t* c, const void* k_new, const void
   return SPLA_OK;
 }
 
-// Sizes the score grid from the host-side bound of the sequence lengths.
-static void plan_score_grid(const spla_cache* c, Params* p) {
+// Sizes the score grid from the host-side bound of the sequence lengths.  A cluster's CTAs sit in one GPC, so the
+// device may hold fewer clusters of a size than its CTA slots suggest; a launch whose clusters do not all fit at
+// once runs in two waves and takes twice as long.  The cluster size is therefore lowered (where the block count
+// leaves a choice) until the occupancy query says that all units' clusters are resident together.
+static void plan_score_grid(spla_cache* c, Params* p) {
   int64_t blocks = (c->len_bound + c->cfg.block_size - 1) / c->cfg.block_size;
   if (blocks < 1) blocks = 1;
   p->cs = 0;
-  int cs = 0, chunk = 0;
-  if (!(c->cfg.flags & SPLA_GENERAL_KERNELS) && plan_score_cluster(p->batch * p->Hkv, blocks, p->NW, p->G, p->d, c->sm_count, &cs, &chunk)) {
-    p->cs = cs;
-    p->chunk = chunk;
-    p->n_chunks_cap = cs;
-    return;
+  const int units = p->batch * p->Hkv;
+  if (!(c->cfg.flags & SPLA_GENERAL_KERNELS)) {
+    int best_cs = 0, best_chunk = 0;
+    for (int cap = 16; cap >= 1; cap /= 2) {
+      int cs = 0, chunk = 0;
+      if (!plan_score_cluster(units, blocks, p->NW, p->G, p->d, c->sm_count, cap, &cs, &chunk)) break;
+      if (best_cs && cs >= best_cs) break;                   // the block count needs at least this size: no choice left
+      best_cs = cs;
+      best_chunk = chunk;
+      if (cs == 1 || (long long)units * cs > 2LL * c->sm_count) break;   // several waves by necessity: nothing to gain
+      if (c->score_occ_cs != cs || c->score_occ_chunk != chunk) {
+        Params probe = *p;
+        probe.cs = cs;
+        probe.chunk = chunk;
+        c->score_occ_n = score_cluster_max_clusters(probe);
+        c->score_occ_cs = cs;
+        c->score_occ_chunk = chunk;
+      }
+      if (c->score_occ_n < 0 || units <= c->score_occ_n) break;   // unknown, or all resident at once
+    }
+    if (best_cs) {
+      p->cs = best_cs;
+      p->chunk = best_chunk;
+      p->n_chunks_cap = best_cs;
+      return;
+    }
   }
   p->chunk = score_chunk_for((long long)p->batch * p->Hkv, blocks * p->NW, c->sm_count);   // in records (windows)
   p->n_chunks_cap = (int)((blocks * p->NW + p->chunk - 1) / p->chunk);
@@ -265,7 +291,7 @@ static cudaError_t launch_score(const Params& p, const void* q, int qb, int* sel
 
 // Cluster size of the tensor-core attend kernel: the largest power of two (at most 16 and at most top_k) for
 // which all CTAs are resident at once; each CTA of a cluster then walks top_k / size selected blocks.
-static int attend_cluster_size(const spla_cache* c) {
+static int attend_cluster_size(spla_cache* c) {
   if (c->cfg.flags & SPLA_GENERAL_KERNELS) return 0;
   const size_t smem = attend_mma_smem_bytes(c->p.B, c->p.d) + 2048;
   long long per_sm = (227 * 1024) / (long long)smem;
@@ -275,6 +301,17 @@ static int attend_cluster_size(const spla_cache* c) {
   const long long U = (long long)c->p.batch * c->p.Hkv;
   int cs = 1;
   while (cs * 2 <= 16 && cs * 2 <= c->p.top_k && U * cs * 2 <= slots) cs *= 2;
+  // all clusters of the launch must be resident together (see plan_score_grid): ask the device
+  for (; cs > 1; cs /= 2) {
+    int lg = 0;
+    while ((1 << lg) < cs) ++lg;
+    if (c->attend_occ[lg] == -2) {
+      Params probe = c->p;
+      probe.acs = cs;
+      c->attend_occ[lg] = attend_mma_max_clusters(probe);
+    }
+    if (c->attend_occ[lg] < 0 || U <= c->attend_occ[lg]) break;
+  }
   return cs;
 }
 

@@ -43,11 +43,36 @@ inline cudaError_t launch_ex(void (*kern)(KArgs...), dim3 grid, dim3 block, size
   return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 
+// How many clusters of `cluster_x` CTAs of this kernel the device holds at once (all CTAs of a cluster sit in one
+// GPC, so this is less than CTA slots / cluster size); -1 if the query fails.
+template <typename... KArgs>
+inline int max_active_clusters(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, int cluster_x) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cluster_x;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) {
+    cudaGetLastError();
+    return -1;
+  }
+  return n;
+}
+
 // score_select.cu
 int score_chunk_for(long long units, long long max_seq_blocks, int sm_count);
 cudaError_t launch_score_select(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream);
 // score_cluster.cu (G <= 8, at most 16 x 1024 blocks per sequence)
-bool plan_score_cluster(int units, long long max_seq_blocks, int NW, int G, int d, int sm_count, int* cs_out, int* chunk_out);
+bool plan_score_cluster(int units, long long max_seq_blocks, int NW, int G, int d, int sm_count, int cs_cap, int* cs_out, int* chunk_out);
+// Clusters of the score kernel (p.cs CTAs each, p.chunk blocks per CTA) the device holds at once; -1 if unknown.
+int score_cluster_max_clusters(const Params& p);
 cudaError_t launch_score_cluster(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new,
                                  cudaStream_t stream);
 struct AttendMaps {                      // TMA tensor maps (CUtensorMap) of the K and V caches, opaque to the host code
@@ -65,6 +90,7 @@ cudaError_t launch_attend_merge(const Params& p, const AttendMaps* maps, const v
                                 float* dbg_o_rla, cudaStream_t stream);
 // attend_mma.cu (bf16 K/V and q, G <= 8)
 size_t attend_mma_smem_bytes(int B, int D);
+int attend_mma_max_clusters(const Params& p);   // clusters of p.acs CTAs resident at once; -1 if unknown
 cudaError_t launch_attend_mma(const Params& p, const AttendMaps& maps, const void* q, const float* rms_weight, float* out,
                               float* dbg_o_sparse, float* dbg_o_rla, cudaStream_t stream);
 // append.cu
