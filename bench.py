@@ -114,7 +114,10 @@ def n_windows(w):
 
 
 def workload_name(w):
-    return w.name + (f"+windows(C={WINDOW[0]},s={WINDOW[1]})" if WINDOW else "") + ("+stats_bf16" if STATS_BF16 else "")
+    from paper_2601_22379_b200 import synth
+    base = synth.BY_NAME[w.name]
+    over = "".join(f"+{k}={getattr(w, k)}" for k in ("batch", "context") if getattr(w, k) != getattr(base, k))
+    return w.name + over + (f"+windows(C={WINDOW[0]},s={WINDOW[1]})" if WINDOW else "") + ("+stats_bf16" if STATS_BF16 else "")
 
 
 def stat_bytes():
@@ -467,6 +470,8 @@ def main():
                          "profiles/score_cluster_kernel_long_128k*.md for the long_128k workload")
     ap.add_argument("--window", default=None, metavar="C,s",
                     help="strided selection windows (the paper's setting is 32,16) instead of whole-block statistics")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (scaling studies; the metric is quoted on the default)")
+    ap.add_argument("--context", type=int, default=0, help="override the workload's context length (scaling studies)")
     ap.add_argument("--stats-bf16", action="store_true",
                     help="store the block statistics as bfloat16 (half the bytes for the score kernel to stream)")
     args = ap.parse_args()
@@ -476,6 +481,10 @@ def main():
     STATS_BF16 = args.stats_bf16
     from paper_2601_22379_b200 import synth
     w = synth.BY_NAME[args.workload]
+    if args.batch > 0:
+        w = w.scaled(batch=args.batch)
+    if args.context > 0:
+        w = w.scaled(context=args.context, context_min=min(w.context_min, args.context))
     if args.impl == "reference":
         run_reference(args, w)
     else:
