@@ -33,6 +33,8 @@ notes of the repository):
     maximum of its windows' Taylor log masses, and the per-head
     normalisation over blocks comes after this pooling;
   * ties are broken by (score descending, block index ascending);
+  * training / prefilling (said only to carry over from decoding): the query
+    at position t sees the cache a decode step at t would see (prefill_unit);
   * 16-bit statistics (an option; the paper does not say in which precision
     the block summaries are kept): mean and variance are computed in full
     precision, rounded once to bfloat16 (round to nearest, ties to even)
@@ -392,6 +394,28 @@ def decode(q, K, V, gamma, seq_lens, *, n_kv_heads, **cfg):
             out[b, h * G:(h + 1) * G] = r["out"]
             units[(b, h)] = r
     return out, units
+
+
+def prefill_unit(q_positions, K, V, gamma_group, first_position: int, **cfg):
+    """Prefill / training-shaped forward of one unit: the output at every query position of a chunk.
+
+    The paper describes the method on the decoding workload and notes that it carries over to training and
+    prefilling (Section 2, opening paragraph).  The reading taken here is the causal one: the query at absolute
+    position t sees exactly the cache a decode step at that position would see, tokens 0..t, with the block
+    statistics, the selection and the recurrent state of that prefix.  q_positions [T, G, d] holds the queries of
+    positions first_position .. first_position + T - 1; K, V [L, d] with L >= first_position + T.
+    Returns out [T, G, d] and the list of selected index arrays.  No GPU counterpart exists yet: this is the
+    reference the next kernel row will be checked against.
+    """
+    q_positions = np.asarray(q_positions, dtype=F64)
+    T = q_positions.shape[0]
+    outs, sels = [], []
+    for i in range(T):
+        n_tok = first_position + i + 1
+        r = decode_unit(q_positions[i], K[:n_tok], V[:n_tok], gamma_group, **cfg)
+        outs.append(r["out"])
+        sels.append(r["sel"])
+    return np.stack(outs), sels
 
 
 # ---------------------------------------------------------------------------

@@ -548,3 +548,45 @@ def test_bf16_statistics_incremental_cache_equals_definitional_form():
         assert np.array_equal(a["sel"], b["sel"])
         np.testing.assert_allclose(a["score"], b["score"], rtol=1e-2, atol=0)   # rounding may flip where Welford and two-pass differ in the last bit
         np.testing.assert_allclose(a["out"], b["out"], rtol=1e-9, atol=1e-12)
+
+
+# ---------------------------------------------------------------------------
+# F  prefill-shaped forward (a reading: the paper only says that the decode formulation carries over)
+# ---------------------------------------------------------------------------
+def test_prefill_forward_is_causal_and_ends_in_the_decode_step():
+    d, B, G, L0, T = 16, 8, 2, 8 * 5 + 3, 21
+    K = RNG.standard_normal((L0 + T, d))
+    V = RNG.standard_normal((L0 + T, d))
+    q = RNG.standard_normal((T, G, d))
+    gamma = RNG.uniform(0.5, 1.5, (G, d))
+    cfg = dict(block_size=B, top_k=4, n_sink=1, n_local=1)
+    out, sels = O.prefill_unit(q, K, V, gamma, L0, **cfg)
+    # the last position is the decode step on the whole cache
+    np.testing.assert_array_equal(out[-1], O.decode_unit(q[-1], K, V, gamma, **cfg)["out"])
+    # causality: what comes after position p cannot change the outputs up to p
+    p = 9
+    K2, V2 = K.copy(), V.copy()
+    K2[L0 + p + 1:] += 5.0
+    V2[L0 + p + 1:] -= 3.0
+    out2, _ = O.prefill_unit(q, K2, V2, gamma, L0, **cfg)
+    np.testing.assert_array_equal(out2[:p + 1], out[:p + 1])
+    assert np.abs(out2[p + 1:] - out[p + 1:]).max() > 1e-3
+    # every position keeps its own (partial) block and the sink block
+    for i, sel in enumerate(sels):
+        nblk = -(-(L0 + i + 1) // B)
+        assert 0 in sel and nblk - 1 in sel and sel.max() == nblk - 1
+
+
+def test_prefill_forward_with_full_selection_is_causal_dense_attention():
+    d, B, G, L0, T = 16, 8, 3, 8 * 2, 13
+    K = RNG.standard_normal((L0 + T, d))
+    V = RNG.standard_normal((L0 + T, d))
+    q = RNG.standard_normal((T, G, d))
+    gamma = np.ones((G, d))
+    out, _ = O.prefill_unit(q, K, V, gamma, L0, block_size=B, top_k=64)
+    # library routine: causal attention of T queries placed at the end of L0 + T keys (boolean mask, float64)
+    qt = torch.from_numpy(q).permute(1, 0, 2)                       # [G, T, d]
+    mask = torch.arange(L0 + T)[None, :] <= (L0 + torch.arange(T))[:, None]
+    want = torch.nn.functional.scaled_dot_product_attention(qt, torch.from_numpy(K)[None].expand(G, -1, -1),
+                                                            torch.from_numpy(V)[None].expand(G, -1, -1), attn_mask=mask)
+    np.testing.assert_allclose(out, want.permute(1, 0, 2).numpy(), rtol=1e-10, atol=1e-12)
