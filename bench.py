@@ -10,8 +10,9 @@ whole job, at the 128K-context configuration, plus the HBM roofline of the domin
 
 Timing: W warm-up steps, then exactly K steps between barrier + synchronize, timed with CUDA events on the
 launching stream, max over ranks.  The steps rotate over R independent caches so that the bytes touched per
-rotation exceed three times the L2 size (cold-L2 protocol).  Steps are replayed from a CUDA graph of 64 steps
-so that the Python launch path is not what is measured.  One JSON line is printed by rank 0.
+rotation exceed three times the L2 size (cold-L2 protocol).  Steps are replayed from a CUDA graph of min(K, 64)
+steps (plus one of the remainder) so that the Python launch path is not what is measured.  One JSON line is printed
+by rank 0.
 """
 from __future__ import annotations
 
@@ -32,8 +33,8 @@ METRIC = "decode_attention_query_heads_per_s"
 UNIT = "query_heads/s"
 L2_BYTES = 126 * 1024 * 1024
 GRAPH_STEPS = 64
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the score kernel from the ncu capture summarised in
-# profiles/score_cluster_kernel_long_128k.md (69.37 MB read + 0.66 MB written)
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from ncu captures of this command
+# on a small case (one cache, a few launches), per workload
 NCU_TRAFFIC = {"long_128k": 70.00e6, "long_128k+windows(C=32,s=16)": 208.8e6, "long_128k+stats_bf16": 35.79e6}
 
 
@@ -60,14 +61,17 @@ def _oracle_worker(args):
         return time.perf_counter() - t0
 
 
-def oracle_throughput(w, n_dec_per_unit: int, repeats: int = 1):
-    """Runs the oracle on one sequence's KV heads (one unit per process).  Returns (query_heads/s list, cores, sample)."""
+def oracle_throughput(w, n_dec_per_unit: int, repeats: int = 1, max_units: int = 0):
+    """Runs the oracle on one sequence's KV heads (one unit per process; at most `max_units` processes when given).
+    Returns (query_heads/s list, cores, sample)."""
     global _ORACLE_UNITS
     import multiprocessing as mp
     import numpy as np
     from paper_2601_22379_b200 import synth
     cores = len(os.sched_getaffinity(0))
     n_units = max(1, min(cores, w.n_kv_heads))
+    if max_units > 0:
+        n_units = min(n_units, max_units)
     K, V = synth.prefill_kv(w, 0, "cpu")
     G = w.group
     gam = synth.gamma(w).double().numpy()
@@ -116,7 +120,7 @@ def n_windows(w):
 def workload_name(w):
     from paper_2601_22379_b200 import synth
     base = synth.BY_NAME[w.name]
-    over = "".join(f"+{k}={getattr(w, k)}" for k in ("batch", "context") if getattr(w, k) != getattr(base, k))
+    over = "".join(f"+{k}={getattr(w, k)}" for k in ("batch", "context", "n_q_heads") if getattr(w, k) != getattr(base, k))
     return w.name + over + (f"+windows(C={WINDOW[0]},s={WINDOW[1]})" if WINDOW else "") + ("+stats_bf16" if STATS_BF16 else "")
 
 
@@ -200,8 +204,10 @@ def run_ours(args, w):
     world, rank, local = replicas.env_world()
     cpu_base = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        vals, cores, sample = oracle_throughput(w, 500, repeats=2)      # before CUDA is initialised (fork)
-        cpu_base = {"value": vals[-1], "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+        vals, cores, sample = oracle_throughput(w, 400, repeats=2)      # before CUDA is initialised (fork)
+        one, _, sample1 = oracle_throughput(w, 300, repeats=1, max_units=1)
+        cpu_base = {"value": vals[-1], "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                    "single_thread": {"value": one[-1], "unit": UNIT, "cores": 1, "sample": sample1}}
 
     build.build()
     torch.cuda.set_device(local)
@@ -216,7 +222,8 @@ def run_ours(args, w):
     if args.caches > 0:                                               # profiling aid: fewer caches, less device memory
         R = args.caches
     n_e2e = max(8, min(steps, 256))
-    per_cache = -(-(steps + warmup + 2 * GRAPH_STEPS + n_e2e) // R) + 2 * GRAPH_STEPS
+    G1 = max(1, min(steps, GRAPH_STEPS))                              # steps per captured graph
+    per_cache = -(-(steps + warmup + 3 * GRAPH_STEPS + n_e2e) // R) + 2 * GRAPH_STEPS
     wl = w.scaled(n_steps=per_cache)
     prefill = runner.generate_prefill(wl, dev)
     caches = []
@@ -238,43 +245,45 @@ def run_ours(args, w):
     kvs = [synth.step_kv(w, s, dev) for s in range(n_in)]
     outs = [torch.empty(w.batch, w.n_q_heads, w.head_dim, dtype=torch.float32, device=dev) for _ in range(R)]
     stream = torch.cuda.Stream(device=dev)
-    counter = {"i": 0}
 
-    def one_step():
-        i = counter["i"]
-        counter["i"] += 1
+    def one_step(i):
         c = caches[i % R]
         k1, v1 = kvs[i % n_in]
         c.append_decode(k1, v1, qs[i % n_in], gamma, out=outs[i % R])    # the step: append, then decode, one call
-        n_app[i % R] += 1
 
     def decode_only(i):
         caches[i % R].decode(qs[i % n_in], gamma, out=outs[i % R])
 
+    def capture(body, n):
+        """A CUDA graph of body(0) .. body(n - 1), replayed once untimed; None for n == 0."""
+        if n <= 0:
+            return None
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(n):
+                body(i)
+        g.replay()
+        return g
+
+    def appended_by(n):                                               # tokens a graph of n steps appends to each cache
+        return [len(range(ci, n, R)) for ci in range(R)]
+
+    n_rep, n_rem = steps // G1, steps % G1
     torch.cuda.synchronize()
     with torch.cuda.stream(stream):
-        for _ in range(warmup):
-            one_step()
-        graph = None
-        saved = list(n_app)
+        for i in range(warmup):                                        # eager warm-up steps (also load the kernels)
+            one_step(i)
+            n_app[i % R] += 1
         set_bounds(exact=False)
-        if steps >= GRAPH_STEPS:
-            counter["i"] = 0
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph, stream=stream):
-                for _ in range(GRAPH_STEPS):
-                    one_step()
-            n_app[:] = saved                                           # capture enqueued nothing
-            graph.replay()                                             # one untimed replay
-            for ci in range(R):
-                n_app[ci] += GRAPH_STEPS // R
-        graph_dec = None
-        if steps >= GRAPH_STEPS:
-            graph_dec = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph_dec, stream=stream):
-                for i in range(GRAPH_STEPS):
-                    decode_only(i)
-            graph_dec.replay()
+        n_launch0 = binding.launch_count()
+        graph = capture(one_step, G1)                                  # (the library counts the kernels it records)
+        launches_per_step = (binding.launch_count() - n_launch0) / G1
+        set_bounds(exact=False)
+        graph_rem = capture(one_step, n_rem)
+        for n in (G1, n_rem):
+            for ci, a in enumerate(appended_by(n)):
+                n_app[ci] += a
+        graph_dec = capture(decode_only, G1)
     torch.cuda.synchronize()
 
     def barrier():
@@ -289,19 +298,19 @@ def run_ours(args, w):
     t0 = time.perf_counter()
     with torch.cuda.stream(stream):
         e0.record(stream)
-        n_rep = steps // GRAPH_STEPS if graph is not None else 0
         for _ in range(n_rep):
             graph.replay()
-        for ci in range(R):
-            n_app[ci] += n_rep * (GRAPH_STEPS // R)
-        set_bounds(exact=True)
-        for _ in range(steps - n_rep * GRAPH_STEPS):
-            one_step()
+        if graph_rem is not None:
+            graph_rem.replay()
         e1.record(stream)
     barrier()
     t1 = time.perf_counter()
     total_ms = e0.elapsed_time(e1)
     clocks = sampler.stop(t0, t1)
+    for ci, a in enumerate(appended_by(G1)):
+        n_app[ci] += n_rep * a
+    for ci, a in enumerate(appended_by(n_rem)):
+        n_app[ci] += a
     for c in caches:
         st = c.sync_status()
         if st != 0:
@@ -310,17 +319,13 @@ def run_ours(args, w):
     # ---- decode-only (no append) for context, same rotation ---------------------------------------------------
     with torch.cuda.stream(stream):
         d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        n_dec_rep = max(1, min(steps // GRAPH_STEPS, 64))
+        n_dec_rep = max(1, min(steps // G1, 64))
         d0.record(stream)
         for r in range(n_dec_rep):
-            if graph_dec is not None:
-                graph_dec.replay()
-            else:
-                for i in range(GRAPH_STEPS):
-                    decode_only(i)
+            graph_dec.replay()
         d1.record(stream)
     torch.cuda.synchronize()
-    dec_ms = d0.elapsed_time(d1) / (n_dec_rep * GRAPH_STEPS)
+    dec_ms = d0.elapsed_time(d1) / (n_dec_rep * G1)
 
     # ---- duration of the dominant kernel (block score + selection): a CUDA graph of back-to-back launches of that
     # kernel alone, rotating over the caches (cold L2), timed with CUDA events on the launching stream -------------
@@ -328,43 +333,21 @@ def run_ours(args, w):
     with torch.cuda.stream(stream):
         for i in range(R):
             caches[i].select(qs[i], sel_bufs[i])                      # warm-up, also loads the kernel
-        graph_sel = None
-        if steps >= GRAPH_STEPS:
-            graph_sel = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph_sel, stream=stream):
-                for i in range(GRAPH_STEPS):
-                    caches[i % R].select(qs[i % n_in], sel_bufs[i % R])
-            graph_sel.replay()
+        graph_sel = capture(lambda i: caches[i % R].select(qs[i % n_in], sel_bufs[i % R]), G1)
         s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        n_sel_rep = max(1, min(steps // GRAPH_STEPS, 64))
+        n_sel_rep = max(1, min(steps // G1, 64))
         s0.record(stream)
         for r in range(n_sel_rep):
-            if graph_sel is not None:
-                graph_sel.replay()
-            else:
-                for i in range(GRAPH_STEPS):
-                    caches[i % R].select(qs[i % n_in], sel_bufs[i % R])
+            graph_sel.replay()
         s1.record(stream)
     torch.cuda.synchronize()
-    sc = s0.elapsed_time(s1) / (n_sel_rep * GRAPH_STEPS)
-
-    # isolated kernel durations with events between the two kernels of one decode (each includes ~6 us of event
-    # and launch latency, measured on an empty kernel; reported for reference only)
-    n_prof = max(8, min(steps, 64))
-    sc_iso, at_iso = [], []
-    with torch.cuda.stream(stream):
-        for i in range(n_prof):
-            a, b = caches[i % R].decode_profile(qs[i % n_in], gamma, outs[i % R])
-            sc_iso.append(a)
-            at_iso.append(b)
-    at = statistics.mean(at_iso)
+    sc = s0.elapsed_time(s1) / (n_sel_rep * G1)
 
     # ---- end to end through the public call with host buffers -----------------------------------------------------
     # Per step: the host writes q, k_t, v_t into a pinned staging buffer; the H2D copy, append and decode are enqueued
-    # (as one captured graph per cache when graphs are in use), the output goes device -> host by the merge kernel's own
-    # stores into a pinned host buffer (no separate copy), and the stream is synchronised, because the caller reads
-    # the output before it can form the next query.
-    # q, k_t and v_t travel in one staging buffer: one host write and one H2D copy per step instead of three
+    # as one captured graph per cache, the output goes device -> host by the merge kernel's own stores into a pinned
+    # host buffer (no separate copy), and the stream is synchronised, because the caller reads the output before it
+    # can form the next query.  q, k_t and v_t travel in one staging buffer: one host write and one H2D copy per step.
     nq, nk = qs[0].numel(), kvs[0][0].numel()
     src = [torch.cat([qs[i].reshape(-1), kvs[i][0].reshape(-1), kvs[i][1].reshape(-1)]).cpu() for i in range(8)]
     hstage = src[0].clone().pin_memory()
@@ -379,70 +362,54 @@ def run_ours(args, w):
         dstage.copy_(hstage, non_blocking=True)
         caches[ci].append_decode(dk, dv, dq, gamma, out=hout)   # the merge kernel stores the output straight into pinned host memory
 
-    e2e_graphs = None
+    e2e_graphs = []
+    set_bounds(exact=False)
     with torch.cuda.stream(stream):
-        if steps >= GRAPH_STEPS:
-            set_bounds(exact=False)
-            e2e_graphs = []
-            for ci in range(R):
-                gph = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(gph, stream=stream):
-                    e2e_body(ci)
-                e2e_graphs.append(gph)
-        else:
-            set_bounds(exact=True)
+        for ci in range(R):
+            gph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gph, stream=stream):
+                e2e_body(ci)
+            e2e_graphs.append(gph)
     barrier()
     with torch.cuda.stream(stream):
         g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         g0.record(stream)
         for i in range(n_e2e):
             hstage.copy_(src[i % 8])                                   # the step's inputs arrive in host memory
-            if e2e_graphs is not None:
-                e2e_graphs[i % R].replay()
-            else:
-                e2e_body(i % R)
+            e2e_graphs[i % R].replay()
             n_app[i % R] += 1
             stream.synchronize()                                       # the caller reads the result before the next step
         g1.record(stream)
     barrier()
     e2e_ms = g0.elapsed_time(g1) / n_e2e
+    set_bounds(exact=True)
+    for c in caches:
+        st = c.sync_status()
+        if st != 0:
+            raise RuntimeError(f"device status {st} after the end-to-end leg")
 
     total_ms, e2e_ms = replicas.max_over_ranks([total_ms, e2e_ms], dev)
     value = replicas.whole_job_rate(w.batch * w.n_q_heads, steps, total_ms)
 
     peak, peak_kind = measured_peaks()
-    # a plain read-only stream over a buffer four times the L2, as a second reference beside the copy peak
-    probe = torch.empty(4 * L2_BYTES, dtype=torch.uint8, device=dev)
-    with torch.cuda.stream(stream):
-        for _ in range(3):
-            binding.probe_read(probe)
-        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        p0.record(stream)
-        for _ in range(10):
-            binding.probe_read(probe)
-        p1.record(stream)
-    torch.cuda.synchronize()
-    read_peak = 10 * probe.numel() / (p0.elapsed_time(p1) * 1e-3) / 1e9
-    del probe
     score_bytes = by["stats"] + by["state"]
     achieved = score_bytes / (sc * 1e-3) / 1e9
     line = base_line(args, w, value, ms_per_step=total_ms / steps)
     line["warmup"] = warmup
     line["config"].update({"l2_protocol": f"rotation over {R} independent caches ({R * by['total'] / 2**20:.0f} MiB per "
                                           f"rotation, > 3x L2) - cold L2", "context_growth_tokens_per_cache": per_cache,
-                           "launch": f"CUDA graph of {GRAPH_STEPS} steps replayed" if graph is not None else "eager"})
+                           "launch": f"CUDA graph of {G1} steps, replayed {n_rep}x" +
+                                     (f", plus one of {n_rem} steps" if n_rem else "")})
     line.update({
         "clocks": clocks,
         "e2e": {"value": w.batch * w.n_q_heads * world / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
-        "gpu_launches": 3 * steps,
+        "gpu_launches": int(round(launches_per_step * steps)),
         "roofline": {"bound": "hbm", "kernel": "score_cluster_kernel (block score + top-k)", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                     "read_stream_GBps": read_peak, "frac_of_read_stream": achieved / read_peak,
                      "bytes_per_launch": score_bytes, "ms_per_launch": sc,
                      "traffic": args.traffic if args.traffic is not None else NCU_TRAFFIC.get(workload_name(w))},
-        "kernels": {"score_select_ms": sc, "score_select_isolated_ms": statistics.mean(sc_iso),
-                    "attend_merge_isolated_ms": at, "decode_minus_score_ms": dec_ms - sc,
+        "kernels": {"score_select_ms": sc, "decode_minus_score_ms": dec_ms - sc,
                     "decode_only_ms": dec_ms, "decode_only_GBps": by["total"] / (dec_ms * 1e-3) / 1e9,
                     "decode_only_frac_of_peak": by["total"] / (dec_ms * 1e-3) / 1e9 / peak,
                     "decode_only_frac_of_8TBps": by["total"] / (dec_ms * 1e-3) / 8e12,
@@ -466,8 +433,10 @@ def main():
     ap.add_argument("--caches", type=int, default=0, help="rotate over this many caches instead of the cold-L2 count "
                     "(for profiler captures, which must hold little device memory)")
     ap.add_argument("--traffic", type=float, default=None,
-                    help="DRAM bytes per launch of the dominant kernel from an ncu capture; default: the figures of "
-                         "profiles/score_cluster_kernel_long_128k*.md for the long_128k workload")
+                    help="DRAM bytes per launch of the dominant kernel from an ncu capture; default: the figure "
+                         "recorded in this file for the workload")
+    ap.add_argument("--q-heads", type=int, default=0, help="override the number of query heads (the group size is "
+                    "q_heads / 8 KV heads; the paper's own model has 40)")
     ap.add_argument("--window", default=None, metavar="C,s",
                     help="strided selection windows (the paper's setting is 32,16) instead of whole-block statistics")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (scaling studies; the metric is quoted on the default)")
@@ -483,6 +452,8 @@ def main():
     w = synth.BY_NAME[args.workload]
     if args.batch > 0:
         w = w.scaled(batch=args.batch)
+    if args.q_heads > 0:
+        w = w.scaled(n_q_heads=args.q_heads)
     if args.context > 0:
         w = w.scaled(context=args.context, context_min=min(w.context_min, args.context))
     if args.impl == "reference":

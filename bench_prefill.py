@@ -1,6 +1,6 @@
 """Times the bulk append (prefill) of a workload: cache write, block statistics, recurrent state, lengths.
 
-    python -m paper_2601_22379_b200.prefill_bench [--workload long_128k] [--batch N] [--reps R] [--general]
+    python bench_prefill.py [--workload long_128k] [--batch N] [--reps R] [--general]
 
 One JSON line: milliseconds per append of the whole context (CUDA events on the launching stream, after a
 warm-up call, each repetition into a fresh cache so that every token is new), tokens/s, and the K/V bytes the
@@ -10,11 +10,17 @@ from __future__ import annotations
 
 import argparse
 import json
+import os
 import statistics
+import sys
 
 import torch
 
-from . import binding, build, runner, synth
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2601_22379_b200 import binding, build, runner, synth  # noqa: E402
 
 
 def main():

@@ -21,7 +21,7 @@
  * General rules
  *   - All device buffers are owned by the caller.  The library allocates no
  *     device memory, frees none, and never synchronises the device except in
- *     spla_sync_status and spla_decode_profile.  Every call enqueues its work on the given stream
+ *     spla_sync_status.  Every call enqueues its work on the given stream
  *     (a cudaStream_t passed as void*; NULL = the legacy default stream) and
  *     returns; results are ready when that stream reaches them.
  *   - Pointers marked DEVICE must be device memory of the current device,
@@ -31,8 +31,9 @@
  *   - Every function returns SPLA_OK (0) or a negative spla_status_t.
  *     Argument errors are detected on the host before anything is launched.
  *     A condition only the device can see (a sequence that would exceed
- *     max_context) skips the offending work without faulting and latches a
- *     status word that spla_sync_status reports.
+ *     max_context, a length or block index outside the cache, a copy that
+ *     did not arrive within the wait limit) skips the offending work without
+ *     faulting and latches a status word that spla_sync_status reports.
  *   - Query head m belongs to KV head m / G, G = n_q_heads / n_kv_heads.
  *   - Order per decode step: spla_append_tokens(k_t, v_t) then
  *     spla_decode(q_t): the query attends to every cached token, its own
@@ -54,7 +55,14 @@ typedef enum {
   SPLA_ERR_INVALID_ARG = -1,  /* NULL pointer, bad shape, misaligned buffer, workspace too small */
   SPLA_ERR_CAPACITY = -2,     /* an append would exceed max_context (host- or device-detected) */
   SPLA_ERR_CUDA = -3,         /* a CUDA runtime call or launch failed; see spla_last_cuda_error */
-  SPLA_ERR_UNSUPPORTED = -4   /* valid request outside what the kernels are built for */
+  SPLA_ERR_UNSUPPORTED = -4,  /* valid request outside what the kernels are built for */
+  SPLA_ERR_TIMEOUT = -5,      /* device-latched: a kernel's bounded wait for one of its own asynchronous copies ran out;
+                                 the kernel skipped the arithmetic that needed the data and returned (no trap, no hang);
+                                 the outputs of that call are undefined */
+  SPLA_ERR_BOUNDS = -6        /* device-latched: a length in seq_lens outside [0, max_context], an invalid entry of a
+                                 caller-given selection, or (SPLA_DEBUG_BOUNDS) a block index / token offset outside
+                                 the cache was met; the access was skipped or the value clamped, nothing out of range
+                                 was addressed */
 } spla_status_t;
 
 typedef enum { SPLA_F32 = 0, SPLA_BF16 = 1 } spla_dtype_t;
@@ -69,6 +77,10 @@ typedef enum { SPLA_F32 = 0, SPLA_BF16 = 1 } spla_dtype_t;
                                    rounded once (to nearest even) when written; the Taylor score of Section 3.1 reads
                                    the rounded values (ln n_i stays exact).  Halves the bytes the score streams; the
                                    paper does not say in which precision its block summaries are kept. */
+#define SPLA_DEBUG_BOUNDS 32u  /* checked mode (a stand-in for a memory checker): every kernel verifies the block index,
+                                   record range or token offset of each access it derives itself before making it;
+                                   a violation skips the access and latches SPLA_ERR_BOUNDS.  Same results otherwise.
+                                   Checks on caller-provided data (seq_lens, sel_in, n_new) are always on. */
 
 typedef struct {
   int32_t batch;          /* sequences per call, >= 1 */
@@ -116,9 +128,8 @@ typedef struct spla_cache spla_cache_t; /* opaque host-side descriptor */
 int spla_query_sizes(const spla_config_t *config, spla_sizes_t *sizes_out);
 
 /*
- * Bind caller-owned buffers to a descriptor (the paper's KV cache k_{1:N}, v_{1:N} "retained in memory to be
- * attended to by all future query vectors", Section 2, together with the block statistics of Section 3.1 and
- * the recurrent state of Eq. rla-impl-1).  Unless SPLA_ADOPT_CONTENTS is set, stats, rla_state, tok_lse,
+ * Bind caller-owned buffers to a descriptor: the KV cache k_{1:N}, v_{1:N} of Section 2, kept for all later
+ * queries, together with the block statistics of Section 3.1 and the recurrent state of Eq. rla-impl-1.  Unless SPLA_ADOPT_CONTENTS is set, stats, rla_state, tok_lse,
  * seq_lens are zeroed on `stream`; the workspace is always initialised.  K/V contents are never cleared.
  * config, buffers: HOST, copied.  *cache_out: HOST, receives a descriptor to release with spla_destroy_cache.
  */
@@ -174,25 +185,23 @@ int spla_select(spla_cache_t *cache, const void *q, int32_t *sel_idx, void *stre
 
 /*
  * Same as spla_decode with the selection given instead of computed (steps 3-5 only): sel_in DEVICE int32
- * [batch][H_kv][top_k], ascending valid block indices padded with -1.  For testing against an oracle when a
- * tie makes several index sets correct, and for callers that select elsewhere.
+ * [batch][H_kv][top_k], valid block indices padded with -1 at the tail.  For testing against an oracle when a
+ * tie makes several index sets correct, and for callers that select elsewhere.  The list is checked on the device:
+ * an entry that is negative before the tail, not below ceil(seq_len / B), or repeated is dropped (the remaining
+ * entries are attended to) and SPLA_ERR_BOUNDS is latched for spla_sync_status; nothing outside the cache is read.
  */
 int spla_decode_selected(spla_cache_t *cache, const void *q, const float *rms_weight, const int32_t *sel_in,
                          float *out, float *dbg_o_sparse, float *dbg_o_rla, void *stream);
 
-/*
- * Measurement aid: spla_decode with a CUDA event recorded on `stream` before, between and after its two
- * kernels, followed by a wait for the last event.  stage_ms: HOST float[2], receives the device time in
- * milliseconds of the score+select kernel and of the attend+merge kernel.  Unlike every other call this one
- * blocks the calling thread, and it may create three CUDA events on its first use for a cache.
- */
-int spla_decode_profile(spla_cache_t *cache, const void *q, const float *rms_weight, float *out, float *stage_ms,
-                        void *stream);
-
 /* Block scores of the last spla_decode: DEVICE fp32 [batch][H_kv][max_blocks] copy-out (entries >= nblk are 0). */
 int spla_copy_scores(spla_cache_t *cache, float *scores_out, void *stream);
 
-/* Waits for `stream`, then returns and clears the device-latched status (SPLA_OK or SPLA_ERR_CAPACITY). */
+/*
+ * Waits for `stream`, then returns and clears the device-latched status: SPLA_OK, or the code of the last condition
+ * a kernel latched since the previous call: SPLA_ERR_CAPACITY (an append skipped a sequence that would overflow),
+ * SPLA_ERR_BOUNDS (a length, selection entry or index outside the cache was clamped or skipped), SPLA_ERR_TIMEOUT (a
+ * bounded wait inside a kernel ran out).  SPLA_ERR_CUDA if the copy or the synchronisation itself fails.
+ */
 int spla_sync_status(spla_cache_t *cache, void *stream);
 
 /*
@@ -212,6 +221,8 @@ int spla_sync_status(spla_cache_t *cache, void *stream);
  *   q:          DEVICE [batch][H_q][d] q_dtype.
  *   sel_idx:    DEVICE int32 [batch][H_kv][top_k] output, ascending, padded with -1.
  *   scores_out: DEVICE fp32 [batch][H_kv][max_blocks] output or NULL (entries past the last block are 0).
+ *   status_out: DEVICE int32 [1] output or NULL: 0, or SPLA_ERR_BOUNDS if a length in seq_lens lay outside
+ *               [0, max_context] (it was clamped; the caller owns that buffer, so a stale one is easy to pass).
  * The call allocates nothing: no cudaMalloc / cudaFree and no allocating library routine.  Every GPU that loads
  * the library carries the SPLA_NOALLOC_SCRATCH_BYTES array until the process exits.  The first call on each
  * device looks up the array's device address (with that device current); make that first call outside any
@@ -221,15 +232,17 @@ int spla_sync_status(spla_cache_t *cache, void *stream);
  */
 #define SPLA_NOALLOC_SCRATCH_BYTES (4u << 20)
 int spla_select_blocks_noalloc(const spla_config_t *config, const float *stats, const int32_t *seq_lens,
-                               const void *q, int32_t *sel_idx, float *scores_out, void *stream);
+                               const void *q, int32_t *sel_idx, float *scores_out, int32_t *status_out, void *stream);
 
 /*
- * Measurement aid with no counterpart in the paper: one read-only pass over `bytes` bytes at `buf` (DEVICE,
- * 16-byte aligned; the contents do not matter and are not changed) by a plain streaming kernel, enqueued on
- * `stream`.  A caller times it with events to learn what a pure read stream reaches on its GPU; the benchmark
- * reports that figure beside the copy bandwidth.  Allocates nothing.
+ * Test hook for the failure path of the kernels' bounded waits (no counterpart in the paper).  Every wait of a decode
+ * kernel on one of its asynchronous copies polls a barrier a bounded number of times (2^22 by default) and, when the
+ * limit is reached, latches SPLA_ERR_TIMEOUT, skips the arithmetic and returns normally.  This call sets that limit
+ * for the decode kernels of `cache` (max_wait_polls > 0; 0 restores the default) and makes their copy barriers expect
+ * extra_expected_bytes more than will ever arrive (>= 0, a multiple of 16; 0 in normal use), so that a test can watch a
+ * wait run out without any fault, trap or endless loop on the device.  HOST values; affects later calls only.
  */
-int spla_probe_read(const void *buf, size_t bytes, void *stream);
+int spla_debug_wait_hook(spla_cache_t *cache, int32_t max_wait_polls, int32_t extra_expected_bytes);
 
 /* Tells the library an upper bound of the current sequence lengths after adopting contents (HOST value). */
 int spla_set_length_bound(spla_cache_t *cache, int32_t max_seq_len);
@@ -242,6 +255,9 @@ const char *spla_status_string(int status);
 
 /* Text of the last CUDA error this library saw on the calling thread ("" if none). */
 const char *spla_last_cuda_error(void);
+
+/* Number of kernels this library has launched (or recorded into a stream capture) from the calling thread so far. */
+unsigned long long spla_launch_count(void);
 
 #ifdef __cplusplus
 }

@@ -13,15 +13,16 @@ from dataclasses import dataclass
 import torch
 
 SPLA_OK, SPLA_ERR_INVALID_ARG, SPLA_ERR_CAPACITY, SPLA_ERR_CUDA, SPLA_ERR_UNSUPPORTED = 0, -1, -2, -3, -4
+SPLA_ERR_TIMEOUT, SPLA_ERR_BOUNDS = -5, -6
 SPLA_F32, SPLA_BF16 = 0, 1
-SPLA_ADOPT_CONTENTS, SPLA_FIRST_ORDER, SPLA_NO_RLA, SPLA_GENERAL_KERNELS, SPLA_STATS_BF16 = 1, 2, 4, 8, 16
+SPLA_ADOPT_CONTENTS, SPLA_FIRST_ORDER, SPLA_NO_RLA, SPLA_GENERAL_KERNELS, SPLA_STATS_BF16, SPLA_DEBUG_BOUNDS = 1, 2, 4, 8, 16, 32
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libspla.so")
 
 EXPORTS = ["spla_query_sizes", "spla_init_cache", "spla_append_tokens", "spla_decode", "spla_decode_selected",
-           "spla_decode_profile", "spla_select_blocks_noalloc", "spla_select", "spla_append_decode",
-           "spla_copy_scores", "spla_probe_read", "spla_sync_status", "spla_set_length_bound", "spla_destroy_cache",
-           "spla_status_string", "spla_last_cuda_error"]
+           "spla_select_blocks_noalloc", "spla_select", "spla_append_decode",
+           "spla_copy_scores", "spla_sync_status", "spla_set_length_bound", "spla_debug_wait_hook", "spla_destroy_cache",
+           "spla_launch_count", "spla_status_string", "spla_last_cuda_error"]
 
 
 class SplaConfig(C.Structure):
@@ -69,15 +70,16 @@ def load(path: str | None = None) -> C.CDLL:
     lib.spla_decode_selected.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.spla_select.argtypes = [vp, vp, vp, vp]
     lib.spla_append_decode.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp]
-    lib.spla_decode_profile.argtypes = [vp, vp, vp, vp, C.POINTER(C.c_float), vp]
-    lib.spla_select_blocks_noalloc.argtypes = [C.POINTER(SplaConfig), vp, vp, vp, vp, vp, vp]
+    lib.spla_select_blocks_noalloc.argtypes = [C.POINTER(SplaConfig), vp, vp, vp, vp, vp, vp, vp]
     lib.spla_copy_scores.argtypes = [vp, vp, vp]
-    lib.spla_probe_read.argtypes = [vp, C.c_size_t, vp]
+    lib.spla_debug_wait_hook.argtypes = [vp, i32, i32]
     lib.spla_sync_status.argtypes = [vp, vp]
     lib.spla_set_length_bound.argtypes = [vp, i32]
     lib.spla_destroy_cache.argtypes = [vp]
-    for name in EXPORTS[:-2]:
+    for name in EXPORTS[:-3]:
         getattr(lib, name).restype = C.c_int
+    lib.spla_launch_count.argtypes = []
+    lib.spla_launch_count.restype = C.c_ulonglong
     lib.spla_status_string.argtypes = [C.c_int]
     lib.spla_status_string.restype = C.c_char_p
     lib.spla_last_cuda_error.argtypes = []
@@ -139,7 +141,8 @@ NOALLOC_SCRATCH_BYTES = 4 << 20
 
 
 def select_blocks_noalloc(cfg: SplaConfig, stats: torch.Tensor, seq_lens: torch.Tensor, q: torch.Tensor,
-                          sel_idx: torch.Tensor, scores_out: torch.Tensor | None = None) -> int:
+                          sel_idx: torch.Tensor, scores_out: torch.Tensor | None = None,
+                          status_out: torch.Tensor | None = None) -> int:
     """Score + select for callers that may not allocate on the device: every tensor is passed in, the kernel's
     scratch is a fixed array inside the library.  Returns the status code (0 = ok) instead of raising, so that a
     caller can fall back to `SplaCache.decode` when the configuration exceeds the fixed scratch.  Calls share
@@ -148,14 +151,12 @@ def select_blocks_noalloc(cfg: SplaConfig, stats: torch.Tensor, seq_lens: torch.
     assert seq_lens.dtype == torch.int32 and sel_idx.dtype == torch.int32 and q.is_contiguous()
     with torch.cuda.device(stats.device):
         return load().spla_select_blocks_noalloc(C.byref(cfg), stats.data_ptr(), seq_lens.data_ptr(), q.data_ptr(),
-                                                 sel_idx.data_ptr(), _ptr(scores_out), _stream())
+                                                 sel_idx.data_ptr(), _ptr(scores_out), _ptr(status_out), _stream())
 
 
-def probe_read(buf: torch.Tensor):
-    """One read-only streaming pass over a device tensor (measurement aid)."""
-    assert buf.is_cuda and buf.is_contiguous()
-    with torch.cuda.device(buf.device):
-        _check(load().spla_probe_read(buf.data_ptr(), buf.numel() * buf.element_size(), _stream()), "spla_probe_read")
+def launch_count() -> int:
+    """Kernels the library has launched (or recorded into a graph capture) from this thread so far."""
+    return int(load().spla_launch_count())
 
 
 class SplaCache:
@@ -269,14 +270,6 @@ class SplaCache:
                    "spla_decode_selected")
         return out
 
-    def decode_profile(self, q, rms_weight, out: torch.Tensor):
-        """Blocking decode that returns (score_select_ms, attend_merge_ms) measured with CUDA events."""
-        ms = (C.c_float * 2)()
-        with torch.cuda.device(self.device):
-            _check(self.lib.spla_decode_profile(self.handle, q.data_ptr(), _ptr(rms_weight), out.data_ptr(), ms,
-                                                _stream()), "spla_decode_profile")
-        return float(ms[0]), float(ms[1])
-
     # -- helpers ------------------------------------------------------------------------------------------
     def scores(self) -> torch.Tensor:
         out = torch.empty(self.cfg.batch, self.cfg.n_kv_heads, self.max_blocks, dtype=torch.float32,
@@ -288,6 +281,10 @@ class SplaCache:
     def sync_status(self) -> int:
         with torch.cuda.device(self.device):
             return self.lib.spla_sync_status(self.handle, _stream())
+
+    def debug_wait_hook(self, max_wait_polls: int, extra_expected_bytes: int):
+        """Test hook: wait limit of the decode kernels' copy barriers and bytes they expect in excess (see spla.h)."""
+        _check(self.lib.spla_debug_wait_hook(self.handle, max_wait_polls, extra_expected_bytes), "spla_debug_wait_hook")
 
     def set_length_bound(self, n: int):
         _check(self.lib.spla_set_length_bound(self.handle, n), "spla_set_length_bound")

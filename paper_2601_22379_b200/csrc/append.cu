@@ -22,7 +22,7 @@ constexpr int kStateUmmaMinTokens = 256;   // appends at least this long take th
 __device__ __forceinline__ int tokens_to_add(const Params& p, const int* n_new, int max_new, int b, int L) {
   int n = n_new ? n_new[b] : max_new;
   n = max(0, min(n, max_new));
-  if (L + n > p.max_context) return -1;      // would overflow: skip this sequence, the caller is told via status
+  if (L < 0 || L + n > p.max_context) return -1;   // would overflow (or a corrupt length): skip this sequence, the caller is told via status
   return n;
 }
 
@@ -127,13 +127,17 @@ __global__ void __launch_bounds__(kStatThreads) append_block_kernel(const Params
   const int L = p.seq_lens[b];
   const int n = tokens_to_add(p, n_new, max_new, b, L);
   if (n < 0) {
-    if (blockIdx.x == 0 && tid == 0) atomicExch(p.status, -2);
+    if (blockIdx.x == 0 && tid == 0) atomicExch(p.status, kStatusCapacity);
     return;
   }
   const int blk = L / p.B + blockIdx.x;
   const int t0 = blk * p.B;
   if (n == 0 || t0 >= L + n) return;                 // CTA-uniform
   const int cnt = min(p.B, L + n - t0);              // tokens the block holds after the append
+  if ((p.flags & kDebugBounds) && (blk < 0 || blk >= p.max_blocks)) {   // checked build: the block must exist (CTA-uniform)
+    if (tid == 0) atomicExch(p.status, kStatusBounds);
+    return;
+  }
   const int t_new = max(0, L - t0);                  // its first new token
 
   const size_t blk_tok0 = (size_t)u * p.max_blocks * p.B + t0;
@@ -291,9 +295,14 @@ __global__ void __launch_bounds__(kFusedThreads, 4) append_fused_kernel(const Pa
 
   if (role < n_copy) {
     // ---- copy role: one warp per token; also the per-token log-sum-exp the decode reads ------------------
-    if (n < 0 && role == 0 && tid == 0) atomicExch(p.status, -2);
+    if (n < 0 && role == 0 && tid == 0) atomicExch(p.status, kStatusCapacity);
     const int i = role * (kFusedThreads / 32) + warp;
-    if (n > 0 && i < n) {
+    bool in_cache = true;
+    if ((p.flags & kDebugBounds) && n > 0 && i < n && L + i >= p.max_blocks * p.B) {   // checked build
+      if (lane == 0) atomicExch(p.status, kStatusBounds);
+      in_cache = false;
+    }
+    if (n > 0 && i < n && in_cache) {
       const size_t pos = unit_tok0 + (size_t)(L + i);
       float k[VEC];
       load_vec<VEC>(kn + (size_t)i * D + lane * VEC, k);
@@ -403,6 +412,7 @@ static cudaError_t launch_typed(const Params& p, const void* k_new, const void* 
     auto kern = append_block_kernel<T, D>;
     if (tile_bytes > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tile_bytes);
     kern<<<dim3((max_new + p.B - 1) / p.B + 1, U), kStatThreads, tile_bytes, stream>>>(p, kn, vn, n_new, max_new);
+    ++g_launch_count;
   }
   if (!(p.flags & 4u)) {
     // long appends of a bf16 cache with d = 128: the rank-n update is a dense contraction, done on the tensor cores
@@ -412,9 +422,11 @@ static cudaError_t launch_typed(const Params& p, const void* k_new, const void* 
       if (e != cudaSuccess) return e;
     } else {
       append_state_kernel<T, D><<<dim3(D / kStateRows, U), D, 0, stream>>>(p, kn, vn, n_new, max_new);
+      ++g_launch_count;
     }
   }
   append_lengths_kernel<<<(p.batch + 127) / 128, 128, 0, stream>>>(p, n_new, max_new);
+  ++g_launch_count;
   return cudaGetLastError();
 }
 

@@ -40,7 +40,7 @@ __device__ __forceinline__ void merge_unit(const Params& p, int u, int n_items, 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = p.G;
   const int b = u / p.Hkv, h = u % p.Hkv;
-  const int nblk_u = (p.seq_lens[b] + p.B - 1) / p.B;
+  const int nblk_u = (checked_len(p, b) + p.B - 1) / p.B;
   const bool rla = !(p.flags & 4u) && p.n_sel[u] < nblk_u;
   float* wt_s = smem;                                // [n_items][G]: exp2(m_it - M) / L
 

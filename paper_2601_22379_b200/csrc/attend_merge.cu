@@ -38,8 +38,14 @@ __global__ void __launch_bounds__(kAttendThreads) attend_merge_kernel(const Para
     return;
   }
   const int blk = p.sel[(size_t)u * p.top_k + item];
-  const int L = p.seq_lens[b];
-  const int n_tok = min(B, L - blk * B);
+  const int L = checked_len(p, b);
+  int n_tok = min(B, L - blk * B);
+  if ((p.flags & kDebugBounds) && (blk < 0 || blk >= p.max_blocks || n_tok <= 0)) {
+    // checked build: a block index that does not name a cached block is reported and the block is treated as empty
+    if (tid == 0) atomicExch(p.status, kStatusBounds);
+    n_tok = 0;
+  }
+  const bool fetch = n_tok > 0;
 
   // shared memory carve-up
   T* Ks = reinterpret_cast<T*>(smem_raw);
@@ -50,11 +56,12 @@ __global__ void __launch_bounds__(kAttendThreads) attend_merge_kernel(const Para
   uint64_t* bar = reinterpret_cast<uint64_t*>(misc + 4 * GP + 2 * NWARP * GP);
   __shared__ int flag_s;
 
-  if (tid == 0) {
+  if (tid == 0 && !fetch) mbar_init(bar, 1);
+  if (tid == 0 && fetch) {
     mbar_init(bar, 1);
     const size_t tile = (size_t)u * p.max_blocks + blk;
     const uint32_t tile_bytes = (uint32_t)((size_t)B * D * sizeof(T));
-    mbar_expect_tx(bar, 2 * tile_bytes + (uint32_t)(B * sizeof(float)));
+    mbar_expect_tx(bar, 2 * tile_bytes + (uint32_t)(B * sizeof(float)) + (uint32_t)p.dbg_tx_extra);
     bulk_g2s(Ks, reinterpret_cast<const T*>(p.k_cache) + tile * B * D, tile_bytes, bar);
     bulk_g2s(Vs, reinterpret_cast<const T*>(p.v_cache) + tile * B * D, tile_bytes, bar);
     bulk_g2s(lse_s, p.tok_lse + tile * B, (uint32_t)(B * sizeof(float)), bar);
@@ -92,10 +99,10 @@ __global__ void __launch_bounds__(kAttendThreads) attend_merge_kernel(const Para
     }
   }
   __syncthreads();                               // barrier initialised before anyone polls it
-  bool arrived = mbar_wait(bar, 0);
-  if (!arrived) {                                // never expected: report it, give the copies a second bounded wait, skip the math
-    if (tid == 0) atomicExch(p.status, -3);
-    mbar_wait(bar, 0);
+  bool arrived = fetch && mbar_wait(bar, 0, p.wait_limit);
+  if (fetch && !arrived) {                                // never expected: report it, give the copies a second bounded wait, skip the math
+    if (tid == 0) atomicExch(p.status, kStatusTimeout);
+    mbar_wait(bar, 0, p.wait_limit);
   }
 
   // ---- pass 1: logits and linear coefficients per token ----------------------------------------------
@@ -210,19 +217,35 @@ __global__ void __launch_bounds__(kAttendThreads) attend_merge_kernel(const Para
   merge_unit<D>(p, u, nsel, rms_weight, out, dbg_sparse, dbg_rla, reinterpret_cast<float*>(smem_raw));
 }
 
-// Copies a caller-given selection into the workspace and counts its valid entries.
-__global__ void adopt_selection_kernel(const Params p, const int* __restrict__ sel_in) {
-  const int u = blockIdx.x;
-  __shared__ int cnt;
-  if (threadIdx.x == 0) cnt = 0;
+// Takes a caller-given selection into the workspace.  The list is not trusted: only entries that name an existing
+// block of the sequence (0 <= index < ceil(L / B)) and that are not repeated are kept, in the order given, packed to
+// the front; the rest of the row is padded with -1.  Anything dropped other than the -1 padding at the tail (a hole,
+// an index past the last block, a duplicate) is reported through the status word, and nothing outside the cache is
+// ever addressed because of it.  One CTA of kMaxTopK threads per unit.
+__global__ void __launch_bounds__(kMaxTopK) adopt_selection_kernel(const Params p, const int* __restrict__ sel_in) {
+  const int u = blockIdx.x, b = u / p.Hkv, t = threadIdx.x;
+  __shared__ int raw_s[kMaxTopK];
+  __shared__ int keep_s[kMaxTopK];
+  const int nblk = (checked_len(p, b) + p.B - 1) / p.B;
+  const int v = t < p.top_k ? sel_in[(size_t)u * p.top_k + t] : -1;
+  raw_s[t] = v;
   __syncthreads();
-  for (int t = threadIdx.x; t < p.top_k; t += blockDim.x) {
-    const int v = sel_in[(size_t)u * p.top_k + t];
-    p.sel[(size_t)u * p.top_k + t] = v;
-    if (v >= 0) atomicAdd(&cnt, 1);
+  bool keep = v >= 0 && v < nblk;
+  for (int j = 0; keep && j < t; ++j) keep = raw_s[j] != v;          // a repeated block would be attended to twice
+  keep_s[t] = keep;
+  __syncthreads();
+  int pos = 0, total = 0, last_given = -1;
+  for (int j = 0; j < p.top_k; ++j) {
+    pos += (j < t) && keep_s[j];
+    total += keep_s[j];
+    if (raw_s[j] != -1) last_given = j;
   }
-  __syncthreads();
-  if (threadIdx.x == 0) p.n_sel[u] = cnt;
+  if (keep) p.sel[(size_t)u * p.top_k + pos] = v;
+  if (t >= total && t < p.top_k) p.sel[(size_t)u * p.top_k + t] = -1;
+  if (t == 0) {
+    p.n_sel[u] = total;
+    if (total != last_given + 1) atomicExch(p.status, kStatusBounds);   // something other than tail padding was dropped
+  }
 }
 
 template <typename T, int D, int GP>
@@ -241,6 +264,7 @@ static cudaError_t launch_one(const Params& p, const void* q, int qb, const floa
   if (e != cudaSuccess) return e;
   dim3 grid(p.top_k, p.batch * p.Hkv);
   kern<<<grid, kAttendThreads, smem, stream>>>(p, q, qb, w, out, ds, dr);
+  ++g_launch_count;
   return cudaGetLastError();
 }
 
@@ -260,7 +284,8 @@ cudaError_t launch_attend_merge(const Params& p, const AttendMaps* maps, const v
                                 const float* rms_weight, const int* sel_in, float* out, float* dbg_o_sparse,
                                 float* dbg_o_rla, cudaStream_t stream) {
   if (sel_in) {
-    adopt_selection_kernel<<<p.batch * p.Hkv, 64, 0, stream>>>(p, sel_in);
+    adopt_selection_kernel<<<p.batch * p.Hkv, kMaxTopK, 0, stream>>>(p, sel_in);
+    ++g_launch_count;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }

@@ -9,8 +9,12 @@
 // where phi(K) is formed element-wise from the very K fragments just used (one ex2 per element, with the cached
 // per-token log-sum-exp), so the selected linear term reads nothing extra.  After the online softmax on rows
 // 0..7 the tile [P ; A] is the left operand of one product with the V tile, which accumulates the softmax
-// numerator and o_tilde together.  The linear coefficients keep ~16 bits: bf16 head plus bf16 remainder (for
-// groups of up to 4 heads the remainder rides in the rows that would otherwise be padding).
+// numerator and o_tilde together.  The linear branch keeps far more than the 8 or 11 bits of one 16-bit operand,
+// because o_bar - o_tilde cancels when most of the context is selected and the RMSNorm then rescales the
+// difference (Section 3.2, "Numerical Stability": the states stay in high precision): phi(q) and phi(k) enter
+// their product as an fp16 head plus an fp16 remainder each, and the coefficients phi(q).phi(k_t) enter the
+// product with V as three bf16 parts.  For groups of up to 4 heads the
+// extra parts ride in the accumulator rows that would otherwise be padding.
 //
 // Merge (Eq. rla-impl-3, Section 3.3): after a hardware cluster barrier CTA g of the cluster pulls head g's
 // partial results from its siblings over distributed shared memory, subtracts o_tilde from o_bar, applies the
@@ -79,6 +83,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
+__device__ __forceinline__ float f16_lo(uint32_t x) { return __low2float(*reinterpret_cast<const __half2*>(&x)); }
+__device__ __forceinline__ float f16_hi(uint32_t x) { return __high2float(*reinterpret_cast<const __half2*>(&x)); }
 __device__ __forceinline__ float bf16_lo(uint32_t x) { return __uint_as_float(x << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
 
@@ -117,36 +123,52 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
   // dependent launch this part overlaps that kernel's tail.  Rows = heads of the group, held in registers.
   // qa: rows 0..7 of the first product (raw q; the softmax scale is applied to the fp32 logits);
   // fa: rows 8..15 of the second product, phi(q) = softmax(phi_scale * q) in fp16.
-  uint32_t qa[KS][2], fa[KS][2];
+  // fl (groups of more than 4 heads only): the fp16 remainder of phi(q), a second left operand; in the packed
+  // layout rows 12..15 of fa carry that remainder for heads 0..3 instead.
+  uint32_t qa[KS][2], fa[KS][2], fl[PACK ? 1 : KS][2];
   {
     const bool hv = g < G;
-    const uint32_t* qrow = reinterpret_cast<const uint32_t*>(q + ((size_t)b * p.Hq + (size_t)h * G + (hv ? g : 0)) * D);
+    const bool rem_row = PACK && g >= 4;                  // this lane's row 8 + g holds the remainder of head g - 4
+    const int hq = rem_row ? g - 4 : g;                   // head whose phi(q) this lane forms
+    const bool hp = hq < G;
+    const uint32_t* qrow = reinterpret_cast<const uint32_t*>(q + ((size_t)b * p.Hq + (size_t)h * G + (hp ? hq : 0)) * D);
     const float a2 = p.phi_scale * kLog2e;
     float mx = -INFINITY;
+    uint32_t qr[KS][2];
 #pragma unroll
     for (int kk = 0; kk < KS; ++kk) {
-      qa[kk][0] = hv ? __ldg(qrow + 8 * kk + t) : 0u;
-      qa[kk][1] = hv ? __ldg(qrow + 8 * kk + 4 + t) : 0u;
+      qr[kk][0] = hp ? __ldg(qrow + 8 * kk + t) : 0u;
+      qr[kk][1] = hp ? __ldg(qrow + 8 * kk + 4 + t) : 0u;
+      qa[kk][0] = hv ? qr[kk][0] : 0u;                    // rows of padding carry zero queries in the exact branch
+      qa[kk][1] = hv ? qr[kk][1] : 0u;
     }
 #pragma unroll
     for (int kk = 0; kk < KS; ++kk)
-      mx = fmaxf(mx, fmaxf(fmaxf(bf16_lo(qa[kk][0]), bf16_hi(qa[kk][0])), fmaxf(bf16_lo(qa[kk][1]), bf16_hi(qa[kk][1]))));
+      mx = fmaxf(mx, fmaxf(fmaxf(bf16_lo(qr[kk][0]), bf16_hi(qr[kk][0])), fmaxf(bf16_lo(qr[kk][1]), bf16_hi(qr[kk][1]))));
     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
     mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
     float e[KS][4], sum = 0.f;
 #pragma unroll
     for (int kk = 0; kk < KS; ++kk) {
-      e[kk][0] = exp2f((bf16_lo(qa[kk][0]) - mx) * a2); e[kk][1] = exp2f((bf16_hi(qa[kk][0]) - mx) * a2);
-      e[kk][2] = exp2f((bf16_lo(qa[kk][1]) - mx) * a2); e[kk][3] = exp2f((bf16_hi(qa[kk][1]) - mx) * a2);
+      e[kk][0] = exp2f((bf16_lo(qr[kk][0]) - mx) * a2); e[kk][1] = exp2f((bf16_hi(qr[kk][0]) - mx) * a2);
+      e[kk][2] = exp2f((bf16_lo(qr[kk][1]) - mx) * a2); e[kk][3] = exp2f((bf16_hi(qr[kk][1]) - mx) * a2);
       sum += (e[kk][0] + e[kk][1]) + (e[kk][2] + e[kk][3]);
     }
     sum += __shfl_xor_sync(0xffffffffu, sum, 1);
     sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-    const float inv = (hv && rla_on) ? 1.f / sum : 0.f;
+    const float inv = (hp && rla_on) ? 1.f / sum : 0.f;
 #pragma unroll
     for (int kk = 0; kk < KS; ++kk) {
-      fa[kk][0] = pack_f16(e[kk][0] * inv, e[kk][1] * inv);
-      fa[kk][1] = pack_f16(e[kk][2] * inv, e[kk][3] * inv);
+      const float f0 = e[kk][0] * inv, f1 = e[kk][1] * inv, f2 = e[kk][2] * inv, f3 = e[kk][3] * inv;
+      const uint32_t h0 = pack_f16(f0, f1), h1 = pack_f16(f2, f3);
+      const uint32_t l0 = pack_f16(f0 - f16_lo(h0), f1 - f16_hi(h0)), l1 = pack_f16(f2 - f16_lo(h1), f3 - f16_hi(h1));
+      if constexpr (PACK) {
+        fa[kk][0] = rem_row ? l0 : h0;
+        fa[kk][1] = rem_row ? l1 : h1;
+      } else {
+        fa[kk][0] = h0; fa[kk][1] = h1;
+        fl[kk][0] = l0; fl[kk][1] = l1;
+      }
     }
   }
   if (tid == 0) {
@@ -156,9 +178,24 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
 
   pdl_wait();                                   // the selection of this step is complete and visible from here on
 
-  const int nsel = __ldcg(p.n_sel + u);
-  const int L = __ldcg(p.seq_lens + b);
+  int nsel = __ldcg(p.n_sel + u);
+  const int L = checked_len(p, b);
   for (int i = tid; i < p.top_k; i += kAttendThreads) sel_s[i] = __ldcg(p.sel + (size_t)u * p.top_k + i);
+  if (p.flags & kDebugBounds) {
+    // checked build: the list must name nsel existing blocks; it is cut at the first entry that does not, and the
+    // status word says so (every CTA of the cluster sees the same list and cuts it at the same place)
+    __shared__ int first_bad_s;
+    if (tid == 0) first_bad_s = min(max(nsel, 0), p.top_k);
+    __syncthreads();
+    const int nblk_chk = (L + B - 1) / B;
+    for (int i = tid; i < min(nsel, p.top_k); i += kAttendThreads)
+      if (sel_s[i] < 0 || sel_s[i] >= nblk_chk) atomicMin(&first_bad_s, i);
+    __syncthreads();
+    if (first_bad_s != nsel) {
+      if (tid == 0 && rank == 0) atomicExch(p.status, kStatusBounds);
+      nsel = first_bad_s;
+    }
+  }
   __syncthreads();                              // selection list and barrier initialisation visible to the CTA
   SPLA_MARK(p, u, 32 + rank, 0);
 
@@ -167,10 +204,10 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
   const int slot_bytes = (2 * tile_bytes + B * 4 + 1023) & ~1023;   // K tile, V tile, per-token lse; the swizzle needs 1 KB alignment
   auto issue = [&](int i) {                                          // thread 0 only
     const int slot = i & 1;
-    const int blk = sel_s[rank + i * CS];
+    const int blk = min(max(sel_s[rank + i * CS], 0), p.max_blocks - 1);   // (a list entry can never address outside the cache)
     const uint32_t base = smem_u32(smem_raw + (size_t)slot * slot_bytes);
     const int row0 = (int)(((size_t)u * p.max_blocks + blk) * B);
-    mbar_expect_tx(&full[slot], (uint32_t)(2 * tile_bytes + B * 4));
+    mbar_expect_tx(&full[slot], (uint32_t)(2 * tile_bytes + B * 4 + p.dbg_tx_extra));
 #pragma unroll
     for (int hh = 0; hh < NH; ++hh) {
       tma_load_2d(base + hh * (B * 128), &map_k, hh * 64, row0, &full[slot]);
@@ -195,7 +232,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
 #pragma unroll 1
   for (int i = 0; i < nb; ++i) {
     const int slot = i & 1;
-    if (!mbar_wait(&full[slot], (i >> 1) & 1)) { if (lane == 0) atomicExch(&err_s, 1); break; }
+    if (!mbar_wait(&full[slot], (i >> 1) & 1, p.wait_limit)) { if (lane == 0) atomicExch(&err_s, 1); break; }
     if (i == 0) SPLA_MARK(p, u, 32 + rank, 2);
     unsigned char* sb = smem_raw + (size_t)slot * slot_bytes;
     const uint32_t ks = smem_u32(sb);
@@ -234,14 +271,30 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
         ldmatrix_x4(kb, krow + (ch >> 3) * half_bytes + (((ch & 7) ^ r8) << 4));
         mma_bf16(sacc[0], qa[kk][0], 0u, qa[kk][1], 0u, kb[0], kb[1]);
         mma_bf16(sacc[1], qa[kk][0], 0u, qa[kk][1], 0u, kb[2], kb[3]);
-        uint32_t pb[4];
+        // phi(k) of the same fragments, as an fp16 head and an fp16 remainder (together 17 or more significant bits)
+        uint32_t pb[4], pl[4];
 #pragma unroll
         for (int x = 0; x < 4; ++x) {
           const float ls = x < 2 ? lse2_0 : lse2_1;
-          pb[x] = pack_f16(ex2(fmaf(bf16_lo(kb[x]), a2, -ls)), ex2(fmaf(bf16_hi(kb[x]), a2, -ls)));
+          const float e0 = ex2(fmaf(bf16_lo(kb[x]), a2, -ls)), e1 = ex2(fmaf(bf16_hi(kb[x]), a2, -ls));
+          pb[x] = pack_f16(e0, e1);
+          pl[x] = pack_f16(e0 - f16_lo(pb[x]), e1 - f16_hi(pb[x]));
         }
         mma_f16(aacc[0], 0u, fa[kk][0], 0u, fa[kk][1], pb[0], pb[1]);
         mma_f16(aacc[1], 0u, fa[kk][0], 0u, fa[kk][1], pb[2], pb[3]);
+        mma_f16(aacc[0], 0u, fa[kk][0], 0u, fa[kk][1], pl[0], pl[1]);
+        mma_f16(aacc[1], 0u, fa[kk][0], 0u, fa[kk][1], pl[2], pl[3]);
+        if constexpr (!PACK) {                         // remainder of phi(q) times the head of phi(k)
+          mma_f16(aacc[0], 0u, fl[kk][0], 0u, fl[kk][1], pb[0], pb[1]);
+          mma_f16(aacc[1], 0u, fl[kk][0], 0u, fl[kk][1], pb[2], pb[3]);
+        }
+      }
+      if constexpr (PACK) {                            // rows 12..15 (remainder of phi(q)) onto rows 8..11
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+          aacc[nt][2] += __shfl_down_sync(0xffffffffu, aacc[nt][2], 16);
+          aacc[nt][3] += __shfl_down_sync(0xffffffffu, aacc[nt][3], 16);
+        }
       }
       // online softmax on rows 0..7; rows 8..15 stay linear.  Tokens past the end of the sequence are masked.
       float mx = -INFINITY;
@@ -269,14 +322,21 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
       }
       l_run = fmaf(l_run, corr, psum);
       // [P ; A] as the left operand of the product with V (bf16, like V).  The linear coefficients are split
-      // into a bf16 head and a bf16 remainder so that o_tilde keeps ~16 bits of them.
-      const uint32_t pa0 = pack_bf16(sacc[0][0], sacc[0][1]), pa2 = pack_bf16(sacc[1][0], sacc[1][1]);
+      // into three bf16 parts (head, remainder, remainder of that) so that o_tilde keeps ~24 bits of them.
+      uint32_t pa0 = pack_bf16(sacc[0][0], sacc[0][1]), pa2 = pack_bf16(sacc[1][0], sacc[1][1]);
       uint32_t pa1 = pack_bf16(sacc[0][2], sacc[0][3]), pa3 = pack_bf16(sacc[1][2], sacc[1][3]);
-      const uint32_t ra1 = pack_bf16(sacc[0][2] - bf16_lo(pa1), sacc[0][3] - bf16_hi(pa1));
-      const uint32_t ra3 = pack_bf16(sacc[1][2] - bf16_lo(pa3), sacc[1][3] - bf16_hi(pa3));
-      if constexpr (PACK) {                            // rows 12..15 <- remainders of heads 0..3 (lanes 16 below)
+      const float r00 = sacc[0][2] - bf16_lo(pa1), r01 = sacc[0][3] - bf16_hi(pa1);
+      const float r10 = sacc[1][2] - bf16_lo(pa3), r11 = sacc[1][3] - bf16_hi(pa3);
+      const uint32_t ra1 = pack_bf16(r00, r01), ra3 = pack_bf16(r10, r11);
+      const uint32_t rb1 = pack_bf16(r00 - bf16_lo(ra1), r01 - bf16_hi(ra1));
+      const uint32_t rb3 = pack_bf16(r10 - bf16_lo(ra3), r11 - bf16_hi(ra3));
+      float corr_o = corr;
+      if constexpr (PACK) {
+        // rows 12..15 <- second parts of heads 0..3, rows 4..7 <- their third parts (from the lanes 16 below);
+        // rows 4..7 then accumulate a linear term and must not take the softmax rescaling
         const uint32_t u1 = __shfl_up_sync(0xffffffffu, ra1, 16), u3 = __shfl_up_sync(0xffffffffu, ra3, 16);
-        if (g >= 4) { pa1 = u1; pa3 = u3; }
+        const uint32_t w1 = __shfl_up_sync(0xffffffffu, rb1, 16), w3 = __shfl_up_sync(0xffffffffu, rb3, 16);
+        if (g >= 4) { pa1 = u1; pa3 = u3; pa0 = w1; pa2 = w3; corr_o = 1.f; }
       }
       const uint32_t vrow = vs + (tok0 + (mi & 1) * 8 + r8) * 128;
 #pragma unroll
@@ -284,14 +344,16 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
         uint32_t vb[4];
         const int ch = 2 * np + (mi >> 1);
         ldmatrix_x4_trans(vb, vrow + (ch >> 3) * half_bytes + (((ch & 7) ^ r8) << 4));
-        o[2 * np][0] *= corr; o[2 * np][1] *= corr;
-        o[2 * np + 1][0] *= corr; o[2 * np + 1][1] *= corr;
+        o[2 * np][0] *= corr_o; o[2 * np][1] *= corr_o;
+        o[2 * np + 1][0] *= corr_o; o[2 * np + 1][1] *= corr_o;
         mma_bf16(o[2 * np], pa0, pa1, pa2, pa3, vb[0], vb[1]);
         mma_bf16(o[2 * np + 1], pa0, pa1, pa2, pa3, vb[2], vb[3]);
         if constexpr (!PACK) {
           if (rla_on) {
             mma_bf16(o[2 * np], 0u, ra1, 0u, ra3, vb[0], vb[1]);
             mma_bf16(o[2 * np + 1], 0u, ra1, 0u, ra3, vb[2], vb[3]);
+            mma_bf16(o[2 * np], 0u, rb1, 0u, rb3, vb[0], vb[1]);
+            mma_bf16(o[2 * np + 1], 0u, rb1, 0u, rb3, vb[2], vb[3]);
           }
         }
       }
@@ -302,7 +364,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
       issue(i + kSlots);
     }
   }
-  if (tid == 0 && err_s) atomicExch(p.status, -3);
+  if (tid == 0 && err_s) atomicExch(p.status, kStatusTimeout);
 
   SPLA_MARK(p, u, 32 + rank, 3);
   // ---- fold the four warps together ------------------------------------------------------------------------
@@ -320,12 +382,13 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
 #pragma unroll
   for (int w = 1; w < NWARP; ++w) M = fmaxf(M, red_m[w * 8 + g]);
   const float f = M > -INFINITY ? ex2(m_run - M) : 0.f;                 // 0 for a warp (or a CTA) that saw no token
+  const float f_o = (PACK && g >= 4) ? 1.f : f;                         // packed rows 4..7 belong to the linear branch
   if (t == 0) red_l[warp * 8 + g] = l_run * f;
   {
     float* ro = red_o + (size_t)warp * 16 * (D + kPad);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-      *reinterpret_cast<float2*>(ro + (size_t)g * (D + kPad) + nt * 8 + 2 * t) = make_float2(o[nt][0] * f, o[nt][1] * f);
+      *reinterpret_cast<float2*>(ro + (size_t)g * (D + kPad) + nt * 8 + 2 * t) = make_float2(o[nt][0] * f_o, o[nt][1] * f_o);
       *reinterpret_cast<float2*>(ro + (size_t)(g + 8) * (D + kPad) + nt * 8 + 2 * t) = make_float2(o[nt][2], o[nt][3]);
     }
   }
@@ -338,7 +401,8 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
 #pragma unroll
       for (int w = 0; w < NWARP; ++w) {
         s += red_o[((size_t)w * 16 + rr) * (D + kPad) + col];
-        if (PACK && br == 1) s += red_o[((size_t)w * 16 + rr + 4) * (D + kPad) + col];
+        if (PACK && br == 1)                                              // the second and third parts of the coefficients
+          s += red_o[((size_t)w * 16 + rr + 4) * (D + kPad) + col] + red_o[((size_t)w * 16 + hd + 4) * (D + kPad) + col];
       }
     }
     mine[idx] = s;

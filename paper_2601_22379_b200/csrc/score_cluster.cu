@@ -260,11 +260,11 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   int L0;
   if (EARLY) {                                    // one read for the whole CTA: the value may change under our feet
     __shared__ int l0_s;
-    if (tid == 0) l0_s = __ldcg(p.seq_lens + b);
+    if (tid == 0) l0_s = cover_len(p, checked_len(p, b), (long long)CS * chunk * p.B);
     __syncthreads();
     L0 = l0_s;
   } else {
-    L0 = __ldcg(p.seq_lens + b);
+    L0 = cover_len(p, checked_len(p, b), (long long)CS * chunk * p.B);
   }
   int L = L0;
   int nblk = (L + p.B - 1) / p.B;
@@ -277,9 +277,13 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
 
   auto issue = [&](int r) {                      // thread 0 only: one bulk copy fills stage r % kStages
     const int s = r % kStages;
-    const int nrec = min(kStageRec, n_stream - r * kStageRec);
+    int nrec = min(kStageRec, n_stream - r * kStageRec);
+    if (p.flags & kDebugBounds) {                // checked build: the copy must stay inside the unit's records
+      const int room = p.max_blocks * NW - (rec_begin + r * kStageRec);
+      if (nrec > room) { atomicExch(p.status, kStatusBounds); nrec = max(room, 0); }
+    }
     const uint32_t bytes = (uint32_t)nrec * SM::kRecBytes;
-    mbar_expect_tx(&full[s], bytes);
+    mbar_expect_tx(&full[s], bytes + (uint32_t)p.dbg_tx_extra);
     bulk_g2s(smem_raw + (size_t)s * SM::kStageBytes, stats_u + (size_t)(rec_begin + r * kStageRec) * 2 * D, bytes, &full[s]);
   };
   // tensor-core path: slot r (16 records) goes to ring position r % kSlots and is consumed by the warp of that
@@ -288,8 +292,13 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
   const int n_slots = (n_stream + kSlotRec - 1) / kSlotRec;
   auto issue_slot = [&](int r) {                // one thread
     const int pos = r % SM::kSlots;
-    const uint32_t bytes = (uint32_t)min(kSlotRec, n_stream - r * kSlotRec) * SM::kRecBytes;
-    mbar_expect_tx(&full[pos], bytes);
+    int nrec = min(kSlotRec, n_stream - r * kSlotRec);
+    if (p.flags & kDebugBounds) {                // checked build: the copy must stay inside the unit's records
+      const int room = p.max_blocks * NW - (rec_begin + r * kSlotRec);
+      if (nrec > room) { atomicExch(p.status, kStatusBounds); nrec = max(room, 0); }
+    }
+    const uint32_t bytes = (uint32_t)nrec * SM::kRecBytes;
+    mbar_expect_tx(&full[pos], bytes + (uint32_t)p.dbg_tx_extra);
     bulk_g2s(smem_raw + (size_t)pos * SM::kSlotBytes, stats_u + (size_t)(rec_begin + r * kSlotRec) * 2 * D, bytes, &full[pos]);
   };
   if (tid == 0) {
@@ -373,7 +382,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
 #pragma unroll 1
       for (int r = warp; r < n_slots; r += SM::kSlots) {          // warp w owns ring position w
         const int pos = r % SM::kSlots;
-        if (!mbar_wait(&full[pos], (r / SM::kSlots) & 1)) { if (lane == 0) atomicExch(&err_s, 1); break; }
+        if (!mbar_wait(&full[pos], (r / SM::kSlots) & 1, p.wait_limit)) { if (lane == 0) atomicExch(&err_s, 1); break; }
         consume_slot(smem_raw + (size_t)pos * SM::kSlotBytes, r * kSlotRec, n_stream);
         __syncwarp();                                              // every lane has its operands: the slot is free
         if (lane == 0 && r + SM::kSlots < n_slots) issue_slot(r + SM::kSlots);
@@ -430,7 +439,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
 #pragma unroll 1
     for (int r = 0; r < (MMA ? 0 : n_rounds); ++r) {
       const int s = r % kStages;
-      if (!mbar_wait(&full[s], (r / kStages) & 1)) { if (lane == 0) atomicExch(&err_s, 1); break; }
+      if (!mbar_wait(&full[s], (r / kStages) & 1, p.wait_limit)) { if (lane == 0) atomicExch(&err_s, 1); break; }
       const int l0 = r * kStageRec + warp * UNR;                       // first record of this warp, CTA-local
       const ST* st = reinterpret_cast<const ST*>(smem_raw + (size_t)s * SM::kStageBytes) + (size_t)(warp * UNR) * 2 * D;
       float mean[PASSES][VECW], var[PASSES][VECW];
@@ -454,7 +463,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[s]);                            // the stage is in registers: hand it back
       if (tid == 0 && r + kStages < n_rounds) {                         // refill it once every warp has done the same
-        if (mbar_wait(&empty[s], (r / kStages) & 1)) issue(r + kStages);
+        if (mbar_wait(&empty[s], (r / kStages) & 1, p.wait_limit)) issue(r + kStages);
         else atomicExch(&err_s, 1);
       }
       __syncwarp();
@@ -465,7 +474,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
       // handful of records) through plain loads into stage 0, one more round
       pdl_wait();
       pdl_launch_dependents();
-      L = __ldcg(p.seq_lens + b);
+      L = cover_len(p, checked_len(p, b), (long long)CS * chunk * p.B);
       nblk = (L + p.B - 1) / p.B;
       blk_begin = min(nblk, cta_blk0);
       nb_my = min(nblk, blk_begin + chunk) - blk_begin;
@@ -565,7 +574,7 @@ __global__ void __launch_bounds__(kCsThreads, 2) score_cluster_kernel(const Para
     part_s[tid * 2] = m;
     part_s[tid * 2 + 1] = s;
   }
-  if (tid == 0 && err_s) atomicExch(p.status, -3);
+  if (tid == 0 && err_s) atomicExch(p.status, kStatusTimeout);
 
   cluster_sync_all();                                                   // ---- sync 1: partial normalisers visible
 

@@ -80,9 +80,9 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
   }
 
   // ------------------------------------------------------------------ score role ----------------------
-  const int L = p.seq_lens[b];
-  const int nblk = (L + p.B - 1) / p.B;
   const int NW = p.NW;                              // selection windows per block; a "record" is one window
+  const int L = cover_len(p, checked_len(p, b), (long long)p.n_chunks_cap * p.chunk / NW * p.B);
+  const int nblk = (L + p.B - 1) / p.B;
   const int nrec = nblk * NW;
   const int chunk = p.chunk;                        // records per CTA
   const int n_chunks = max(1, (nrec + chunk - 1) / chunk);
@@ -133,7 +133,12 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
 #pragma unroll
     for (int r = 0; r < UNR; ++r) {
       const int i = base + round * kRound + r;
-      load_record<VEC>(p.stats, stats_u + (size_t)i * 2 * D, rec_bf16, D, lane, i < nrec, mean[buf][r], var[buf][r]);
+      bool valid = i < nrec;
+      if ((p.flags & kDebugBounds) && valid && i >= p.max_blocks * NW) {   // checked build: the record must exist
+        atomicExch(p.status, kStatusBounds);
+        valid = false;
+      }
+      load_record<VEC>(p.stats, stats_u + (size_t)i * 2 * D, rec_bf16, D, lane, valid, mean[buf][r], var[buf][r]);
     }
   };
   auto compute_round = [&](int round, int buf) {
@@ -440,6 +445,7 @@ static cudaError_t launch_one(const Params& p, const void* q, int q_is_bf16, int
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   kern<<<grid, kScoreThreads, smem, stream>>>(p, q, q_is_bf16, sel_user);
+  ++g_launch_count;
   return cudaGetLastError();
 }
 

@@ -28,9 +28,10 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratch
 
 std::mutex g_setup_mutex;
 void* g_scratch_dev_ptr[kMaxDevices] = {};   // per device: device address of g_noalloc_scratch
+int g_sm_count[kMaxDevices] = {};            // per device: multiprocessor count (sizes the grid; the query allocates nothing)
 
 // Once per device, with that device current: resolve the device address of the scratch array.
-cudaError_t scratch_for_current_device(void** ptr_out) {
+cudaError_t scratch_for_current_device(void** ptr_out, int* sm_count_out) {
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
@@ -41,8 +42,10 @@ cudaError_t scratch_for_current_device(void** ptr_out) {
     e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
     if (e != cudaSuccess) return e;
     g_scratch_dev_ptr[dev] = ptr;
+    g_sm_count[dev] = device_sm_count();
   }
   *ptr_out = g_scratch_dev_ptr[dev];
+  *sm_count_out = g_sm_count[dev];
   return cudaSuccess;
 }
 
@@ -51,7 +54,8 @@ size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 }  // namespace
 
 extern "C" int spla_select_blocks_noalloc(const spla_config_t* cfg, const float* stats, const int32_t* seq_lens,
-                                          const void* q, int32_t* sel_idx, float* scores_out, void* stream) {
+                                          const void* q, int32_t* sel_idx, float* scores_out, int32_t* status_out,
+                                          void* stream) {
   if (!cfg || !stats || !seq_lens || !q || !sel_idx) return SPLA_ERR_INVALID_ARG;
   spla_sizes_t sz;
   const int rc = spla_query_sizes(cfg, &sz);                 // validates the configuration (host only)
@@ -77,8 +81,9 @@ extern "C" int spla_select_blocks_noalloc(const spla_config_t* cfg, const float*
   if (off > kNoAllocScratchBytes) return SPLA_ERR_UNSUPPORTED;   // beyond the fixed scratch: use spla_decode
 
   void* base_v = nullptr;
-  cudaError_t e = scratch_for_current_device(&base_v);
-  if (e != cudaSuccess) return SPLA_ERR_CUDA;
+  int sm_count = 148;
+  cudaError_t e = scratch_for_current_device(&base_v, &sm_count);
+  if (e != cudaSuccess) return cuda_fail(e, "spla_select_blocks_noalloc/scratch address");
   char* base = reinterpret_cast<char*>(base_v);
 
   Params p;
@@ -92,7 +97,7 @@ extern "C" int spla_select_blocks_noalloc(const spla_config_t* cfg, const float*
   p.kv_bf16 = cfg->kv_dtype == SPLA_BF16;
   p.sm_scale = cfg->sm_scale == 0.f ? 1.0f / sqrtf((float)cfg->head_dim) : cfg->sm_scale;
   p.phi_scale = 1.f; p.rms_eps = 1e-6f;
-  p.chunk = score_chunk_for((long long)U, (long long)max_blocks, 148);
+  p.chunk = score_chunk_for((long long)U, (long long)max_blocks, sm_count);
   p.n_chunks_cap = (int)((max_blocks + p.chunk - 1) / p.chunk);
   p.stats = const_cast<float*>(stats);
   p.seq_lens = const_cast<int*>(seq_lens);
@@ -108,5 +113,7 @@ extern "C" int spla_select_blocks_noalloc(const spla_config_t* cfg, const float*
   if (e == cudaSuccess) e = launch_score_select(p, q, cfg->q_dtype == SPLA_BF16, sel_idx, s);
   if (e == cudaSuccess && scores_out)
     e = cudaMemcpyAsync(scores_out, base + o_scores, U * max_blocks * 4, cudaMemcpyDeviceToDevice, s);
-  return e == cudaSuccess ? SPLA_OK : SPLA_ERR_CUDA;
+  if (e == cudaSuccess && status_out)
+    e = cudaMemcpyAsync(status_out, base + o_status, sizeof(int), cudaMemcpyDeviceToDevice, s);
+  return e == cudaSuccess ? SPLA_OK : cuda_fail(e, "spla_select_blocks_noalloc");
 }

@@ -20,8 +20,6 @@ struct spla_cache {
   // clusters the device holds at once, as last queried: score kernel for (cs, chunk), attend kernel per log2(acs)
   int score_occ_cs = 0, score_occ_chunk = 0, score_occ_n = -1;
   int attend_occ[5] = {-2, -2, -2, -2, -2};
-  cudaEvent_t ev[3];   // created on first use by spla_decode_profile
-  bool have_ev;
   int sm_count;
   AttendMaps maps;
   AttendMaps state_maps;   // the same caches in boxes of 64 tokens, for the tensor-core state kernel
@@ -29,10 +27,19 @@ struct spla_cache {
 
 static thread_local char g_cuda_err[256] = "";
 
-static int cuda_fail(cudaError_t e, const char* where) {
+namespace spla {
+thread_local unsigned long long g_launch_count = 0;
+int cuda_fail(cudaError_t e, const char* where) {
   snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", where, cudaGetErrorString(e));
   return SPLA_ERR_CUDA;
 }
+int device_sm_count() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+    return n;
+  return 148;
+}
+}  // namespace spla
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -73,7 +80,8 @@ static int validate_config(const spla_config_t* c) {
   if ((c->kv_dtype != SPLA_F32 && c->kv_dtype != SPLA_BF16) || (c->q_dtype != SPLA_F32 && c->q_dtype != SPLA_BF16))
     return SPLA_ERR_INVALID_ARG;
   if (c->sm_scale < 0.f || c->phi_scale < 0.f || c->rms_eps < 0.f) return SPLA_ERR_INVALID_ARG;
-  if (c->flags & ~(SPLA_ADOPT_CONTENTS | SPLA_FIRST_ORDER | SPLA_NO_RLA | SPLA_GENERAL_KERNELS | SPLA_STATS_BF16)) return SPLA_ERR_INVALID_ARG;
+  if (c->flags & ~(SPLA_ADOPT_CONTENTS | SPLA_FIRST_ORDER | SPLA_NO_RLA | SPLA_GENERAL_KERNELS | SPLA_STATS_BF16 | SPLA_DEBUG_BOUNDS))
+    return SPLA_ERR_INVALID_ARG;
   const int G = c->n_q_heads / c->n_kv_heads;
   if (G > kMaxGroup) return SPLA_ERR_UNSUPPORTED;
   if (c->head_dim != 64 && c->head_dim != 128) return SPLA_ERR_UNSUPPORTED;
@@ -159,14 +167,7 @@ extern "C" int spla_init_cache(const spla_config_t* config, const spla_buffers_t
   if (!c) return SPLA_ERR_INVALID_ARG;
   c->cfg = *config;
   c->buf = *b;
-  c->have_ev = false;
-  c->sm_count = 148;
-  {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-      c->sm_count = n;
-  }
+  c->sm_count = device_sm_count();
   if (c->cfg.sm_scale == 0.f) c->cfg.sm_scale = 1.0f / sqrtf((float)config->head_dim);
   if (c->cfg.phi_scale == 0.f) c->cfg.phi_scale = 1.0f;
   if (c->cfg.rms_eps == 0.f) c->cfg.rms_eps = 1e-6f;
@@ -359,41 +360,6 @@ extern "C" int spla_append_decode(spla_cache_t* c, const void* k_new, const void
   return SPLA_OK;
 }
 
-// Keeps the stream busy for a few tens of microseconds (bounded) so that the launches that follow are already
-// queued when it ends; otherwise the event timestamps would include the host's submission latency.
-__global__ void profile_delay_kernel() {
-  for (int i = 0; i < 60; ++i) __nanosleep(1000);
-}
-
-extern "C" int spla_decode_profile(spla_cache_t* c, const void* q, const float* rms_weight, float* out,
-                                   float* stage_ms, void* stream) {
-  if (!c || !q || !out || !stage_ms) return SPLA_ERR_INVALID_ARG;
-  if (!rms_weight && !(c->cfg.flags & SPLA_NO_RLA)) return SPLA_ERR_INVALID_ARG;
-  if (!aligned(q, 16) || !aligned(out, 16)) return SPLA_ERR_INVALID_ARG;
-  cudaError_t e = cudaSuccess;
-  if (!c->have_ev) {
-    for (int i = 0; i < 3 && e == cudaSuccess; ++i) e = cudaEventCreate(&c->ev[i]);
-    if (e != cudaSuccess) return cuda_fail(e, "spla_decode_profile/events");
-    c->have_ev = true;
-  }
-  Params p = c->p;
-  plan_score_grid(c, &p);
-  p.acs = attend_cluster_size(c);
-  const int qb = c->cfg.q_dtype == SPLA_BF16;
-  cudaStream_t s = (cudaStream_t)stream;
-  profile_delay_kernel<<<1, 1, 0, s>>>();
-  e = cudaEventRecord(c->ev[0], s);
-  if (e == cudaSuccess) e = launch_score(p, q, qb, nullptr, s);
-  if (e == cudaSuccess) e = cudaEventRecord(c->ev[1], s);
-  if (e == cudaSuccess) e = launch_attend_merge(p, &c->maps, q, qb, rms_weight, nullptr, out, nullptr, nullptr, s);
-  if (e == cudaSuccess) e = cudaEventRecord(c->ev[2], s);
-  if (e == cudaSuccess) e = cudaEventSynchronize(c->ev[2]);
-  if (e == cudaSuccess) e = cudaEventElapsedTime(&stage_ms[0], c->ev[0], c->ev[1]);
-  if (e == cudaSuccess) e = cudaEventElapsedTime(&stage_ms[1], c->ev[1], c->ev[2]);
-  if (e != cudaSuccess) return cuda_fail(e, "spla_decode_profile");
-  return SPLA_OK;
-}
-
 extern "C" int spla_select(spla_cache_t* c, const void* q, int32_t* sel_idx, void* stream) {
   if (!c || !q || !sel_idx) return SPLA_ERR_INVALID_ARG;
   if (!aligned(q, 16)) return SPLA_ERR_INVALID_ARG;
@@ -441,9 +407,14 @@ extern "C" int spla_sync_status(spla_cache_t* c, void* stream) {
   return st;
 }
 
+extern "C" int spla_debug_wait_hook(spla_cache_t* c, int32_t max_wait_polls, int32_t extra_expected_bytes) {
+  if (!c || max_wait_polls < 0 || extra_expected_bytes < 0 || (extra_expected_bytes % 16)) return SPLA_ERR_INVALID_ARG;
+  c->p.wait_limit = max_wait_polls;
+  c->p.dbg_tx_extra = extra_expected_bytes;
+  return SPLA_OK;
+}
+
 extern "C" int spla_destroy_cache(spla_cache_t* c) {
-  if (c && c->have_ev)
-    for (int i = 0; i < 3; ++i) cudaEventDestroy(c->ev[i]);
   delete c;
   return SPLA_OK;
 }
@@ -455,8 +426,12 @@ extern "C" const char* spla_status_string(int status) {
     case SPLA_ERR_CAPACITY: return "cache capacity exceeded";
     case SPLA_ERR_CUDA: return "CUDA error";
     case SPLA_ERR_UNSUPPORTED: return "unsupported configuration";
+    case SPLA_ERR_TIMEOUT: return "a kernel's bounded wait ran out";
+    case SPLA_ERR_BOUNDS: return "length or index outside the cache (clamped or skipped on the device)";
     default: return "unknown status";
   }
 }
 
 extern "C" const char* spla_last_cuda_error(void) { return g_cuda_err; }
+
+extern "C" unsigned long long spla_launch_count(void) { return g_launch_count; }

@@ -17,6 +17,12 @@ constexpr int kMaxGroup = 16;
 constexpr int kMaxWindows = 8;          // selection windows per block, at most
 constexpr int kMaxTopK = 64;
 constexpr unsigned kStatsBf16 = 16u;     // Params::flags bit: statistics records are bfloat16 (SPLA_STATS_BF16)
+constexpr unsigned kDebugBounds = 32u;   // Params::flags bit: every block index / token offset is checked (SPLA_DEBUG_BOUNDS)
+// Values a kernel may latch into the status word (the spla_status_t codes of the same meaning)
+constexpr int kStatusCapacity = -2;      // an append would overflow max_context: that sequence was skipped
+constexpr int kStatusTimeout = -5;       // a bounded wait on a copy barrier ran out: the math was skipped
+constexpr int kStatusBounds = -6;        // an index or length outside the cache was met: the access was skipped
+constexpr int kWaitLimitDefault = 1 << 22;
 constexpr int kMaxBlocks = 32768;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -55,6 +61,8 @@ struct Params {
   int* state_ticket;   // [U]
   int* status;         // [1]
   int max_chunks;
+  int wait_limit;                       // iterations a bounded barrier wait polls before it gives up (0: kWaitLimitDefault)
+  int dbg_tx_extra;                     // test hook: bytes added to what the decode kernels' copy barriers expect (0 in use)
 #ifdef SPLA_TRACE
   unsigned long long* trace;  // development builds only: [unit][64 CTAs][8 marks] of %globaltimer values
 #endif
@@ -146,10 +154,11 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                "l"(src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
 }
-// Bounded wait: returns false if the phase did not complete within the iteration limit.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+// Bounded wait: returns false if the phase did not complete within `limit` polls (0: the default limit).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int limit = 0) {
   const uint32_t addr = smem_u32(bar);
-  for (int it = 0; it < (1 << 22); ++it) {
+  if (limit <= 0) limit = kWaitLimitDefault;
+  for (int it = 0; it < limit; ++it) {
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -162,6 +171,29 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     if (it > 64) __nanosleep(64);
   }
   return false;
+}
+
+// The cached length of sequence b as the decode kernels use it.  seq_lens is a caller-owned buffer (and may have been
+// adopted with its contents): a value outside [0, max_context] would size loops and shared-memory arrays wrongly, so
+// it is clamped and reported through the status word instead of being trusted.
+__device__ __forceinline__ int checked_len(const Params& p, int b) {
+  int L = __ldcg(p.seq_lens + b);
+  if ((unsigned)L > (unsigned)p.max_context) {
+    atomicExch(p.status, kStatusBounds);
+    L = L < 0 ? 0 : p.max_context;
+  }
+  return L;
+}
+
+// A score launch is sized on the host from an upper bound of the lengths.  A length above what the launch covers (the
+// host's bound was wrong, or seq_lens was overwritten) is cut to the covered part and reported, so that every block
+// the selection may name has been scored.
+__device__ __forceinline__ int cover_len(const Params& p, int L, long long cover_tokens) {
+  if ((long long)L > cover_tokens) {
+    atomicExch(p.status, kStatusBounds);
+    L = (int)cover_tokens;
+  }
+  return L;
 }
 
 // Development aid, compiled in only with -DSPLA_TRACE (python -m paper_2601_22379_b200.build --trace): thread 0 of

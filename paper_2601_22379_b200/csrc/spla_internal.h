@@ -13,6 +13,9 @@ inline int padded_group(int G) {
   return gp;
 }
 
+// Kernels this library has launched from the calling thread (spla_launch_count): bumped at every launch site.
+extern thread_local unsigned long long g_launch_count;
+
 // Launch with optional thread-block-cluster shape and programmatic dependent launch: with `pdl` the grid may
 // start while the preceding kernel of the stream drains; it must execute griddepcontrol.wait before it touches
 // anything that kernel produces (every kernel launched this way does so in its prologue).
@@ -40,6 +43,7 @@ inline cudaError_t launch_ex(void (*kern)(KArgs...), dim3 grid, dim3 block, size
   }
   cfg.attrs = attr;
   cfg.numAttrs = n;
+  ++g_launch_count;
   return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 
@@ -66,6 +70,9 @@ inline int max_active_clusters(void (*kern)(KArgs...), dim3 grid, dim3 block, si
   return n;
 }
 
+// spla_api.cu: records the text of a failed CUDA call for spla_last_cuda_error and returns SPLA_ERR_CUDA
+int cuda_fail(cudaError_t e, const char* where);
+int device_sm_count();   // multiprocessors of the current device (148 if the query fails)
 // score_select.cu
 int score_chunk_for(long long units, long long max_seq_blocks, int sm_count);
 cudaError_t launch_score_select(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream);

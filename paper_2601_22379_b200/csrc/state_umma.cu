@@ -326,7 +326,7 @@ __global__ void __launch_bounds__(kSuThreads, 1)
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kSuTmemCols) : "memory");
   }
-  if (tid == 0 && abort_s) atomicExch(p.status, -3);
+  if (tid == 0 && abort_s) atomicExch(p.status, kStatusTimeout);
   if (S == 1) return;
 
   // ------------------------------------------------------------------ last CTA of the unit: partials -> S_bar ----
@@ -373,6 +373,7 @@ cudaError_t launch_state_umma(const Params& p, const AttendMaps* maps, const int
   if (e != cudaSuccess) return e;
   state_umma_kernel<<<dim3(S, U), kSuThreads, kSuSmemBytes, stream>>>(
       p, *reinterpret_cast<const CUtensorMap*>(maps->k), *reinterpret_cast<const CUtensorMap*>(maps->v), n_new, max_new);
+  ++g_launch_count;
   return cudaGetLastError();
 }
 

@@ -63,7 +63,7 @@ def test_query_sizes_follow_the_documented_layouts(lib):
     (dict(batch=0), binding.SPLA_ERR_INVALID_ARG),
     (dict(n_sink_blocks=20, n_local_blocks=20), binding.SPLA_ERR_INVALID_ARG),
     (dict(flags=64), binding.SPLA_ERR_INVALID_ARG),
-    (dict(flags=32), binding.SPLA_ERR_INVALID_ARG),
+    (dict(flags=128), binding.SPLA_ERR_INVALID_ARG),
     (dict(sm_scale=-1.0), binding.SPLA_ERR_INVALID_ARG),
     (dict(head_dim=96), binding.SPLA_ERR_UNSUPPORTED),
     (dict(block_size=48), binding.SPLA_ERR_UNSUPPORTED),

@@ -163,6 +163,30 @@ def _sample_units(w, n, seed=0):
     return [allu[i] for i in idx]
 
 
+def _check_all_selections(w, cache, q, K, V, lens_h, window=None):
+    """Steps a1-a2 for EVERY unit at full size: the library's index set against the oracle's score-only path
+    (block statistics -> grouped BlockScore -> Select; Section 3.1 Eq. taylor-2nd, Section 2.2, Section 2.1), which
+    needs no attention and is therefore cheap enough to run on all units."""
+    assert window is None
+    sel = cache.select(q)
+    torch.cuda.synchronize()
+    assert cache.sync_status() == 0
+    sel = sel.cpu().numpy()
+    G = w.group
+    scale = 1.0 / np.sqrt(w.head_dim)
+    n_same = 0
+    for b in range(w.batch):
+        L = int(lens_h[b])
+        for h in range(w.n_kv_heads):
+            mean, var, n = O.block_statistics(K[b, h, :L].double().cpu().numpy(), w.block_size)
+            qh = q[b, h * G:(h + 1) * G].double().cpu().numpy() * scale
+            _, _, score = O.block_scores(qh, mean, var, n)
+            ref = {"sel": O.select_blocks(score, w.top_k, w.n_sink, w.n_local), "score": score}
+            n_same += parity.check_selection(sel[b, h], ref, w.top_k, w.n_sink, w.n_local)
+    assert n_same >= 0.9 * w.batch * w.n_kv_heads          # tie-band swaps are rare
+    return n_same
+
+
 def test_config1_tiny_ref_full_16_steps():
     w = synth.CONFIGS[0]
     cache, K, V, lens = runner.build_cache(w, DEV)
@@ -199,13 +223,15 @@ def test_config2_gqa_32k_full_three_query_seeds():
                 assert set(nb[b, h].tolist()) <= set(sel[b, h].tolist())
 
 
-def _stepped_full(w, n_units, check_steps, window=None, flags=0):
+def _stepped_full(w, n_units, check_steps, window=None, flags=0, all_selections=False):
     cache, K, V, lens = runner.build_cache(w, DEV, window=window, flags=flags)
     stats_bf16 = bool(flags & binding.SPLA_STATS_BF16)
     tie_band = parity.TIE_BAND_STATS_BF16 if stats_bf16 else parity.TIE_BAND
     gamma = synth.gamma(w).to(DEV)
     gam = gamma.double().cpu().numpy()
     lens_h = lens.cpu().numpy()
+    if all_selections:                                     # every unit's index set on the prefilled cache
+        _check_all_selections(w, cache, synth.step_queries(w, 0, DEV), K, V, lens_h)
     units = _sample_units(w, n_units, 1)
     G = w.group
     orc = {}
@@ -236,7 +262,14 @@ def _stepped_full(w, n_units, check_steps, window=None, flags=0):
 
 
 def test_config3_long_128k_full_64_steps():
-    _stepped_full(synth.CONFIGS[2], n_units=3, check_steps={0, 1, 31, 62, 63})
+    _stepped_full(synth.CONFIGS[2], n_units=3, check_steps={0, 1, 31, 62, 63}, all_selections=True)
+
+
+def test_long_128k_full_size_with_the_group_size_of_the_papers_model():
+    """40 query heads over 8 KV heads (G = 5, Table 1 of the paper) at the full 128K context: all selections, and
+    sampled units' outputs over a few steps."""
+    w = synth.CONFIGS[2].scaled(n_q_heads=40, n_steps=6)
+    _stepped_full(w, n_units=2, check_steps={0, 5}, all_selections=True)
 
 
 def test_config4_very_long_1m_full():
@@ -245,10 +278,11 @@ def test_config4_very_long_1m_full():
     gamma = synth.gamma(w).to(DEV)
     q = synth.step_queries(w, 0, DEV)
     _check_units(w, cache, q, gamma, K, V, lens.cpu().numpy(), _sample_units(w, 2, 4), w.n_sink, w.n_local)
+    _check_all_selections(w, cache, q, K, V, lens.cpu().numpy())
 
 
 def test_config5_ragged_serving_full_256_steps():
-    _stepped_full(synth.CONFIGS[4], n_units=4, check_steps={0, 63, 64, 255})
+    _stepped_full(synth.CONFIGS[4], n_units=4, check_steps={0, 63, 64, 255}, all_selections=True)
 
 
 # ---------------------------------------------------------------------------------------------------------

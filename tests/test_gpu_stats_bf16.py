@@ -152,7 +152,7 @@ def test_noalloc_entry_rejects_bf16_statistics():
     cfg = cache.cfg
     rc = binding.load().spla_select_blocks_noalloc(
         ctypes.byref(cfg), cache.bufs.stats.data_ptr(), cache.bufs.seq_lens.data_ptr(), q.data_ptr(),
-        cache.new_sel_buffer().data_ptr(), None, None)          # rejected on the host: nothing is launched
+        cache.new_sel_buffer().data_ptr(), None, None, None)          # rejected on the host: nothing is launched
     assert rc == binding.SPLA_ERR_UNSUPPORTED
 
 

@@ -217,6 +217,16 @@ def _softmax_rows(x):
     return scipy.special.softmax(x, axis=-1)
 
 
+def test_selected_tokens_against_a_hand_written_list():
+    """Blocks 1 and 3 of a 14-token context in blocks of 4: block 1 holds tokens 4..7, block 3 is the partial
+    last block with tokens 12 and 13; the -1 padding names nothing (Section 2.1, Eq. dense: the tokens of the
+    blocks in the index set)."""
+    np.testing.assert_array_equal(O.selected_tokens(np.array([1, 3, -1]), 14, 4), [4, 5, 6, 7, 12, 13])
+    np.testing.assert_array_equal(O.selected_tokens(np.array([0, -1, -1]), 3, 4), [0, 1, 2])
+    np.testing.assert_array_equal(O.selected_tokens(np.array([-1, -1]), 9, 4), [])
+    np.testing.assert_array_equal(O.selected_tokens(np.array([0, 2]), 12, 4), [0, 1, 2, 3, 8, 9, 10, 11])
+
+
 def test_p2_subtraction_equals_explicit_sum_over_unselected_blocks():
     d, B, L, G = 12, 8, 8 * 9 + 5, 3
     K, V = RNG.standard_normal((L, d)), RNG.standard_normal((L, d))

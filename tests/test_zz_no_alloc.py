@@ -56,6 +56,30 @@ def test_noalloc_rejects_what_does_not_fit_its_fixed_scratch():
     dummy = torch.zeros(64, dtype=torch.float32, device=DEV)
     idx = torch.zeros(64, dtype=torch.int32, device=DEV)
     rc = binding.load().spla_select_blocks_noalloc(big, dummy.data_ptr(), idx.data_ptr(), dummy.data_ptr(),
-                                                   idx.data_ptr(), None, None)
+                                                   idx.data_ptr(), None, None, None)
     assert rc == binding.SPLA_ERR_UNSUPPORTED
-    assert binding.load().spla_select_blocks_noalloc(big, None, None, None, None, None, None) == binding.SPLA_ERR_INVALID_ARG
+    assert binding.load().spla_select_blocks_noalloc(big, None, None, None, None, None, None, None) == binding.SPLA_ERR_INVALID_ARG
+
+
+def test_noalloc_clamps_a_length_beyond_the_capacity_and_says_so():
+    """seq_lens is the caller's buffer: a stale value above max_context must neither overrun the fixed scratch nor
+    the kernel's shared arrays.  It is clamped to the capacity and reported through status_out."""
+    w = synth.BY_NAME["gqa_32k"].scaled(batch=2, context=64 * 20, n_needles=0)
+    cache, K, V, lens = runner.build_cache(w, DEV)
+    q = synth.step_queries(w, 0, DEV)
+    sel = cache.new_sel_buffer()
+    status = torch.full((1,), 77, dtype=torch.int32, device=DEV)
+    assert binding.select_blocks_noalloc(cache.cfg, cache.bufs.stats, cache.bufs.seq_lens, q, sel, None, status) == binding.SPLA_OK
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    bad = cache.bufs.seq_lens.clone()
+    bad[1] = cache.cfg.max_context + 12345
+    sel.fill_(-7)
+    assert binding.select_blocks_noalloc(cache.cfg, cache.bufs.stats, bad, q, sel, None, status) == binding.SPLA_OK
+    torch.cuda.synchronize()
+    assert status.item() == binding.SPLA_ERR_BOUNDS
+    s = sel.cpu().numpy()
+    assert ((s >= -1) & (s < cache.max_blocks)).all()                 # a clean selection inside the cache for every unit
+    ref = cache.new_sel_buffer()
+    cache.select(q, ref)
+    assert torch.equal(sel[0], ref[0])                                # the untouched sequence selects as before
