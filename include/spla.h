@@ -193,6 +193,31 @@ int spla_select(spla_cache_t *cache, const void *q, int32_t *sel_idx, void *stre
 int spla_decode_selected(spla_cache_t *cache, const void *q, const float *rms_weight, const int32_t *sel_in,
                          float *out, float *dbg_o_sparse, float *dbg_o_rla, void *stream);
 
+/*
+ * Prefill- / training-shaped forward.  The paper develops the method on the decode step and says that it carries over
+ * to training and prefilling (Section 2, opening paragraph; Section 3.3 "Kernel Design": its kernels serve both).  The
+ * reading taken here is the causal one: T new tokens per sequence are appended, and the output of each of the T query
+ * positions is what spla_append_decode would give if the tokens were appended one at a time - position i sees tokens
+ * 0 .. L + i, with the block statistics (its own block as far as it is filled), the selection and the recurrent
+ * state S_bar of that prefix.  Afterwards the cache is as after spla_append_tokens(k_new, v_new, NULL, T).
+ *   k_new, v_new: DEVICE [batch][H_kv][T][d] kv_dtype (every sequence takes all T tokens).
+ *   q:            DEVICE [batch][T][H_q][d] q_dtype, unscaled.
+ *   rms_weight:   DEVICE [H_q][d] fp32 (may be NULL with SPLA_NO_RLA).
+ *   out:          DEVICE [batch][T][H_q][d] fp32.
+ *   sel_idx:      DEVICE int32 [batch][T][H_kv][top_k] or NULL: the blocks each position selected.
+ *   workspace:    DEVICE scratch, 256-byte aligned, of at least the `min_bytes` that spla_query_prefill_workspace
+ *                 reports for this T; with more (up to `good_bytes`) more positions are processed per kernel launch.
+ * Built on the general kernels (any group size up to 16, fp32 or bf16, d 64 or 128); strided selection windows are not
+ * supported (SPLA_ERR_UNSUPPORTED).  Returns SPLA_ERR_CAPACITY, with nothing enqueued, if the chunk does not fit.
+ */
+int spla_prefill(spla_cache_t *cache, const void *k_new, const void *v_new, const void *q, int32_t T,
+                 const float *rms_weight, float *out, int32_t *sel_idx, void *workspace, size_t workspace_bytes,
+                 void *stream);
+
+/* Workspace of spla_prefill for chunks of T tokens: the least it runs with, and a size that lets it work efficiently.
+ * HOST pointers; either may be NULL. */
+int spla_query_prefill_workspace(const spla_config_t *config, int32_t T, size_t *min_bytes, size_t *good_bytes);
+
 /* Block scores of the last spla_decode: DEVICE fp32 [batch][H_kv][max_blocks] copy-out (entries >= nblk are 0). */
 int spla_copy_scores(spla_cache_t *cache, float *scores_out, void *stream);
 

@@ -20,7 +20,8 @@ SPLA_ADOPT_CONTENTS, SPLA_FIRST_ORDER, SPLA_NO_RLA, SPLA_GENERAL_KERNELS, SPLA_S
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libspla.so")
 
 EXPORTS = ["spla_query_sizes", "spla_init_cache", "spla_append_tokens", "spla_decode", "spla_decode_selected",
-           "spla_select_blocks_noalloc", "spla_select", "spla_append_decode",
+           "spla_select_blocks_noalloc", "spla_select", "spla_append_decode", "spla_prefill",
+           "spla_query_prefill_workspace",
            "spla_copy_scores", "spla_sync_status", "spla_set_length_bound", "spla_debug_wait_hook", "spla_destroy_cache",
            "spla_launch_count", "spla_status_string", "spla_last_cuda_error"]
 
@@ -71,6 +72,8 @@ def load(path: str | None = None) -> C.CDLL:
     lib.spla_select.argtypes = [vp, vp, vp, vp]
     lib.spla_append_decode.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.spla_select_blocks_noalloc.argtypes = [C.POINTER(SplaConfig), vp, vp, vp, vp, vp, vp, vp]
+    lib.spla_prefill.argtypes = [vp, vp, vp, vp, i32, vp, vp, vp, vp, C.c_size_t, vp]
+    lib.spla_query_prefill_workspace.argtypes = [C.POINTER(SplaConfig), i32, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     lib.spla_copy_scores.argtypes = [vp, vp, vp]
     lib.spla_debug_wait_hook.argtypes = [vp, i32, i32]
     lib.spla_sync_status.argtypes = [vp, vp]
@@ -246,6 +249,29 @@ class SplaCache:
                                                k_new.shape[2], q.data_ptr(), _ptr(rms_weight), out.data_ptr(),
                                                _ptr(sel_idx), _ptr(dbg_o_sparse), _ptr(dbg_o_rla), _stream()),
                    "spla_append_decode")
+        return out
+
+    def prefill(self, k_new: torch.Tensor, v_new: torch.Tensor, q: torch.Tensor, rms_weight, out=None, sel_idx=None,
+                workspace_bytes: int | None = None) -> torch.Tensor:
+        """Prefill-shaped forward: appends T tokens per sequence and returns the output of every position.
+        k_new, v_new [batch, H_kv, T, d]; q [batch, T, H_q, d]; out [batch, T, H_q, d] fp32;
+        sel_idx (optional) [batch, T, H_kv, top_k] int32.  `workspace_bytes`: scratch to use (default: the size the
+        library recommends; at least the minimum it reports)."""
+        cfg = self.cfg
+        T = k_new.shape[2]
+        assert k_new.is_cuda and k_new.is_contiguous() and v_new.is_contiguous() and k_new.shape == v_new.shape
+        assert k_new.dtype == self.kv_torch_dtype and tuple(k_new.shape[:2]) == (cfg.batch, cfg.n_kv_heads)
+        assert q.is_contiguous() and q.dtype == self.q_torch_dtype and tuple(q.shape) == (cfg.batch, T, cfg.n_q_heads, cfg.head_dim)
+        lo, good = C.c_size_t(), C.c_size_t()
+        _check(self.lib.spla_query_prefill_workspace(C.byref(cfg), T, C.byref(lo), C.byref(good)), "spla_query_prefill_workspace")
+        nbytes = good.value if workspace_bytes is None else max(int(workspace_bytes), lo.value)
+        ws = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        if out is None:
+            out = torch.empty(cfg.batch, T, cfg.n_q_heads, cfg.head_dim, dtype=torch.float32, device=self.device)
+        with torch.cuda.device(self.device):
+            _check(self.lib.spla_prefill(self.handle, k_new.data_ptr(), v_new.data_ptr(), q.data_ptr(), T, _ptr(rms_weight),
+                                         out.data_ptr(), _ptr(sel_idx), ws.data_ptr(), nbytes, _stream()), "spla_prefill")
+        self._prefill_ws = ws                                  # keep the scratch alive until the stream has used it
         return out
 
     def select(self, q: torch.Tensor, sel_idx: torch.Tensor | None = None) -> torch.Tensor:

@@ -30,24 +30,25 @@ __device__ __forceinline__ bool arrive_last(int* ticket, int expected, int* flag
 // When every block of the sequence is selected the unselected set is empty and o_bar - o_tilde is exactly zero;
 // the difference of the two computed sums would only be rounding noise (which the RMSNorm would blow up), so
 // the residual is set to zero in that case.
+// `vu` indexes the workspace arrays, `ur` says which cache unit / query rows / length it stands for.
 template <int D>
-__device__ __forceinline__ void merge_unit(const Params& p, int u, int n_items, const float* __restrict__ rms_weight,
-                                           float* __restrict__ out, float* __restrict__ dbg_sparse,
-                                           float* __restrict__ dbg_rla, float* smem) {
+__device__ __forceinline__ void merge_unit(const Params& p, int vu, const UnitRef& ur, int n_items,
+                                           const float* __restrict__ rms_weight, float* __restrict__ out,
+                                           float* __restrict__ dbg_sparse, float* __restrict__ dbg_rla, float* smem) {
   constexpr int C4 = D / 4;                          // threads per head, one float4 of columns each
   constexpr int HG = kAttendThreads / C4;            // heads in flight
   constexpr int IU = 8;                              // items whose loads are in flight together
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = p.G;
-  const int b = u / p.Hkv, h = u % p.Hkv;
-  const int nblk_u = (checked_len(p, b) + p.B - 1) / p.B;
-  const bool rla = !(p.flags & 4u) && p.n_sel[u] < nblk_u;
+  const int h = ur.h;
+  const int nblk_u = (ur.L + p.B - 1) / p.B;
+  const bool rla = !(p.flags & 4u) && p.n_sel[vu] < nblk_u;
   float* wt_s = smem;                                // [n_items][G]: exp2(m_it - M) / L
 
   // The first batch of partial results is requested before the weights are formed: the two are independent
   // and each costs one L2 round trip.
   const int hg = tid / C4, c4 = tid % C4;
-  const float* parts = p.att_acc + (size_t)u * p.top_k * 2 * G * D;
+  const float* parts = p.att_acc + (size_t)vu * p.top_k * 2 * G * D;
   float4 a[IU], t[IU];
   auto fetch = [&](int g, int it0) {
 #pragma unroll
@@ -66,7 +67,7 @@ __device__ __forceinline__ void merge_unit(const Params& p, int u, int n_items, 
   if (hg < G) fetch(hg, 0);
 
   // softmax weights of the items: one warp per head, lanes over items
-  const float* ml_u = p.att_ml + (size_t)u * p.top_k * G * 2;
+  const float* ml_u = p.att_ml + (size_t)vu * p.top_k * G * 2;
   for (int g = warp; g < G; g += kAttendThreads / 32) {
     float m[2], l[2];
 #pragma unroll
@@ -92,10 +93,12 @@ __device__ __forceinline__ void merge_unit(const Params& p, int u, int n_items, 
     const bool live = g < G;
     float4 osp = make_float4(0.f, 0.f, 0.f, 0.f), otil = osp, obar = osp;
     if (live) {
-      if (rla) {
+      if (rla && ur.t >= 0) {                      // prefill: o_bar of this position, from the chunk scan
+        obar = __ldcg(reinterpret_cast<const float4*>(p.vobar + (((size_t)ur.u * p.vTtot + ur.t) * G + g) * D) + c4);
+      } else if (rla) {
 #pragma unroll
         for (int s = 0; s < kStateSplits; ++s) {
-          const float4 v = __ldcg(reinterpret_cast<const float4*>(p.obar_part + (((size_t)u * kStateSplits + s) * G + g) * D) + c4);
+          const float4 v = __ldcg(reinterpret_cast<const float4*>(p.obar_part + (((size_t)vu * kStateSplits + s) * G + g) * D) + c4);
           obar.x += v.x; obar.y += v.y; obar.z += v.z; obar.w += v.w;
         }
       }
@@ -116,7 +119,7 @@ __device__ __forceinline__ void merge_unit(const Params& p, int u, int n_items, 
 #pragma unroll
     for (int o = C4 / 2; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);   // over the C4 lanes of this head
     if (live) {
-      const size_t o = ((size_t)b * p.Hq + (size_t)h * G + g) * D + c4 * 4;
+      const size_t o = (ur.qrow + g) * D + c4 * 4;
       float4 res = osp;
       if (rla) {
         const float inv_rms = rsqrtf(sq / D + p.rms_eps);
@@ -133,10 +136,9 @@ __device__ __forceinline__ void merge_unit(const Params& p, int u, int n_items, 
 
 // Empty sequence: the output of the unit is zero.
 template <int D>
-__device__ __forceinline__ void write_zero_unit(const Params& p, int u, float* out, float* dbg_sparse, float* dbg_rla) {
-  const int b = u / p.Hkv, h = u % p.Hkv;
+__device__ __forceinline__ void write_zero_unit(const Params& p, const UnitRef& ur, float* out, float* dbg_sparse, float* dbg_rla) {
   for (int idx = threadIdx.x; idx < p.G * D; idx += blockDim.x) {
-    const size_t o = ((size_t)b * p.Hq + (size_t)h * p.G) * D + idx;
+    const size_t o = ur.qrow * D + idx;
     out[o] = 0.f;
     if (dbg_sparse) dbg_sparse[o] = 0.f;
     if (dbg_rla) dbg_rla[o] = 0.f;

@@ -26,19 +26,20 @@ __global__ void __launch_bounds__(kAttendThreads) attend_merge_kernel(const Para
   constexpr int TS = kAttendThreads / D;        // token slices in the value pass
   extern __shared__ __align__(128) unsigned char smem_raw[];
 
-  const int u = blockIdx.y, item = blockIdx.x;
-  const int b = u / p.Hkv, h = u % p.Hkv;
+  const int vu = blockIdx.y, item = blockIdx.x;     // vu: index into the workspace (a virtual unit in a prefill launch)
+  const UnitRef ur = unit_ref(p, vu);
+  const int u = ur.u;                               // the cache's unit
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = p.G, B = p.B;
   const bool rla = !(p.flags & 4u);
 
-  const int nsel = p.n_sel[u];
+  const int nsel = p.n_sel[vu];
   if (item >= nsel) {
-    if (nsel == 0 && item == 0) write_zero_unit<D>(p, u, out, dbg_sparse, dbg_rla);   // empty sequence
+    if (nsel == 0 && item == 0) write_zero_unit<D>(p, ur, out, dbg_sparse, dbg_rla);   // empty sequence
     return;
   }
-  const int blk = p.sel[(size_t)u * p.top_k + item];
-  const int L = checked_len(p, b);
+  const int blk = p.sel[(size_t)vu * p.top_k + item];
+  const int L = ur.L;
   int n_tok = min(B, L - blk * B);
   if ((p.flags & kDebugBounds) && (blk < 0 || blk >= p.max_blocks || n_tok <= 0)) {
     // checked build: a block index that does not name a cached block is reported and the block is treated as empty
@@ -75,7 +76,7 @@ __global__ void __launch_bounds__(kAttendThreads) attend_merge_kernel(const Para
   for (int g = 0; g < GP; ++g) {
     if (g < G) {
       float x[VEC];
-      const size_t qoff = ((size_t)b * p.Hq + (size_t)h * G + g) * D + lane * VEC;
+      const size_t qoff = (ur.qrow + g) * D + lane * VEC;
       if (q_is_bf16) load_vec<VEC>(reinterpret_cast<const __nv_bfloat16*>(q_raw) + qoff, x);
       else load_vec<VEC>(reinterpret_cast<const float*>(q_raw) + qoff, x);
       float mx = -INFINITY;
@@ -196,7 +197,7 @@ __global__ void __launch_bounds__(kAttendThreads) attend_merge_kernel(const Para
   }
 
   // ---- partial results of this block -------------------------------------------------------------------
-  float* part = p.att_acc + ((size_t)u * p.top_k + item) * 2 * G * D;
+  float* part = p.att_acc + ((size_t)vu * p.top_k + item) * 2 * G * D;
   if (ts == 0) {
 #pragma unroll
     for (int g = 0; g < GP; ++g) {
@@ -207,14 +208,14 @@ __global__ void __launch_bounds__(kAttendThreads) attend_merge_kernel(const Para
     }
   }
   if (tid < G) {
-    float* ml = p.att_ml + (((size_t)u * p.top_k + item) * G + tid) * 2;
+    float* ml = p.att_ml + (((size_t)vu * p.top_k + item) * G + tid) * 2;
     ml[0] = my_m;
     ml[1] = my_l;
   }
-  if (!arrive_last(&p.attend_ticket[u], nsel, &flag_s)) return;
+  if (!arrive_last(&p.attend_ticket[vu], nsel, &flag_s)) return;
 
   // ---- merge (last CTA of the unit) ---------------------------------------------------------------------
-  merge_unit<D>(p, u, nsel, rms_weight, out, dbg_sparse, dbg_rla, reinterpret_cast<float*>(smem_raw));
+  merge_unit<D>(p, vu, ur, nsel, rms_weight, out, dbg_sparse, dbg_rla, reinterpret_cast<float*>(smem_raw));
 }
 
 // Takes a caller-given selection into the workspace.  The list is not trusted: only entries that name an existing
@@ -262,7 +263,7 @@ static cudaError_t launch_one(const Params& p, const void* q, int qb, const floa
   auto kern = attend_merge_kernel<T, D, GP>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  dim3 grid(p.top_k, p.batch * p.Hkv);
+  dim3 grid(p.top_k, p.batch * p.Hkv * (p.vT > 0 ? p.vT : 1));
   kern<<<grid, kAttendThreads, smem, stream>>>(p, q, qb, w, out, ds, dr);
   ++g_launch_count;
   return cudaGetLastError();

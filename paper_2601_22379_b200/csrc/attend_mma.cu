@@ -1,9 +1,12 @@
 // Sparse attention + fused residual-linear term for bf16 K/V on tensor cores (GQA groups of up to 8 heads).
 //
 // The CTAs that serve one (sequence, KV head) unit form a thread-block cluster; CTA r of the cluster walks the
-// selected blocks r, r + CS, r + 2 CS, ... through a two-slot shared-memory ring that TMA fills (tiled tensor
-// copies with the 128-byte swizzle, so the ldmatrix reads below are bank-conflict free).  Each warp takes
-// 16-token slices.  Per slice the query group is the M side of two thin products that share one accumulator,
+// selected blocks r, r + CS, r + 2 CS, ... through a shared-memory ring that TMA fills (tiled tensor copies with
+// the 128-byte swizzle, so the ldmatrix reads below are bank-conflict free).  A CTA holds NG groups of four warps;
+// group j takes every NG-th block of the CTA's list and its warps take the block's 16-token slices.  Two shapes are
+// built: one group and a two-slot ring for launches with many units (two CTAs share an SM), and two groups with a
+// ring as deep as shared memory allows for launches that fit the machine with one CTA per SM, where what counts is
+// how many tiles are in flight at once.  Per slice the query group is the M side of two thin products that share one accumulator,
 //     rows 0..7  :  S = Q K^T            (exact branch,  Section 2.2 of the paper, Eq. gqa-sparse)
 //     rows 8..15 :  A = phi(Q) phi(K)^T  (linear branch, Section 3.2, Eq. rla-impl-2)
 // where phi(K) is formed element-wise from the very K fragments just used (one ex2 per element, with the cached
@@ -28,7 +31,7 @@ namespace spla {
 
 namespace {
 
-constexpr int kSlots = 2;
+constexpr int kMaxSlots = 12;      // ring positions at most (the launch says how many are used)
 
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -94,17 +97,18 @@ constexpr int kPad = 8;   // floats of padding per row of the cross-warp reducti
 
 // PACK: the group has at most 4 heads, so accumulator rows 4..7 and 12..15 are padding; rows 12..15 then carry
 // the bf16 remainder of the linear coefficients and no extra products are needed for it.
-template <int D, bool PACK>
-__global__ void __launch_bounds__(kAttendThreads, 2)
+template <int D, bool PACK, int NG>
+__global__ void __launch_bounds__(NG * kAttendThreads, NG == 1 ? 2 : 1)
     attend_mma_kernel(const Params p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                       const __nv_bfloat16* __restrict__ q, const float* __restrict__ rms_weight, float* __restrict__ out,
                       float* __restrict__ dbg_sparse, float* __restrict__ dbg_rla) {
   constexpr int KS = D / 16;        // k-steps of the two QK-type products
   constexpr int NT = D / 8;         // n-tiles of the PV-type product
   constexpr int NH = D / 64;        // 64-column halves of a tile (one TMA box each)
-  constexpr int NWARP = kAttendThreads / 32;
+  constexpr int NTHR = NG * kAttendThreads;
+  constexpr int NWARP = NTHR / 32;
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  __shared__ __align__(8) uint64_t full[kSlots];
+  __shared__ __align__(8) uint64_t full[kMaxSlots];
   __shared__ float red_s[NWARP];
   __shared__ int sel_s[kMaxTopK];
   __shared__ int err_s;
@@ -113,9 +117,15 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
   const int rank = blockIdx.x, CS = gridDim.x;
   const int b = u / p.Hkv, h = u % p.Hkv;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int gi = warp >> 2, wg = warp & 3, gtid = tid & (kAttendThreads - 1);   // group, warp in group, thread in group
   const int g = lane >> 2, t = lane & 3;
   const int G = p.G, B = p.B;
   const bool rla_on = !(p.flags & 4u);
+  const int ns = NG == 1 ? 2 : p.aslots;        // ring positions in use (a multiple of NG: a group refills what it frees)
+  auto group_sync = [&]() {                    // barrier over the four warps of this group
+    if constexpr (NG == 1) __syncthreads();
+    else asm volatile("bar.sync %0, %1;" ::"r"(1 + gi), "r"(kAttendThreads) : "memory");
+  };
 
   SPLA_MARK(p, u, 32 + rank, 1);
   pdl_launch_dependents();
@@ -123,9 +133,11 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
   // dependent launch this part overlaps that kernel's tail.  Rows = heads of the group, held in registers.
   // qa: rows 0..7 of the first product (raw q; the softmax scale is applied to the fp32 logits);
   // fa: rows 8..15 of the second product, phi(q) = softmax(phi_scale * q) in fp16.
-  // fl (groups of more than 4 heads only): the fp16 remainder of phi(q), a second left operand; in the packed
-  // layout rows 12..15 of fa carry that remainder for heads 0..3 instead.
-  uint32_t qa[KS][2], fa[KS][2], fl[PACK ? 1 : KS][2];
+  // fl_s (groups of more than 4 heads only): the fp16 remainder of phi(q), a second left operand, kept in shared
+  // memory (the same for every warp) to stay clear of the register limit; in the packed layout rows 12..15 of fa
+  // carry that remainder for heads 0..3 instead.
+  __shared__ uint32_t fl_s[PACK ? 1 : KS][2][32];
+  uint32_t qa[KS][2], fa[KS][2];
   {
     const bool hv = g < G;
     const bool rem_row = PACK && g >= 4;                  // this lane's row 8 + g holds the remainder of head g - 4
@@ -167,12 +179,12 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
         fa[kk][1] = rem_row ? l1 : h1;
       } else {
         fa[kk][0] = h0; fa[kk][1] = h1;
-        fl[kk][0] = l0; fl[kk][1] = l1;
+        if (warp == 0) { fl_s[kk][0][lane] = l0; fl_s[kk][1][lane] = l1; }   // (visible after the barrier below)
       }
     }
   }
   if (tid == 0) {
-    for (int s = 0; s < kSlots; ++s) mbar_init(&full[s], 1);
+    for (int s = 0; s < kMaxSlots; ++s) mbar_init(&full[s], 1);
     err_s = 0;
   }
 
@@ -180,7 +192,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
 
   int nsel = __ldcg(p.n_sel + u);
   const int L = checked_len(p, b);
-  for (int i = tid; i < p.top_k; i += kAttendThreads) sel_s[i] = __ldcg(p.sel + (size_t)u * p.top_k + i);
+  for (int i = tid; i < p.top_k; i += NTHR) sel_s[i] = __ldcg(p.sel + (size_t)u * p.top_k + i);
   if (p.flags & kDebugBounds) {
     // checked build: the list must name nsel existing blocks; it is cut at the first entry that does not, and the
     // status word says so (every CTA of the cluster sees the same list and cuts it at the same place)
@@ -188,7 +200,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
     if (tid == 0) first_bad_s = min(max(nsel, 0), p.top_k);
     __syncthreads();
     const int nblk_chk = (L + B - 1) / B;
-    for (int i = tid; i < min(nsel, p.top_k); i += kAttendThreads)
+    for (int i = tid; i < min(nsel, p.top_k); i += NTHR)
       if (sel_s[i] < 0 || sel_s[i] >= nblk_chk) atomicMin(&first_bad_s, i);
     __syncthreads();
     if (first_bad_s != nsel) {
@@ -202,8 +214,8 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
   const int nb = nsel > rank ? (nsel - rank + CS - 1) / CS : 0;     // my blocks: j = rank + i * CS
   const int tile_bytes = B * D * 2;
   const int slot_bytes = (2 * tile_bytes + B * 4 + 1023) & ~1023;   // K tile, V tile, per-token lse; the swizzle needs 1 KB alignment
-  auto issue = [&](int i) {                                          // thread 0 only
-    const int slot = i & 1;
+  auto issue = [&](int i) {                                          // one thread
+    const int slot = i % ns;
     const int blk = min(max(sel_s[rank + i * CS], 0), p.max_blocks - 1);   // (a list entry can never address outside the cache)
     const uint32_t base = smem_u32(smem_raw + (size_t)slot * slot_bytes);
     const int row0 = (int)(((size_t)u * p.max_blocks + blk) * B);
@@ -216,7 +228,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
     bulk_g2s(smem_raw + (size_t)slot * slot_bytes + 2 * tile_bytes, p.tok_lse + (size_t)row0, (uint32_t)(B * 4), &full[slot]);
   };
   if (tid == 0)
-    for (int i = 0; i < min(kSlots, nb); ++i) issue(i);
+    for (int i = 0; i < min(ns, nb); ++i) issue(i);
 
   // ---- per-warp running state over its slices -----------------------------------------------------------
   float m_run = -INFINITY, l_run = 0.f;      // row g of the exact branch (l: this lane's share)
@@ -229,10 +241,16 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
   const int mi = lane >> 3, r8 = lane & 7;   // ldmatrix: which 8x8 matrix this lane addresses, and which row
   const int half_bytes = B * 128;
 
+  // A wait that runs out marks the warp dead: it skips the arithmetic from then on but still joins every barrier of
+  // its group, so that the barrier counts match whatever the other warps saw.
+  bool dead = false;
 #pragma unroll 1
-  for (int i = 0; i < nb; ++i) {
-    const int slot = i & 1;
-    if (!mbar_wait(&full[slot], (i >> 1) & 1, p.wait_limit)) { if (lane == 0) atomicExch(&err_s, 1); break; }
+  for (int i = gi; i < nb; i += NG) {
+    const int slot = i % ns;
+    if (!dead && !__all_sync(0xffffffffu, mbar_wait(&full[slot], (i / ns) & 1, p.wait_limit))) {
+      dead = true;
+      if (lane == 0) atomicExch(&err_s, 1);
+    }
     if (i == 0) SPLA_MARK(p, u, 32 + rank, 2);
     unsigned char* sb = smem_raw + (size_t)slot * slot_bytes;
     const uint32_t ks = smem_u32(sb);
@@ -243,17 +261,17 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
     if (ntok < B) {
       // the open block of the sequence: rows past its end hold whatever the cache memory holds; the value rows
       // must be zero so that (probability 0) x (garbage) cannot produce a NaN
-      for (int idx = tid; idx < (B - ntok) * (D / 8); idx += kAttendThreads) {
+      for (int idx = gtid; idx < (B - ntok) * (D / 8) && !dead; idx += kAttendThreads) {
         const int row = ntok + idx / (D / 8), ch = idx % (D / 8);
         *reinterpret_cast<uint4*>(sb + tile_bytes + (ch >> 3) * half_bytes + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) =
             make_uint4(0u, 0u, 0u, 0u);
       }
-      __syncthreads();
+      group_sync();
     }
 #pragma unroll 1
-    for (int sl = warp; sl < spb; sl += NWARP) {
+    for (int sl = wg; sl < spb; sl += 4) {
       const int tok0 = sl * 16;
-      if (tok0 >= ntok) break;
+      if (tok0 >= ntok || dead) break;
       const float lse2_0 = lse_s[tok0 + g] * kLog2e, lse2_1 = lse_s[tok0 + 8 + g] * kLog2e;
       // two accumulator tiles per n-tile (one per product) so that the dependent chain of each is half as long;
       // rows 0..7 of the first and rows 8..15 of the second are the meaningful halves
@@ -285,8 +303,9 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
         mma_f16(aacc[0], 0u, fa[kk][0], 0u, fa[kk][1], pl[0], pl[1]);
         mma_f16(aacc[1], 0u, fa[kk][0], 0u, fa[kk][1], pl[2], pl[3]);
         if constexpr (!PACK) {                         // remainder of phi(q) times the head of phi(k)
-          mma_f16(aacc[0], 0u, fl[kk][0], 0u, fl[kk][1], pb[0], pb[1]);
-          mma_f16(aacc[1], 0u, fl[kk][0], 0u, fl[kk][1], pb[2], pb[3]);
+          const uint32_t fl0 = fl_s[kk][0][lane], fl1 = fl_s[kk][1][lane];
+          mma_f16(aacc[0], 0u, fl0, 0u, fl1, pb[0], pb[1]);
+          mma_f16(aacc[1], 0u, fl0, 0u, fl1, pb[2], pb[3]);
         }
       }
       if constexpr (PACK) {                            // rows 12..15 (remainder of phi(q)) onto rows 8..11
@@ -358,10 +377,10 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
         }
       }
     }
-    __syncthreads();                                   // every warp is done with this slot
-    if (tid == 0 && i + kSlots < nb) {
+    group_sync();                                      // every warp of the group is done with this slot
+    if (gtid == 0 && i + ns < nb && !dead) {
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy reads before the async-proxy refill
-      issue(i + kSlots);
+      issue(i + ns);
     }
   }
   if (tid == 0 && err_s) atomicExch(p.status, kStatusTimeout);
@@ -393,7 +412,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
     }
   }
   __syncthreads();
-  for (int idx = tid; idx < 2 * 8 * D; idx += kAttendThreads) {
+  for (int idx = tid; idx < 2 * 8 * D; idx += NTHR) {
     const int br = idx / (8 * D), hd = (idx / D) % 8, col = idx % D;    // branch, head, column
     float s = 0.f;
     if (hd < G) {
@@ -468,54 +487,65 @@ __global__ void __launch_bounds__(kAttendThreads, 2)
   cluster_sync_all();                                // ---- nobody leaves while a sibling may still read its memory
 }
 
-size_t attend_mma_smem_bytes(int B, int D) {
-  const size_t ring = (size_t)kSlots * ((2 * (size_t)B * D * 2 + (size_t)B * 4 + 1023) / 1024 * 1024);
-  const size_t fold = (size_t)((kAttendThreads / 32) * (16 * (D + kPad) + 16) + 2 * 8 * D + 16) * sizeof(float);
+// Ring positions of the two-group shape: as many as fit beside the static shared memory, an even number.
+int attend_mma_slots(int B, int D) {
+  const size_t slot = (2 * (size_t)B * D * 2 + (size_t)B * 4 + 1023) / 1024 * 1024;
+  int n = (int)((size_t)(222 * 1024) / slot);
+  if (n > kMaxSlots) n = kMaxSlots;
+  return n & ~1;
+}
+
+// `groups` = 1: two ring positions; 2: attend_mma_slots() positions.
+size_t attend_mma_smem_bytes(int B, int D, int groups) {
+  const int slots = groups == 1 ? 2 : attend_mma_slots(B, D);
+  const size_t ring = (size_t)slots * ((2 * (size_t)B * D * 2 + (size_t)B * 4 + 1023) / 1024 * 1024);
+  const size_t fold = (size_t)(groups * (kAttendThreads / 32) * (16 * (D + kPad) + 16) + 2 * 8 * D + 16) * sizeof(float);
   return ring > fold ? ring : fold;
+}
+
+template <int D, bool PACK, int NG>
+static cudaError_t launch_shape(const Params& p, const AttendMaps& maps, const void* q, const float* w, float* out, float* ds,
+                                float* dr, cudaStream_t stream, int* occupancy) {
+  const size_t smem = attend_mma_smem_bytes(p.B, D, NG);
+  const dim3 grid(p.acs, p.batch * p.Hkv);
+  auto kern = attend_mma_kernel<D, PACK, NG>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e == cudaSuccess && p.acs > 8) e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+  if (e != cudaSuccess) return e;
+  if (occupancy) {
+    *occupancy = max_active_clusters(kern, grid, dim3(NG * kAttendThreads), smem, p.acs);
+    return cudaSuccess;
+  }
+  const CUtensorMap& mk = *reinterpret_cast<const CUtensorMap*>(maps.k);
+  const CUtensorMap& mv = *reinterpret_cast<const CUtensorMap*>(maps.v);
+  return launch_ex(kern, grid, dim3(NG * kAttendThreads), smem, stream, p.acs, true, p, mk, mv,
+                   reinterpret_cast<const __nv_bfloat16*>(q), w, out, ds, dr);
 }
 
 template <int D>
 static cudaError_t launch_mma(const Params& p, const AttendMaps& maps, const void* q, const float* w, float* out, float* ds,
-                              float* dr, cudaStream_t stream) {
-  const size_t smem = attend_mma_smem_bytes(p.B, D);
-  const dim3 grid(p.acs, p.batch * p.Hkv);
-  const CUtensorMap& mk = *reinterpret_cast<const CUtensorMap*>(maps.k);
-  const CUtensorMap& mv = *reinterpret_cast<const CUtensorMap*>(maps.v);
-  const __nv_bfloat16* qb = reinterpret_cast<const __nv_bfloat16*>(q);
-  if (p.G <= 4) {
-    auto kern = attend_mma_kernel<D, true>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess && p.acs > 8) e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-    if (e != cudaSuccess) return e;
-    return launch_ex(kern, grid, dim3(kAttendThreads), smem, stream, p.acs, true, p, mk, mv, qb, w, out, ds, dr);
-  }
-  auto kern = attend_mma_kernel<D, false>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e == cudaSuccess && p.acs > 8) e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-  if (e != cudaSuccess) return e;
-  return launch_ex(kern, grid, dim3(kAttendThreads), smem, stream, p.acs, true, p, mk, mv, qb, w, out, ds, dr);
+                              float* dr, cudaStream_t stream, int* occ) {
+  if (p.agroups == 2)
+    return p.G <= 4 ? launch_shape<D, true, 2>(p, maps, q, w, out, ds, dr, stream, occ)
+                    : launch_shape<D, false, 2>(p, maps, q, w, out, ds, dr, stream, occ);
+  return p.G <= 4 ? launch_shape<D, true, 1>(p, maps, q, w, out, ds, dr, stream, occ)
+                  : launch_shape<D, false, 1>(p, maps, q, w, out, ds, dr, stream, occ);
 }
 
-template <int D>
-static int max_clusters_mma(const Params& p) {
-  const size_t smem = attend_mma_smem_bytes(p.B, D);
-  const dim3 grid(p.acs, p.batch * p.Hkv);
-  auto query = [&](auto kern) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess && p.acs > 8) e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-    if (e != cudaSuccess) { cudaGetLastError(); return -1; }
-    return max_active_clusters(kern, grid, dim3(kAttendThreads), smem, p.acs);
-  };
-  return p.G <= 4 ? query(attend_mma_kernel<D, true>) : query(attend_mma_kernel<D, false>);
+// Clusters of p.acs CTAs (of p.agroups warp groups) of the attend kernel the device holds at once; -1 if the query fails.
+int attend_mma_max_clusters(const Params& p) {
+  int n = -1;
+  AttendMaps none;
+  const cudaError_t e = p.d == 128 ? launch_mma<128>(p, none, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, &n)
+                                   : launch_mma<64>(p, none, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, &n);
+  if (e != cudaSuccess) { cudaGetLastError(); return -1; }
+  return n;
 }
-
-// Clusters of p.acs CTAs of the attend kernel the device holds at once; -1 if the query fails.
-int attend_mma_max_clusters(const Params& p) { return p.d == 128 ? max_clusters_mma<128>(p) : max_clusters_mma<64>(p); }
 
 cudaError_t launch_attend_mma(const Params& p, const AttendMaps& maps, const void* q, const float* rms_weight, float* out,
                               float* dbg_o_sparse, float* dbg_o_rla, cudaStream_t stream) {
-  return p.d == 128 ? launch_mma<128>(p, maps, q, rms_weight, out, dbg_o_sparse, dbg_o_rla, stream)
-                    : launch_mma<64>(p, maps, q, rms_weight, out, dbg_o_sparse, dbg_o_rla, stream);
+  return p.d == 128 ? launch_mma<128>(p, maps, q, rms_weight, out, dbg_o_sparse, dbg_o_rla, stream, nullptr)
+                    : launch_mma<64>(p, maps, q, rms_weight, out, dbg_o_sparse, dbg_o_rla, stream, nullptr);
 }
 
 }  // namespace spla

@@ -67,8 +67,9 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
   constexpr int NWARP = kScoreThreads / 32;
   extern __shared__ __align__(16) unsigned char smem_raw[];
 
-  const int u = blockIdx.y;
-  const int b = u / p.Hkv, h = u % p.Hkv;
+  const int vu = blockIdx.y;                        // index into the workspace arrays (a virtual unit in a prefill launch)
+  const UnitRef ur = unit_ref(p, vu);
+  const int u = ur.u;                               // the cache's unit: statistics, K/V, state
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = p.G;
   const int c = blockIdx.x;
@@ -81,7 +82,7 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
 
   // ------------------------------------------------------------------ score role ----------------------
   const int NW = p.NW;                              // selection windows per block; a "record" is one window
-  const int L = cover_len(p, checked_len(p, b), (long long)p.n_chunks_cap * p.chunk / NW * p.B);
+  const int L = cover_len(p, ur.L, (long long)p.n_chunks_cap * p.chunk / NW * p.B);
   const int nblk = (L + p.B - 1) / p.B;
   const int nrec = nblk * NW;
   const int chunk = p.chunk;                        // records per CTA
@@ -95,7 +96,7 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
   for (int g = 0; g < GP; ++g) {
     if (g < G) {
       float x[VEC];
-      const size_t qoff = ((size_t)b * p.Hq + (size_t)h * G + g) * D + lane * VEC;
+      const size_t qoff = (ur.qrow + g) * D + lane * VEC;
       if (q_is_bf16) load_vec<VEC>(reinterpret_cast<const __nv_bfloat16*>(q_raw) + qoff, x);
       else load_vec<VEC>(reinterpret_cast<const float*>(q_raw) + qoff, x);
 #pragma unroll
@@ -112,7 +113,10 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
   const size_t ell_stride = (size_t)p.max_blocks * NW;
   const size_t stats_u = (size_t)u * ell_stride * 2 * D;      // first element of the unit's records
   const bool rec_bf16 = (p.flags & kStatsBf16) != 0;
-  float* ell_u = p.ell + (size_t)u * G * ell_stride;
+  float* ell_u = p.ell + (size_t)vu * G * ell_stride;
+  // prefill: a position's own (last) block holds fewer tokens than the cache's record of it describes: its
+  // statistics as of that position come from the per-position table (whole-block statistics only)
+  const float* own_rec = ur.t >= 0 ? p.vstats + ((size_t)u * p.vTtot + ur.t) * 2 * D : nullptr;
   // After the warp reduction lanes 0..15 hold the mean dots and lanes 16..31 the variance dots, value index
   // lane / LPV, each replicated on LPV lanes.  Copy lane `sub` finalises record `sub` of the batch, so the
   // log / exp work of FB records runs side by side instead of one record at a time.
@@ -138,7 +142,8 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
         atomicExch(p.status, kStatusBounds);
         valid = false;
       }
-      load_record<VEC>(p.stats, stats_u + (size_t)i * 2 * D, rec_bf16, D, lane, valid, mean[buf][r], var[buf][r]);
+      if (own_rec && i == nblk - 1) load_record<VEC>(own_rec, 0, false, D, lane, valid, mean[buf][r], var[buf][r]);
+      else load_record<VEC>(p.stats, stats_u + (size_t)i * 2 * D, rec_bf16, D, lane, valid, mean[buf][r], var[buf][r]);
     }
   };
   auto compute_round = [&](int round, int buf) {
@@ -219,16 +224,16 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
     float m = -INFINITY, s = 0.f;
 #pragma unroll
     for (int w = 0; w < NWARP; ++w) lse_merge(m, s, wred[(w * GP + tid) * 2], wred[(w * GP + tid) * 2 + 1]);
-    float* cp = p.chunk_part + (((size_t)u * p.max_chunks + c) * G + tid) * 2;
+    float* cp = p.chunk_part + (((size_t)vu * p.max_chunks + c) * G + tid) * 2;
     cp[0] = m;
     cp[1] = s;
   }
   __syncthreads();                                       // every thread's stores precede thread 0's fence
   if (tid == 0) {
     __threadfence();
-    const int t = atomicAdd(&p.score_ticket[u], 1);
+    const int t = atomicAdd(&p.score_ticket[vu], 1);
     is_last_s = (t == n_chunks - 1);
-    if (is_last_s) p.score_ticket[u] = 0;                // ready for the next decode step
+    if (is_last_s) p.score_ticket[vu] = 0;               // ready for the next decode step
     __threadfence();
   }
   __syncthreads();
@@ -298,7 +303,7 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
     float m = -INFINITY, s = 0.f;
 #pragma unroll 4
     for (int cc = lane; cc < n_chunks; cc += 32) {
-      const float2 ms = __ldcg(reinterpret_cast<const float2*>(p.chunk_part + (((size_t)u * p.max_chunks + cc) * G + g) * 2));
+      const float2 ms = __ldcg(reinterpret_cast<const float2*>(p.chunk_part + (((size_t)vu * p.max_chunks + cc) * G + g) * 2));
       lse_merge(m, s, ms.x, ms.y);
     }
     const float M = warp_max(m);
@@ -310,7 +315,7 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
 
   SPLA_MARK(p, u, c, 4);
   const int k_eff = min(p.top_k, nblk);
-  float* scores_u = p.scores + (size_t)u * p.max_blocks;
+  float* scores_u = p.scores + (size_t)vu * p.max_blocks;
   float lse_r[GP];
 #pragma unroll
   for (int g = 0; g < GP; ++g) lse_r[g] = g < G ? lse_s[g] : 0.f;
@@ -408,8 +413,8 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
   __syncthreads();
   int gt_before = s_gt - n_gt, eq_before = s_eq - n_eq;
   for (int w = 0; w < warp; ++w) { gt_before += wtot[0][w]; eq_before += wtot[1][w]; }
-  int* sel_u = p.sel + (size_t)u * p.top_k;
-  int* sel_o = sel_user ? sel_user + (size_t)u * p.top_k : nullptr;
+  int* sel_u = p.sel + (size_t)vu * p.top_k;
+  int* sel_o = sel_user ? sel_user + (ur.qrow / G) * p.top_k : nullptr;   // [batch][H_kv][k], or [batch][T][H_kv][k]
   if (k_eff > 0 && n_gt + n_eq > 0) {
     for (int i = i0; i < i1; ++i) {
       const uint32_t key = keys[i];
@@ -427,14 +432,14 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
     sel_u[t] = -1;
     if (sel_o) sel_o[t] = -1;
   }
-  if (tid == 0) p.n_sel[u] = k_eff;
+  if (tid == 0) p.n_sel[vu] = k_eff;
   SPLA_MARK(p, u, c, 7);
 }
 
 template <int D, int GP>
 static cudaError_t launch_one(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream) {
-  const int U = p.batch * p.Hkv;
-  const bool rla = !(p.flags & 4u);
+  const int U = p.batch * p.Hkv * (p.vT > 0 ? p.vT : 1);
+  const bool rla = !(p.flags & 4u) && p.vT == 0;          // (a prefill launch gets o_bar from the chunk scan instead)
   dim3 grid(p.n_chunks_cap + (rla ? kStateSplits : 0), U);
   size_t smem = (size_t)p.max_blocks * sizeof(uint32_t);
   const size_t smem_state = (size_t)(GP * D + (kScoreThreads / D) * GP * D) * sizeof(float);

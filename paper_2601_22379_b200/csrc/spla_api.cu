@@ -18,8 +18,9 @@ struct spla_cache {
   Params p;
   int64_t len_bound;   // host-side upper bound of the longest sequence
   // clusters the device holds at once, as last queried: score kernel for (cs, chunk), attend kernel per log2(acs)
-  int score_occ_cs = 0, score_occ_chunk = 0, score_occ_n = -1;
-  int attend_occ[5] = {-2, -2, -2, -2, -2};
+  int score_occ_cs[2] = {0, 0}, score_occ_chunk[2] = {0, 0}, score_occ_n[2] = {-1, -1};   // [0]: 8-warp build, [1]: 16-warp
+  int attend_occ[2][5] = {{-2, -2, -2, -2, -2}, {-2, -2, -2, -2, -2}};   // [groups - 1][log2 cluster size]
+  int plan_override = 0;   // 0: planner's choice; 1: two CTAs per SM shapes; (development switch)
   int sm_count;
   AttendMaps maps;
   AttendMaps state_maps;   // the same caches in boxes of 64 tokens, for the tensor-core state kernel
@@ -168,6 +169,7 @@ extern "C" int spla_init_cache(const spla_config_t* config, const spla_buffers_t
   c->cfg = *config;
   c->buf = *b;
   c->sm_count = device_sm_count();
+  c->plan_override = getenv("SPLA_PLAN") ? atoi(getenv("SPLA_PLAN")) : 0;   // TEMPORARY development switch
   if (c->cfg.sm_scale == 0.f) c->cfg.sm_scale = 1.0f / sqrtf((float)config->head_dim);
   if (c->cfg.phi_scale == 0.f) c->cfg.phi_scale = 1.0f;
   if (c->cfg.rms_eps == 0.f) c->cfg.rms_eps = 1e-6f;
@@ -251,37 +253,52 @@ extern "C" int spla_append_tokens(spla_cache_t* c, const void* k_new, const void
 // device may hold fewer clusters of a size than its CTA slots suggest; a launch whose clusters do not all fit at
 // once runs in two waves and takes twice as long.  The cluster size is therefore lowered (where the block count
 // leaves a choice) until the occupancy query says that all units' clusters are resident together.
+// Returns true with p->cs / chunk / swarps set if the cluster kernel of `warps` warps per CTA can serve the launch;
+// for the 16-warp build (one CTA per SM) only if all its clusters are resident at once.
+static bool plan_score_size(spla_cache* c, Params* p, int64_t blocks, int warps) {
+  const int units = p->batch * p->Hkv;
+  const int wi = warps == 16 ? 1 : 0;
+  const long long slots = (long long)(warps == 16 ? 1 : 2) * c->sm_count;
+  int best_cs = 0, best_chunk = 0, occ = -1;
+  for (int cap = 16; cap >= 1; cap /= 2) {
+    int cs = 0, chunk = 0;
+    if (!plan_score_cluster(units, blocks, p->NW, p->G, p->d, c->sm_count, cap, warps, &cs, &chunk)) break;
+    if (best_cs && cs >= best_cs) break;                   // the block count needs at least this size: no choice left
+    best_cs = cs;
+    best_chunk = chunk;
+    occ = -1;
+    if (cs == 1 || (long long)units * cs > slots) break;   // several waves by necessity: nothing to gain
+    if (c->score_occ_cs[wi] != cs || c->score_occ_chunk[wi] != chunk) {
+      Params probe = *p;
+      probe.cs = cs;
+      probe.chunk = chunk;
+      probe.swarps = warps;
+      c->score_occ_n[wi] = score_cluster_max_clusters(probe);
+      c->score_occ_cs[wi] = cs;
+      c->score_occ_chunk[wi] = chunk;
+    }
+    occ = c->score_occ_n[wi];
+    if (occ < 0 || units <= occ) break;                    // unknown, or all resident at once
+  }
+  if (!best_cs) return false;
+  if (warps == 16 && ((long long)units * best_cs > slots || (occ >= 0 && units > occ))) return false;
+  p->cs = best_cs;
+  p->chunk = best_chunk;
+  p->n_chunks_cap = best_cs;
+  p->swarps = warps;
+  return true;
+}
+
 static void plan_score_grid(spla_cache* c, Params* p) {
   int64_t blocks = (c->len_bound + c->cfg.block_size - 1) / c->cfg.block_size;
   if (blocks < 1) blocks = 1;
   p->cs = 0;
-  const int units = p->batch * p->Hkv;
+  p->swarps = 8;
   if (!(c->cfg.flags & SPLA_GENERAL_KERNELS)) {
-    int best_cs = 0, best_chunk = 0;
-    for (int cap = 16; cap >= 1; cap /= 2) {
-      int cs = 0, chunk = 0;
-      if (!plan_score_cluster(units, blocks, p->NW, p->G, p->d, c->sm_count, cap, &cs, &chunk)) break;
-      if (best_cs && cs >= best_cs) break;                   // the block count needs at least this size: no choice left
-      best_cs = cs;
-      best_chunk = chunk;
-      if (cs == 1 || (long long)units * cs > 2LL * c->sm_count) break;   // several waves by necessity: nothing to gain
-      if (c->score_occ_cs != cs || c->score_occ_chunk != chunk) {
-        Params probe = *p;
-        probe.cs = cs;
-        probe.chunk = chunk;
-        c->score_occ_n = score_cluster_max_clusters(probe);
-        c->score_occ_cs = cs;
-        c->score_occ_chunk = chunk;
-      }
-      if (c->score_occ_n < 0 || units <= c->score_occ_n) break;   // unknown, or all resident at once
-    }
-    if (best_cs) {
-      p->cs = best_cs;
-      p->chunk = best_chunk;
-      p->n_chunks_cap = best_cs;
-      return;
-    }
+    if (c->plan_override != 1 && plan_score_size(c, p, blocks, 16)) return;
+    if (plan_score_size(c, p, blocks, 8)) return;
   }
+  p->cs = 0;
   p->chunk = score_chunk_for((long long)p->batch * p->Hkv, blocks * p->NW, c->sm_count);   // in records (windows)
   p->n_chunks_cap = (int)((blocks * p->NW + p->chunk - 1) / p->chunk);
 }
@@ -290,30 +307,52 @@ static cudaError_t launch_score(const Params& p, const void* q, int qb, int* sel
   return p.cs > 0 ? launch_score_cluster(p, q, qb, sel_user, pending_new, s) : launch_score_select(p, q, qb, sel_user, s);
 }
 
-// Cluster size of the tensor-core attend kernel: the largest power of two (at most 16 and at most top_k) for
-// which all CTAs are resident at once; each CTA of a cluster then walks top_k / size selected blocks.
-static int attend_cluster_size(spla_cache* c) {
-  if (c->cfg.flags & SPLA_GENERAL_KERNELS) return 0;
-  const size_t smem = attend_mma_smem_bytes(c->p.B, c->p.d) + 2048;
+// Shape of the tensor-core attend launch, written to p->acs / agroups / aslots.  The cluster size is the largest power
+// of two (at most 16 and at most top_k) for which all CTAs are resident at once; each CTA of a cluster then walks
+// top_k / size selected blocks.  Launches that fit the machine with one CTA per SM take the two-group shape (eight
+// warps, a ring as deep as shared memory allows); the others one group per CTA and two CTAs per SM.
+static void plan_attend(spla_cache* c, Params* p) {
+  p->acs = 0; p->agroups = 1; p->aslots = 2;
+  if (c->cfg.flags & SPLA_GENERAL_KERNELS) return;
+  const long long U = (long long)c->p.batch * c->p.Hkv;
+  auto resident = [&](int cs, int groups) {       // clusters of this shape the device holds at once (cached)
+    int lg = 0;
+    while ((1 << lg) < cs) ++lg;
+    int& slot = c->attend_occ[groups - 1][lg];
+    if (slot == -2) {
+      Params probe = c->p;
+      probe.acs = cs; probe.agroups = groups; probe.aslots = attend_mma_slots(c->p.B, c->p.d);
+      slot = attend_mma_max_clusters(probe);
+    }
+    return slot;
+  };
+  const int plan_env = c->plan_override;
+  if (plan_env != 1 && attend_mma_slots(c->p.B, c->p.d) >= 2 && U <= c->sm_count) {
+    int cs = 1;
+    while (cs * 2 <= 16 && cs * 2 <= c->p.top_k && U * cs * 2 <= c->sm_count) cs *= 2;
+    for (; cs > 1; cs /= 2) {
+      const int occ = resident(cs, 2);
+      if (occ < 0 || U <= occ) break;
+    }
+    const int occ1 = resident(cs, 2);
+    if ((occ1 < 0 || U <= occ1) && (U * cs * 2 > c->sm_count || cs == 16 || cs * 2 > c->p.top_k)) {
+      p->acs = cs; p->agroups = 2; p->aslots = attend_mma_slots(c->p.B, c->p.d);
+      return;
+    }
+  }
+  const size_t smem = attend_mma_smem_bytes(c->p.B, c->p.d, 1) + 2048;
   long long per_sm = (227 * 1024) / (long long)smem;
   if (per_sm > 2) per_sm = 2;                     // the kernel is compiled for two CTAs per SM (no register spills)
-  if (per_sm < 1) return 0;                       // the tiles do not fit: use the general kernel
+  if (per_sm < 1) return;                         // the tiles do not fit: use the general kernel
   const long long slots = per_sm * c->sm_count;
-  const long long U = (long long)c->p.batch * c->p.Hkv;
   int cs = 1;
   while (cs * 2 <= 16 && cs * 2 <= c->p.top_k && U * cs * 2 <= slots) cs *= 2;
   // all clusters of the launch must be resident together (see plan_score_grid): ask the device
   for (; cs > 1; cs /= 2) {
-    int lg = 0;
-    while ((1 << lg) < cs) ++lg;
-    if (c->attend_occ[lg] == -2) {
-      Params probe = c->p;
-      probe.acs = cs;
-      c->attend_occ[lg] = attend_mma_max_clusters(probe);
-    }
-    if (c->attend_occ[lg] < 0 || U <= c->attend_occ[lg]) break;
+    const int occ = resident(cs, 1);
+    if (occ < 0 || U <= occ) break;
   }
-  return cs;
+  p->acs = cs;
 }
 
 
@@ -324,7 +363,7 @@ extern "C" int spla_decode(spla_cache_t* c, const void* q, const float* rms_weig
   if (!aligned(q, 16) || !aligned(out, 16)) return SPLA_ERR_INVALID_ARG;
   Params p = c->p;
   plan_score_grid(c, &p);
-  p.acs = attend_cluster_size(c);
+  plan_attend(c, &p);
   const int qb = c->cfg.q_dtype == SPLA_BF16;
   cudaStream_t s = (cudaStream_t)stream;
   cudaError_t e = launch_score(p, q, qb, sel_idx, s);
@@ -348,7 +387,7 @@ extern "C" int spla_append_decode(spla_cache_t* c, const void* k_new, const void
   if (rc != SPLA_OK) return rc;
   Params p = c->p;
   plan_score_grid(c, &p);
-  p.acs = attend_cluster_size(c);
+  plan_attend(c, &p);
   const int qb = c->cfg.q_dtype == SPLA_BF16;
   cudaStream_t s = (cudaStream_t)stream;
   // only the fused decode-step append kernel opens the dependent launch early enough for this to matter
@@ -378,7 +417,7 @@ extern "C" int spla_decode_selected(spla_cache_t* c, const void* q, const float*
   p.n_chunks_cap = 0;                      // only the o_bar CTAs of the first kernel run
   p.chunk = kScoreChunkMin;
   p.cs = 0;
-  p.acs = attend_cluster_size(c);
+  plan_attend(c, &p);
   const int qb = c->cfg.q_dtype == SPLA_BF16;
   cudaStream_t s = (cudaStream_t)stream;
   cudaError_t e = cudaSuccess;
@@ -386,6 +425,123 @@ extern "C" int spla_decode_selected(spla_cache_t* c, const void* q, const float*
   if (e != cudaSuccess) return cuda_fail(e, "spla_decode_selected/o_bar");
   e = launch_attend_merge(p, &c->maps, q, qb, rms_weight, sel_in, out, dbg_o_sparse, dbg_o_rla, s);
   if (e != cudaSuccess) return cuda_fail(e, "spla_decode_selected/attend_merge");
+  return SPLA_OK;
+}
+
+// ---- prefill-shaped forward --------------------------------------------------------------------------------------
+// Workspace of spla_prefill: the per-position tables for the whole chunk, then the decode kernels' scratch for one
+// batch of `tb` positions (U * tb virtual units).
+struct PrefillLayout {
+  size_t vstats, vobar, ell, chunk_part, scores, sel, n_sel, att_acc, att_ml, tickets, tickets_bytes, total;
+  int max_chunks;
+};
+
+static PrefillLayout prefill_layout(const spla_config_t* c, int T, int tb) {
+  PrefillLayout w;
+  const size_t U = (size_t)c->batch * c->n_kv_heads, G = c->n_q_heads / c->n_kv_heads, d = c->head_dim;
+  const size_t max_blocks = ((size_t)c->max_context + c->block_size - 1) / c->block_size;
+  const size_t V = U * (size_t)tb;                 // virtual units per launch
+  w.max_chunks = (int)((max_blocks + kScoreChunkMin - 1) / kScoreChunkMin);
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  w.vstats = take(U * T * 2 * d * 4);
+  w.vobar = take(U * T * G * d * 4);
+  w.ell = take(V * G * max_blocks * 4);
+  w.chunk_part = take(V * w.max_chunks * G * 2 * 4);
+  w.scores = take(V * max_blocks * 4);
+  w.sel = take(V * c->top_k * 4);
+  w.n_sel = take(V * 4);
+  w.att_acc = take(V * c->top_k * 2 * G * d * 4);
+  w.att_ml = take(V * c->top_k * G * 2 * 4);
+  w.tickets = take(2 * V * 4);                      // score tickets, then attend tickets: zeroed by every call
+  w.tickets_bytes = 2 * V * 4;
+  w.total = off;
+  return w;
+}
+
+static int prefill_batch_cap(const spla_config_t* c) {   // virtual units are the grid's y dimension
+  const long long U = (long long)c->batch * c->n_kv_heads;
+  return (int)(65535 / U);
+}
+
+extern "C" int spla_query_prefill_workspace(const spla_config_t* config, int32_t T, size_t* min_bytes, size_t* good_bytes) {
+  int rc = validate_config(config);
+  if (rc) return rc;
+  if (T < 1 || (!min_bytes && !good_bytes)) return SPLA_ERR_INVALID_ARG;
+  if (prefill_batch_cap(config) < 1) return SPLA_ERR_UNSUPPORTED;
+  const size_t one = prefill_layout(config, T, 1).total;
+  if (min_bytes) *min_bytes = one;
+  if (good_bytes) {
+    // about 256 MB of per-batch scratch, at most the whole chunk at once
+    const size_t per_pos = prefill_layout(config, T, 2).total - one;
+    long long tb = (long long)((256ull << 20) / (per_pos ? per_pos : 1));
+    if (tb < 1) tb = 1;
+    if (tb > T) tb = T;
+    if (tb > prefill_batch_cap(config)) tb = prefill_batch_cap(config);
+    *good_bytes = prefill_layout(config, T, (int)tb).total;
+  }
+  return SPLA_OK;
+}
+
+extern "C" int spla_prefill(spla_cache_t* c, const void* k_new, const void* v_new, const void* q, int32_t T,
+                            const float* rms_weight, float* out, int32_t* sel_idx, void* workspace, size_t workspace_bytes,
+                            void* stream) {
+  if (!c || !k_new || !v_new || !q || !out || !workspace || T < 1) return SPLA_ERR_INVALID_ARG;
+  if (!rms_weight && !(c->cfg.flags & SPLA_NO_RLA)) return SPLA_ERR_INVALID_ARG;
+  if (!aligned(k_new, 16) || !aligned(v_new, 16) || !aligned(q, 16) || !aligned(out, 16) || !aligned(workspace, 256))
+    return SPLA_ERR_INVALID_ARG;
+  if (c->p.NW != 1) return SPLA_ERR_UNSUPPORTED;                 // whole-block statistics only
+  if (c->len_bound + T > c->cfg.max_context) return SPLA_ERR_CAPACITY;
+  // positions per launch: as many as the workspace holds
+  const int cap = prefill_batch_cap(&c->cfg);
+  if (cap < 1) return SPLA_ERR_UNSUPPORTED;
+  const size_t one = prefill_layout(&c->cfg, T, 1).total;
+  if (workspace_bytes < one) return SPLA_ERR_INVALID_ARG;
+  const size_t per_pos = prefill_layout(&c->cfg, T, 2).total - one;
+  long long tb = 1 + (long long)((workspace_bytes - one) / (per_pos ? per_pos : 1));
+  if (tb > T) tb = T;
+  if (tb > cap) tb = cap;
+  while (tb > 1 && prefill_layout(&c->cfg, T, (int)tb).total > workspace_bytes) --tb;   // (alignment padding)
+  const PrefillLayout w = prefill_layout(&c->cfg, T, (int)tb);
+  char* ws = reinterpret_cast<char*>(workspace);
+  cudaStream_t s = (cudaStream_t)stream;
+  const int qb = c->cfg.q_dtype == SPLA_BF16;
+
+  // 1. the chunk goes into the cache: K/V, per-token log-sum-exp, block statistics, lengths; the state is left for the
+  //    scan (which needs S_bar as it was before the chunk)
+  {
+    Params pa = c->p;
+    pa.flags |= SPLA_NO_RLA;
+    cudaError_t e = launch_append(pa, k_new, v_new, nullptr, T, nullptr, s);
+    if (e != cudaSuccess) return cuda_fail(e, "spla_prefill/append");
+    c->len_bound += T;
+  }
+  // 2. per-position statistics of the growing block, o_bar of every position, S_bar advanced over the chunk
+  float* vstats = reinterpret_cast<float*>(ws + w.vstats);
+  float* vobar = reinterpret_cast<float*>(ws + w.vobar);
+  cudaError_t e = launch_prefill_prepare(c->p, T, q, qb, vstats, vobar, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ws + w.tickets, 0, w.tickets_bytes, s);
+  if (e != cudaSuccess) return cuda_fail(e, "spla_prefill/prepare");
+  // 3. score, select, attend, merge: the general decode kernels over virtual units, a batch of positions per launch
+  Params pv = c->p;
+  pv.ell = (float*)(ws + w.ell); pv.chunk_part = (float*)(ws + w.chunk_part); pv.scores = (float*)(ws + w.scores);
+  pv.sel = (int*)(ws + w.sel); pv.n_sel = (int*)(ws + w.n_sel);
+  pv.att_acc = (float*)(ws + w.att_acc); pv.att_ml = (float*)(ws + w.att_ml);
+  pv.score_ticket = (int*)(ws + w.tickets); pv.attend_ticket = pv.score_ticket + (size_t)c->p.batch * c->p.Hkv * tb;
+  pv.max_chunks = w.max_chunks;
+  pv.vTtot = T; pv.vstats = vstats; pv.vobar = vobar;
+  pv.cs = 0; pv.acs = 0;
+  int64_t blocks = (c->len_bound + c->cfg.block_size - 1) / c->cfg.block_size;
+  if (blocks < 1) blocks = 1;
+  for (int t0 = 0; t0 < T; t0 += (int)tb) {
+    pv.vt0 = t0;
+    pv.vT = (int)(tb < T - t0 ? tb : T - t0);
+    pv.chunk = score_chunk_for((long long)pv.batch * pv.Hkv * pv.vT, blocks, c->sm_count);
+    pv.n_chunks_cap = (int)((blocks + pv.chunk - 1) / pv.chunk);
+    e = launch_score_select(pv, q, qb, sel_idx, s);
+    if (e == cudaSuccess) e = launch_attend_merge(pv, nullptr, q, qb, rms_weight, nullptr, out, nullptr, nullptr, s);
+    if (e != cudaSuccess) return cuda_fail(e, "spla_prefill/decode kernels");
+  }
   return SPLA_OK;
 }
 

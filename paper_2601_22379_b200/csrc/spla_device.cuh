@@ -38,6 +38,9 @@ struct Params {
   int chunk;                            // block records per score CTA
   int cs;                               // score kernel, cluster edition: CTAs per unit (0 = general kernel)
   int acs;                              // tensor-core attend kernel: CTAs (cluster size) per unit
+  int agroups;                          //   warp groups per CTA (1: two CTAs per SM, two-slot ring; 2: one CTA per SM, deep ring)
+  int aslots;                           //   ring positions of the two-group shape
+  int swarps;                           // cluster score kernel: warps per CTA (8: two CTAs per SM; 16: one CTA per SM)
   // caller buffers
   void* k_cache;
   void* v_cache;
@@ -61,6 +64,13 @@ struct Params {
   int* state_ticket;   // [U]
   int* status;         // [1]
   int max_chunks;
+  // Prefill-shaped forward (general kernels only): the grid's second dimension then counts *virtual* units, one per
+  // (sequence, KV head, query position of the current batch of positions); vT == 0 in decode.
+  int vT;                               // query positions per launch (0: decode)
+  int vt0;                              // first position of this launch within the chunk
+  int vTtot;                            // positions of the whole chunk (stride of q / out / vstats / vobar)
+  const float* vstats;                  // [U][vTtot][2][d] statistics of each position's own (last, partial) block as of that position
+  const float* vobar;                   // [U][vTtot][G][d] o_bar = phi(q_t) S_bar_t of every position
   int wait_limit;                       // iterations a bounded barrier wait polls before it gives up (0: kWaitLimitDefault)
   int dbg_tx_extra;                     // test hook: bytes added to what the decode kernels' copy barriers expect (0 in use)
 #ifdef SPLA_TRACE
@@ -183,6 +193,25 @@ __device__ __forceinline__ int checked_len(const Params& p, int b) {
     L = L < 0 ? 0 : p.max_context;
   }
   return L;
+}
+
+// What one value of the grid's unit dimension stands for.  Decode: unit u = (sequence b, KV head h), all cached
+// tokens.  Prefill-shaped forward: a virtual unit = (u, position t of the chunk); it sees the first L tokens only,
+// L = the cached length minus the chunk positions after t, which is what a decode step at that position would see.
+struct UnitRef {
+  int u, b, h, t, L;
+  size_t qrow;                          // row of the group's first head in q / out (rows of d elements)
+};
+__device__ __forceinline__ UnitRef unit_ref(const Params& p, int vu) {
+  UnitRef r;
+  if (p.vT > 0) { r.u = vu / p.vT; r.t = p.vt0 + vu % p.vT; }
+  else { r.u = vu; r.t = -1; }
+  r.b = r.u / p.Hkv;
+  r.h = r.u % p.Hkv;
+  r.L = checked_len(p, r.b);
+  if (r.t >= 0) r.L = max(0, r.L - (p.vTtot - 1 - r.t));
+  r.qrow = ((size_t)r.b * (r.t >= 0 ? p.vTtot : 1) + (size_t)max(r.t, 0)) * p.Hq + (size_t)r.h * p.G;
+  return r;
 }
 
 // A score launch is sized on the host from an upper bound of the lengths.  A length above what the launch covers (the

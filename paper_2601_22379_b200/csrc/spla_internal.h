@@ -77,7 +77,8 @@ int device_sm_count();   // multiprocessors of the current device (148 if the qu
 int score_chunk_for(long long units, long long max_seq_blocks, int sm_count);
 cudaError_t launch_score_select(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream);
 // score_cluster.cu (G <= 8, at most 16 x 1024 blocks per sequence)
-bool plan_score_cluster(int units, long long max_seq_blocks, int NW, int G, int d, int sm_count, int cs_cap, int* cs_out, int* chunk_out);
+bool plan_score_cluster(int units, long long max_seq_blocks, int NW, int G, int d, int sm_count, int cs_cap, int warps,
+                        int* cs_out, int* chunk_out);
 // Clusters of the score kernel (p.cs CTAs each, p.chunk blocks per CTA) the device holds at once; -1 if unknown.
 int score_cluster_max_clusters(const Params& p);
 cudaError_t launch_score_cluster(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new,
@@ -96,10 +97,14 @@ cudaError_t launch_attend_merge(const Params& p, const AttendMaps* maps, const v
                                 const float* rms_weight, const int* sel_in, float* out, float* dbg_o_sparse,
                                 float* dbg_o_rla, cudaStream_t stream);
 // attend_mma.cu (bf16 K/V and q, G <= 8)
-size_t attend_mma_smem_bytes(int B, int D);
-int attend_mma_max_clusters(const Params& p);   // clusters of p.acs CTAs resident at once; -1 if unknown
+size_t attend_mma_smem_bytes(int B, int D, int groups);
+int attend_mma_slots(int B, int D);             // ring positions of the two-group shape
+int attend_mma_max_clusters(const Params& p);   // clusters of p.acs CTAs (p.agroups groups each) resident at once; -1 if unknown
 cudaError_t launch_attend_mma(const Params& p, const AttendMaps& maps, const void* q, const float* rms_weight, float* out,
                               float* dbg_o_sparse, float* dbg_o_rla, cudaStream_t stream);
+// prefill.cu: prefix statistics of every chunk position's own block and the chunk scan (o_bar per position; advances S_bar)
+cudaError_t launch_prefill_prepare(const Params& p, int Ttot, const void* q, int q_is_bf16, float* vstats, float* vobar,
+                                   cudaStream_t stream);
 // append.cu
 // `state_maps` (may be null): tensor maps with boxes of 64 tokens; when given, bulk appends of a bf16 cache with
 // d = 128 update S_bar on the tensor cores instead of the FMA kernel.
