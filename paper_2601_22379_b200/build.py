@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ_DIR = os.path.join(HERE, "build")
 LIB_PATH = os.path.join(HERE, "libspla.so")
-SOURCES = ["spla_api.cu", "score_select.cu", "score_cluster.cu", "score_cluster16.cu", "attend_merge.cu", "attend_mma.cu", "append.cu", "state_umma.cu", "prefill.cu", "select_noalloc.cu"]
+SOURCES = ["spla_api.cu", "score_select.cu", "score_cluster.cu", "decode_fused.cu", "decode_fused_d128f.cu", "decode_fused_d128h.cu", "decode_fused_d64f.cu", "decode_fused_d64h.cu", "attend_merge.cu", "attend_mma.cu", "append.cu", "state_umma.cu", "prefill.cu", "select_noalloc.cu"]
 ARCH_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

@@ -1,11 +1,7 @@
-// The 8-warp build of the cluster score kernel (two CTAs per SM), the launch planner and the dispatch between the
-// two build sizes.
+// The cluster score + select kernel as a launch of its own, and the planner of its grid.
 #include "score_cluster.cuh"
 
 namespace spla {
-
-cudaError_t launch_score_cluster16(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new,
-                                   cudaStream_t stream, int* occ);   // score_cluster16.cu
 
 // Decides whether the cluster kernel can serve a launch and with which cluster size / records per CTA.
 // Returns false when the general kernel has to be used (very long sequences, groups above 8).
@@ -36,14 +32,12 @@ bool plan_score_cluster(int units, long long max_seq_blocks, int NW, int G, int 
 // and may stream the older blocks' statistics before that append has completed.
 cudaError_t launch_score_cluster(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new,
                                  cudaStream_t stream) {
-  if (p.swarps == 16) return launch_score_cluster16(p, q, q_is_bf16, sel_user, pending_new, stream, nullptr);
   return launch_size<8>(p, q, q_is_bf16, sel_user, pending_new, stream, nullptr);
 }
 
 int score_cluster_max_clusters(const Params& p) {
   int n = -1;
-  const cudaError_t e = p.swarps == 16 ? launch_score_cluster16(p, nullptr, 0, nullptr, 0, nullptr, &n)
-                                       : launch_size<8>(p, nullptr, 0, nullptr, 0, nullptr, &n);
+  const cudaError_t e = launch_size<8>(p, nullptr, 0, nullptr, 0, nullptr, &n);
   if (e != cudaSuccess) { cudaGetLastError(); return -1; }
   return n;
 }

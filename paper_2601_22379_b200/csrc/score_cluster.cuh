@@ -16,9 +16,8 @@
 // Ordering everywhere is (score descending, block index ascending).  The only waits are the two hardware
 // barriers and bounded mbarrier polls.  No multicast is used.
 //
-// The kernel is built in two sizes (template parameter NWP, the warps per CTA): 8 warps with a 96 KB ring, two CTAs
-// per SM, for launches with many units; 16 warps with a 192 KB ring, one CTA per SM, for launches whose clusters all
-// fit the machine at once - there every SM streams with the same number of warps and twice the bytes in flight.
+// The body is a device function: it is the whole of the score + select kernel (spla_select, and spla_decode where the
+// fused kernel does not apply) and the first half of the fused decode kernel (decode_fused.cuh).
 #pragma once
 
 #include "spla_internal.h"
@@ -34,22 +33,6 @@ constexpr int kStages = 3;
 constexpr int kMaxCluster = 16;
 constexpr int kSlotRec = 16;                             // records per slot of the tensor-core streaming path
 
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ uint32_t map_to_rank(uint32_t smem_addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ float ld_dsmem_f32(uint32_t addr) {
-  float v;
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
-  return v;
-}
-__device__ __forceinline__ void st_dsmem_u32(uint32_t addr, uint32_t v) {
-  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
-}
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -65,19 +48,6 @@ __device__ __forceinline__ void lse_merge(float& m, float& s, float m2, float s2
   const float nm = fmaxf(m, m2);
   if (nm > -INFINITY) s = s * __expf(m - nm) + s2 * __expf(m2 - nm);
   m = nm;
-}
-
-// Warp-level tensor-core product D += A B with fp32 accumulators.  Fragment layout (PTX ISA, mma.m16n8k16;
-// g = lane / 4, t = lane % 4): A rows g and g + 8, B column g, D rows g and g + 8 at columns 2t, 2t + 1.
-__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                         uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<const uint32_t*>(&v);
 }
 
 // Sums N per-lane values over aligned groups of W lanes (W = 16 or 32, N <= W a power of two) by halving:
@@ -142,10 +112,11 @@ struct Smem {
 // more, so their statistics are streamed while the append still runs; only then does the kernel wait for the
 // append, read the final length and take the few remaining blocks (those the append wrote to) from global memory.
 // ST: element type of the statistics records (float, or __nv_bfloat16 with half the bytes to stream).
+// On return the selection of the unit is in p.sel / p.n_sel (and sel_user), written by the cluster's leader, and the
+// o_bar partials in p.obar_part; every thread of every CTA of the cluster returns (nobody has left the kernel).
 template <int D, int GP, bool WIN, bool EARLY, typename ST, int NWP>
-__global__ void __launch_bounds__(NWP * 32, NWP == 8 ? 2 : 1) score_cluster_kernel(const Params p, const void* __restrict__ q_raw,
-                                                                                   int q_is_bf16, int* __restrict__ sel_user,
-                                                                                   int pending_new) {
+__device__ __forceinline__ void score_cluster_body(const Params& p, const void* __restrict__ q_raw, int q_is_bf16,
+                                                   int* __restrict__ sel_user, int pending_new, unsigned char* smem_raw) {
   using SM = Smem<D, GP, ST, NWP>;
   constexpr int kCsConsumers = NWP;             // warps; all consume, lane 0 of warp 0 also feeds the ring
   constexpr int kCsThreads = NWP * 32;
@@ -159,7 +130,6 @@ __global__ void __launch_bounds__(NWP * 32, NWP == 8 ? 2 : 1) score_cluster_kern
   constexpr int LPV = W / NV;                   // lanes holding a copy of each reduced value
   constexpr int FB = LPV < PASSES ? LPV : PASSES;
   static_assert(LPV >= 1, "group too large for the lane layout");
-  extern __shared__ __align__(1024) unsigned char smem_raw[];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int CS = gridDim.x;
@@ -671,12 +641,12 @@ __global__ void __launch_bounds__(NWP * 32, NWP == 8 ? 2 : 1) score_cluster_kern
     // The siblings are done with the selection; while the leader finishes it they compute the part of the
     // residual branch that needs no selection, o_bar = phi(q) S_bar, one slice of the state's rows each.
     if (rla)
-      for (int s = rank - 1; s < kStateSplits; s += CS - 1)
+      for (int s = rank - 1; s < kStateSplits; s += CS - 1) {
+        __syncthreads();                       // (the slices of one CTA reuse the same shared memory)
         state_role<D, GP, kCsThreads>(p, u, s, q_raw, q_is_bf16, reinterpret_cast<float*>(smem_raw));
+      }
     SPLA_MARK(p, u, rank, 7);
-    return;
-  }
-
+  } else {
   // ------------------------------------------------------------------ phase C (leader) ----------------------
   const uint32_t* cand_key = reinterpret_cast<const uint32_t*>(smem_raw + SM::kCandKey);
   const int* cand_idx = reinterpret_cast<const int*>(smem_raw + SM::kCandIdx);
@@ -785,6 +755,15 @@ __global__ void __launch_bounds__(NWP * 32, NWP == 8 ? 2 : 1) score_cluster_kern
       __syncthreads();
       state_role<D, GP, kCsThreads>(p, u, s, q_raw, q_is_bf16, reinterpret_cast<float*>(smem_raw));
     }
+  }   // leader
+}
+
+template <int D, int GP, bool WIN, bool EARLY, typename ST, int NWP>
+__global__ void __launch_bounds__(NWP * 32, 2) score_cluster_kernel(const Params p, const void* __restrict__ q_raw,
+                                                                    int q_is_bf16, int* __restrict__ sel_user,
+                                                                    int pending_new) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  score_cluster_body<D, GP, WIN, EARLY, ST, NWP>(p, q_raw, q_is_bf16, sel_user, pending_new, smem_raw);
 }
 
 // `occupancy` non-null: nothing is launched; it receives the number of clusters of this launch that the device holds

@@ -18,9 +18,9 @@ struct spla_cache {
   Params p;
   int64_t len_bound;   // host-side upper bound of the longest sequence
   // clusters the device holds at once, as last queried: score kernel for (cs, chunk), attend kernel per log2(acs)
-  int score_occ_cs[2] = {0, 0}, score_occ_chunk[2] = {0, 0}, score_occ_n[2] = {-1, -1};   // [0]: 8-warp build, [1]: 16-warp
-  int attend_occ[2][5] = {{-2, -2, -2, -2, -2}, {-2, -2, -2, -2, -2}};   // [groups - 1][log2 cluster size]
-  int plan_override = 0;   // 0: planner's choice; 1: two CTAs per SM shapes; (development switch)
+  int score_occ_cs[2] = {0, 0}, score_occ_chunk[2] = {0, 0}, score_occ_n[2] = {-1, -1};   // [0]: score kernel, [1]: fused decode kernel
+  int attend_occ[5] = {-2, -2, -2, -2, -2};   // by log2 of the cluster size
+  int plan_override = 0;   // 0: planner's choice; 1: never the fused decode kernel (development switch)
   int sm_count;
   AttendMaps maps;
   AttendMaps state_maps;   // the same caches in boxes of 64 tokens, for the tensor-core state kernel
@@ -253,93 +253,74 @@ extern "C" int spla_append_tokens(spla_cache_t* c, const void* k_new, const void
 // device may hold fewer clusters of a size than its CTA slots suggest; a launch whose clusters do not all fit at
 // once runs in two waves and takes twice as long.  The cluster size is therefore lowered (where the block count
 // leaves a choice) until the occupancy query says that all units' clusters are resident together.
-// Returns true with p->cs / chunk / swarps set if the cluster kernel of `warps` warps per CTA can serve the launch;
-// for the 16-warp build (one CTA per SM) only if all its clusters are resident at once.
-static bool plan_score_size(spla_cache* c, Params* p, int64_t blocks, int warps) {
+// `fused`: the plan is for the fused decode kernel (score + attend in one launch), whose occupancy is asked for.
+// Returns true with p->cs / chunk set if a cluster kernel can serve the launch.
+static bool plan_score_clusters(spla_cache* c, Params* p, int64_t blocks, bool fused) {
   const int units = p->batch * p->Hkv;
-  const int wi = warps == 16 ? 1 : 0;
-  const long long slots = (long long)(warps == 16 ? 1 : 2) * c->sm_count;
-  int best_cs = 0, best_chunk = 0, occ = -1;
+  const int wi = fused ? 1 : 0;
+  // CTAs per SM: two, unless the attend phase's K/V ring (blocks of 128 tokens at d = 128) takes more than half an SM
+  int per_sm = 2;
+  if (fused && attend_mma_smem_bytes(p->B, p->d, 1) + 4096 > (size_t)113 * 1024) per_sm = 1;
+  const long long slots = (long long)per_sm * c->sm_count;
+  int best_cs = 0, best_chunk = 0;
   for (int cap = 16; cap >= 1; cap /= 2) {
     int cs = 0, chunk = 0;
-    if (!plan_score_cluster(units, blocks, p->NW, p->G, p->d, c->sm_count, cap, warps, &cs, &chunk)) break;
+    if (!plan_score_cluster(units, blocks, p->NW, p->G, p->d, per_sm * c->sm_count / 2, cap, 8, &cs, &chunk)) break;
     if (best_cs && cs >= best_cs) break;                   // the block count needs at least this size: no choice left
     best_cs = cs;
     best_chunk = chunk;
-    occ = -1;
     if (cs == 1 || (long long)units * cs > slots) break;   // several waves by necessity: nothing to gain
     if (c->score_occ_cs[wi] != cs || c->score_occ_chunk[wi] != chunk) {
       Params probe = *p;
       probe.cs = cs;
       probe.chunk = chunk;
-      probe.swarps = warps;
-      c->score_occ_n[wi] = score_cluster_max_clusters(probe);
+      probe.swarps = 8;
+      c->score_occ_n[wi] = fused ? decode_fused_max_clusters(probe) : score_cluster_max_clusters(probe);
       c->score_occ_cs[wi] = cs;
       c->score_occ_chunk[wi] = chunk;
     }
-    occ = c->score_occ_n[wi];
+    const int occ = c->score_occ_n[wi];
     if (occ < 0 || units <= occ) break;                    // unknown, or all resident at once
   }
   if (!best_cs) return false;
-  if (warps == 16 && ((long long)units * best_cs > slots || (occ >= 0 && units > occ))) return false;
   p->cs = best_cs;
   p->chunk = best_chunk;
   p->n_chunks_cap = best_cs;
-  p->swarps = warps;
+  p->swarps = 8;
   return true;
 }
 
-static void plan_score_grid(spla_cache* c, Params* p) {
+// `fused`: plan for the fused decode kernel if a cluster plan exists (p->cs > 0 on return), else for the general kernel.
+static void plan_score_grid(spla_cache* c, Params* p, bool fused = false) {
   int64_t blocks = (c->len_bound + c->cfg.block_size - 1) / c->cfg.block_size;
   if (blocks < 1) blocks = 1;
   p->cs = 0;
   p->swarps = 8;
-  if (!(c->cfg.flags & SPLA_GENERAL_KERNELS)) {
-    if (c->plan_override != 1 && plan_score_size(c, p, blocks, 16)) return;
-    if (plan_score_size(c, p, blocks, 8)) return;
-  }
+  if (!(c->cfg.flags & SPLA_GENERAL_KERNELS) && plan_score_clusters(c, p, blocks, fused)) return;
   p->cs = 0;
   p->chunk = score_chunk_for((long long)p->batch * p->Hkv, blocks * p->NW, c->sm_count);   // in records (windows)
   p->n_chunks_cap = (int)((blocks * p->NW + p->chunk - 1) / p->chunk);
 }
 
+// The fused decode kernel serves bf16 caches and queries with groups of up to 8 heads (what the tensor-core attend
+// phase is built for) whenever the cluster score plan exists.
+static bool fused_eligible(const spla_cache* c) {
+  return c->plan_override != 1 && !(c->cfg.flags & SPLA_GENERAL_KERNELS) && c->p.kv_bf16 && c->cfg.q_dtype == SPLA_BF16 &&
+         c->p.G <= 8 && c->maps.valid && attend_mma_smem_bytes(c->p.B, c->p.d, 1) + 4096 <= (size_t)113 * 1024;
+}
+
+
 static cudaError_t launch_score(const Params& p, const void* q, int qb, int* sel_user, cudaStream_t s, int pending_new = 0) {
   return p.cs > 0 ? launch_score_cluster(p, q, qb, sel_user, pending_new, s) : launch_score_select(p, q, qb, sel_user, s);
 }
 
-// Shape of the tensor-core attend launch, written to p->acs / agroups / aslots.  The cluster size is the largest power
-// of two (at most 16 and at most top_k) for which all CTAs are resident at once; each CTA of a cluster then walks
-// top_k / size selected blocks.  Launches that fit the machine with one CTA per SM take the two-group shape (eight
-// warps, a ring as deep as shared memory allows); the others one group per CTA and two CTAs per SM.
+// Cluster size of the tensor-core attend kernel as a launch of its own, written to p->acs: the largest power of two (at
+// most 16 and at most top_k) for which all CTAs are resident at once; each CTA of a cluster then walks top_k / size
+// selected blocks.
 static void plan_attend(spla_cache* c, Params* p) {
   p->acs = 0; p->agroups = 1; p->aslots = 2;
   if (c->cfg.flags & SPLA_GENERAL_KERNELS) return;
   const long long U = (long long)c->p.batch * c->p.Hkv;
-  auto resident = [&](int cs, int groups) {       // clusters of this shape the device holds at once (cached)
-    int lg = 0;
-    while ((1 << lg) < cs) ++lg;
-    int& slot = c->attend_occ[groups - 1][lg];
-    if (slot == -2) {
-      Params probe = c->p;
-      probe.acs = cs; probe.agroups = groups; probe.aslots = attend_mma_slots(c->p.B, c->p.d);
-      slot = attend_mma_max_clusters(probe);
-    }
-    return slot;
-  };
-  const int plan_env = c->plan_override;
-  if (plan_env != 1 && attend_mma_slots(c->p.B, c->p.d) >= 2 && U <= c->sm_count) {
-    int cs = 1;
-    while (cs * 2 <= 16 && cs * 2 <= c->p.top_k && U * cs * 2 <= c->sm_count) cs *= 2;
-    for (; cs > 1; cs /= 2) {
-      const int occ = resident(cs, 2);
-      if (occ < 0 || U <= occ) break;
-    }
-    const int occ1 = resident(cs, 2);
-    if ((occ1 < 0 || U <= occ1) && (U * cs * 2 > c->sm_count || cs == 16 || cs * 2 > c->p.top_k)) {
-      p->acs = cs; p->agroups = 2; p->aslots = attend_mma_slots(c->p.B, c->p.d);
-      return;
-    }
-  }
   const size_t smem = attend_mma_smem_bytes(c->p.B, c->p.d, 1) + 2048;
   long long per_sm = (227 * 1024) / (long long)smem;
   if (per_sm > 2) per_sm = 2;                     // the kernel is compiled for two CTAs per SM (no register spills)
@@ -347,30 +328,48 @@ static void plan_attend(spla_cache* c, Params* p) {
   const long long slots = per_sm * c->sm_count;
   int cs = 1;
   while (cs * 2 <= 16 && cs * 2 <= c->p.top_k && U * cs * 2 <= slots) cs *= 2;
-  // all clusters of the launch must be resident together (see plan_score_grid): ask the device
+  // all clusters of the launch must be resident together (see plan_score_clusters): ask the device
   for (; cs > 1; cs /= 2) {
-    const int occ = resident(cs, 1);
-    if (occ < 0 || U <= occ) break;
+    int lg = 0;
+    while ((1 << lg) < cs) ++lg;
+    if (c->attend_occ[lg] == -2) {
+      Params probe = c->p;
+      probe.acs = cs; probe.agroups = 1; probe.aslots = 2;
+      c->attend_occ[lg] = attend_mma_max_clusters(probe);
+    }
+    if (c->attend_occ[lg] < 0 || U <= c->attend_occ[lg]) break;
   }
   p->acs = cs;
 }
 
+// Steps a1-a5 for every unit: the fused kernel where it applies, else score + select and attend + merge as two launches.
+static int launch_decode(spla_cache* c, const void* q, const float* rms_weight, float* out, int32_t* sel_idx,
+                         float* dbg_o_sparse, float* dbg_o_rla, int pending, cudaStream_t s, const char* where) {
+  Params p = c->p;
+  const int qb = c->cfg.q_dtype == SPLA_BF16;
+  cudaError_t e;
+  if (fused_eligible(c)) {
+    // (a launch of several waves keeps the two-kernel form: measured faster there, the phases of different waves
+    // would otherwise compete for the same SMs)
+    plan_score_grid(c, &p, true);
+    if (p.cs > 0 && (long long)p.batch * p.Hkv * p.cs <= 2LL * c->sm_count) {
+      e = launch_decode_fused(p, c->maps, q, rms_weight, out, dbg_o_sparse, dbg_o_rla, sel_idx, pending, s);
+      return e == cudaSuccess ? SPLA_OK : cuda_fail(e, where);
+    }
+  }
+  plan_score_grid(c, &p, false);
+  plan_attend(c, &p);
+  e = launch_score(p, q, qb, sel_idx, s, pending);
+  if (e == cudaSuccess) e = launch_attend_merge(p, &c->maps, q, qb, rms_weight, nullptr, out, dbg_o_sparse, dbg_o_rla, s);
+  return e == cudaSuccess ? SPLA_OK : cuda_fail(e, where);
+}
 
 extern "C" int spla_decode(spla_cache_t* c, const void* q, const float* rms_weight, float* out, int32_t* sel_idx,
                            float* dbg_o_sparse, float* dbg_o_rla, void* stream) {
   if (!c || !q || !out) return SPLA_ERR_INVALID_ARG;
   if (!rms_weight && !(c->cfg.flags & SPLA_NO_RLA)) return SPLA_ERR_INVALID_ARG;
   if (!aligned(q, 16) || !aligned(out, 16)) return SPLA_ERR_INVALID_ARG;
-  Params p = c->p;
-  plan_score_grid(c, &p);
-  plan_attend(c, &p);
-  const int qb = c->cfg.q_dtype == SPLA_BF16;
-  cudaStream_t s = (cudaStream_t)stream;
-  cudaError_t e = launch_score(p, q, qb, sel_idx, s);
-  if (e != cudaSuccess) return cuda_fail(e, "spla_decode/score_select");
-  e = launch_attend_merge(p, &c->maps, q, qb, rms_weight, nullptr, out, dbg_o_sparse, dbg_o_rla, s);
-  if (e != cudaSuccess) return cuda_fail(e, "spla_decode/attend_merge");
-  return SPLA_OK;
+  return launch_decode(c, q, rms_weight, out, sel_idx, dbg_o_sparse, dbg_o_rla, 0, (cudaStream_t)stream, "spla_decode");
 }
 
 // One decode step, append then decode, as one call.  Because the score kernel then directly follows this step's
@@ -385,18 +384,10 @@ extern "C" int spla_append_decode(spla_cache_t* c, const void* k_new, const void
   if (!aligned(q, 16) || !aligned(out, 16)) return SPLA_ERR_INVALID_ARG;
   const int rc = spla_append_tokens(c, k_new, v_new, n_new, max_new, stream);
   if (rc != SPLA_OK) return rc;
-  Params p = c->p;
-  plan_score_grid(c, &p);
-  plan_attend(c, &p);
-  const int qb = c->cfg.q_dtype == SPLA_BF16;
-  cudaStream_t s = (cudaStream_t)stream;
   // only the fused decode-step append kernel opens the dependent launch early enough for this to matter
   const int pending = (max_new <= 32) ? max_new : 0;
-  cudaError_t e = launch_score(p, q, qb, sel_idx, s, pending);
-  if (e != cudaSuccess) return cuda_fail(e, "spla_append_decode/score_select");
-  e = launch_attend_merge(p, &c->maps, q, qb, rms_weight, nullptr, out, dbg_o_sparse, dbg_o_rla, s);
-  if (e != cudaSuccess) return cuda_fail(e, "spla_append_decode/attend_merge");
-  return SPLA_OK;
+  return launch_decode(c, q, rms_weight, out, sel_idx, dbg_o_sparse, dbg_o_rla, pending, (cudaStream_t)stream,
+                       "spla_append_decode");
 }
 
 extern "C" int spla_select(spla_cache_t* c, const void* q, int32_t* sel_idx, void* stream) {

@@ -105,6 +105,11 @@ cudaError_t launch_attend_mma(const Params& p, const AttendMaps& maps, const voi
 // prefill.cu: prefix statistics of every chunk position's own block and the chunk scan (o_bar per position; advances S_bar)
 cudaError_t launch_prefill_prepare(const Params& p, int Ttot, const void* q, int q_is_bf16, float* vstats, float* vobar,
                                    cudaStream_t stream);
+// decode_fused.cu: score + select + attend + merge of one decode step as one cluster kernel (bf16 K/V and q, G <= 8;
+// the cluster plan in p.cs / p.chunk).  pending_new as for launch_score_cluster.
+cudaError_t launch_decode_fused(const Params& p, const AttendMaps& maps, const void* q, const float* rms_weight, float* out,
+                                float* dbg_o_sparse, float* dbg_o_rla, int* sel_user, int pending_new, cudaStream_t stream);
+int decode_fused_max_clusters(const Params& p);   // clusters of p.cs CTAs resident at once; -1 if unknown
 // append.cu
 // `state_maps` (may be null): tensor maps with boxes of 64 tokens; when given, bulk appends of a bf16 cache with
 // d = 128 update S_bar on the tensor cores instead of the FMA kernel.

@@ -102,11 +102,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t addr, float (&v)[32]) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
-  const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);        // a in the low half
-  return *reinterpret_cast<const uint32_t*>(&h);
-}
-
 #ifdef SPLA_TRACE
 #define SU_MARK(i, k)                                                                       \
   do {                                                                                      \
