@@ -83,7 +83,8 @@ template <int D, bool PACK, int NG, bool FUSED>
 __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorMap& map_k, const CUtensorMap& map_v,
                                                 const __nv_bfloat16* __restrict__ q, const float* __restrict__ rms_weight,
                                                 float* __restrict__ out, float* __restrict__ dbg_sparse,
-                                                float* __restrict__ dbg_rla, unsigned char* smem_raw) {
+                                                float* __restrict__ dbg_rla, unsigned char* smem_raw,
+                                                const int* sel_share = nullptr) {
   constexpr int KS = D / 16;        // k-steps of the two QK-type products
   constexpr int NT = D / 8;         // n-tiles of the PV-type product
   constexpr int NH = D / 64;        // 64-column halves of a tile (one TMA box each)
@@ -179,9 +180,11 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
 
   if constexpr (!FUSED) pdl_wait();             // the selection of this step is complete and visible from here on
 
-  int nsel = __ldcg(p.n_sel + u);
-  const int L = checked_len(p, b);
-  for (int i = tid; i < p.top_k; i += NTHR) sel_s[i] = __ldcg(p.sel + (size_t)u * p.top_k + i);
+  // the selection, its size and the length: from the workspace, or (fused kernel) from where the score phase's leader
+  // left them in this CTA's shared memory
+  int nsel = sel_share ? sel_share[kMaxTopK] : __ldcg(p.n_sel + u);
+  const int L = sel_share ? sel_share[kMaxTopK + 1] : checked_len(p, b);
+  for (int i = tid; i < p.top_k; i += NTHR) sel_s[i] = sel_share ? (i < nsel ? sel_share[i] : -1) : __ldcg(p.sel + (size_t)u * p.top_k + i);
   if (p.flags & kDebugBounds) {
     // checked build: the list must name nsel existing blocks; it is cut at the first entry that does not, and the
     // status word says so (every CTA of the cluster sees the same list and cuts it at the same place)

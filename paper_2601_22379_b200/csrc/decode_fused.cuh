@@ -28,11 +28,21 @@ __global__ void __launch_bounds__(256, 2)
                         const __nv_bfloat16* __restrict__ q, const float* __restrict__ rms_weight, float* __restrict__ out,
                         float* __restrict__ dbg_sparse, float* __restrict__ dbg_rla, int* __restrict__ sel_user, int pending_new) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  score_cluster_body<D, GP, WIN, EARLY, ST, 8>(p, q, 1, sel_user, pending_new, smem_raw);
-  cluster_sync_all();      // p.sel / p.n_sel (leader) and p.obar_part (siblings) are visible; phase 1's shared memory is dead
+  __shared__ int sel_share[kMaxTopK + 2];   // the unit's selection, its size, the length: written in every CTA by the leader
+  if (threadIdx.x == 0) {                   // the K/V tensor maps are needed late: have them fetched now
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
+  }
+  score_cluster_body<D, GP, WIN, EARLY, ST, 8>(p, q, 1, sel_user, pending_new, smem_raw, sel_share);
+  // Phase 2's tiles arrive through the asynchronous proxy (TMA) in shared memory that phase 1 has just read and written
+  // through the generic proxy (the statistics ring, the selection's work arrays, the o_bar scratch): every thread orders
+  // its accesses before them.
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __threadfence();         // the o_bar partials went to global memory: performed device-wide before the barrier releases them
+  cluster_sync_all();      // the selection (every CTA's sel_share) and p.obar_part (siblings) are visible; phase 1's shared memory is dead
   if ((threadIdx.x >> 5) < 4) {
     warpgroup_reg_inc<232>();
-    attend_mma_body<D, (GP <= 4), 1, true>(p, map_k, map_v, q, rms_weight, out, dbg_sparse, dbg_rla, smem_raw);
+    attend_mma_body<D, (GP <= 4), 1, true>(p, map_k, map_v, q, rms_weight, out, dbg_sparse, dbg_rla, smem_raw, sel_share);
   } else {
     warpgroup_reg_dec<24>();
     cluster_sync_all();    // the two cluster barriers of phase 2 count every thread of the cluster

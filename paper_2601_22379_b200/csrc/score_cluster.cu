@@ -3,29 +3,18 @@
 
 namespace spla {
 
-// Decides whether the cluster kernel can serve a launch and with which cluster size / records per CTA.
-// Returns false when the general kernel has to be used (very long sequences, groups above 8).
-// `cs_cap` bounds the cluster size from above where the block count leaves a choice (the caller lowers it when the
-// device cannot hold all clusters of the first choice at once).  `warps` is the build size (8 or 16): the 16-warp
-// build holds one CTA per SM, so the machine is full with half as many CTAs.
-bool plan_score_cluster(int units, long long max_seq_blocks, int NW, int G, int d, int sm_count, int cs_cap, int warps,
-                        int* cs_out, int* chunk_out) {
-  if (G > 8) return false;
+// Blocks per CTA when `cs` CTAs share a sequence of at most max_seq_blocks blocks, or 0 if the cluster kernel cannot
+// serve that (groups above 8, more than 1024 blocks per CTA, shared memory).  The share is the exact quotient rounded
+// up to a multiple of 8, so that the CTAs of a cluster stream equal amounts.
+int score_cluster_chunk(long long max_seq_blocks, int cs, int NW, int G, int d) {
+  if (G > 8 || cs < 1 || cs > kMaxCluster) return 0;
   if (max_seq_blocks < 1) max_seq_blocks = 1;
-  if (cs_cap > kMaxCluster) cs_cap = kMaxCluster;
-  const int per_sm = warps == 16 ? 1 : 2;
-  const long long per_cta_max = warps == 16 ? 1024 : 576;                     // keep the local ranking short
-  int cs = 1;
-  while (cs < kMaxCluster && max_seq_blocks > per_cta_max * cs) cs *= 2;
-  while (cs < cs_cap && (long long)units * cs * 2 <= (long long)per_sm * sm_count) cs *= 2;   // fill the machine once
-  const long long chunk = (max_seq_blocks + cs - 1) / cs;
-  const int chunk32 = (int)((chunk + 31) / 32 * 32);
-  if (chunk32 > 1024) return false;
-  const size_t ring = (size_t)kStages * warps * kRecPerWarp * 2 * d * 4;
-  if (ring + 4096 + (size_t)G * chunk32 * 4 > (size_t)(warps == 16 ? 226 : 200) * 1024) return false;
-  *cs_out = cs;
-  *chunk_out = chunk32;
-  return true;
+  const long long chunk = ((max_seq_blocks + cs - 1) / cs + 7) / 8 * 8;
+  if (chunk > 1024) return 0;
+  const size_t ring = (size_t)kStages * 8 * kRecPerWarp * 2 * d * 4;
+  if (ring + 4096 + (size_t)G * chunk * 4 > (size_t)200 * 1024) return 0;
+  (void)NW;
+  return (int)chunk;
 }
 
 // pending_new > 0: the kernel directly follows, in the stream, an append of at most that many tokens per sequence

@@ -92,7 +92,11 @@ struct Smem {
   static constexpr int kScratch = (kSelTmp + kMaxTopK * 4 + 15) / 16 * 16; // TopkScratch
   static constexpr int kWorkEnd = (kScratch + (int)sizeof(TopkScratch) + 1023) / 1024 * 1024;
   // the ring, padded where the work arrays need more than its stages
-  static constexpr int kRingBytes = kStreamBytes > kWorkEnd ? kStreamBytes : kWorkEnd;
+  // ... and, for the fused decode kernel, padded to 68 KB: the attend phase lays its K/V tile ring (at most 66 KB) over
+  // this area, and the tile copies must stay clear of the fixed region below, which holds this phase's mbarrier
+  // objects (never invalidated: overwriting them with tile data corrupted value rows, found with NaN-filled memory)
+  static constexpr int kRingBytes0 = kStreamBytes > kWorkEnd ? kStreamBytes : kWorkEnd;
+  static constexpr int kRingBytes = kRingBytes0 > 68 * 1024 ? kRingBytes0 : 68 * 1024;
   // fixed region after the ring:
   static constexpr int kPart = kRingBytes;                          // float [GP][2]  this CTA's (max, sum)
   static constexpr int kAllPart = kPart + GP * 2 * 4;               // float [16][GP][2]
@@ -115,8 +119,11 @@ struct Smem {
 // On return the selection of the unit is in p.sel / p.n_sel (and sel_user), written by the cluster's leader, and the
 // o_bar partials in p.obar_part; every thread of every CTA of the cluster returns (nobody has left the kernel).
 template <int D, int GP, bool WIN, bool EARLY, typename ST, int NWP>
+// `sel_share` (fused kernel only, else null): a shared-memory array of kMaxTopK + 2 ints at the same place in every CTA
+// of the cluster; the leader also writes the selection there, in every CTA, followed by the count and the length.
 __device__ __forceinline__ void score_cluster_body(const Params& p, const void* __restrict__ q_raw, int q_is_bf16,
-                                                   int* __restrict__ sel_user, int pending_new, unsigned char* smem_raw) {
+                                                   int* __restrict__ sel_user, int pending_new, unsigned char* smem_raw,
+                                                   int* sel_share = nullptr) {
   using SM = Smem<D, GP, ST, NWP>;
   constexpr int kCsConsumers = NWP;             // warps; all consume, lane 0 of warp 0 also feeds the ring
   constexpr int kCsThreads = NWP * 32;
@@ -179,6 +186,7 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
   constexpr int NJ = D * (int)sizeof(ST) / 64;   // 16-byte chunks per thread and record half
   const int g8 = lane >> 2, t4 = lane & 3;
   uint32_t bq[MMA ? NJ : 1][4], bv[MMA ? NJ : 1][4];
+  float qm[GP][VECW], qv[GP][VECW];
   if constexpr (MMA) {
     const int head = g8 >> 1, part = g8 & 1;
 #pragma unroll
@@ -214,7 +222,6 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
       }
     }
   }
-  float qm[GP][VECW], qv[GP][VECW];
 #pragma unroll
   for (int g = 0; g < GP && !MMA; ++g) {
     if (g < G) {
@@ -380,10 +387,12 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
             for (int g = 0; g < GP; ++g) {
               // packed fp32 FMAs (two products per instruction): even and odd channels accumulate side by side
               float2 am = make_float2(0.f, 0.f), av = make_float2(0.f, 0.f);
+              if (GP <= 4 || g < G) {              // (groups of 5 to 7 heads: the padded heads' products are skipped)
 #pragma unroll
-              for (int v = 0; v < VECW; v += 2) {
-                am = __ffma2_rn(make_float2(qm[g][v], qm[g][v + 1]), make_float2(mean[p0 + pp][v], mean[p0 + pp][v + 1]), am);
-                av = __ffma2_rn(make_float2(qv[g][v], qv[g][v + 1]), make_float2(var[p0 + pp][v], var[p0 + pp][v + 1]), av);
+                for (int v = 0; v < VECW; v += 2) {
+                  am = __ffma2_rn(make_float2(qm[g][v], qm[g][v + 1]), make_float2(mean[p0 + pp][v], mean[p0 + pp][v + 1]), am);
+                  av = __ffma2_rn(make_float2(qv[g][v], qv[g][v + 1]), make_float2(var[p0 + pp][v], var[p0 + pp][v + 1]), av);
+                }
               }
               vals[g] = am.x + am.y;
               vals[GP + g] = av.x + av.y;
@@ -743,12 +752,21 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
       for (int j = 0; j < k_eff; ++j) pos += sel_tmp[j] < ia;
       sel_u[pos] = ia;
       if (sel_o) sel_o[pos] = ia;
+      if (sel_share)
+        for (int r = 0; r < CS; ++r) st_dsmem_u32(map_to_rank(smem_u32(sel_share + pos), (uint32_t)r), (uint32_t)ia);
     } else {
       sel_u[s] = -1;
       if (sel_o) sel_o[s] = -1;
     }
   }
-  if (tid == 0) p.n_sel[u] = k_eff;
+  if (tid == 0) {
+    p.n_sel[u] = k_eff;
+    if (sel_share)
+      for (int r = 0; r < CS; ++r) {
+        st_dsmem_u32(map_to_rank(smem_u32(sel_share + kMaxTopK), (uint32_t)r), (uint32_t)k_eff);
+        st_dsmem_u32(map_to_rank(smem_u32(sel_share + kMaxTopK + 1), (uint32_t)r), (uint32_t)L);
+      }
+  }
   SPLA_MARK(p, u, rank, 7);
   if (rla && CS == 1)
     for (int s = 0; s < kStateSplits; ++s) {

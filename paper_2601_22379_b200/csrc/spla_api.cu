@@ -18,7 +18,7 @@ struct spla_cache {
   Params p;
   int64_t len_bound;   // host-side upper bound of the longest sequence
   // clusters the device holds at once, as last queried: score kernel for (cs, chunk), attend kernel per log2(acs)
-  int score_occ_cs[2] = {0, 0}, score_occ_chunk[2] = {0, 0}, score_occ_n[2] = {-1, -1};   // [0]: score kernel, [1]: fused decode kernel
+  int score_occ_chunk[2][17] = {}, score_occ_n[2][17] = {};   // resident clusters as last queried, by [kernel: score / fused decode][cluster size]
   int attend_occ[5] = {-2, -2, -2, -2, -2};   // by log2 of the cluster size
   int plan_override = 0;   // 0: planner's choice; 1: never the fused decode kernel (development switch)
   int sm_count;
@@ -249,43 +249,51 @@ extern "C" int spla_append_tokens(spla_cache_t* c, const void* k_new, const void
   return SPLA_OK;
 }
 
-// Sizes the score grid from the host-side bound of the sequence lengths.  A cluster's CTAs sit in one GPC, so the
-// device may hold fewer clusters of a size than its CTA slots suggest; a launch whose clusters do not all fit at
-// once runs in two waves and takes twice as long.  The cluster size is therefore lowered (where the block count
-// leaves a choice) until the occupancy query says that all units' clusters are resident together.
+// Sizes the score grid from the host-side bound of the sequence lengths: the CTAs per unit (cluster size) and the
+// blocks per CTA.  Wanted: as many CTAs as the device holds at once (two per SM), so that every SM streams, but all
+// of them resident together - a cluster's CTAs sit in one GPC, so the device may hold fewer clusters of a size than
+// its CTA slots suggest, and a launch whose clusters do not all fit runs in two waves and takes twice as long.  The
+// cluster size need not be a power of two (32 units x 9 CTAs fill 148 SMs where 32 x 8 leave 40 of them half empty).
+// Candidates go from the largest that fits the slots down to the smallest the block count allows; the first whose
+// clusters the occupancy query reports as all resident is taken.
 // `fused`: the plan is for the fused decode kernel (score + attend in one launch), whose occupancy is asked for.
 // Returns true with p->cs / chunk set if a cluster kernel can serve the launch.
 static bool plan_score_clusters(spla_cache* c, Params* p, int64_t blocks, bool fused) {
   const int units = p->batch * p->Hkv;
   const int wi = fused ? 1 : 0;
-  // CTAs per SM: two, unless the attend phase's K/V ring (blocks of 128 tokens at d = 128) takes more than half an SM
-  int per_sm = 2;
-  if (fused && attend_mma_smem_bytes(p->B, p->d, 1) + 4096 > (size_t)113 * 1024) per_sm = 1;
-  const long long slots = (long long)per_sm * c->sm_count;
-  int best_cs = 0, best_chunk = 0;
-  for (int cap = 16; cap >= 1; cap /= 2) {
-    int cs = 0, chunk = 0;
-    if (!plan_score_cluster(units, blocks, p->NW, p->G, p->d, per_sm * c->sm_count / 2, cap, 8, &cs, &chunk)) break;
-    if (best_cs && cs >= best_cs) break;                   // the block count needs at least this size: no choice left
-    best_cs = cs;
-    best_chunk = chunk;
-    if (cs == 1 || (long long)units * cs > slots) break;   // several waves by necessity: nothing to gain
-    if (c->score_occ_cs[wi] != cs || c->score_occ_chunk[wi] != chunk) {
+  const long long slots = 2LL * c->sm_count;
+  int cs_lo = 1;                                            // keep the local ranking short: at most 576 blocks per CTA
+  while (cs_lo < 16 && blocks > 576LL * cs_lo) ++cs_lo;
+  while (cs_lo < 16 && !score_cluster_chunk(blocks, cs_lo, p->NW, p->G, p->d)) ++cs_lo;
+  if (!score_cluster_chunk(blocks, cs_lo, p->NW, p->G, p->d)) return false;
+  int cs_hi = (int)(slots / units);
+  if (cs_hi > 16) cs_hi = 16;
+  if (cs_hi < cs_lo) cs_hi = cs_lo;                         // several waves by necessity
+  int pick = cs_lo;
+  for (int cs = cs_hi; cs >= cs_lo; --cs) {
+    const int chunk = score_cluster_chunk(blocks, cs, p->NW, p->G, p->d);
+    if (!chunk) continue;
+    if (c->plan_override == 2 && (cs & (cs - 1)) && cs > cs_lo) continue;   // (development switch: powers of two only)
+    if (cs == 1 || (long long)units * cs > slots) { pick = cs; break; }   // nothing to ask
+    if (c->score_occ_chunk[wi][cs] != chunk) {
       Params probe = *p;
       probe.cs = cs;
       probe.chunk = chunk;
       probe.swarps = 8;
-      c->score_occ_n[wi] = fused ? decode_fused_max_clusters(probe) : score_cluster_max_clusters(probe);
-      c->score_occ_cs[wi] = cs;
-      c->score_occ_chunk[wi] = chunk;
+      c->score_occ_n[wi][cs] = fused ? decode_fused_max_clusters(probe) : score_cluster_max_clusters(probe);
+      c->score_occ_chunk[wi][cs] = chunk;
     }
-    const int occ = c->score_occ_n[wi];
-    if (occ < 0 || units <= occ) break;                    // unknown, or all resident at once
+    const int occ = c->score_occ_n[wi][cs];
+    if (units <= occ || (occ < 0 && (cs & (cs - 1)) == 0)) { pick = cs; break; }   // all resident (or unknown, for the portable sizes)
   }
-  if (!best_cs) return false;
-  p->cs = best_cs;
-  p->chunk = best_chunk;
-  p->n_chunks_cap = best_cs;
+  p->cs = pick;
+  if (getenv("SPLA_PLAN_PRINT")) {   // TEMPORARY
+    fprintf(stderr, "plan fused=%d units=%d blocks=%lld cs_lo=%d cs_hi=%d pick=%d occ:", (int)fused, units, (long long)blocks, cs_lo, cs_hi, pick);
+    for (int cs = 1; cs <= 16; ++cs) fprintf(stderr, " %d", c->score_occ_chunk[wi][cs] ? c->score_occ_n[wi][cs] : -9);
+    fprintf(stderr, "\n");
+  }
+  p->chunk = score_cluster_chunk(blocks, pick, p->NW, p->G, p->d);
+  p->n_chunks_cap = pick;
   p->swarps = 8;
   return true;
 }
@@ -343,10 +351,15 @@ static void plan_attend(spla_cache* c, Params* p) {
 }
 
 // Steps a1-a5 for every unit: the fused kernel where it applies, else score + select and attend + merge as two launches.
+// pending > 0: the call directly follows, in the stream, this step's append of at most that many tokens per sequence;
+// the score phase then streams the statistics of the blocks that were complete before it while it still runs.
+// (Starting that stream early in a plain spla_decode as well, before the wait for whatever kernel precedes, with the
+// query read after the wait, was measured and is not done: decode at 128K 39.6 against 38.8 us.)
 static int launch_decode(spla_cache* c, const void* q, const float* rms_weight, float* out, int32_t* sel_idx,
                          float* dbg_o_sparse, float* dbg_o_rla, int pending, cudaStream_t s, const char* where) {
   Params p = c->p;
   const int qb = c->cfg.q_dtype == SPLA_BF16;
+  if (c->plan_override == 3) pending = 0;       // (development switch)
   cudaError_t e;
   if (fused_eligible(c)) {
     // (a launch of several waves keeps the two-kernel form: measured faster there, the phases of different waves
@@ -384,10 +397,10 @@ extern "C" int spla_append_decode(spla_cache_t* c, const void* k_new, const void
   if (!aligned(q, 16) || !aligned(out, 16)) return SPLA_ERR_INVALID_ARG;
   const int rc = spla_append_tokens(c, k_new, v_new, n_new, max_new, stream);
   if (rc != SPLA_OK) return rc;
-  // only the fused decode-step append kernel opens the dependent launch early enough for this to matter
-  const int pending = (max_new <= 32) ? max_new : 0;
-  return launch_decode(c, q, rms_weight, out, sel_idx, dbg_o_sparse, dbg_o_rla, pending, (cudaStream_t)stream,
-                       "spla_append_decode");
+  // only the fused decode-step append kernel (at most 32 tokens) opens the dependent launch early enough for the
+  // early stream to matter
+  return launch_decode(c, q, rms_weight, out, sel_idx, dbg_o_sparse, dbg_o_rla, max_new <= 32 ? max_new : 0,
+                       (cudaStream_t)stream, "spla_append_decode");
 }
 
 extern "C" int spla_select(spla_cache_t* c, const void* q, int32_t* sel_idx, void* stream) {

@@ -77,8 +77,7 @@ int device_sm_count();   // multiprocessors of the current device (148 if the qu
 int score_chunk_for(long long units, long long max_seq_blocks, int sm_count);
 cudaError_t launch_score_select(const Params& p, const void* q, int q_is_bf16, int* sel_user, cudaStream_t stream);
 // score_cluster.cu (G <= 8, at most 16 x 1024 blocks per sequence)
-bool plan_score_cluster(int units, long long max_seq_blocks, int NW, int G, int d, int sm_count, int cs_cap, int warps,
-                        int* cs_out, int* chunk_out);
+int score_cluster_chunk(long long max_seq_blocks, int cs, int NW, int G, int d);   // blocks per CTA, 0: not servable
 // Clusters of the score kernel (p.cs CTAs each, p.chunk blocks per CTA) the device holds at once; -1 if unknown.
 int score_cluster_max_clusters(const Params& p);
 cudaError_t launch_score_cluster(const Params& p, const void* q, int q_is_bf16, int* sel_user, int pending_new,

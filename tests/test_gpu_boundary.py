@@ -155,3 +155,31 @@ def test_near_complete_selection_keeps_the_strict_tolerance():
                 parity.compare_unit(w, res, out[b], osp[b], orla[b], sel[b, h], h, n_sink=1, n_local=1, rerun=run)
                 worst = max(worst, np.linalg.norm(res["o_bar"]) / max(np.linalg.norm(res["o_rla"]), 1e-30))
     assert worst > 3.0                                        # the cases do cancel
+
+
+@pytest.mark.parametrize("flags,window", [(0, None), (binding.SPLA_STATS_BF16, None), (binding.SPLA_STATS_BF16, (32, 16)),
+                                          (0, (32, 16)), (binding.SPLA_GENERAL_KERNELS, None)])
+def test_what_lies_beyond_the_end_of_a_sequence_never_reaches_the_results(flags, window):
+    """The caches are caller memory and are never cleared: past the last token of a sequence they hold whatever was
+    there before.  Here that is NaN everywhere (a large NaN-filled tensor is freed just before the caches are
+    allocated, so that they reuse its memory).  Steps across a block boundary - the new block then holds one valid
+    token and 63 rows of NaN - must give finite outputs, the same from the one-call step as from separate calls."""
+    junk = torch.full((3 << 30,), float("nan"), dtype=torch.bfloat16, device=DEV)
+    del junk
+    torch.cuda.synchronize()
+    w = synth.BY_NAME["long_128k"].scaled(batch=2, context=64 * 40 + 60, n_steps=8)
+    a, K, V, lens = runner.build_cache(w, DEV, flags=flags, window=window)
+    b, _, _, _ = runner.build_cache(w, DEV, flags=flags, window=window, prefill=(K, V, lens))
+    assert torch.isnan(a.bufs.k_cache.float()).any()          # the poison is where the test wants it
+    gamma = synth.gamma(w).to(DEV)
+    for step in range(w.n_steps):
+        k1, v1 = synth.step_kv(w, step, DEV)
+        q = synth.step_queries(w, step, DEV)
+        sa, sb = a.new_sel_buffer(), b.new_sel_buffer()
+        a.append_tokens(k1, v1)
+        oa = a.decode(q, gamma, sel_idx=sa)
+        ob = b.append_decode(k1, v1, q, gamma, sel_idx=sb)
+        torch.cuda.synchronize()
+        assert a.sync_status() == 0 and b.sync_status() == 0
+        assert torch.isfinite(oa).all() and torch.isfinite(ob).all(), f"step {step}"
+        assert torch.equal(sa, sb) and torch.equal(oa, ob), f"step {step}"

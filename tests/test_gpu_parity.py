@@ -425,7 +425,10 @@ def test_select_then_decode_selected_equals_decode():
     out_b = cache.decode_selected(q, gamma, sel_b)
     torch.cuda.synchronize()
     assert torch.equal(sel_a, sel_b)
-    np.testing.assert_allclose(out_b.cpu().numpy(), out_a.cpu().numpy(), rtol=1e-6, atol=1e-6)
+    # the two routes may split a unit's blocks over a different number of CTAs: the softmax weights are then rounded to
+    # bf16 against other running maxima, so the outputs agree to bf16 accuracy (1e-4 .. 1e-3), not to fp32 accuracy
+    a, b = out_a.cpu().numpy(), out_b.cpu().numpy()
+    assert parity.rel_l2(b, a) < 1e-3 and parity.max_abs(b, a) < 2e-3
 
 
 def test_scores_are_normalised_and_match_oracle():
