@@ -39,8 +39,7 @@ def needs_build() -> bool:
     return any(os.path.getmtime(f) > t for f in _deps())
 
 
-def build(force: bool = False, verbose: bool = False, trace: bool = False) -> str:
-    """trace=True compiles the development time-line marks in (-DSPLA_TRACE); never used by tests or the bench."""
+def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB_PATH
     os.makedirs(OBJ_DIR, exist_ok=True)
@@ -48,7 +47,7 @@ def build(force: bool = False, verbose: bool = False, trace: bool = False) -> st
 
     def compile_one(src: str) -> tuple[str, str]:
         obj = os.path.join(OBJ_DIR, src.replace(".cu", ".o"))
-        cmd = [nvcc, *ARCH_FLAGS, *NVCC_FLAGS, *(["-DSPLA_TRACE"] if trace else []), "-c", os.path.join(CSRC, src), "-o", obj]
+        cmd = [nvcc, *ARCH_FLAGS, *NVCC_FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
         r = subprocess.run(cmd, capture_output=True, text=True)
         if r.returncode != 0:
             raise RuntimeError(f"nvcc failed on {src}:\n{r.stdout}\n{r.stderr}")
@@ -70,6 +69,5 @@ def build(force: bool = False, verbose: bool = False, trace: bool = False) -> st
 
 
 if __name__ == "__main__":
-    path = build(force="--force" in sys.argv or "--trace" in sys.argv, verbose="--verbose" in sys.argv,
-                 trace="--trace" in sys.argv)
+    path = build(force="--force" in sys.argv, verbose="--verbose" in sys.argv)
     print(path)

@@ -266,7 +266,6 @@ __global__ void __launch_bounds__(kFusedThreads, 4) append_fused_kernel(const Pa
 
   pdl_wait();                                      // the preceding decode still reads the cache and the lengths
   pdl_launch_dependents();
-  SPLA_MARK(p, u, blockIdx.x, 0);
   const int L = p.seq_lens[b];
   const int n = tokens_to_add(p, n_new, max_new, b, L);
   const T* kn = k_new + (size_t)u * max_new * D;
@@ -388,7 +387,6 @@ __global__ void __launch_bounds__(kFusedThreads, 4) append_fused_kernel(const Pa
     }
   }
 
-  SPLA_MARK(p, u, blockIdx.x, 2);
 }
 
 template <typename T, int D>

@@ -12,18 +12,9 @@ __global__ void __launch_bounds__(NG * kAttendThreads, NG == 1 ? 2 : 1)
   attend_mma_body<D, PACK, NG, false>(p, map_k, map_v, q, rms_weight, out, dbg_sparse, dbg_rla, smem_raw);
 }
 
-// Ring positions of the two-group shape: as many as fit beside the static shared memory, an even number.
-int attend_mma_slots(int B, int D) {
-  const size_t slot = (2 * (size_t)B * D * 2 + (size_t)B * 4 + 1023) / 1024 * 1024;
-  int n = (int)((size_t)(222 * 1024) / slot);
-  if (n > kMaxSlots) n = kMaxSlots;
-  return n & ~1;
-}
-
-// `groups` = 1: two ring positions; 2: attend_mma_slots() positions.
+// Dynamic shared memory of the kernel: the two-slot tile ring, reused for the cross-warp fold.
 size_t attend_mma_smem_bytes(int B, int D, int groups) {
-  const int slots = groups == 1 ? 2 : attend_mma_slots(B, D);
-  const size_t ring = (size_t)slots * ((2 * (size_t)B * D * 2 + (size_t)B * 4 + 1023) / 1024 * 1024);
+  const size_t ring = (size_t)(2 * groups) * ((2 * (size_t)B * D * 2 + (size_t)B * 4 + 1023) / 1024 * 1024);
   const size_t fold = (size_t)(groups * (kAttendThreads / 32) * (16 * (D + kPad) + 16) + 2 * 8 * D + 16) * sizeof(float);
   return ring > fold ? ring : fold;
 }
@@ -54,7 +45,7 @@ static cudaError_t launch_mma(const Params& p, const AttendMaps& maps, const voi
                   : launch_shape<D, false, 1>(p, maps, q, w, out, ds, dr, stream, occ);
 }
 
-// Clusters of p.acs CTAs (of p.agroups warp groups) of the attend kernel the device holds at once; -1 if the query fails.
+// Clusters of p.acs CTAs of the attend kernel the device holds at once; -1 if the query fails.
 int attend_mma_max_clusters(const Params& p) {
   int n = -1;
   AttendMaps none;

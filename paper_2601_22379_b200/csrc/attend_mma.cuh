@@ -38,7 +38,7 @@ namespace spla {
 
 namespace {
 
-constexpr int kMaxSlots = 12;      // ring positions at most (the launch says how many are used)
+constexpr int kMaxSlots = 4;       // ring positions at most (two per warp group)
 
 // Tiled TMA load of one box (never multicast): coordinates {x = element column, y = row}.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
@@ -103,7 +103,7 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
   const int g = lane >> 2, t = lane & 3;
   const int G = p.G, B = p.B;
   const bool rla_on = !(p.flags & 4u);
-  const int ns = NG == 1 ? 2 : p.aslots;        // ring positions in use (a multiple of NG: a group refills what it frees)
+  constexpr int ns = 2 * NG;                    // ring positions in use (a multiple of NG: a group refills what it frees)
   auto cta_sync = [&]() {                      // barrier over the threads that run this body
     if constexpr (FUSED) asm volatile("bar.sync 1, %0;" ::"n"(NG * kAttendThreads) : "memory");
     else __syncthreads();
@@ -113,7 +113,6 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
     else asm volatile("bar.sync %0, %1;" ::"r"(2 + gi), "r"(kAttendThreads) : "memory");
   };
 
-  SPLA_MARK(p, u, 32 + rank, 1);
   if constexpr (!FUSED) pdl_launch_dependents();
   // ---- query fragments first: they depend on nothing the preceding kernel writes, so under programmatic
   // dependent launch this part overlaps that kernel's tail.  Rows = heads of the group, held in registers.
@@ -201,7 +200,6 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
     }
   }
   cta_sync();                              // selection list and barrier initialisation visible to the CTA
-  SPLA_MARK(p, u, 32 + rank, 0);
 
   const int nb = nsel > rank ? (nsel - rank + CS - 1) / CS : 0;     // my blocks: j = rank + i * CS
   const int tile_bytes = B * D * 2;
@@ -247,7 +245,6 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
       dead = true;
       if (lane == 0) atomicExch(&err_s, 1);
     }
-    if (i == 0) SPLA_MARK(p, u, 32 + rank, 2);
     unsigned char* sb = smem_raw + (size_t)slot * slot_bytes;
     const uint32_t ks = smem_u32(sb);
     const uint32_t vs = ks + tile_bytes;
@@ -381,7 +378,6 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
   }
   if (tid == 0 && err_s) atomicExch(p.status, kStatusTimeout);
 
-  SPLA_MARK(p, u, 32 + rank, 3);
   // ---- fold the four warps together ------------------------------------------------------------------------
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
@@ -431,10 +427,8 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
     mine_ml[tid * 2] = Mg;
     mine_ml[tid * 2 + 1] = Lg;
   }
-  SPLA_MARK(p, u, 32 + rank, 4);
 
   cluster_sync_all();                                // ---- every CTA's partial result is in its shared memory
-  SPLA_MARK(p, u, 32 + rank, 5);
 
   // ---- merge: CTA r of the cluster owns heads r, r + CS, ...; one thread per output column ---------------
   const int nblk_u = (L + B - 1) / B;
@@ -479,7 +473,6 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
       if (dbg_rla) dbg_rla[oidx] = r_;
     }
   }
-  SPLA_MARK(p, u, 32 + rank, 6);
   cluster_sync_all();                                // ---- nobody leaves while a sibling may still read its memory
 }
 

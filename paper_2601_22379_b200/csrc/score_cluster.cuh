@@ -164,7 +164,6 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
     else { for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kCsConsumers); } }
     err_s = 0;
   }
-  SPLA_MARK(p, blockIdx.y, 30, 0);
   if (!EARLY) {
     pdl_wait();                                 // everything the preceding kernels wrote (statistics, lengths, q) is visible
     pdl_launch_dependents();                    // only now may the next kernel begin its prologue: it reads q before its own wait
@@ -290,7 +289,6 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
     if constexpr (MMA) { for (int r = 0; r < min(SM::kSlots, n_slots); ++r) issue_slot(r); }
     else { for (int r = 0; r < min(kStages, n_rounds); ++r) issue(r); }
   }
-  SPLA_MARK(p, u, rank, 0);
 #pragma unroll
   for (int g = 0; g < GP && !MMA; ++g) {
 #pragma unroll
@@ -302,7 +300,6 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
   if (WIN)                                      // pooled slots start below every key
     for (int x = tid; x < G * chunk; x += kCsThreads) reinterpret_cast<uint32_t*>(ell_s)[x] = 0u;
   __syncthreads();                              // the barrier initialisation is visible to every consumer
-  SPLA_MARK(p, u, rank, 1);
 
   {
     // After the group reduction the first W/2 lanes of a group hold the mean dots and the others the variance
@@ -504,7 +501,6 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
         }
       }
     }
-    SPLA_MARK(p, u, rank, 2);
     if (WIN) {
       // the pooled keys back to floats, and this CTA's (max, sum exp) per head from them; lane 0 of every warp
       // then holds the warp's pair
@@ -566,7 +562,6 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
   cluster_sync_all();                                                   // ---- sync 1: partial normalisers visible
 
   // ------------------------------------------------------------------ phase B -------------------------------
-  SPLA_MARK(p, u, rank, 3);
   // Log-sum-exp of every head over the whole cluster, by each warp on its own (no block barrier): lane p
   // fetches the (max, sum) pair of CTA p / GP and head p % GP over distributed shared memory, then the lanes
   // of one head are folded with shuffles.
@@ -634,17 +629,14 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
     }
   }
   __syncthreads();
-  SPLA_MARK(p, u, rank, 4);
 
   // this CTA's best min(k_eff, n_my) blocks go to the leader's candidate table
   {
     const int cnt = select_topk(keys, nb_my, k_eff, [&](int li) { return blk_begin + li; }, push, scratch);
     if (tid == 0) st_dsmem_u32(map_to_rank(smem_u32(smem_raw + SM::kCandCnt), 0u) + (uint32_t)rank * 4, (uint32_t)cnt);
   }
-  SPLA_MARK(p, u, rank, 5);
 
   cluster_sync_all();                                                   // ---- sync 2: candidates are in the leader
-  SPLA_MARK(p, u, rank, 6);
   const bool rla = !(p.flags & 4u);
   if (rank != 0) {
     // The siblings are done with the selection; while the leader finishes it they compute the part of the
@@ -654,7 +646,6 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
         __syncthreads();                       // (the slices of one CTA reuse the same shared memory)
         state_role<D, GP, kCsThreads>(p, u, s, q_raw, q_is_bf16, reinterpret_cast<float*>(smem_raw));
       }
-    SPLA_MARK(p, u, rank, 7);
   } else {
   // ------------------------------------------------------------------ phase C (leader) ----------------------
   const uint32_t* cand_key = reinterpret_cast<const uint32_t*>(smem_raw + SM::kCandKey);
@@ -717,7 +708,6 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
   const int total = *n_surv;
   auto keep = [&](int slot, uint32_t, int idx) { sel_tmp[slot] = idx; };
   auto flat_of = [&](int c) { return flat_idx[c]; };
-  SPLA_MARK(p, u, 31, 0);
   if (total <= kCsThreads) {
     // few survivors (the usual case): every thread ranks its candidates against all others by counting, reading the
     // table with broadcast 128-bit loads; no shared-memory atomics, one barrier
@@ -740,7 +730,6 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
     topk_prepare(flat_key, total, flat_of, keep, scratch);
     select_topk(flat_key, total, k_eff, flat_of, keep, scratch);
   }
-  SPLA_MARK(p, u, 31, 2);
 
   int* sel_u = p.sel + (size_t)u * p.top_k;
   int* sel_o = sel_user ? sel_user + (size_t)u * p.top_k : nullptr;
@@ -767,7 +756,6 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
         st_dsmem_u32(map_to_rank(smem_u32(sel_share + kMaxTopK + 1), (uint32_t)r), (uint32_t)L);
       }
   }
-  SPLA_MARK(p, u, rank, 7);
   if (rla && CS == 1)
     for (int s = 0; s < kStateSplits; ++s) {
       __syncthreads();

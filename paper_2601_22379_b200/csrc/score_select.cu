@@ -88,7 +88,6 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
   const int chunk = p.chunk;                        // records per CTA
   const int n_chunks = max(1, (nrec + chunk - 1) / chunk);
   if (c >= n_chunks) return;
-  SPLA_MARK(p, u, c, 0);
 
   // q_hat slices for the mean dot and 1/2 q_hat^2 for the variance dot, in registers.
   float qm[GP][VEC], qv[GP][VEC];
@@ -194,7 +193,6 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
     }
   };
 
-  SPLA_MARK(p, u, c, 1);
   load_round(0, 0);
 #pragma unroll 1
   for (int round = 0; round < rounds; round += 2) {
@@ -206,7 +204,6 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
     }
   }
 
-  SPLA_MARK(p, u, c, 2);
   // per-chunk (max, sum exp) per head: fold the FB finalising lanes, then the warps
 #pragma unroll
   for (int o = 1; o < FB; o <<= 1) {
@@ -237,7 +234,6 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
     __threadfence();
   }
   __syncthreads();
-  SPLA_MARK(p, u, c, 3);
   if (!is_last_s) return;
 
   // ------------------------------------------------------------------ selection (one CTA per unit) ----
@@ -313,7 +309,6 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
   }
   __syncthreads();
 
-  SPLA_MARK(p, u, c, 4);
   const int k_eff = min(p.top_k, nblk);
   float* scores_u = p.scores + (size_t)vu * p.max_blocks;
   float lse_r[GP];
@@ -337,7 +332,6 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
   }
   __syncthreads();
 
-  SPLA_MARK(p, u, c, 5);
   // radix select: the k_eff-th largest key, 8 bits per pass.  A warp whose active lanes all hold the same
   // digit (the rule in the exponent pass) adds its count once; otherwise each lane adds for itself.
   uint32_t prefix = 0, mask = 0;
@@ -393,7 +387,6 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
   }
   const uint32_t T = prefix;   // threshold key; kk = how many keys equal to T are taken (lowest indices first)
 
-  SPLA_MARK(p, u, c, 6);
   // index-ordered compaction
   const int per = (nblk + kScoreThreads - 1) / kScoreThreads;
   const int i0 = tid * per, i1 = min(nblk, i0 + per);
@@ -433,7 +426,6 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
     if (sel_o) sel_o[t] = -1;
   }
   if (tid == 0) p.n_sel[vu] = k_eff;
-  SPLA_MARK(p, u, c, 7);
 }
 
 template <int D, int GP>

@@ -20,7 +20,6 @@ struct spla_cache {
   // clusters the device holds at once, as last queried: score kernel for (cs, chunk), attend kernel per log2(acs)
   int score_occ_chunk[2][17] = {}, score_occ_n[2][17] = {};   // resident clusters as last queried, by [kernel: score / fused decode][cluster size]
   int attend_occ[5] = {-2, -2, -2, -2, -2};   // by log2 of the cluster size
-  int plan_override = 0;   // 0: planner's choice; 1: never the fused decode kernel (development switch)
   int sm_count;
   AttendMaps maps;
   AttendMaps state_maps;   // the same caches in boxes of 64 tokens, for the tensor-core state kernel
@@ -169,7 +168,6 @@ extern "C" int spla_init_cache(const spla_config_t* config, const spla_buffers_t
   c->cfg = *config;
   c->buf = *b;
   c->sm_count = device_sm_count();
-  c->plan_override = getenv("SPLA_PLAN") ? atoi(getenv("SPLA_PLAN")) : 0;   // TEMPORARY development switch
   if (c->cfg.sm_scale == 0.f) c->cfg.sm_scale = 1.0f / sqrtf((float)config->head_dim);
   if (c->cfg.phi_scale == 0.f) c->cfg.phi_scale = 1.0f;
   if (c->cfg.rms_eps == 0.f) c->cfg.rms_eps = 1e-6f;
@@ -198,9 +196,6 @@ extern "C" int spla_init_cache(const spla_config_t* config, const spla_buffers_t
   p.state_part = (float*)(ws + w.state_part); p.state_ticket = (int*)(ws + w.state_ticket);
   p.status = (int*)(ws + w.status);
   p.max_chunks = w.max_chunks;
-#ifdef SPLA_TRACE
-  p.trace = getenv("SPLA_TRACE_PTR") ? (unsigned long long*)strtoull(getenv("SPLA_TRACE_PTR"), nullptr, 0) : nullptr;
-#endif
   p.acs = 0;
 
   c->maps.valid = false;
@@ -273,13 +268,11 @@ static bool plan_score_clusters(spla_cache* c, Params* p, int64_t blocks, bool f
   for (int cs = cs_hi; cs >= cs_lo; --cs) {
     const int chunk = score_cluster_chunk(blocks, cs, p->NW, p->G, p->d);
     if (!chunk) continue;
-    if (c->plan_override == 2 && (cs & (cs - 1)) && cs > cs_lo) continue;   // (development switch: powers of two only)
     if (cs == 1 || (long long)units * cs > slots) { pick = cs; break; }   // nothing to ask
     if (c->score_occ_chunk[wi][cs] != chunk) {
       Params probe = *p;
       probe.cs = cs;
       probe.chunk = chunk;
-      probe.swarps = 8;
       c->score_occ_n[wi][cs] = fused ? decode_fused_max_clusters(probe) : score_cluster_max_clusters(probe);
       c->score_occ_chunk[wi][cs] = chunk;
     }
@@ -287,14 +280,8 @@ static bool plan_score_clusters(spla_cache* c, Params* p, int64_t blocks, bool f
     if (units <= occ || (occ < 0 && (cs & (cs - 1)) == 0)) { pick = cs; break; }   // all resident (or unknown, for the portable sizes)
   }
   p->cs = pick;
-  if (getenv("SPLA_PLAN_PRINT")) {   // TEMPORARY
-    fprintf(stderr, "plan fused=%d units=%d blocks=%lld cs_lo=%d cs_hi=%d pick=%d occ:", (int)fused, units, (long long)blocks, cs_lo, cs_hi, pick);
-    for (int cs = 1; cs <= 16; ++cs) fprintf(stderr, " %d", c->score_occ_chunk[wi][cs] ? c->score_occ_n[wi][cs] : -9);
-    fprintf(stderr, "\n");
-  }
   p->chunk = score_cluster_chunk(blocks, pick, p->NW, p->G, p->d);
   p->n_chunks_cap = pick;
-  p->swarps = 8;
   return true;
 }
 
@@ -303,7 +290,6 @@ static void plan_score_grid(spla_cache* c, Params* p, bool fused = false) {
   int64_t blocks = (c->len_bound + c->cfg.block_size - 1) / c->cfg.block_size;
   if (blocks < 1) blocks = 1;
   p->cs = 0;
-  p->swarps = 8;
   if (!(c->cfg.flags & SPLA_GENERAL_KERNELS) && plan_score_clusters(c, p, blocks, fused)) return;
   p->cs = 0;
   p->chunk = score_chunk_for((long long)p->batch * p->Hkv, blocks * p->NW, c->sm_count);   // in records (windows)
@@ -313,7 +299,7 @@ static void plan_score_grid(spla_cache* c, Params* p, bool fused = false) {
 // The fused decode kernel serves bf16 caches and queries with groups of up to 8 heads (what the tensor-core attend
 // phase is built for) whenever the cluster score plan exists.
 static bool fused_eligible(const spla_cache* c) {
-  return c->plan_override != 1 && !(c->cfg.flags & SPLA_GENERAL_KERNELS) && c->p.kv_bf16 && c->cfg.q_dtype == SPLA_BF16 &&
+  return !(c->cfg.flags & SPLA_GENERAL_KERNELS) && c->p.kv_bf16 && c->cfg.q_dtype == SPLA_BF16 &&
          c->p.G <= 8 && c->maps.valid && attend_mma_smem_bytes(c->p.B, c->p.d, 1) + 4096 <= (size_t)113 * 1024;
 }
 
@@ -326,7 +312,7 @@ static cudaError_t launch_score(const Params& p, const void* q, int qb, int* sel
 // most 16 and at most top_k) for which all CTAs are resident at once; each CTA of a cluster then walks top_k / size
 // selected blocks.
 static void plan_attend(spla_cache* c, Params* p) {
-  p->acs = 0; p->agroups = 1; p->aslots = 2;
+  p->acs = 0;
   if (c->cfg.flags & SPLA_GENERAL_KERNELS) return;
   const long long U = (long long)c->p.batch * c->p.Hkv;
   const size_t smem = attend_mma_smem_bytes(c->p.B, c->p.d, 1) + 2048;
@@ -342,7 +328,7 @@ static void plan_attend(spla_cache* c, Params* p) {
     while ((1 << lg) < cs) ++lg;
     if (c->attend_occ[lg] == -2) {
       Params probe = c->p;
-      probe.acs = cs; probe.agroups = 1; probe.aslots = 2;
+      probe.acs = cs;
       c->attend_occ[lg] = attend_mma_max_clusters(probe);
     }
     if (c->attend_occ[lg] < 0 || U <= c->attend_occ[lg]) break;
@@ -359,7 +345,6 @@ static int launch_decode(spla_cache* c, const void* q, const float* rms_weight, 
                          float* dbg_o_sparse, float* dbg_o_rla, int pending, cudaStream_t s, const char* where) {
   Params p = c->p;
   const int qb = c->cfg.q_dtype == SPLA_BF16;
-  if (c->plan_override == 3) pending = 0;       // (development switch)
   cudaError_t e;
   if (fused_eligible(c)) {
     // (a launch of several waves keeps the two-kernel form: measured faster there, the phases of different waves

@@ -38,9 +38,6 @@ struct Params {
   int chunk;                            // block records per score CTA
   int cs;                               // score kernel, cluster edition: CTAs per unit (0 = general kernel)
   int acs;                              // tensor-core attend kernel: CTAs (cluster size) per unit
-  int agroups;                          //   warp groups per CTA (1: two CTAs per SM, two-slot ring; 2: one CTA per SM, deep ring)
-  int aslots;                           //   ring positions of the two-group shape
-  int swarps;                           // cluster score kernel: warps per CTA (8: two CTAs per SM; 16: one CTA per SM)
   // caller buffers
   void* k_cache;
   void* v_cache;
@@ -73,9 +70,6 @@ struct Params {
   const float* vobar;                   // [U][vTtot][G][d] o_bar = phi(q_t) S_bar_t of every position
   int wait_limit;                       // iterations a bounded barrier wait polls before it gives up (0: kWaitLimitDefault)
   int dbg_tx_extra;                     // test hook: bytes added to what the decode kernels' copy barriers expect (0 in use)
-#ifdef SPLA_TRACE
-  unsigned long long* trace;  // development builds only: [unit][64 CTAs][8 marks] of %globaltimer values
-#endif
 };
 
 __device__ __forceinline__ float to_float(float x) { return x; }
@@ -262,21 +256,6 @@ __device__ __forceinline__ int cover_len(const Params& p, int L, long long cover
   }
   return L;
 }
-
-// Development aid, compiled in only with -DSPLA_TRACE (python -m paper_2601_22379_b200.build --trace): thread 0 of
-// a CTA stores %globaltimer at numbered marks so that the phases of a kernel can be laid out on a time line.
-#ifdef SPLA_TRACE
-#define SPLA_MARK(p, unit, cta, k)                                                        \
-  do {                                                                                    \
-    if ((p).trace && threadIdx.x == 0 && (cta) < 64) {                                    \
-      unsigned long long t_;                                                              \
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                              \
-      (p).trace[((size_t)(unit) * 64 + (cta)) * 8 + (k)] = t_;                            \
-    }                                                                                     \
-  } while (0)
-#else
-#define SPLA_MARK(p, unit, cta, k) do { } while (0)
-#endif
 
 // Programmatic dependent launch: wait for the preceding grid's memory, allow the next grid to start.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

@@ -97,8 +97,7 @@ cudaError_t launch_attend_merge(const Params& p, const AttendMaps* maps, const v
                                 float* dbg_o_rla, cudaStream_t stream);
 // attend_mma.cu (bf16 K/V and q, G <= 8)
 size_t attend_mma_smem_bytes(int B, int D, int groups);
-int attend_mma_slots(int B, int D);             // ring positions of the two-group shape
-int attend_mma_max_clusters(const Params& p);   // clusters of p.acs CTAs (p.agroups groups each) resident at once; -1 if unknown
+int attend_mma_max_clusters(const Params& p);   // clusters of p.acs CTAs resident at once; -1 if unknown
 cudaError_t launch_attend_mma(const Params& p, const AttendMaps& maps, const void* q, const float* rms_weight, float* out,
                               float* dbg_o_sparse, float* dbg_o_rla, cudaStream_t stream);
 // prefill.cu: prefix statistics of every chunk position's own block and the chunk scan (o_bar per position; advances S_bar)

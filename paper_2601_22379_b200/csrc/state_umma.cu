@@ -102,18 +102,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t addr, float (&v)[32]) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-#ifdef SPLA_TRACE
-#define SU_MARK(i, k)                                                                       \
-  do {                                                                                      \
-    if (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && (i) < 32) {                        \
-      unsigned long long t_;                                                                \
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                \
-      p.trace[(size_t)(i) * 8 + (k)] = t_;                                                  \
-    }                                                                                       \
-  } while (0)
-#else
-#define SU_MARK(i, k) do { } while (0)
-#endif
 
 }  // namespace
 
@@ -170,7 +158,6 @@ __global__ void __launch_bounds__(kSuThreads, 1)
           if (i >= kSuStages && !mbar_wait(&empty[s], ((i / kSuStages) - 1) & 1)) { atomicExch(&abort_s, 1); break; }
           const uint32_t base = smem_u32(smem_raw + (size_t)s * kSuStageBytes);
           const int row = (int)(unit_tok0 + (size_t)L + (size_t)(t_begin + i) * kSuTile);
-          SU_MARK(i, 0);
           mbar_expect_tx(&full[s], 2 * kSuTileBytes);
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
@@ -191,7 +178,6 @@ __global__ void __launch_bounds__(kSuThreads, 1)
           const bool first = i % kSuGroup == 0, last = i % kSuGroup == kSuGroup - 1 || i == my_tiles - 1;
           if (first && g >= 2 && !mbar_wait(&acc_empty[ab], ((g >> 1) - 1) & 1)) { atomicExch(&abort_s, 1); break; }
           if (!mbar_wait(&ready[s], (i / kSuStages) & 1)) { atomicExch(&abort_s, 1); break; }
-          SU_MARK(i, 3);
           tc_fence_after();
           const uint32_t base = smem_u32(smem_raw + (size_t)s * kSuStageBytes);
 #pragma unroll
@@ -201,7 +187,6 @@ __global__ void __launch_bounds__(kSuThreads, 1)
               umma_bf16(tmem + ab * kSuD, umma_desc(base + part * kSuTileBytes + kk * 2048),
                         umma_desc(base + 2 * kSuTileBytes + kk * 2048), (!first || part > 0 || kk > 0) ? 1u : 0u);
           umma_commit(&empty[s]);                        // the stage may be refilled once these have read it
-          SU_MARK(i, 4);
           if (last) umma_commit(&acc_full[ab]);          // and the group's sum may be drained
         }
       }
@@ -262,7 +247,6 @@ __global__ void __launch_bounds__(kSuThreads, 1)
         }
         load_lse(i + 2);
         if (!mbar_wait(&full[s], (i / kSuStages) & 1)) { ok = false; break; }
-        if (tg == 0) SU_MARK(i, 1);
         unsigned char* st = smem_raw + (size_t)s * kSuStageBytes + tg * 16;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -291,10 +275,8 @@ __global__ void __launch_bounds__(kSuThreads, 1)
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the tensor core's reads
         __syncwarp();
         if (lane == 0) mbar_arrive1(&ready[s]);
-        if (tg == 0) SU_MARK(i, 2);
         // one accumulator group behind the issuer: by now those instructions have long completed
         while (ok && drained < i / kSuGroup) { drain(drained); ++drained; }
-        if (tg == 0) SU_MARK(i, 5);
         if (!ok) break;
       }
       while (ok && !*abort_flag && drained < n_groups) { drain(drained); ++drained; }
