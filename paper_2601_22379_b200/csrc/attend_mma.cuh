@@ -204,21 +204,25 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
   const int nb = nsel > rank ? (nsel - rank + CS - 1) / CS : 0;     // my blocks: j = rank + i * CS
   const int tile_bytes = B * D * 2;
   const int slot_bytes = (2 * tile_bytes + B * 4 + 1023) & ~1023;   // K tile, V tile, per-token lse; the swizzle needs 1 KB alignment
-  auto issue = [&](int i) {                                          // one thread
+  // The copies of tile i of this CTA (K and V in 64-column halves, the tokens' log-sum-exp): `part` < 0 issues all of
+  // them from one thread; otherwise the caller spreads the parts 0 .. kTileParts - 1 over lanes (part 0 also announces
+  // the bytes; the barrier's transaction count may run ahead of that announcement).
+  constexpr int kTileParts = 2 * NH + 1;
+  auto issue = [&](int i, int part = -1) {
     const int slot = i % ns;
     const int blk = min(max(sel_s[rank + i * CS], 0), p.max_blocks - 1);   // (a list entry can never address outside the cache)
     const uint32_t base = smem_u32(smem_raw + (size_t)slot * slot_bytes);
     const int row0 = (int)(((size_t)u * p.max_blocks + blk) * B);
-    mbar_expect_tx(&full[slot], (uint32_t)(2 * tile_bytes + B * 4 + p.dbg_tx_extra));
+    if (part <= 0) mbar_expect_tx(&full[slot], (uint32_t)(2 * tile_bytes + B * 4 + p.dbg_tx_extra));
 #pragma unroll
     for (int hh = 0; hh < NH; ++hh) {
-      tma_load_2d(base + hh * (B * 128), &map_k, hh * 64, row0, &full[slot]);
-      tma_load_2d(base + tile_bytes + hh * (B * 128), &map_v, hh * 64, row0, &full[slot]);
+      if (part < 0 || part == 2 * hh) tma_load_2d(base + hh * (B * 128), &map_k, hh * 64, row0, &full[slot]);
+      if (part < 0 || part == 2 * hh + 1) tma_load_2d(base + tile_bytes + hh * (B * 128), &map_v, hh * 64, row0, &full[slot]);
     }
-    bulk_g2s(smem_raw + (size_t)slot * slot_bytes + 2 * tile_bytes, p.tok_lse + (size_t)row0, (uint32_t)(B * 4), &full[slot]);
+    if (part < 0 || part == 2 * NH)
+      bulk_g2s(smem_raw + (size_t)slot * slot_bytes + 2 * tile_bytes, p.tok_lse + (size_t)row0, (uint32_t)(B * 4), &full[slot]);
   };
-  if (tid == 0)
-    for (int i = 0; i < min(ns, nb); ++i) issue(i);
+  if (tid < ns * kTileParts && tid / kTileParts < nb) issue(tid / kTileParts, tid % kTileParts);   // the first tiles, one copy per lane
   if constexpr (FUSED) {
     make_fragments();
     if constexpr (!PACK) cta_sync();          // fl_s is read by every warp
@@ -404,19 +408,21 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
     }
   }
   cta_sync();
-  for (int idx = tid; idx < 2 * 8 * D; idx += NTHR) {
-    const int br = idx / (8 * D), hd = (idx / D) % 8, col = idx % D;    // branch, head, column
-    float s = 0.f;
-    if (hd < G) {
-      const int rr = br * 8 + hd;
+  for (int idx = tid; idx < 2 * G * (D / 4); idx += NTHR) {             // four columns per thread and step
+    const int br = idx / (G * (D / 4)), hd = (idx / (D / 4)) % G, c4 = (idx % (D / 4)) * 4;   // branch, head, first column
+    const int rr = br * 8 + hd;
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-      for (int w = 0; w < NWARP; ++w) {
-        s += red_o[((size_t)w * 16 + rr) * (D + kPad) + col];
-        if (PACK && br == 1)                                              // the second and third parts of the coefficients
-          s += red_o[((size_t)w * 16 + rr + 4) * (D + kPad) + col] + red_o[((size_t)w * 16 + hd + 4) * (D + kPad) + col];
+    for (int w = 0; w < NWARP; ++w) {
+      const float4 a = *reinterpret_cast<const float4*>(red_o + ((size_t)w * 16 + rr) * (D + kPad) + c4);
+      s.x += a.x; s.y += a.y; s.z += a.z; s.w += a.w;
+      if (PACK && br == 1) {                                              // the second and third parts of the coefficients
+        const float4 b2 = *reinterpret_cast<const float4*>(red_o + ((size_t)w * 16 + rr + 4) * (D + kPad) + c4);
+        const float4 b3 = *reinterpret_cast<const float4*>(red_o + ((size_t)w * 16 + hd + 4) * (D + kPad) + c4);
+        s.x += b2.x + b3.x; s.y += b2.y + b3.y; s.z += b2.z + b3.z; s.w += b2.w + b3.w;
       }
     }
-    mine[idx] = s;
+    *reinterpret_cast<float4*>(mine + (size_t)rr * D + c4) = s;
   }
   if (tid < 8) {
     float Mg = red_m[tid], Lg = 0.f;
@@ -437,24 +443,42 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
     const int col = tid;
     float o_sp = 0.f, o_til = 0.f, o_bar = 0.f;
     if (nsel > 0) {
-      float Mx = -INFINITY;
-      for (int r = 0; r < CS; ++r) Mx = fmaxf(Mx, ld_dsmem_f32(map_to_rank(smem_u32(mine_ml + hd * 2), (uint32_t)r)));
-      float Ls = 0.f;
-      for (int r = 0; r < CS; ++r) {
-        const uint32_t rm = map_to_rank(smem_u32(mine_ml + hd * 2), (uint32_t)r);
-        const float w = ex2(ld_dsmem_f32(rm) - Mx);
-        Ls = fmaf(w, ld_dsmem_f32(rm + 4), Ls);
-        if (col < D) {
-          o_sp = fmaf(w, ld_dsmem_f32(map_to_rank(smem_u32(mine + hd * D + col), (uint32_t)r)), o_sp);
-          if (rla) o_til += ld_dsmem_f32(map_to_rank(smem_u32(mine + (8 + hd) * D + col), (uint32_t)r));
+      // every load is issued before the first is used: the o_bar partials from global memory, then the siblings'
+      // partial results over distributed shared memory (one round trip instead of one per sibling)
+      float ob[kStateSplits];
+#pragma unroll
+      for (int s = 0; s < kStateSplits; ++s)
+        ob[s] = (rla && col < D) ? __ldcg(p.obar_part + (((size_t)u * kStateSplits + s) * G + hd) * D + col) : 0.f;
+      constexpr int kMaxCS = 16;
+      float mr[kMaxCS], lr[kMaxCS], osp[kMaxCS], otl[kMaxCS];
+#pragma unroll
+      for (int r = 0; r < kMaxCS; ++r) {
+        mr[r] = -INFINITY; lr[r] = 0.f; osp[r] = 0.f; otl[r] = 0.f;
+        if (r < CS) {
+          const uint32_t rm = map_to_rank(smem_u32(mine_ml + hd * 2), (uint32_t)r);
+          mr[r] = ld_dsmem_f32(rm);
+          lr[r] = ld_dsmem_f32(rm + 4);
+          if (col < D) {
+            osp[r] = ld_dsmem_f32(map_to_rank(smem_u32(mine + hd * D + col), (uint32_t)r));
+            if (rla) otl[r] = ld_dsmem_f32(map_to_rank(smem_u32(mine + (8 + hd) * D + col), (uint32_t)r));
+          }
         }
       }
-      o_sp /= Ls;
-      if (rla && col < D) {
+      float Mx = -INFINITY;
 #pragma unroll
-        for (int s = 0; s < kStateSplits; ++s)
-          o_bar += __ldcg(p.obar_part + (((size_t)u * kStateSplits + s) * G + hd) * D + col);
-      }
+      for (int r = 0; r < kMaxCS; ++r) Mx = fmaxf(Mx, mr[r]);
+      float Ls = 0.f;
+#pragma unroll
+      for (int r = 0; r < kMaxCS; ++r)
+        if (r < CS) {
+          const float w = ex2(mr[r] - Mx);
+          Ls = fmaf(w, lr[r], Ls);
+          o_sp = fmaf(w, osp[r], o_sp);
+          o_til += otl[r];
+        }
+      o_sp /= Ls;
+#pragma unroll
+      for (int s = 0; s < kStateSplits; ++s) o_bar += ob[s];
     }
     const float r_ = (rla && col < D) ? o_bar - o_til : 0.f;
     float sq = warp_sum(r_ * r_);

@@ -3,12 +3,13 @@
 //
 //   phase 1  block score and top-k selection (Section 3.1, Eq. taylor-2nd; Section 2.2 grouped BlockScore;
 //            Section 2.1 Select) and o_bar = phi(q) S_bar (Section 3.2, Eq. rla-impl-1): the body of the cluster
-//            score kernel, all eight warps of every CTA;
-//   barrier  hardware cluster barrier: the leader's index set and the siblings' o_bar partials are visible to
-//            the whole cluster;
+//            score kernel, all eight warps of every CTA.  It ends with the selection of the unit (best block first) in
+//            every CTA's own shared memory (each CTA computes it from its copy of the unit's keys), so nothing is handed
+//            over and no cluster barrier stands between the phases;
 //   phase 2  exact attention over the selected blocks with the selected linear term from the same tiles
 //            (Section 2.2, Eq. gqa-sparse; Section 3.2, Eq. rla-impl-2), the subtraction and the RMSNorm merge
-//            (Eq. rla-impl-3, Section 3.3): the body of the tensor-core attend kernel, on the first four warps.
+//            (Eq. rla-impl-3, Section 3.3): the body of the tensor-core attend kernel, on the first four warps, which
+//            are also the ones that selected; the other four finish o_bar meanwhile and then only join the barriers.
 // The two phases want different register budgets (about 120 registers x 8 warps, then about 220 x 4 warps).  After
 // phase 1 the second warp group hands its registers back to the CTA's pool and the first takes them (setmaxnreg),
 // so both phases run at two CTAs per SM without spilling.  What the fusion removes: one kernel boundary per step
@@ -28,23 +29,24 @@ __global__ void __launch_bounds__(256, 2)
                         const __nv_bfloat16* __restrict__ q, const float* __restrict__ rms_weight, float* __restrict__ out,
                         float* __restrict__ dbg_sparse, float* __restrict__ dbg_rla, int* __restrict__ sel_user, int pending_new) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  __shared__ int sel_share[kMaxTopK + 2];   // the unit's selection, its size, the length: written in every CTA by the leader
+  __shared__ __align__(16) int sel_share[kMaxTopK + 2];   // the unit's selection, its size, the length: phase 1 leaves them here
   if (threadIdx.x == 0) {                   // the K/V tensor maps are needed late: have them fetched now
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
   }
   score_cluster_body<D, GP, WIN, EARLY, ST, 8>(p, q, 1, sel_user, pending_new, smem_raw, sel_share);
-  // Phase 2's tiles arrive through the asynchronous proxy (TMA) in shared memory that phase 1 has just read and written
-  // through the generic proxy (the statistics ring, the selection's work arrays, the o_bar scratch): every thread orders
-  // its accesses before them.
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  __threadfence();         // the o_bar partials went to global memory: performed device-wide before the barrier releases them
-  cluster_sync_all();      // the selection (every CTA's sel_share) and p.obar_part (siblings) are visible; phase 1's shared memory is dead
   if ((threadIdx.x >> 5) < 4) {
+    // Phase 2's tiles arrive through the asynchronous proxy (TMA) in shared memory that these warps have just read and
+    // written through the generic proxy (the key table, the selection's work arrays): each of them orders its accesses
+    // before the copies, then they meet.  (What all eight warps did there earlier was ordered before phase 1's last
+    // cluster barrier.)
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("bar.sync 1, 128;" ::: "memory");
     warpgroup_reg_inc<232>();
     attend_mma_body<D, (GP <= 4), 1, true>(p, map_k, map_v, q, rms_weight, out, dbg_sparse, dbg_rla, smem_raw, sel_share);
   } else {
     warpgroup_reg_dec<24>();
+    __threadfence();       // the o_bar partials went to global memory: performed device-wide before the barrier releases them
     cluster_sync_all();    // the two cluster barriers of phase 2 count every thread of the cluster
     cluster_sync_all();
   }

@@ -1,20 +1,23 @@
 // Block score + selection, cluster edition: the CTAs that score one (sequence, KV head) unit form a thread-block
 // cluster, so the selection no longer runs as a serial tail in one CTA behind a global-memory hand-off.
 //
-//   phase A  every CTA streams its share of the unit's statistics records through a ring of shared-memory
-//            stages filled by bulk asynchronous copies (full/empty mbarriers; one thread feeds the ring) and keeps the
-//            Taylor log masses ell^m_i (Section 3.1 of the paper, Eq. taylor-2nd, diagonal covariance) and its
-//            per-head (max, sum exp) in shared memory;
-//   sync 1   hardware cluster barrier;
-//   phase B  every CTA reads the partial normalisers of its siblings over distributed shared memory, forms the
-//            aggregated BlockScore of its own blocks (Section 2.2: per-head softmax over blocks, summed over the
-//            group), picks its best min(k, n) blocks and pushes them into the leader CTA's memory;
-//   sync 2   hardware cluster barrier;
-//   phase C  the leader picks the top k of the <= 16 x 64 candidates (forced sink / local blocks carry the
-//            maximal key; Section 4 "Sparsity Specifications") and writes them in ascending order, while its
-//            siblings compute o_bar = phi(q) S_bar, the part of the residual branch that needs no selection.
-// Ordering everywhere is (score descending, block index ascending).  The only waits are the two hardware
-// barriers and bounded mbarrier polls.  No multicast is used.
+//   phase A     every CTA streams its share of the unit's statistics records through a ring of shared-memory
+//               stages filled by bulk asynchronous copies (full/empty mbarriers; one thread feeds the ring) and keeps
+//               the Taylor log masses ell^m_i (Section 3.1 of the paper, Eq. taylor-2nd, diagonal covariance) in shared
+//               memory;
+//   exchange 1  its per-head (max, sum exp) goes into every CTA of the cluster as asynchronous stores (st.async) that
+//               count their bytes on a barrier of the receiver; a CTA goes on when all partials have reached it;
+//   phase B     warps 0-3 form the normalisers and the aggregated BlockScore of the CTA's own blocks (Section 2.2:
+//               per-head softmax over blocks, summed over the group); warps 4-7 compute o_bar = phi(q) S_bar, the
+//               part of the residual branch that needs no selection, from here on;
+//   exchange 2  each score goes, as an integer key, into the key table of every CTA that selects (all of them in the
+//               fused decode kernel, the first otherwise), again as counted asynchronous stores;
+//   phase C     warps 0-3 of a selecting CTA pick the top k on their own (Section 2.1 Select; the forced sink / local
+//               blocks of Section 4 "Sparsity Specifications" are known from their indices).  No leader, no hand-off:
+//               the selection of a unit is computed in as many copies as CTAs use it, which costs less than sending it.
+// Ordering everywhere is (score descending, block index ascending).  No barrier of the whole cluster lies on the path:
+// one is announced at the start and completed before the first exchange (everybody's barriers exist), and the kernel
+// of its own closes with one.  All waits are bounded mbarrier polls or CTA barriers.  No multicast is used.
 //
 // The body is a device function: it is the whole of the score + select kernel (spla_select, and spla_decode where the
 // fused kernel does not apply) and the first half of the fused decode kernel (decode_fused.cuh).
@@ -82,28 +85,32 @@ struct Smem {
   static constexpr int kSlots = NWP;                               // one ring position per warp
   static constexpr int kStreamBytes = kMma ? kSlots * kSlotBytes : kStages * kStageBytes;
   // after streaming the ring is dead and holds the selection's work arrays:
-  static constexpr int kKeys = 0;                                   // uint32 [1024]        this CTA's block keys
-  static constexpr int kCandKey = kKeys + 1024 * 4;                 // uint32 [16][64]      (the leader's copy is the live one)
-  static constexpr int kCandIdx = kCandKey + kMaxCluster * kMaxTopK * 4;
-  static constexpr int kCandCnt = kCandIdx + kMaxCluster * kMaxTopK * 4;   // int [16]
-  static constexpr int kFlatKey = kCandCnt + 64;                    // uint32 [1024]
-  static constexpr int kFlatIdx = kFlatKey + kMaxCluster * kMaxTopK * 4;
-  static constexpr int kSelTmp = kFlatIdx + kMaxCluster * kMaxTopK * 4;    // int [64]
-  static constexpr int kScratch = (kSelTmp + kMaxTopK * 4 + 15) / 16 * 16; // TopkScratch
+  static constexpr int kKeys = 0;                                   // uint32 [16 x 1024]   the keys of the whole unit, by block index
+  static constexpr int kFlatCap = 512;                              // survivors that are ranked by counting
+  static constexpr int kFlat = kKeys + kMaxCluster * 1024 * 4;      // uint64 [kFlatCap + 4]  (key, complement of the index)
+  static constexpr int kLaneMax = kFlat + (kFlatCap + 4) * 8;       // uint32 [128]         best key of every pair of selecting threads (64 used)
+  static constexpr int kSelTmp = kLaneMax + 128 * 4;                // int [64]             the picks, best first (where the caller gives no array)
+  static constexpr int kSelOut = kSelTmp + kMaxTopK * 4;            // int [64 + 2]         work array of the histogram selection
+  static constexpr int kScratch = (kSelOut + (kMaxTopK + 2) * 4 + 15) / 16 * 16;   // TopkScratch
   static constexpr int kWorkEnd = (kScratch + (int)sizeof(TopkScratch) + 1023) / 1024 * 1024;
-  // the ring, padded where the work arrays need more than its stages
-  // ... and, for the fused decode kernel, padded to 68 KB: the attend phase lays its K/V tile ring (at most 66 KB) over
-  // this area, and the tile copies must stay clear of the fixed region below, which holds this phase's mbarrier
-  // objects (never invalidated: overwriting them with tile data corrupted value rows, found with NaN-filled memory)
-  static constexpr int kRingBytes0 = kStreamBytes > kWorkEnd ? kStreamBytes : kWorkEnd;
-  static constexpr int kRingBytes = kRingBytes0 > 68 * 1024 ? kRingBytes0 : 68 * 1024;
+  // ... followed by the scratch of the o_bar role, which runs beside the selection
+  static constexpr int kStateScratch = kWorkEnd;                    // float [GP * D + (128 / D) * GP * D]
+  static constexpr int kStateBytes = (GP * D + (128 / D > 0 ? 128 / D : 1) * GP * D) * 4;
+  static constexpr int kAreaEnd = (kStateScratch + kStateBytes + 1023) / 1024 * 1024;
+  // The ring area is padded to hold all of that.  The fused decode kernel relies on it too: its attend phase lays the
+  // K/V tile ring (at most 66 KB) over this area, and the tile copies must stay clear of the fixed region below, which
+  // holds this phase's mbarrier objects (never invalidated: overwriting them with tile data corrupted value rows, found
+  // with NaN-filled memory), and of the o_bar scratch, which may still be in use when the first tiles arrive.
+  static constexpr int kRingBytes = kStreamBytes > kAreaEnd ? kStreamBytes : kAreaEnd;
+  static_assert(kStateScratch >= 68 * 1024, "the attend phase's tile ring must end below the o_bar scratch");
   // fixed region after the ring:
   static constexpr int kPart = kRingBytes;                          // float [GP][2]  this CTA's (max, sum)
   static constexpr int kAllPart = kPart + GP * 2 * 4;               // float [16][GP][2]
   static constexpr int kLse = kAllPart + kMaxCluster * GP * 2 * 4;  // float [GP]
   static constexpr int kWred = kLse + GP * 4;                       // float [NWP][GP][2]
   static constexpr int kBars = (kWred + NWP * GP * 2 * 4 + 7) / 8 * 8;            // uint64: full / empty per stage, or one per slot
-  static constexpr int kNumBars = NWP > 2 * kStages ? NWP : 2 * kStages;
+  static constexpr int kRingBars = kMma ? NWP : 2 * kStages;
+  static constexpr int kNumBars = kRingBars + 2;                    // ... and one each for the two exchanges of the cluster
   static constexpr int kEll = (kBars + kNumBars * 8 + 15) / 16 * 16;               // float [G][chunk]
 };
 
@@ -116,11 +123,12 @@ struct Smem {
 // more, so their statistics are streamed while the append still runs; only then does the kernel wait for the
 // append, read the final length and take the few remaining blocks (those the append wrote to) from global memory.
 // ST: element type of the statistics records (float, or __nv_bfloat16 with half the bytes to stream).
-// On return the selection of the unit is in p.sel / p.n_sel (and sel_user), written by the cluster's leader, and the
-// o_bar partials in p.obar_part; every thread of every CTA of the cluster returns (nobody has left the kernel).
+// On return the selection of the unit is in p.sel / p.n_sel (and sel_user), written by the cluster's first CTA, and the
+// o_bar partials are in p.obar_part or on their way there (warps 4-7 return on their own, without a barrier with the
+// selecting warps 0-3); every thread of every CTA of the cluster returns (nobody has left the kernel).
 template <int D, int GP, bool WIN, bool EARLY, typename ST, int NWP>
-// `sel_share` (fused kernel only, else null): a shared-memory array of kMaxTopK + 2 ints at the same place in every CTA
-// of the cluster; the leader also writes the selection there, in every CTA, followed by the count and the length.
+// `sel_share` (fused kernel only, else null): a shared-memory array of kMaxTopK + 2 ints; warps 0-3 of every CTA leave
+// the selection there, in ascending order, followed by the count and the length, and have met on a barrier since.
 __device__ __forceinline__ void score_cluster_body(const Params& p, const void* __restrict__ q_raw, int q_is_bf16,
                                                    int* __restrict__ sel_user, int pending_new, unsigned char* smem_raw,
                                                    int* sel_share = nullptr) {
@@ -151,6 +159,8 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
   float* wred = reinterpret_cast<float*>(smem_raw + SM::kWred);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw + SM::kBars);
   uint64_t* empty = full + kStages;
+  uint64_t* pbar = full + SM::kRingBars;        // completes when every CTA's partial normalisers have arrived here
+  uint64_t* kbar = pbar + 1;                    // completes when every CTA's keys have arrived here
   float* ell_s = reinterpret_cast<float*>(smem_raw + SM::kEll);          // [G][chunk] log mass per block
   __shared__ int err_s;
 
@@ -162,8 +172,11 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
   if (tid == 0) {                               // nothing here depends on the preceding kernel
     if constexpr (SM::kMma) { for (int s = 0; s < SM::kSlots; ++s) mbar_init(&full[s], 1); }
     else { for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kCsConsumers); } }
+    mbar_init(pbar, 1);
+    mbar_init(kbar, 1);
     err_s = 0;
   }
+  cluster_arrive();                             // the siblings may store here once everybody's barriers exist: completed before the first exchange
   if (!EARLY) {
     pdl_wait();                                 // everything the preceding kernels wrote (statistics, lengths, q) is visible
     pdl_launch_dependents();                    // only now may the next kernel begin its prologue: it reads q before its own wait
@@ -549,31 +562,85 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
       wred[(warp * GP + my_g) * 2 + 1] = run_sum;
     }
   }
+  // (fused decode kernel: TMA tiles will overwrite the ring area; what all eight warps did there is ordered before
+  // those copies here, the barrier passes the order on)
+  if (sel_share) asm volatile("fence.proxy.async;" ::: "memory");
   __syncthreads();
+  cluster_wait();                               // every CTA of the cluster has its barriers in place (announced at the top)
+
+  // ---- exchange 1: this CTA's (max, sum exp) of every head goes into every CTA of the cluster, as asynchronous
+  // stores that count their bytes on the receiver's barrier: a CTA goes on as soon as all partials have reached it,
+  // without a barrier of the whole cluster.  (All partials here also means: every CTA is done with its ring.)
+  const bool key_dest = sel_share || rank == 0;   // a kernel of its own: only the first CTA selects
   if (tid < G) {
     float m = -INFINITY, s = 0.f;
 #pragma unroll
     for (int w = 0; w < kCsConsumers; ++w) lse_merge(m, s, wred[(w * GP + tid) * 2], wred[(w * GP + tid) * 2 + 1]);
-    part_s[tid * 2] = m;
-    part_s[tid * 2 + 1] = s;
+    const uint32_t mine = smem_u32(all_part + ((size_t)rank * GP + tid) * 2), bar = smem_u32(pbar);
+    for (int r = 0; r < CS; ++r)
+      st_async_v2(map_to_rank(mine, (uint32_t)r), __float_as_uint(m), __float_as_uint(s), map_to_rank(bar, (uint32_t)r));
+  }
+  const int nblk_pad = min(nblk, CS * chunk);
+  if (tid == 32) {
+    mbar_expect_tx(pbar, (uint32_t)(CS * G * 8));
+    if (key_dest) {                               // the keys arrive two at a time: every CTA sends ceil(its blocks / 2) pairs
+      uint32_t bytes = 0;
+      for (int r = 0; r < CS; ++r) bytes += (uint32_t)((max(0, min(nblk_pad, (r + 1) * chunk) - min(nblk_pad, r * chunk)) + 1) / 2) * 8u;
+      mbar_expect_tx(kbar, bytes);
+    }
   }
   if (tid == 0 && err_s) atomicExch(p.status, kStatusTimeout);
+  const bool rla = !(p.flags & 4u);
+  const int n = nblk;
+  const int k_eff = min(p.top_k, n);
+  int* sel_tmp = sel_share ? sel_share : reinterpret_cast<int*>(smem_raw + SM::kSelTmp);   // the picks, best first
 
-  cluster_sync_all();                                                   // ---- sync 1: partial normalisers visible
+  if (warp >= 4) {
+    // Warps 4-7: o_bar = phi(q) S_bar (one slice of the state's rows per CTA) beside the scoring and the selection;
+    // then, in the first CTA, the selection in ascending order for the workspace and the caller.
+    if (!sel_share) cluster_arrive();             // (closing barrier of the kernel of its own, see below: these warps send nothing)
+    if (rla)
+      for (int s = rank; s < kStateSplits; s += CS) {
+        if (s != rank) asm volatile("bar.sync 2, 128;" ::: "memory");   // (the slices of one CTA reuse the same scratch)
+        state_role<D, GP, 128>(p, u, s, q_raw, q_is_bf16, reinterpret_cast<float*>(smem_raw + SM::kStateScratch), tid - 128, 2);
+      }
+    if (rank == 0) {
+      asm volatile("bar.sync 3, 256;" ::: "memory");                    // warps 0-3 have the picks
+      int* sel_u = p.sel + (size_t)u * p.top_k;
+      int* sel_o = sel_user ? sel_user + (size_t)u * p.top_k : nullptr;
+      for (int s = tid - 128; s < p.top_k; s += 128) {
+        if (s < k_eff) {
+          const int ia = sel_tmp[s];
+          int pos = 0;
+#pragma unroll 4
+          for (int j = 0; j < k_eff; j += 4) {                          // (padded with entries that precede nothing)
+            const int4 ii = *reinterpret_cast<const int4*>(sel_tmp + j);
+            pos += (ii.x < ia) + (ii.y < ia) + (ii.z < ia) + (ii.w < ia);
+          }
+          sel_u[pos] = ia;
+          if (sel_o) sel_o[pos] = ia;
+        } else {
+          sel_u[s] = -1;
+          if (sel_o) sel_o[s] = -1;
+        }
+      }
+      if (tid == 128) p.n_sel[u] = k_eff;
+    }
+    if (!sel_share) cluster_wait();
+    return;
+  }
 
-  // ------------------------------------------------------------------ phase B -------------------------------
-  // Log-sum-exp of every head over the whole cluster, by each warp on its own (no block barrier): lane p
-  // fetches the (max, sum) pair of CTA p / GP and head p % GP over distributed shared memory, then the lanes
-  // of one head are folded with shuffles.
+  // ------------------------------------------------------------------ phase B (warps 0-3) -------------------
+  const TopkGroup selg{tid, 128, 1};
+  if (!mbar_wait(pbar, 0, p.wait_limit) && lane == 0) atomicExch(p.status, kStatusTimeout);
+  // Log-sum-exp of every head over the whole cluster, by each warp on its own (no block barrier): lane p takes the
+  // (max, sum) pair of CTA p / GP and head p % GP, then the lanes of one head are folded with shuffles.
   float lse_r[GP];
   {
     float m = -INFINITY, sm = 0.f;
     for (int pr = lane; pr < CS * GP; pr += 32) {
-      const int r = pr / GP, g = pr % GP;
-      if (g < G) {
-        const uint32_t remote = map_to_rank(smem_u32(part_s + g * 2), (uint32_t)r);
-        lse_merge(m, sm, ld_dsmem_f32(remote), ld_dsmem_f32(remote + 4));
-      }
+      const int g = pr % GP;
+      if (g < G) lse_merge(m, sm, all_part[pr * 2], all_part[pr * 2 + 1]);
     }
 #pragma unroll
     for (int o = GP; o < 32; o <<= 1) {
@@ -585,183 +652,165 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
     for (int g = 0; g < GP; ++g) lse_r[g] = __shfl_sync(0xffffffffu, lse, g);
   }
 
+  // ---- exchange 2: the aggregated score of this CTA's blocks goes to global memory (spla_copy_scores) and, as an
+  // integer key, into the key table of every selecting CTA (two blocks per thread and store; the share of a CTA is a
+  // multiple of 8 blocks; entries past the sequence's last block are never read)
   uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw + SM::kKeys);
-  TopkScratch* scratch = reinterpret_cast<TopkScratch*>(smem_raw + SM::kScratch);
-  const int k_eff = min(p.top_k, nblk);
-  const uint32_t cand_key0 = map_to_rank(smem_u32(smem_raw + SM::kCandKey), 0u) + (uint32_t)rank * kMaxTopK * 4;
-  const uint32_t cand_idx0 = map_to_rank(smem_u32(smem_raw + SM::kCandIdx), 0u) + (uint32_t)rank * kMaxTopK * 4;
-  auto push = [&](int slot, uint32_t key, int idx) {                  // into the leader's candidate table
-    st_dsmem_u32(cand_key0 + (uint32_t)slot * 4, key);
-    st_dsmem_u32(cand_idx0 + (uint32_t)slot * 4, (uint32_t)idx);
-  };
-  if (tid == 0) { scratch->lo = 0xffffffffu; scratch->hi = 0u; scratch->n_forced = 0; scratch->n_emit = 0; }
-  __syncthreads();
   {
-    // aggregated score of this CTA's blocks; the statistics the selection needs are gathered on the way
     float* scores_u = p.scores + (size_t)u * p.max_blocks;
-    uint32_t mn = 0xffffffffu, mx = 0u;
-    int nf = 0;
-    for (int li = tid; li < nb_my; li += kCsThreads) {
-      float sc = 0.f;
+    const uint32_t keys0 = smem_u32(keys), bar = smem_u32(kbar);
+    const int n_dest = sel_share ? CS : 1;
+    for (int li = tid * 2; li < nb_my; li += 128 * 2) {
+      float sc0 = 0.f, sc1 = 0.f;
 #pragma unroll
       for (int g = 0; g < GP; ++g)
-        if (g < G) sc += __expf(ell_s[g * chunk + li] - lse_r[g]);
+        if (g < G) {
+          const float2 e = *reinterpret_cast<const float2*>(ell_s + g * chunk + li);
+          sc0 += __expf(e.x - lse_r[g]);
+          sc1 += __expf(e.y - lse_r[g]);
+        }
       const int i = blk_begin + li;
-      scores_u[i] = sc;
-      const bool forced = (i < p.n_sink) || (i >= nblk - p.n_local);
-      const uint32_t key = forced ? 0xffffffffu : __float_as_uint(sc);
-      keys[li] = key;
-      if (forced) {
-        ++nf;
-        push(atomicAdd(&scratch->n_emit, 1), key, i);
-      } else {
-        mn = min(mn, key);
-        mx = max(mx, key);
-      }
-    }
-    mn = __reduce_min_sync(0xffffffffu, mn);
-    mx = __reduce_max_sync(0xffffffffu, mx);
-    nf = __reduce_add_sync(0xffffffffu, nf);
-    if (lane == 0) {
-      atomicMin(&scratch->lo, mn);
-      atomicMax(&scratch->hi, mx);
-      if (nf) atomicAdd(&scratch->n_forced, nf);
+      scores_u[i] = sc0;
+      if (li + 1 < nb_my) scores_u[i + 1] = sc1; else sc1 = 0.f;
+      for (int r = 0; r < n_dest; ++r)
+        st_async_v2(map_to_rank(keys0 + (uint32_t)i * 4u, (uint32_t)r), __float_as_uint(sc0), __float_as_uint(sc1),
+                    map_to_rank(bar, (uint32_t)r));
     }
   }
-  __syncthreads();
-
-  // this CTA's best min(k_eff, n_my) blocks go to the leader's candidate table
-  {
-    const int cnt = select_topk(keys, nb_my, k_eff, [&](int li) { return blk_begin + li; }, push, scratch);
-    if (tid == 0) st_dsmem_u32(map_to_rank(smem_u32(smem_raw + SM::kCandCnt), 0u) + (uint32_t)rank * 4, (uint32_t)cnt);
+  // As a kernel of its own the cluster closes with a barrier that every thread announces once it has sent its last
+  // store and completes before it leaves: no CTA is gone while a sibling may still store into it, even after a wait
+  // that gave up.  (In the fused decode kernel the barriers of the attend phase do that.)
+  if (!sel_share) cluster_arrive();
+  if (!key_dest) {
+    cluster_wait();
+    return;
   }
 
-  cluster_sync_all();                                                   // ---- sync 2: candidates are in the leader
-  const bool rla = !(p.flags & 4u);
-  if (rank != 0) {
-    // The siblings are done with the selection; while the leader finishes it they compute the part of the
-    // residual branch that needs no selection, o_bar = phi(q) S_bar, one slice of the state's rows each.
-    if (rla)
-      for (int s = rank - 1; s < kStateSplits; s += CS - 1) {
-        __syncthreads();                       // (the slices of one CTA reuse the same shared memory)
-        state_role<D, GP, kCsThreads>(p, u, s, q_raw, q_is_bf16, reinterpret_cast<float*>(smem_raw));
-      }
-  } else {
-  // ------------------------------------------------------------------ phase C (leader) ----------------------
-  const uint32_t* cand_key = reinterpret_cast<const uint32_t*>(smem_raw + SM::kCandKey);
-  const int* cand_idx = reinterpret_cast<const int*>(smem_raw + SM::kCandIdx);
-  const int* cand_cnt = reinterpret_cast<const int*>(smem_raw + SM::kCandCnt);
-  uint32_t* flat_key = reinterpret_cast<uint32_t*>(smem_raw + SM::kFlatKey);
-  int* flat_idx = reinterpret_cast<int*>(smem_raw + SM::kFlatIdx);
-  int* sel_tmp = reinterpret_cast<int*>(smem_raw + SM::kSelTmp);
-  // Two lower bounds of the k_eff-th best key, so that most of the table drops out before any ranking.  With n_full
-  // CTAs that sent a full list of k_eff candidates: (a) the smallest key of any one full list (that list alone holds
-  // k_eff keys from there upwards: good when one part of the sequence dominates); (b) the smallest, over the full
-  // lists, of each list's q-th best key, q = ceil(k_eff / n_full) (n_full q >= k_eff keys lie at or above it: good
-  // when the lists look alike).  The larger of the two is used.
-  uint32_t* list_min = reinterpret_cast<uint32_t*>(scratch->hist);      // [kMaxCluster] bound (a) per list
-  uint32_t* list_qth = list_min + kMaxCluster;                          // [kMaxCluster] q-th best per list
-  int* n_surv = scratch->hist + 2 * kMaxCluster;                        // survivor counter
-  int n_full = 0;
-  for (int r = 0; r < CS; ++r) n_full += cand_cnt[r] == k_eff;
-  const int quota = n_full > 0 ? (k_eff + n_full - 1) / n_full : 0;
-  for (int r = warp; r < CS; r += kCsConsumers) {
-    const int cnt = cand_cnt[r];
-    const bool is_full = cnt == k_eff;
-    uint32_t v0 = lane < cnt ? cand_key[r * kMaxTopK + lane] : (is_full ? 0xffffffffu : 0u);
-    uint32_t v1 = lane + 32 < cnt ? cand_key[r * kMaxTopK + lane + 32] : (is_full ? 0xffffffffu : 0u);
-    const uint32_t lmin = __reduce_min_sync(0xffffffffu, min(v0, v1));  // (the padding of a full list is neutral here)
-    if (lane >= cnt) v0 = 0u;
-    if (lane + 32 >= cnt) v1 = 0u;
-    uint32_t m = 0xffffffffu;                                           // "no bound from this list" for the minimum below
-    if (is_full && quota <= 8) {
-      for (int round = 0; round < quota; ++round) {                     // knock the largest out, quota times
-        m = __reduce_max_sync(0xffffffffu, max(v0, v1));
-        const uint32_t in0 = __ballot_sync(0xffffffffu, v0 == m);
-        const uint32_t in1 = __ballot_sync(0xffffffffu, v1 == m);
-        if (in0) { if (lane == __ffs(in0) - 1) v0 = 0u; }
-        else if (lane == __ffs(in1) - 1) v1 = 0u;
-      }
-    }
-    if (lane == 0) { list_min[r] = is_full ? lmin : 0u; list_qth[r] = m; }
+  // the selection's fixed parts need no key: the forced blocks behind the `need` ranked ones, padding that precedes
+  // nothing behind them, an empty survivor table
+  unsigned long long* flat = reinterpret_cast<unsigned long long*>(smem_raw + SM::kFlat);
+  const int n_forced = (p.n_sink + p.n_local >= n) ? n : p.n_sink + p.n_local;
+  const int need = k_eff - n_forced;
+  const int n_sink = p.n_sink, local0 = n - p.n_local;             // free blocks: n_sink <= i < local0
+  for (int s = tid; s < kMaxTopK; s += 128) {
+    int v = 0x7fffffff;
+    if (k_eff == n) { if (s < k_eff) v = s; }                      // everything is selected
+    else if (s >= max(need, 0) && s < k_eff) { const int f = s - max(need, 0); v = f < n_sink ? f : local0 + (f - n_sink); }
+    sel_tmp[s] = v;
   }
-  if (tid == 0) *n_surv = 0;
-  __syncthreads();
-  uint32_t bound_a = 0u, bound_b = 0xffffffffu;
-  for (int r = 0; r < CS; ++r) { bound_a = max(bound_a, list_min[r]); bound_b = min(bound_b, list_qth[r]); }
-  if (bound_b == 0xffffffffu) bound_b = 0u;                             // no full list, or too large a quota
-  const uint32_t bound = max(bound_a, bound_b);
-  for (int c0 = 0; c0 < CS * kMaxTopK; c0 += kCsThreads) {             // the survivors, in no particular order
-    const int c = c0 + tid, r = c / kMaxTopK, sl = c % kMaxTopK;
-    const bool live = c < CS * kMaxTopK && sl < cand_cnt[r] && cand_key[c] >= bound;
-    const uint32_t vote = __ballot_sync(0xffffffffu, live);
-    int base = 0;
-    if (lane == 0 && vote) base = atomicAdd(n_surv, __popc(vote));
-    base = __shfl_sync(0xffffffffu, base, 0);
-    if (live) {
-      const int dst = base + __popc(vote & ((1u << lane) - 1u));
-      flat_key[dst] = cand_key[c];
-      flat_idx[dst] = cand_idx[c];
-    }
-  }
-  __syncthreads();
-  const int total = *n_surv;
-  auto keep = [&](int slot, uint32_t, int idx) { sel_tmp[slot] = idx; };
-  auto flat_of = [&](int c) { return flat_idx[c]; };
-  if (total <= kCsThreads) {
-    // few survivors (the usual case): every thread ranks its candidates against all others by counting, reading the
-    // table with broadcast 128-bit loads; no shared-memory atomics, one barrier
-    if (tid < 4) { flat_key[total + tid] = 0u; flat_idx[total + tid] = 0x7fffffff; }   // padding that precedes nothing
-    __syncthreads();
-    for (int c = tid; c < total; c += kCsThreads) {
-      const uint32_t a = flat_key[c];
-      const int ia = flat_idx[c];
-      int rk = 0;
-      for (int j = 0; j < total; j += 4) {
-        const uint4 kk = *reinterpret_cast<const uint4*>(flat_key + j);
-        const int4 ii = *reinterpret_cast<const int4*>(flat_idx + j);
-        rk += pair_before(kk.x, ii.x, a, ia) + pair_before(kk.y, ii.y, a, ia) + pair_before(kk.z, ii.z, a, ia) +
-              pair_before(kk.w, ii.w, a, ia);
-      }
-      if (rk < k_eff) sel_tmp[rk] = ia;
-    }
-    __syncthreads();
-  } else {
-    topk_prepare(flat_key, total, flat_of, keep, scratch);
-    select_topk(flat_key, total, k_eff, flat_of, keep, scratch);
-  }
+  for (int s = tid; s < SM::kFlatCap + 4; s += 128) flat[s] = 0ull;
+  if (tid == 0 && sel_share) { sel_share[kMaxTopK] = k_eff; sel_share[kMaxTopK + 1] = L; }
 
-  int* sel_u = p.sel + (size_t)u * p.top_k;
-  int* sel_o = sel_user ? sel_user + (size_t)u * p.top_k : nullptr;
-  for (int s = tid; s < p.top_k; s += kCsThreads) {
-    if (s < k_eff) {
-      const int ia = sel_tmp[s];
-      int pos = 0;
+  if (!mbar_wait(kbar, 0, p.wait_limit) && lane == 0) atomicExch(p.status, kStatusTimeout);   // ---- all keys are here
+
+  // ------------------------------------------------------------------ phase C (warps 0-3) -------------------
+  // Top k_eff of the unit's n blocks.  The forced blocks (the first n_sink, the last n_local) are known from their
+  // indices; `need` free blocks remain to be picked.  Thread t looks at the free blocks t, t + 128, ...; every pair of
+  // threads notes the best key it sees; the need-th best of these 64 is a lower bound of the need-th best key overall
+  // (they are 64 different blocks), and with evenly spread keys little more than `need` keys reach it.  The survivors
+  // are ranked by counting, as 64-bit words (key, complement of the index) that one comparison orders; the picks stay
+  // in that order (best first, then the forced blocks): every CTA computes the same list, and the attention does not
+  // care.  Where too many survive (equal scores) or the sequence has more than 128 x 64 blocks, the histogram selection
+  // runs over the whole table instead and its picks are put in ascending order.
+  if (k_eff < n && need > 0) {
+    uint32_t* pair_max = reinterpret_cast<uint32_t*>(smem_raw + SM::kLaneMax);
+    TopkScratch* scratch = reinterpret_cast<TopkScratch*>(smem_raw + SM::kScratch);
+    int* n_surv = &scratch->n_small;
+    uint32_t* bound_s = &scratch->lo;
+    const int n_free = local0 - n_sink;
+    const int nr = (n_free + 127) / 128;                              // free blocks per thread
+    const uint32_t* my_keys = keys + n_sink + tid;
+    const int my_n = n_free > tid ? (n_free - tid + 127) / 128 : 0;   // ... of this thread
+    int total = SM::kFlatCap + 1;
+    if (nr <= 64) {
+      uint32_t mx = 0u;
 #pragma unroll 8
-      for (int j = 0; j < k_eff; ++j) pos += sel_tmp[j] < ia;
-      sel_u[pos] = ia;
-      if (sel_o) sel_o[pos] = ia;
-      if (sel_share)
-        for (int r = 0; r < CS; ++r) st_dsmem_u32(map_to_rank(smem_u32(sel_share + pos), (uint32_t)r), (uint32_t)ia);
-    } else {
-      sel_u[s] = -1;
-      if (sel_o) sel_o[s] = -1;
-    }
-  }
-  if (tid == 0) {
-    p.n_sel[u] = k_eff;
-    if (sel_share)
-      for (int r = 0; r < CS; ++r) {
-        st_dsmem_u32(map_to_rank(smem_u32(sel_share + kMaxTopK), (uint32_t)r), (uint32_t)k_eff);
-        st_dsmem_u32(map_to_rank(smem_u32(sel_share + kMaxTopK + 1), (uint32_t)r), (uint32_t)L);
+      for (int r = 0; r < my_n; ++r) mx = max(mx, my_keys[128 * r]);
+      mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      // made unique and comparable in one go: the low six bits give way to the pair's number (rounding the key down
+      // keeps the bound a lower bound)
+      const int pr = tid >> 1, half = tid & 1;
+      const uint32_t mine = (mx & ~63u) | (uint32_t)(63 - pr);
+      if (!half) pair_max[pr] = mine;
+      if (tid == 0) *n_surv = 0;
+      selg.sync();
+      {
+        int rk = 0;                               // rank of this pair's best key among the 64, half of them per thread
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+          const uint4 kk = *reinterpret_cast<const uint4*>(pair_max + half * 32 + j);
+          rk += (kk.x > mine) + (kk.y > mine) + (kk.z > mine) + (kk.w > mine);
+        }
+        rk += __shfl_xor_sync(0xffffffffu, rk, 1);
+        if (!half && rk == need - 1) *bound_s = mine & ~63u;
       }
-  }
-  if (rla && CS == 1)
-    for (int s = 0; s < kStateSplits; ++s) {
-      __syncthreads();
-      state_role<D, GP, kCsThreads>(p, u, s, q_raw, q_is_bf16, reinterpret_cast<float*>(smem_raw));
+      selg.sync();
+      const uint32_t bound = *bound_s;
+      {
+        // the survivors, in no particular order: mark, count, reserve a range per warp, write
+        unsigned long long mask = 0ull;
+#pragma unroll 8
+        for (int r = 0; r < my_n; ++r) mask |= (unsigned long long)(my_keys[128 * r] >= bound) << r;
+        const int cnt = __popcll(mask);
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int t = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += t;
+        }
+        int base = 0;
+        if (lane == 31) base = atomicAdd(n_surv, incl);
+        int dst = __shfl_sync(0xffffffffu, base, 31) + incl - cnt;
+        while (mask) {
+          const int r = __ffsll((long long)mask) - 1;
+          mask &= mask - 1ull;
+          if (dst < SM::kFlatCap)
+            flat[dst] = ((unsigned long long)my_keys[128 * r] << 32) | (uint32_t)(0x7fffffff - (n_sink + tid + 128 * r));
+          ++dst;
+        }
+      }
+      selg.sync();
+      total = *n_surv;
     }
-  }   // leader
+    if (total <= SM::kFlatCap) {
+      // P = 4, 2 or 1 neighbouring lanes share a candidate and a part of the table each (broadcast 128-bit loads; the
+      // empty entries behind the survivors precede nothing)
+      const int lg = total <= 32 ? 2 : total <= 64 ? 1 : 0, P = 1 << lg;
+      const int span = ((total + P - 1) / P + 1) & ~1;                // entries per part, even
+      for (int c0 = 0; c0 < total; c0 += 128 >> lg) {
+        const int c = c0 + (tid >> lg), part = tid & (P - 1);
+        const unsigned long long a = c < total ? flat[c] : ~0ull;
+        int rk = 0;
+#pragma unroll 4
+        for (int j = part * span; j < (part + 1) * span; j += 2) {
+          const ulonglong2 kk = *reinterpret_cast<const ulonglong2*>(flat + j);
+          rk += (kk.x > a) + (kk.y > a);
+        }
+        if (lg >= 1) rk += __shfl_xor_sync(0xffffffffu, rk, 1);
+        if (lg >= 2) rk += __shfl_xor_sync(0xffffffffu, rk, 2);
+        if (part == 0 && c < total && rk < need) sel_tmp[rk] = 0x7fffffff - (int)(uint32_t)a;
+      }
+    } else {
+      // forced blocks get the maximal key and the histogram selection picks all k_eff, in no reproducible order:
+      // they are put in ascending order, so that every CTA of the cluster holds the same list
+      for (int i = tid; i < n_forced; i += 128) keys[i < n_sink ? i : local0 + (i - n_sink)] = 0xffffffffu;
+      int* pick = reinterpret_cast<int*>(smem_raw + SM::kSelOut);
+      selg.sync();
+      auto keep = [&](int slot, uint32_t, int idx) { pick[slot] = idx; };
+      auto same = [&](int i) { return i; };
+      topk_prepare(keys, n, same, keep, scratch, selg);
+      select_topk(keys, n, k_eff, same, keep, scratch, selg);
+      for (int s = tid; s < k_eff; s += 128) {
+        const int ia = pick[s];
+        int pos = 0;
+        for (int j = 0; j < k_eff; ++j) pos += pick[j] < ia;
+        sel_tmp[pos] = ia;
+      }
+    }
+  }
+  selg.sync();
+  if (rank == 0) asm volatile("bar.arrive 3, 256;" ::: "memory");       // warps 4-7 write the list out
+  if (!sel_share) cluster_wait();
 }
 
 template <int D, int GP, bool WIN, bool EARLY, typename ST, int NWP>

@@ -76,7 +76,7 @@ __global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_k
 
   // ------------------------------------------------------------------ o_bar role ----------------------
   if (c >= p.n_chunks_cap) {
-    state_role<D, GP, kScoreThreads>(p, u, c - p.n_chunks_cap, q_raw, q_is_bf16, reinterpret_cast<float*>(smem_raw));
+    state_role<D, GP, kScoreThreads>(p, u, c - p.n_chunks_cap, q_raw, q_is_bf16, reinterpret_cast<float*>(smem_raw), (int)threadIdx.x, 0);
     return;
   }
 

@@ -6,15 +6,22 @@
 
 namespace spla {
 
-// NT threads take part (the CTA may be larger; the others only join the barriers).
+// NT threads take part.  bar_id 0: they are the first NT threads of the CTA, whose other threads only join the
+// barriers.  Otherwise they are NT consecutive threads (whole warps) with local numbers `tid` = 0 .. NT - 1 that meet
+// on the named barrier `bar_id`, and the rest of the CTA is elsewhere.
 // smem: (GP * D + (NT / D) * GP * D) floats.
 template <int D, int GP, int NT>
 __device__ __forceinline__ void state_role(const Params& p, int u, int s, const void* __restrict__ q_raw, int q_is_bf16,
-                                           float* smem) {
+                                           float* smem, const int tid, const int bar_id) {
+  auto meet = [&]() {
+    if (bar_id == 0) __syncthreads();
+    else asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(NT) : "memory");
+  };
+  const int stride = bar_id == 0 ? (int)blockDim.x : NT;
   constexpr int VEC = D / 32;
   constexpr int RG = NT / D;                             // row groups working side by side
   constexpr int ROWS = D / kStateSplits / RG;            // rows per thread
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int lane = tid & 31, warp = tid >> 5;
   const int b = u / p.Hkv, h = u % p.Hkv, G = p.G;
   const bool act = tid < NT;
   float* phiq = smem;                                    // [GP][D]
@@ -22,9 +29,10 @@ __device__ __forceinline__ void state_role(const Params& p, int u, int s, const 
   const float a2 = p.phi_scale * kLog2e;
   const int rg = tid / D, j = tid % D;
   const float* S = p.state + (size_t)u * D * D + (size_t)(s * (D / kStateSplits) + rg) * D + j;
-  float sv[ROWS];
+  constexpr int RB = ROWS > 16 ? 16 : ROWS;              // rows in flight per thread (bounds the registers)
+  float sv[RB];
 #pragma unroll
-  for (int r = 0; r < ROWS; ++r) sv[r] = act ? __ldcs(S + (size_t)r * RG * D) : 0.f;   // all loads in flight before use
+  for (int r = 0; r < RB; ++r) sv[r] = act ? __ldcs(S + (size_t)r * RG * D) : 0.f;   // in flight while phi(q) is formed
   for (int g = warp; g < G; g += NT / 32) {
     float x[VEC];
     const size_t qoff = ((size_t)b * p.Hq + (size_t)h * G + g) * D + lane * VEC;
@@ -42,23 +50,30 @@ __device__ __forceinline__ void state_role(const Params& p, int u, int s, const 
 #pragma unroll
     for (int v = 0; v < VEC; ++v) phiq[g * D + lane * VEC + v] = x[v] * inv;
   }
-  __syncthreads();
+  meet();
   if (act) {
     float acc[GP];
 #pragma unroll
     for (int g = 0; g < GP; ++g) acc[g] = 0.f;
 #pragma unroll
-    for (int r = 0; r < ROWS; ++r) {
-      const int row = s * (D / kStateSplits) + rg + r * RG;
+    for (int r0 = 0; r0 < ROWS; r0 += RB) {
+      if (r0 > 0) {
 #pragma unroll
-      for (int g = 0; g < GP; ++g)
-        if (g < G) acc[g] = fmaf(phiq[g * D + row], sv[r], acc[g]);
+        for (int r = 0; r < RB; ++r) sv[r] = __ldcs(S + (size_t)(r0 + r) * RG * D);
+      }
+#pragma unroll
+      for (int r = 0; r < RB; ++r) {
+        const int row = s * (D / kStateSplits) + rg + (r0 + r) * RG;
+#pragma unroll
+        for (int g = 0; g < GP; ++g)
+          if (g < G) acc[g] = fmaf(phiq[g * D + row], sv[r], acc[g]);
+      }
     }
 #pragma unroll
     for (int g = 0; g < GP; ++g) red[(rg * GP + g) * D + j] = acc[g];
   }
-  __syncthreads();
-  for (int idx = tid; idx < G * D; idx += blockDim.x) {
+  meet();
+  for (int idx = tid; idx < G * D; idx += stride) {
     const int g = idx / D, jj = idx % D;
     float t = 0.f;
 #pragma unroll

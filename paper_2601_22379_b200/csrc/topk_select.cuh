@@ -24,15 +24,27 @@ struct TopkScratch {                // shared memory work area
   int code_t, above, bin_count;
 };
 
+// The threads that run a selection together: the whole CTA (barrier id 0), or its first `nthreads` threads (whole
+// warps) meeting on a named barrier of their own while the rest of the CTA does something else.
+struct TopkGroup {
+  int tid, nthreads, bar_id;
+  __device__ __forceinline__ void sync() const {
+    if (bar_id == 0) __syncthreads();
+    else asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(nthreads) : "memory");
+  }
+};
+__device__ __forceinline__ TopkGroup topk_whole_cta() { return TopkGroup{(int)threadIdx.x, (int)blockDim.x, 0}; }
+
 __device__ __forceinline__ bool pair_before(uint32_t ka, int ia, uint32_t kb, int ib) { return ka > kb || (ka == kb && ia < ib); }
 
 // Statistics pass for callers that have not gathered them while producing the keys: emits the forced pairs and
 // leaves lo / hi / n_forced / n_emit in the scratch.  Ends with a barrier.
 template <class IdxFn, class EmitFn>
-__device__ __forceinline__ void topk_prepare(const uint32_t* key, int n, IdxFn idx_of, EmitFn emit, TopkScratch* sc) {
-  const int tid = threadIdx.x, lane = tid & 31, nthreads = blockDim.x;
+__device__ __forceinline__ void topk_prepare(const uint32_t* key, int n, IdxFn idx_of, EmitFn emit, TopkScratch* sc,
+                                             const TopkGroup grp = topk_whole_cta()) {
+  const int tid = grp.tid, lane = tid & 31, nthreads = grp.nthreads;
   if (tid == 0) { sc->lo = 0xffffffffu; sc->hi = 0u; sc->n_forced = 0; sc->n_emit = 0; }
-  __syncthreads();
+  grp.sync();
   uint32_t mn = 0xffffffffu, mx = 0u;
   int nf = 0;
   for (int i = tid; i < n; i += nthreads) {
@@ -53,16 +65,17 @@ __device__ __forceinline__ void topk_prepare(const uint32_t* key, int n, IdxFn i
     atomicMax(&sc->hi, mx);
     if (nf) atomicAdd(&sc->n_forced, nf);
   }
-  __syncthreads();
+  grp.sync();
 }
 
 // Requires sc->lo, sc->hi, sc->n_forced, sc->n_emit to describe `key` (forced pairs already emitted) and a
 // barrier since they were written.  `emit(slot, key, idx)` stores one selected pair (slots in no particular
-// order); `idx_of(i)` maps position i of `key` to the pair's index.  All threads of the CTA must call this.
+// order); `idx_of(i)` maps position i of `key` to the pair's index.  All threads of the group must call this.
 // Returns min(k, n).
 template <class IdxFn, class EmitFn>
-__device__ __forceinline__ int select_topk(const uint32_t* key, int n, int k, IdxFn idx_of, EmitFn emit, TopkScratch* sc) {
-  const int tid = threadIdx.x, lane = tid & 31, nthreads = blockDim.x;
+__device__ __forceinline__ int select_topk(const uint32_t* key, int n, int k, IdxFn idx_of, EmitFn emit, TopkScratch* sc,
+                                          const TopkGroup grp = topk_whole_cta()) {
+  const int tid = grp.tid, lane = tid & 31, nthreads = grp.nthreads;
   k = min(k, n);
   if (k <= 0) return 0;
   const int n_forced = sc->n_forced;
@@ -72,7 +85,7 @@ __device__ __forceinline__ int select_topk(const uint32_t* key, int n, int k, Id
   if (need >= n - n_forced) {                 // everything is selected
     for (int i = tid; i < n; i += nthreads)
       if (key[i] != 0xffffffffu) emit(atomicAdd(&sc->n_emit, 1), key[i], idx_of(i));
-    __syncthreads();
+    grp.sync();
     return k;
   }
 
@@ -82,7 +95,7 @@ __device__ __forceinline__ int select_topk(const uint32_t* key, int n, int k, Id
     shift = range < 256u ? 0 : (32 - __clz(range)) - 8;
     for (int i = tid; i < 256 + 32; i += nthreads) sc->hist[i] = 0;
     if (tid == 0) sc->n_small = 0;
-    __syncthreads();
+    grp.sync();
     for (int i = tid; i < n; i += nthreads) {
       const uint32_t x = key[i];
       if (x >= lo && x <= hi) {
@@ -90,7 +103,7 @@ __device__ __forceinline__ int select_topk(const uint32_t* key, int n, int k, Id
         atomicAdd(&sc->hist[c + (c >> 3)], 1);
       }
     }
-    __syncthreads();
+    grp.sync();
     if (tid < 32) {                           // the bin of the need-th largest live key
       int bins[8], tot = 0;
 #pragma unroll
@@ -111,7 +124,7 @@ __device__ __forceinline__ int select_topk(const uint32_t* key, int n, int k, Id
         }
       }
     }
-    __syncthreads();
+    grp.sync();
     const uint32_t code_t = (uint32_t)sc->code_t;
     bin_count = sc->bin_count;
     const bool last = bin_count <= kSelSmall || shift == 0;
@@ -133,7 +146,7 @@ __device__ __forceinline__ int select_topk(const uint32_t* key, int n, int k, Id
     const uint32_t span = shift == 0 ? 0u : ((1u << shift) - 1u);
     hi = min(hi, lo2 + span);
     lo = lo2;
-    __syncthreads();                          // small_* complete; code_t / above may be rewritten by the next pass
+    grp.sync();                          // small_* complete; code_t / above may be rewritten by the next pass
     if (last) break;
   }
 
@@ -162,7 +175,7 @@ __device__ __forceinline__ int select_topk(const uint32_t* key, int n, int k, Id
       if (rk < need) emit(atomicAdd(&sc->n_emit, 1), lo, ia);
     }
   }
-  __syncthreads();
+  grp.sync();
   return k;
 }
 
