@@ -57,9 +57,10 @@ __global__ void __launch_bounds__(kAttendThreads) attend_merge_kernel(const Para
   uint64_t* bar = reinterpret_cast<uint64_t*>(misc + 4 * GP + 2 * NWARP * GP);
   __shared__ int flag_s;
 
-  if (tid == 0 && !fetch) mbar_init(bar, 1);
+  if (tid == 0 && !fetch) { mbar_init(bar, 1); mbar_init_done(); }
   if (tid == 0 && fetch) {
     mbar_init(bar, 1);
+    mbar_init_done();
     const size_t tile = (size_t)u * p.max_blocks + blk;
     const uint32_t tile_bytes = (uint32_t)((size_t)B * D * sizeof(T));
     mbar_expect_tx(bar, 2 * tile_bytes + (uint32_t)(B * sizeof(float)) + (uint32_t)p.dbg_tx_extra);

@@ -84,13 +84,14 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
                                                 const __nv_bfloat16* __restrict__ q, const float* __restrict__ rms_weight,
                                                 float* __restrict__ out, float* __restrict__ dbg_sparse,
                                                 float* __restrict__ dbg_rla, unsigned char* smem_raw,
-                                                const int* sel_share = nullptr) {
+                                                const int* sel_share = nullptr, uint64_t* full_ext = nullptr) {
   constexpr int KS = D / 16;        // k-steps of the two QK-type products
   constexpr int NT = D / 8;         // n-tiles of the PV-type product
   constexpr int NH = D / 64;        // 64-column halves of a tile (one TMA box each)
   constexpr int NTHR = NG * kAttendThreads;
   constexpr int NWARP = NTHR / 32;
-  __shared__ __align__(8) uint64_t full[kMaxSlots];
+  __shared__ __align__(8) uint64_t full_own[kMaxSlots];
+  uint64_t* full = full_ext ? full_ext : full_own;      // (the fused kernel initialises its tile barriers at its start)
   __shared__ float red_s[NWARP];
   __shared__ int sel_s[kMaxTopK];
   __shared__ int err_s;
@@ -173,7 +174,10 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
   // requested first and the fragments are formed while they are on their way.
   if constexpr (!FUSED) make_fragments();
   if (tid == 0) {
-    for (int s = 0; s < kMaxSlots; ++s) mbar_init(&full[s], 1);
+    if (!full_ext) {
+      for (int s = 0; s < kMaxSlots; ++s) mbar_init(&full[s], 1);
+      mbar_init_done();
+    }
     err_s = 0;
   }
 
@@ -382,6 +386,9 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
   }
   if (tid == 0 && err_s) atomicExch(p.status, kStatusTimeout);
 
+  // (a kernel input the merge needs at its very end: requested now, it arrives under the fold)
+  const float gamma0 = (rank < G && tid < D) ? __ldg(rms_weight + ((size_t)h * G + rank) * D + tid) : 0.f;
+
   // ---- fold the four warps together ------------------------------------------------------------------------
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
   l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
@@ -391,19 +398,14 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
   float* red_l = red_m + NWARP * 8;                                     // [NWARP][8]
   float* mine = red_l + NWARP * 8;                                      // [2][8][D]   this CTA's partial result
   float* mine_ml = mine + 2 * 8 * D;                                    // [8][2]      (max, sum) of the exact branch
-  if (t == 0) red_m[warp * 8 + g] = m_run;
-  cta_sync();
-  float M = red_m[g];
-#pragma unroll
-  for (int w = 1; w < NWARP; ++w) M = fmaxf(M, red_m[w * 8 + g]);
-  const float f = M > -INFINITY ? ex2(m_run - M) : 0.f;                 // 0 for a warp (or a CTA) that saw no token
-  const float f_o = (PACK && g >= 4) ? 1.f : f;                         // packed rows 4..7 belong to the linear branch
-  if (t == 0) red_l[warp * 8 + g] = l_run * f;
+  // every warp leaves its rows as they are, with its running maximum and sum; the combiner rescales (one barrier less
+  // than agreeing on the maximum first)
+  if (t == 0) { red_m[warp * 8 + g] = m_run; red_l[warp * 8 + g] = l_run; }
   {
     float* ro = red_o + (size_t)warp * 16 * (D + kPad);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-      *reinterpret_cast<float2*>(ro + (size_t)g * (D + kPad) + nt * 8 + 2 * t) = make_float2(o[nt][0] * f_o, o[nt][1] * f_o);
+      *reinterpret_cast<float2*>(ro + (size_t)g * (D + kPad) + nt * 8 + 2 * t) = make_float2(o[nt][0], o[nt][1]);
       *reinterpret_cast<float2*>(ro + (size_t)(g + 8) * (D + kPad) + nt * 8 + 2 * t) = make_float2(o[nt][2], o[nt][3]);
     }
   }
@@ -411,11 +413,19 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
   for (int idx = tid; idx < 2 * G * (D / 4); idx += NTHR) {             // four columns per thread and step
     const int br = idx / (G * (D / 4)), hd = (idx / (D / 4)) % G, c4 = (idx % (D / 4)) * 4;   // branch, head, first column
     const int rr = br * 8 + hd;
+    float fw[NWARP];                                                    // 0 for a warp that saw no token
+    {
+      float M = red_m[hd];
+#pragma unroll
+      for (int w = 1; w < NWARP; ++w) M = fmaxf(M, red_m[w * 8 + hd]);
+#pragma unroll
+      for (int w = 0; w < NWARP; ++w) fw[w] = (br == 0 && M > -INFINITY) ? ex2(red_m[w * 8 + hd] - M) : (br == 0 ? 0.f : 1.f);
+    }
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
     for (int w = 0; w < NWARP; ++w) {
       const float4 a = *reinterpret_cast<const float4*>(red_o + ((size_t)w * 16 + rr) * (D + kPad) + c4);
-      s.x += a.x; s.y += a.y; s.z += a.z; s.w += a.w;
+      s.x += a.x * fw[w]; s.y += a.y * fw[w]; s.z += a.z * fw[w]; s.w += a.w * fw[w];
       if (PACK && br == 1) {                                              // the second and third parts of the coefficients
         const float4 b2 = *reinterpret_cast<const float4*>(red_o + ((size_t)w * 16 + rr + 4) * (D + kPad) + c4);
         const float4 b3 = *reinterpret_cast<const float4*>(red_o + ((size_t)w * 16 + hd + 4) * (D + kPad) + c4);
@@ -429,7 +439,7 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
 #pragma unroll
     for (int w = 1; w < NWARP; ++w) Mg = fmaxf(Mg, red_m[w * 8 + tid]);
 #pragma unroll
-    for (int w = 0; w < NWARP; ++w) Lg += red_l[w * 8 + tid];
+    for (int w = 0; w < NWARP; ++w) Lg += Mg > -INFINITY ? red_l[w * 8 + tid] * ex2(red_m[w * 8 + tid] - Mg) : 0.f;
     mine_ml[tid * 2] = Mg;
     mine_ml[tid * 2 + 1] = Lg;
   }
@@ -491,7 +501,8 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
     if (col < D) {
       const size_t oidx = ((size_t)b * p.Hq + (size_t)h * G + hd) * D + col;
       float res = o_sp;
-      if (rla) res += rms_weight[((size_t)h * G + hd) * D + col] * r_ * rsqrtf(tot / D + p.rms_eps);
+      const float gamma = hd == rank ? gamma0 : rms_weight[((size_t)h * G + hd) * D + col];
+      if (rla) res += gamma * r_ * rsqrtf(tot / D + p.rms_eps);
       out[oidx] = res;
       if (dbg_sparse) dbg_sparse[oidx] = o_sp;
       if (dbg_rla) dbg_rla[oidx] = r_;

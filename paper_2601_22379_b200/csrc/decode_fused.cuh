@@ -30,9 +30,11 @@ __global__ void __launch_bounds__(256, 2)
                         float* __restrict__ dbg_sparse, float* __restrict__ dbg_rla, int* __restrict__ sel_user, int pending_new) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   __shared__ __align__(16) int sel_share[kMaxTopK + 2];   // the unit's selection, its size, the length: phase 1 leaves them here
+  __shared__ __align__(8) uint64_t tile_full[kMaxSlots];   // the attend phase's tile barriers
   if (threadIdx.x == 0) {                   // the K/V tensor maps are needed late: have them fetched now
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
+    for (int s = 0; s < kMaxSlots; ++s) mbar_init(&tile_full[s], 1);   // (phase 1's initialisation fence, same thread, covers them)
   }
   score_cluster_body<D, GP, WIN, EARLY, ST, 8>(p, q, 1, sel_user, pending_new, smem_raw, sel_share);
   if ((threadIdx.x >> 5) < 4) {
@@ -43,9 +45,10 @@ __global__ void __launch_bounds__(256, 2)
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("bar.sync 1, 128;" ::: "memory");
     warpgroup_reg_inc<232>();
-    attend_mma_body<D, (GP <= 4), 1, true>(p, map_k, map_v, q, rms_weight, out, dbg_sparse, dbg_rla, smem_raw, sel_share);
+    attend_mma_body<D, (GP <= 4), 1, true>(p, map_k, map_v, q, rms_weight, out, dbg_sparse, dbg_rla, smem_raw, sel_share, tile_full);
   } else {
     warpgroup_reg_dec<24>();
+    if (blockIdx.x == 0) write_selection(p, blockIdx.y, sel_share, -1, sel_user, (int)threadIdx.x - 128);
     __threadfence();       // the o_bar partials went to global memory: performed device-wide before the barrier releases them
     cluster_sync_all();    // the two cluster barriers of phase 2 count every thread of the cluster
     cluster_sync_all();

@@ -126,6 +126,32 @@ struct Smem {
 // On return the selection of the unit is in p.sel / p.n_sel (and sel_user), written by the cluster's first CTA, and the
 // o_bar partials are in p.obar_part or on their way there (warps 4-7 return on their own, without a barrier with the
 // selecting warps 0-3); every thread of every CTA of the cluster returns (nobody has left the kernel).
+// The picks of a unit, held best first in shared memory (`picks`, padded to a multiple of four with entries that precede
+// nothing), go to the workspace and the caller's array in ascending order.  Run by warps 4-7 of the unit's first CTA
+// (`t` = 0 .. 127), which first wait for warps 0-3 to announce the list on named barrier 3.  k_eff < 0: the count
+// follows the list, at picks[kMaxTopK].
+__device__ __forceinline__ void write_selection(const Params& p, int u, const int* picks, int k_eff, int* __restrict__ sel_user,
+                                                int t) {
+  asm volatile("bar.sync 3, 256;" ::: "memory");
+  if (k_eff < 0) k_eff = picks[kMaxTopK];
+  int* sel_u = p.sel + (size_t)u * p.top_k;
+  int* sel_o = sel_user ? sel_user + (size_t)u * p.top_k : nullptr;
+  for (int s = t; s < p.top_k; s += 128) {
+    int pos = s, ia = -1;
+    if (s < k_eff) {
+      ia = picks[s];
+      pos = 0;
+      for (int j = 0; j < k_eff; j += 4) {
+        const int4 ii = *reinterpret_cast<const int4*>(picks + j);
+        pos += (ii.x < ia) + (ii.y < ia) + (ii.z < ia) + (ii.w < ia);
+      }
+    }
+    sel_u[pos] = ia;
+    if (sel_o) sel_o[pos] = ia;
+  }
+  if (t == 0) p.n_sel[u] = k_eff;
+}
+
 template <int D, int GP, bool WIN, bool EARLY, typename ST, int NWP>
 // `sel_share` (fused kernel only, else null): a shared-memory array of kMaxTopK + 2 ints; warps 0-3 of every CTA leave
 // the selection there, in ascending order, followed by the count and the length, and have met on a barrier since.
@@ -174,6 +200,7 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
     else { for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kCsConsumers); } }
     mbar_init(pbar, 1);
     mbar_init(kbar, 1);
+    mbar_init_done();
     err_s = 0;
   }
   cluster_arrive();                             // the siblings may store here once everybody's barriers exist: completed before the first exchange
@@ -564,7 +591,7 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
   }
   // (fused decode kernel: TMA tiles will overwrite the ring area; what all eight warps did there is ordered before
   // those copies here, the barrier passes the order on)
-  if (sel_share) asm volatile("fence.proxy.async;" ::: "memory");
+  if (sel_share) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncthreads();
   cluster_wait();                               // every CTA of the cluster has its barriers in place (announced at the top)
 
@@ -572,13 +599,21 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
   // stores that count their bytes on the receiver's barrier: a CTA goes on as soon as all partials have reached it,
   // without a barrier of the whole cluster.  (All partials here also means: every CTA is done with its ring.)
   const bool key_dest = sel_share || rank == 0;   // a kernel of its own: only the first CTA selects
-  if (tid < G) {
+  if (warp == 0) {
+    // lane w * GP + g takes the pair of warp w and head g; the warps of a head are folded with shuffles (32 / GP >= 8
+    // warps fit a pass for groups of up to four heads, else two passes); lanes 0 .. G - 1 then send head `lane`
     float m = -INFINITY, s = 0.f;
+    for (int e = lane; e < kCsConsumers * GP; e += 32) lse_merge(m, s, wred[e * 2], wred[e * 2 + 1]);
 #pragma unroll
-    for (int w = 0; w < kCsConsumers; ++w) lse_merge(m, s, wred[(w * GP + tid) * 2], wred[(w * GP + tid) * 2 + 1]);
-    const uint32_t mine = smem_u32(all_part + ((size_t)rank * GP + tid) * 2), bar = smem_u32(pbar);
-    for (int r = 0; r < CS; ++r)
-      st_async_v2(map_to_rank(mine, (uint32_t)r), __float_as_uint(m), __float_as_uint(s), map_to_rank(bar, (uint32_t)r));
+    for (int o = GP; o < 32; o <<= 1) {
+      const float m2 = __shfl_xor_sync(0xffffffffu, m, o), s2 = __shfl_xor_sync(0xffffffffu, s, o);
+      lse_merge(m, s, m2, s2);
+    }
+    if (lane < G) {
+      const uint32_t mine = smem_u32(all_part + ((size_t)rank * GP + lane) * 2), bar = smem_u32(pbar);
+      for (int r = 0; r < CS; ++r)
+        st_async_v2(map_to_rank(mine, (uint32_t)r), __float_as_uint(m), __float_as_uint(s), map_to_rank(bar, (uint32_t)r));
+    }
   }
   const int nblk_pad = min(nblk, CS * chunk);
   if (tid == 32) {
@@ -604,28 +639,8 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
         if (s != rank) asm volatile("bar.sync 2, 128;" ::: "memory");   // (the slices of one CTA reuse the same scratch)
         state_role<D, GP, 128>(p, u, s, q_raw, q_is_bf16, reinterpret_cast<float*>(smem_raw + SM::kStateScratch), tid - 128, 2);
       }
-    if (rank == 0) {
-      asm volatile("bar.sync 3, 256;" ::: "memory");                    // warps 0-3 have the picks
-      int* sel_u = p.sel + (size_t)u * p.top_k;
-      int* sel_o = sel_user ? sel_user + (size_t)u * p.top_k : nullptr;
-      for (int s = tid - 128; s < p.top_k; s += 128) {
-        if (s < k_eff) {
-          const int ia = sel_tmp[s];
-          int pos = 0;
-#pragma unroll 4
-          for (int j = 0; j < k_eff; j += 4) {                          // (padded with entries that precede nothing)
-            const int4 ii = *reinterpret_cast<const int4*>(sel_tmp + j);
-            pos += (ii.x < ia) + (ii.y < ia) + (ii.z < ia) + (ii.w < ia);
-          }
-          sel_u[pos] = ia;
-          if (sel_o) sel_o[pos] = ia;
-        } else {
-          sel_u[s] = -1;
-          if (sel_o) sel_o[s] = -1;
-        }
-      }
-      if (tid == 128) p.n_sel[u] = k_eff;
-    }
+    // (the fused decode kernel calls this itself, once these warps have given their registers to the others)
+    if (rank == 0 && !sel_share) write_selection(p, u, sel_tmp, k_eff, sel_user, tid - 128);
     if (!sel_share) cluster_wait();
     return;
   }
@@ -699,21 +714,22 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
     sel_tmp[s] = v;
   }
   for (int s = tid; s < SM::kFlatCap + 4; s += 128) flat[s] = 0ull;
-  if (tid == 0 && sel_share) { sel_share[kMaxTopK] = k_eff; sel_share[kMaxTopK + 1] = L; }
+  if (tid == 0) {
+    reinterpret_cast<TopkScratch*>(smem_raw + SM::kScratch)->n_small = 0;   // (the survivor count)
+    if (sel_share) { sel_share[kMaxTopK] = k_eff; sel_share[kMaxTopK + 1] = L; }
+  }
 
   if (!mbar_wait(kbar, 0, p.wait_limit) && lane == 0) atomicExch(p.status, kStatusTimeout);   // ---- all keys are here
 
   // ------------------------------------------------------------------ phase C (warps 0-3) -------------------
   // Top k_eff of the unit's n blocks.  The forced blocks (the first n_sink, the last n_local) are known from their
-  // indices; `need` free blocks remain to be picked.  Thread t looks at the free blocks t, t + 128, ...; every pair of
-  // threads notes the best key it sees; the need-th best of these 64 is a lower bound of the need-th best key overall
-  // (they are 64 different blocks), and with evenly spread keys little more than `need` keys reach it.  The survivors
+  // indices; `need` free blocks remain to be picked.  The need-th best of 64 sampled maxima is a lower bound of the
+  // need-th best key overall (they belong to different blocks), and little more than `need` keys reach it.  The survivors
   // are ranked by counting, as 64-bit words (key, complement of the index) that one comparison orders; the picks stay
   // in that order (best first, then the forced blocks): every CTA computes the same list, and the attention does not
   // care.  Where too many survive (equal scores) or the sequence has more than 128 x 64 blocks, the histogram selection
   // runs over the whole table instead and its picks are put in ascending order.
   if (k_eff < n && need > 0) {
-    uint32_t* pair_max = reinterpret_cast<uint32_t*>(smem_raw + SM::kLaneMax);
     TopkScratch* scratch = reinterpret_cast<TopkScratch*>(smem_raw + SM::kScratch);
     int* n_surv = &scratch->n_small;
     uint32_t* bound_s = &scratch->lo;
@@ -723,17 +739,18 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
     const int my_n = n_free > tid ? (n_free - tid + 127) / 128 : 0;   // ... of this thread
     int total = SM::kFlatCap + 1;
     if (nr <= 64) {
+      // Thread t looks at the free blocks t, t + 128, ... (spread over the whole sequence, whatever its structure);
+      // every pair of threads notes the best key it sees, made unique and comparable in one go: the low six bits give
+      // way to the pair's number (rounding the key down keeps the bound a lower bound).
+      uint32_t* pair_max = reinterpret_cast<uint32_t*>(smem_raw + SM::kLaneMax);
       uint32_t mx = 0u;
 #pragma unroll 8
       for (int r = 0; r < my_n; ++r) mx = max(mx, my_keys[128 * r]);
       mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-      // made unique and comparable in one go: the low six bits give way to the pair's number (rounding the key down
-      // keeps the bound a lower bound)
       const int pr = tid >> 1, half = tid & 1;
       const uint32_t mine = (mx & ~63u) | (uint32_t)(63 - pr);
       if (!half) pair_max[pr] = mine;
-      if (tid == 0) *n_surv = 0;
-      selg.sync();
+      selg.sync();                                // (also: the survivor count was cleared before the keys came)
       {
         int rk = 0;                               // rank of this pair's best key among the 64, half of them per thread
 #pragma unroll
@@ -776,7 +793,7 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
       // P = 4, 2 or 1 neighbouring lanes share a candidate and a part of the table each (broadcast 128-bit loads; the
       // empty entries behind the survivors precede nothing)
       const int lg = total <= 32 ? 2 : total <= 64 ? 1 : 0, P = 1 << lg;
-      const int span = ((total + P - 1) / P + 1) & ~1;                // entries per part, even
+      const int span = (((total + P - 1) >> lg) + 1) & ~1;            // entries per part, even
       for (int c0 = 0; c0 < total; c0 += 128 >> lg) {
         const int c = c0 + (tid >> lg), part = tid & (P - 1);
         const unsigned long long a = c < total ? flat[c] : ~0ull;

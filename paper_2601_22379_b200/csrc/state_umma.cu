@@ -136,6 +136,7 @@ __global__ void __launch_bounds__(kSuThreads, 1)
   if (tid == 0) {
     for (int s = 0; s < kSuStages; ++s) { mbar_init(&full[s], 1); mbar_init(&ready[s], kSuTransformWarps / 2); mbar_init(&empty[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], kSuTransformWarps); }
+    mbar_init_done();
     abort_s = 0;
   }
   if (warp == 1) {                                       // tensor memory for the 128 x 128 fp32 accumulator
