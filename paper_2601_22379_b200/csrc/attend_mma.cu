@@ -12,12 +12,9 @@ __global__ void __launch_bounds__(NG * kAttendThreads, NG == 1 ? 2 : 1)
   attend_mma_body<D, PACK, NG, false>(p, map_k, map_v, q, rms_weight, out, dbg_sparse, dbg_rla, smem_raw);
 }
 
-// Dynamic shared memory of the kernel: the two-slot tile ring, reused for the cross-warp fold.
-size_t attend_mma_smem_bytes(int B, int D, int groups) {
-  const size_t ring = (size_t)(2 * groups) * ((2 * (size_t)B * D * 2 + (size_t)B * 4 + 1023) / 1024 * 1024);
-  const size_t fold = (size_t)(groups * (kAttendThreads / 32) * (16 * (D + kPad) + 16) + 2 * 8 * D + 16) * sizeof(float);
-  return ring > fold ? ring : fold;
-}
+// Dynamic shared memory of the kernel: the two-slot tile ring, reused for the cross-warp fold, and the receive area of
+// the merge behind it.
+size_t attend_mma_smem_bytes(int B, int D, int groups) { return attend_mma_ring_bytes(B, D, groups) + attend_mma_recv_bytes(D); }
 
 template <int D, bool PACK, int NG>
 static cudaError_t launch_shape(const Params& p, const AttendMaps& maps, const void* q, const float* w, float* out, float* ds,

@@ -19,9 +19,11 @@
 // product with V as three bf16 parts.  For groups of up to 4 heads the
 // extra parts ride in the accumulator rows that would otherwise be padding.
 //
-// Merge (Eq. rla-impl-3, Section 3.3): after a hardware cluster barrier CTA g of the cluster pulls head g's
-// partial results from its siblings over distributed shared memory, subtracts o_tilde from o_bar, applies the
-// RMSNorm and writes the output.  The only waits are two cluster barriers and bounded mbarrier polls.
+// Merge (Eq. rla-impl-3, Section 3.3): every CTA sends its partial results of head g into CTA g % CS of the cluster as
+// asynchronous stores (st.async) that count their bytes on a barrier there; that CTA goes on when all of them have
+// arrived, subtracts o_tilde from o_bar, applies the RMSNorm and writes the output.  No barrier of the whole cluster
+// lies on the path (one closes the kernel: nobody leaves while a sibling may still store into it); all waits are
+// bounded mbarrier polls or CTA barriers.
 //
 // The body is a device function: it is the whole of the attend + merge kernel (spla_decode_selected, and spla_decode
 // where the fused kernel does not apply) and the second half of the fused decode kernel (decode_fused.cuh), where it
@@ -75,6 +77,14 @@ __device__ __forceinline__ float bf16_hi(uint32_t x) { return __uint_as_float(x 
 
 constexpr int kPad = 8;   // floats of padding per row of the cross-warp reduction buffer
 
+// Bytes of the tile ring (reused for the cross-warp fold); as a kernel of its own the receive area of the merge follows.
+__host__ __device__ constexpr size_t attend_mma_ring_bytes(int B, int D, int groups) {
+  const size_t ring = (size_t)(2 * groups) * ((2 * (size_t)B * D * 2 + (size_t)B * 4 + 1023) / 1024 * 1024);
+  const size_t fold = (size_t)(groups * (kAttendThreads / 32) * (16 * (D + kPad) + 16)) * sizeof(float);
+  return (ring > fold ? ring : fold);
+}
+constexpr size_t attend_mma_recv_bytes(int D) { return (size_t)16 * (2 * D + 2) * 4; }
+
 }  // namespace
 
 // PACK: the group has at most 4 heads, so accumulator rows 4..7 and 12..15 are padding; rows 12..15 then carry
@@ -84,14 +94,16 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
                                                 const __nv_bfloat16* __restrict__ q, const float* __restrict__ rms_weight,
                                                 float* __restrict__ out, float* __restrict__ dbg_sparse,
                                                 float* __restrict__ dbg_rla, unsigned char* smem_raw,
-                                                const int* sel_share = nullptr, uint64_t* full_ext = nullptr) {
+                                                const int* sel_share = nullptr, uint64_t* full_ext = nullptr,
+                                                unsigned char* recv_raw = nullptr, const float* obar_local = nullptr) {
   constexpr int KS = D / 16;        // k-steps of the two QK-type products
   constexpr int NT = D / 8;         // n-tiles of the PV-type product
   constexpr int NH = D / 64;        // 64-column halves of a tile (one TMA box each)
   constexpr int NTHR = NG * kAttendThreads;
   constexpr int NWARP = NTHR / 32;
-  __shared__ __align__(8) uint64_t full_own[kMaxSlots];
-  uint64_t* full = full_ext ? full_ext : full_own;      // (the fused kernel initialises its tile barriers at its start)
+  __shared__ __align__(8) uint64_t full_own[kMaxSlots + 1];
+  uint64_t* full = full_ext ? full_ext : full_own;      // (the fused kernel initialises its barriers at its start)
+  uint64_t* mbar_merge = full + kMaxSlots;              // completes when every sibling's partial results have arrived here
   __shared__ float red_s[NWARP];
   __shared__ int sel_s[kMaxTopK];
   __shared__ int err_s;
@@ -175,11 +187,14 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
   if constexpr (!FUSED) make_fragments();
   if (tid == 0) {
     if (!full_ext) {
-      for (int s = 0; s < kMaxSlots; ++s) mbar_init(&full[s], 1);
+      for (int s = 0; s <= kMaxSlots; ++s) mbar_init(&full[s], 1);
       mbar_init_done();
     }
     err_s = 0;
   }
+  // As a kernel of its own: the siblings may store here once everybody's merge barrier exists; announced now,
+  // completed before the first such store.  (In the fused kernel the score phase has done that.)
+  if constexpr (!FUSED) cluster_arrive();
 
   if constexpr (!FUSED) pdl_wait();             // the selection of this step is complete and visible from here on
 
@@ -396,8 +411,15 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
   float* red_o = reinterpret_cast<float*>(smem_raw);                    // [NWARP][16][D + kPad]
   float* red_m = red_o + NWARP * 16 * (D + kPad);                       // [NWARP][8]
   float* red_l = red_m + NWARP * 8;                                     // [NWARP][8]
-  float* mine = red_l + NWARP * 8;                                      // [2][8][D]   this CTA's partial result
-  float* mine_ml = mine + 2 * 8 * D;                                    // [8][2]      (max, sum) of the exact branch
+  // Where the partial results of head hd go: into the CTA that merges it, hd % CS, entry (hd / CS) * CS + sender of
+  // its receive area (at most 16 entries: [2][D] floats each, then the (max, sum) pairs), as asynchronous stores that
+  // count their bytes on that CTA's merge barrier.
+  constexpr int kRecvEntries = 16;
+  float* recv = recv_raw ? reinterpret_cast<float*>(recv_raw)
+                         : reinterpret_cast<float*>(smem_raw + attend_mma_ring_bytes(B, D, NG));   // [16][2][D], [16][2]
+  float* recv_ml = recv + kRecvEntries * 2 * D;
+  const int my_heads = G > rank ? (G - rank + CS - 1) / CS : 0;         // heads this CTA merges
+  if (tid == 0 && my_heads > 0) mbar_expect_tx(mbar_merge, (uint32_t)(my_heads * CS * (2 * D * 4 + 8)));
   // every warp leaves its rows as they are, with its running maximum and sum; the combiner rescales (one barrier less
   // than agreeing on the maximum first)
   if (t == 0) { red_m[warp * 8 + g] = m_run; red_l[warp * 8 + g] = l_run; }
@@ -410,6 +432,8 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
     }
   }
   cta_sync();
+  if constexpr (!FUSED) cluster_wait();         // (every CTA's merge barrier exists: announced at the top)
+  const uint32_t recv0 = smem_u32(recv), recv_ml0 = smem_u32(recv_ml), bar0 = smem_u32(mbar_merge);
   for (int idx = tid; idx < 2 * G * (D / 4); idx += NTHR) {             // four columns per thread and step
     const int br = idx / (G * (D / 4)), hd = (idx / (D / 4)) % G, c4 = (idx % (D / 4)) * 4;   // branch, head, first column
     const int rr = br * 8 + hd;
@@ -432,83 +456,89 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
         s.x += b2.x + b3.x; s.y += b2.y + b3.y; s.z += b2.z + b3.z; s.w += b2.w + b3.w;
       }
     }
-    *reinterpret_cast<float4*>(mine + (size_t)rr * D + c4) = s;
+    const uint32_t dest = (uint32_t)(hd % CS);
+    const int entry = (hd / CS) * CS + rank;
+    st_async_v4(map_to_rank(recv0 + (uint32_t)(((entry * 2 + br) * D + c4) * 4), dest), s.x, s.y, s.z, s.w,
+                map_to_rank(bar0, dest));
   }
-  if (tid < 8) {
+  if (tid < G) {
     float Mg = red_m[tid], Lg = 0.f;
 #pragma unroll
     for (int w = 1; w < NWARP; ++w) Mg = fmaxf(Mg, red_m[w * 8 + tid]);
 #pragma unroll
     for (int w = 0; w < NWARP; ++w) Lg += Mg > -INFINITY ? red_l[w * 8 + tid] * ex2(red_m[w * 8 + tid] - Mg) : 0.f;
-    mine_ml[tid * 2] = Mg;
-    mine_ml[tid * 2 + 1] = Lg;
+    const uint32_t dest = (uint32_t)(tid % CS);
+    const int entry = (tid / CS) * CS + rank;
+    st_async_v2(map_to_rank(recv_ml0 + (uint32_t)(entry * 8), dest), __float_as_uint(Mg), __float_as_uint(Lg),
+                map_to_rank(bar0, dest));
   }
-
-  cluster_sync_all();                                // ---- every CTA's partial result is in its shared memory
 
   // ---- merge: CTA r of the cluster owns heads r, r + CS, ...; one thread per output column ---------------
   const int nblk_u = (L + B - 1) / B;
   const bool rla = rla_on && nsel < nblk_u;          // everything selected: the residual is exactly zero
-  for (int hd = rank; hd < G; hd += CS) {
-    const int col = tid;
-    float o_sp = 0.f, o_til = 0.f, o_bar = 0.f;
-    if (nsel > 0) {
-      // every load is issued before the first is used: the o_bar partials from global memory, then the siblings'
-      // partial results over distributed shared memory (one round trip instead of one per sibling)
-      float ob[kStateSplits];
+  if (my_heads > 0) {
+    // as a kernel of its own o_bar comes from the workspace (written by the preceding kernel): requested before the wait
+    float ob0[kStateSplits];
 #pragma unroll
-      for (int s = 0; s < kStateSplits; ++s)
-        ob[s] = (rla && col < D) ? __ldcg(p.obar_part + (((size_t)u * kStateSplits + s) * G + hd) * D + col) : 0.f;
-      constexpr int kMaxCS = 16;
-      float mr[kMaxCS], lr[kMaxCS], osp[kMaxCS], otl[kMaxCS];
-#pragma unroll
-      for (int r = 0; r < kMaxCS; ++r) {
-        mr[r] = -INFINITY; lr[r] = 0.f; osp[r] = 0.f; otl[r] = 0.f;
-        if (r < CS) {
-          const uint32_t rm = map_to_rank(smem_u32(mine_ml + hd * 2), (uint32_t)r);
-          mr[r] = ld_dsmem_f32(rm);
-          lr[r] = ld_dsmem_f32(rm + 4);
+    for (int s = 0; s < kStateSplits; ++s)
+      ob0[s] = (!FUSED && rla && tid < D) ? __ldcg(p.obar_part + (((size_t)u * kStateSplits + s) * G + rank) * D + tid) : 0.f;
+    if (!__all_sync(0xffffffffu, mbar_wait(mbar_merge, 0, p.wait_limit)) && lane == 0) atomicExch(p.status, kStatusTimeout);
+    if constexpr (FUSED) asm volatile("bar.sync 2, 256;" ::: "memory");   // warps 4-7 have left o_bar of this CTA's heads
+    for (int hd = rank, hi = 0; hd < G; hd += CS, ++hi) {
+      const int col = tid;
+      float o_sp = 0.f, o_til = 0.f, o_bar = 0.f;
+      if (nsel > 0) {
+        const float* e_ml = recv_ml + (size_t)hi * CS * 2;
+        const float* e_o = recv + (size_t)hi * CS * 2 * D;
+        float Mx = -INFINITY;
+        for (int r = 0; r < CS; ++r) Mx = fmaxf(Mx, e_ml[r * 2]);
+        float Ls = 0.f;
+        for (int r = 0; r < CS; ++r) {
+          const float w = ex2(e_ml[r * 2] - Mx);
+          Ls = fmaf(w, e_ml[r * 2 + 1], Ls);
           if (col < D) {
-            osp[r] = ld_dsmem_f32(map_to_rank(smem_u32(mine + hd * D + col), (uint32_t)r));
-            if (rla) otl[r] = ld_dsmem_f32(map_to_rank(smem_u32(mine + (8 + hd) * D + col), (uint32_t)r));
+            o_sp = fmaf(w, e_o[(size_t)(r * 2) * D + col], o_sp);
+            if (rla) o_til += e_o[(size_t)(r * 2 + 1) * D + col];
+          }
+        }
+        o_sp /= Ls;
+        if (rla && col < D) {
+          if constexpr (FUSED) {
+            o_bar = obar_local[(size_t)hi * D + col];
+          } else if (hi == 0) {
+#pragma unroll
+            for (int s = 0; s < kStateSplits; ++s) o_bar += ob0[s];
+          } else {
+#pragma unroll
+            for (int s = 0; s < kStateSplits; ++s)
+              o_bar += __ldcg(p.obar_part + (((size_t)u * kStateSplits + s) * G + hd) * D + col);
           }
         }
       }
-      float Mx = -INFINITY;
+      const float r_ = (rla && col < D) ? o_bar - o_til : 0.f;
+      float sq = warp_sum(r_ * r_);
+      cta_sync();
+      if (lane == 0) red_s[warp] = sq;
+      cta_sync();
+      float tot = 0.f;
 #pragma unroll
-      for (int r = 0; r < kMaxCS; ++r) Mx = fmaxf(Mx, mr[r]);
-      float Ls = 0.f;
-#pragma unroll
-      for (int r = 0; r < kMaxCS; ++r)
-        if (r < CS) {
-          const float w = ex2(mr[r] - Mx);
-          Ls = fmaf(w, lr[r], Ls);
-          o_sp = fmaf(w, osp[r], o_sp);
-          o_til += otl[r];
-        }
-      o_sp /= Ls;
-#pragma unroll
-      for (int s = 0; s < kStateSplits; ++s) o_bar += ob[s];
+      for (int w = 0; w < NWARP; ++w) tot += red_s[w];
+      if (col < D) {
+        const size_t oidx = ((size_t)b * p.Hq + (size_t)h * G + hd) * D + col;
+        float res = o_sp;
+        const float gamma = hd == rank ? gamma0 : rms_weight[((size_t)h * G + hd) * D + col];
+        if (rla) res += gamma * r_ * rsqrtf(tot / D + p.rms_eps);
+        out[oidx] = res;
+        if (dbg_sparse) dbg_sparse[oidx] = o_sp;
+        if (dbg_rla) dbg_rla[oidx] = r_;
+      }
     }
-    const float r_ = (rla && col < D) ? o_bar - o_til : 0.f;
-    float sq = warp_sum(r_ * r_);
-    cta_sync();
-    if (lane == 0) red_s[warp] = sq;
-    cta_sync();
-    float tot = 0.f;
-#pragma unroll
-    for (int w = 0; w < NWARP; ++w) tot += red_s[w];
-    if (col < D) {
-      const size_t oidx = ((size_t)b * p.Hq + (size_t)h * G + hd) * D + col;
-      float res = o_sp;
-      const float gamma = hd == rank ? gamma0 : rms_weight[((size_t)h * G + hd) * D + col];
-      if (rla) res += gamma * r_ * rsqrtf(tot / D + p.rms_eps);
-      out[oidx] = res;
-      if (dbg_sparse) dbg_sparse[oidx] = o_sp;
-      if (dbg_rla) dbg_rla[oidx] = r_;
-    }
+  } else if constexpr (FUSED) {
+    asm volatile("bar.sync 2, 256;" ::: "memory");   // (the barrier with warps 4-7 counts every thread)
   }
-  cluster_sync_all();                                // ---- nobody leaves while a sibling may still read its memory
+  // ---- the closing barrier: nobody leaves while a sibling may still store into it; and the CTAs of a cluster leave
+  // together (when some left earlier than others, the next launch's clusters no longer all found room at once)
+  cluster_sync_all();
 }
 
 }  // namespace spla

@@ -30,13 +30,15 @@ __global__ void __launch_bounds__(256, 2)
                         float* __restrict__ dbg_sparse, float* __restrict__ dbg_rla, int* __restrict__ sel_user, int pending_new) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   __shared__ __align__(16) int sel_share[kMaxTopK + 2];   // the unit's selection, its size, the length: phase 1 leaves them here
-  __shared__ __align__(8) uint64_t tile_full[kMaxSlots];   // the attend phase's tile barriers
+  __shared__ __align__(8) uint64_t tile_full[kMaxSlots + 1];   // the attend phase's tile barriers and its merge barrier
+  // o_bar of the heads this CTA merges (at most 8 x D floats): behind the working space of the role that computes it
+  float* obar_s = reinterpret_cast<float*>(smem_raw + Smem<D, GP, ST, 8>::kStateScratch + 2048);
   if (threadIdx.x == 0) {                   // the K/V tensor maps are needed late: have them fetched now
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
-    for (int s = 0; s < kMaxSlots; ++s) mbar_init(&tile_full[s], 1);   // (phase 1's initialisation fence, same thread, covers them)
+    for (int s = 0; s <= kMaxSlots; ++s) mbar_init(&tile_full[s], 1);  // (phase 1's initialisation fence, same thread, covers them)
   }
-  score_cluster_body<D, GP, WIN, EARLY, ST, 8>(p, q, 1, sel_user, pending_new, smem_raw, sel_share);
+  score_cluster_body<D, GP, WIN, EARLY, ST, 8>(p, q, 1, sel_user, pending_new, smem_raw, sel_share, obar_s);
   if ((threadIdx.x >> 5) < 4) {
     // Phase 2's tiles arrive through the asynchronous proxy (TMA) in shared memory that these warps have just read and
     // written through the generic proxy (the key table, the selection's work arrays): each of them orders its accesses
@@ -45,13 +47,16 @@ __global__ void __launch_bounds__(256, 2)
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("bar.sync 1, 128;" ::: "memory");
     warpgroup_reg_inc<232>();
-    attend_mma_body<D, (GP <= 4), 1, true>(p, map_k, map_v, q, rms_weight, out, dbg_sparse, dbg_rla, smem_raw, sel_share, tile_full);
+    attend_mma_body<D, (GP <= 4), 1, true>(p, map_k, map_v, q, rms_weight, out, dbg_sparse, dbg_rla, smem_raw, sel_share, tile_full,
+                                           smem_raw + Smem<D, GP, ST, 8>::kMergeRecv, obar_s);
   } else {
     warpgroup_reg_dec<24>();
+    if (threadIdx.x == 128) {               // the tiles are a microsecond or two away: have the tensor maps at hand again
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
+    }
     if (blockIdx.x == 0) write_selection(p, blockIdx.y, sel_share, -1, sel_user, (int)threadIdx.x - 128);
-    __threadfence();       // the o_bar partials went to global memory: performed device-wide before the barrier releases them
-    cluster_sync_all();    // the two cluster barriers of phase 2 count every thread of the cluster
-    cluster_sync_all();
+    cluster_sync_all();    // the closing barrier of phase 2 counts every thread of the cluster
   }
 }
 
@@ -61,7 +66,7 @@ static cudaError_t fused_launch_win(const Params& p, const AttendMaps& maps, con
   using SM = Smem<D, GP, ST, 8>;
   const int U = p.batch * p.Hkv;
   size_t smem = (size_t)SM::kEll + (size_t)p.G * p.chunk * sizeof(float);
-  const size_t smem_attend = attend_mma_smem_bytes(p.B, D, 1);
+  const size_t smem_attend = attend_mma_ring_bytes(p.B, D, 1);     // (the merge's receive area lies in phase 1's layout)
   if (smem_attend > smem) smem = smem_attend;
   auto kern = decode_fused_kernel<D, GP, WIN, EARLY, ST>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

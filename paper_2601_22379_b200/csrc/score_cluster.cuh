@@ -95,13 +95,16 @@ struct Smem {
   static constexpr int kWorkEnd = (kScratch + (int)sizeof(TopkScratch) + 1023) / 1024 * 1024;
   // ... followed by the scratch of the o_bar role, which runs beside the selection
   static constexpr int kStateScratch = kWorkEnd;                    // float [GP * D + (128 / D) * GP * D]
-  static constexpr int kStateBytes = (GP * D + (128 / D > 0 ? 128 / D : 1) * GP * D) * 4;
+  static constexpr int kStateBytes0 = (GP * D + (128 / D > 0 ? 128 / D : 1) * GP * D) * 4;
+  static constexpr int kStateBytes = kStateBytes0 > 2048 + 8 * D * 4 ? kStateBytes0 : 2048 + 8 * D * 4;   // (fused kernel: 2 KB of working space, then o_bar of up to 8 heads)
   static constexpr int kAreaEnd = (kStateScratch + kStateBytes + 1023) / 1024 * 1024;
   // The ring area is padded to hold all of that.  The fused decode kernel relies on it too: its attend phase lays the
   // K/V tile ring (at most 66 KB) over this area, and the tile copies must stay clear of the fixed region below, which
   // holds this phase's mbarrier objects (never invalidated: overwriting them with tile data corrupted value rows, found
   // with NaN-filled memory), and of the o_bar scratch, which may still be in use when the first tiles arrive.
-  static constexpr int kRingBytes = kStreamBytes > kAreaEnd ? kStreamBytes : kAreaEnd;
+  static constexpr int kMergeRecv = kAreaEnd;                       // the attend phase's receive area (fused kernel)
+  static constexpr int kMergeRecvBytes = (16 * (2 * D + 2) * 4 + 1023) / 1024 * 1024;
+  static constexpr int kRingBytes = kStreamBytes > kMergeRecv + kMergeRecvBytes ? kStreamBytes : kMergeRecv + kMergeRecvBytes;
   static_assert(kStateScratch >= 68 * 1024, "the attend phase's tile ring must end below the o_bar scratch");
   // fixed region after the ring:
   static constexpr int kPart = kRingBytes;                          // float [GP][2]  this CTA's (max, sum)
@@ -154,10 +157,11 @@ __device__ __forceinline__ void write_selection(const Params& p, int u, const in
 
 template <int D, int GP, bool WIN, bool EARLY, typename ST, int NWP>
 // `sel_share` (fused kernel only, else null): a shared-memory array of kMaxTopK + 2 ints; warps 0-3 of every CTA leave
-// the selection there, in ascending order, followed by the count and the length, and have met on a barrier since.
+// the selection there, best block first, followed by the count and the length, and have met on a barrier since.
+// `obar_local` (fused kernel only, else null): shared memory for o_bar of the heads this CTA merges, [heads][D].
 __device__ __forceinline__ void score_cluster_body(const Params& p, const void* __restrict__ q_raw, int q_is_bf16,
                                                    int* __restrict__ sel_user, int pending_new, unsigned char* smem_raw,
-                                                   int* sel_share = nullptr) {
+                                                   int* sel_share = nullptr, float* obar_local = nullptr) {
   using SM = Smem<D, GP, ST, NWP>;
   constexpr int kCsConsumers = NWP;             // warps; all consume, lane 0 of warp 0 also feeds the ring
   constexpr int kCsThreads = NWP * 32;
@@ -634,11 +638,19 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
     // Warps 4-7: o_bar = phi(q) S_bar (one slice of the state's rows per CTA) beside the scoring and the selection;
     // then, in the first CTA, the selection in ascending order for the workspace and the caller.
     if (!sel_share) cluster_arrive();             // (closing barrier of the kernel of its own, see below: these warps send nothing)
-    if (rla)
+    if (rla && obar_local) {
+      // fused decode kernel: this CTA will merge heads rank, rank + CS, ... and computes their o_bar in full, into its
+      // own shared memory
+      for (int hd = rank, i = 0; hd < G; hd += CS, ++i)
+        state_head<D, 128>(p, u, hd, q_raw, q_is_bf16, obar_local + (size_t)i * D,
+                           reinterpret_cast<float*>(smem_raw + SM::kStateScratch), tid - 128, 2);
+    } else if (rla) {
       for (int s = rank; s < kStateSplits; s += CS) {
         if (s != rank) asm volatile("bar.sync 2, 128;" ::: "memory");   // (the slices of one CTA reuse the same scratch)
         state_role<D, GP, 128>(p, u, s, q_raw, q_is_bf16, reinterpret_cast<float*>(smem_raw + SM::kStateScratch), tid - 128, 2);
       }
+    }
+    if (obar_local) asm volatile("bar.arrive 2, 256;" ::: "memory");   // o_bar of this CTA's heads is in place (warps 0-3 wait there before the merge)
     // (the fused decode kernel calls this itself, once these warps have given their registers to the others)
     if (rank == 0 && !sel_share) write_selection(p, u, sel_tmp, k_eff, sel_user, tid - 128);
     if (!sel_share) cluster_wait();

@@ -189,6 +189,11 @@ __device__ __forceinline__ void st_async_v2(uint32_t addr, uint32_t a, uint32_t 
                "r"(b), "r"(bar)
                : "memory");
 }
+__device__ __forceinline__ void st_async_v4(uint32_t addr, float a, float b, float c, float d, uint32_t bar) {   // 16 bytes, 16-byte aligned
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(addr),
+               "f"(a), "f"(b), "f"(c), "f"(d), "r"(bar)
+               : "memory");
+}
 // the two halves of the same barrier, for warps that have work to do between announcing and needing it (.aligned:
 // executed by whole warps)
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }

@@ -82,4 +82,65 @@ __device__ __forceinline__ void state_role(const Params& p, int u, int s, const 
   }
 }
 
+// o_bar of ONE query head over all rows of the state, left in shared memory (`obar`, D floats): the fused decode
+// kernel's form, where the CTA that merges a head computes that head's o_bar itself, so that it neither travels nor has
+// to be made visible to another CTA.  NT threads with local numbers `tid` meet on the named barrier `bar_id`.
+// smem: (D + (NT / D) * D) floats.
+template <int D, int NT>
+__device__ __forceinline__ void state_head(const Params& p, int u, int head, const void* __restrict__ q_raw, int q_is_bf16,
+                                           float* __restrict__ obar, float* smem, const int tid, const int bar_id) {
+  auto meet = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(NT) : "memory"); };
+  constexpr int VEC = D / 32;
+  constexpr int RG = NT / D;                             // row groups working side by side
+  constexpr int ROWS = D / RG;                           // rows per thread
+  constexpr int RB = ROWS < 32 ? ROWS : 32;              // rows in flight per thread (the role is latency-bound: few, deep batches)
+  const int lane = tid & 31, warp = tid >> 5;
+  const int b = u / p.Hkv, h = u % p.Hkv;
+  float* phiq = smem;                                    // [D]
+  float* red = phiq + D;                                 // [RG][D]
+  const int rg = tid / D, j = tid % D;
+  const float* S = p.state + (size_t)u * D * D + (size_t)rg * D + j;
+  float sv[RB];
+#pragma unroll
+  for (int r = 0; r < RB; ++r) sv[r] = __ldcs(S + (size_t)r * RG * D);       // in flight while phi(q) is formed
+  if (warp == 0) {
+    const float a2 = p.phi_scale * kLog2e;
+    float x[VEC];
+    const size_t qoff = ((size_t)b * p.Hq + (size_t)h * p.G + head) * D + lane * VEC;
+    if (q_is_bf16) load_vec<VEC>(reinterpret_cast<const __nv_bfloat16*>(q_raw) + qoff, x);
+    else load_vec<VEC>(reinterpret_cast<const float*>(q_raw) + qoff, x);
+    float mx = -INFINITY;
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) { x[v] *= a2; mx = fmaxf(mx, x[v]); }
+    mx = warp_max(mx);
+    float sum = 0.f;
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) { x[v] = exp2f(x[v] - mx); sum += x[v]; }
+    sum = warp_sum(sum);
+    const float inv = 1.f / sum;
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) phiq[lane * VEC + v] = x[v] * inv;
+  }
+  meet();
+  float acc = 0.f;
+#pragma unroll 1
+  for (int r0 = 0; r0 < ROWS; r0 += RB) {
+    if (r0 > 0) {
+#pragma unroll
+      for (int r = 0; r < RB; ++r) sv[r] = __ldcs(S + (size_t)(r0 + r) * RG * D);
+    }
+#pragma unroll
+    for (int r = 0; r < RB; ++r) acc = fmaf(phiq[rg + (r0 + r) * RG], sv[r], acc);
+  }
+  red[rg * D + j] = acc;
+  meet();
+  if (tid < D) {
+    float t = 0.f;
+#pragma unroll
+    for (int r2 = 0; r2 < RG; ++r2) t += red[r2 * D + tid];
+    obar[tid] = t;
+  }
+  meet();                                                // (the scratch may be reused)
+}
+
 }  // namespace spla
