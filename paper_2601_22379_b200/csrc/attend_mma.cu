@@ -19,7 +19,7 @@ size_t attend_mma_smem_bytes(int B, int D, int groups) { return attend_mma_ring_
 template <int D, bool PACK, int NG>
 static cudaError_t launch_shape(const Params& p, const AttendMaps& maps, const void* q, const float* w, float* out, float* ds,
                                 float* dr, cudaStream_t stream, int* occupancy) {
-  const size_t smem = attend_mma_smem_bytes(p.B, D, NG);
+  const size_t smem = attend_mma_smem_bytes(p.tile_rows, D, NG);
   const dim3 grid(p.acs, p.batch * p.Hkv);
   auto kern = attend_mma_kernel<D, PACK, NG>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -115,6 +115,7 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
   const int gi = warp >> 2, wg = warp & 3, gtid = tid & (kAttendThreads - 1);   // group, warp in group, thread in group
   const int g = lane >> 2, t = lane & 3;
   const int G = p.G, B = p.B;
+  const int TB = p.tile_rows, TPB = B / TB;   // rows of a K/V tile, tiles per block (blocks of 128 tokens at d = 128 come as two tiles)
   const bool rla_on = !(p.flags & 4u);
   constexpr int ns = 2 * NG;                    // ring positions in use (a multiple of NG: a group refills what it frees)
   auto cta_sync = [&]() {                      // barrier over the threads that run this body
@@ -220,26 +221,28 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
   }
   cta_sync();                              // selection list and barrier initialisation visible to the CTA
 
-  const int nb = nsel > rank ? (nsel - rank + CS - 1) / CS : 0;     // my blocks: j = rank + i * CS
-  const int tile_bytes = B * D * 2;
-  const int slot_bytes = (2 * tile_bytes + B * 4 + 1023) & ~1023;   // K tile, V tile, per-token lse; the swizzle needs 1 KB alignment
+  const int n_tiles = nsel * TPB;                                    // tile j: part j % TPB of pick j / TPB
+  const int nb = n_tiles > rank ? (n_tiles - rank + CS - 1) / CS : 0;   // my tiles: j = rank + i * CS
+  const int tile_bytes = TB * D * 2;
+  const int slot_bytes = (2 * tile_bytes + TB * 4 + 1023) & ~1023;  // K tile, V tile, per-token lse; the swizzle needs 1 KB alignment
   // The copies of tile i of this CTA (K and V in 64-column halves, the tokens' log-sum-exp): `part` < 0 issues all of
   // them from one thread; otherwise the caller spreads the parts 0 .. kTileParts - 1 over lanes (part 0 also announces
   // the bytes; the barrier's transaction count may run ahead of that announcement).
   constexpr int kTileParts = 2 * NH + 1;
   auto issue = [&](int i, int part = -1) {
     const int slot = i % ns;
-    const int blk = min(max(sel_s[rank + i * CS], 0), p.max_blocks - 1);   // (a list entry can never address outside the cache)
+    const int j = rank + i * CS;
+    const int blk = min(max(sel_s[j / TPB], 0), p.max_blocks - 1);   // (a list entry can never address outside the cache)
     const uint32_t base = smem_u32(smem_raw + (size_t)slot * slot_bytes);
-    const int row0 = (int)(((size_t)u * p.max_blocks + blk) * B);
-    if (part <= 0) mbar_expect_tx(&full[slot], (uint32_t)(2 * tile_bytes + B * 4 + p.dbg_tx_extra));
+    const int row0 = (int)(((size_t)u * p.max_blocks + blk) * B) + (j % TPB) * TB;
+    if (part <= 0) mbar_expect_tx(&full[slot], (uint32_t)(2 * tile_bytes + TB * 4 + p.dbg_tx_extra));
 #pragma unroll
     for (int hh = 0; hh < NH; ++hh) {
-      if (part < 0 || part == 2 * hh) tma_load_2d(base + hh * (B * 128), &map_k, hh * 64, row0, &full[slot]);
-      if (part < 0 || part == 2 * hh + 1) tma_load_2d(base + tile_bytes + hh * (B * 128), &map_v, hh * 64, row0, &full[slot]);
+      if (part < 0 || part == 2 * hh) tma_load_2d(base + hh * (TB * 128), &map_k, hh * 64, row0, &full[slot]);
+      if (part < 0 || part == 2 * hh + 1) tma_load_2d(base + tile_bytes + hh * (TB * 128), &map_v, hh * 64, row0, &full[slot]);
     }
     if (part < 0 || part == 2 * NH)
-      bulk_g2s(smem_raw + (size_t)slot * slot_bytes + 2 * tile_bytes, p.tok_lse + (size_t)row0, (uint32_t)(B * 4), &full[slot]);
+      bulk_g2s(smem_raw + (size_t)slot * slot_bytes + 2 * tile_bytes, p.tok_lse + (size_t)row0, (uint32_t)(TB * 4), &full[slot]);
   };
   if (tid < ns * kTileParts && tid / kTileParts < nb) issue(tid / kTileParts, tid % kTileParts);   // the first tiles, one copy per lane
   if constexpr (FUSED) {
@@ -254,9 +257,9 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
   for (int nt = 0; nt < NT; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
   const float sc2 = p.sm_scale * kLog2e;
   const float a2 = p.phi_scale * kLog2e;
-  const int spb = B / 16;                    // slices per block
+  const int spb = TB / 16;                   // slices per tile
   const int mi = lane >> 3, r8 = lane & 7;   // ldmatrix: which 8x8 matrix this lane addresses, and which row
-  const int half_bytes = B * 128;
+  const int half_bytes = TB * 128;
 
   // A wait that runs out marks the warp dead: it skips the arithmetic from then on but still joins every barrier of
   // its group, so that the barrier counts match whatever the other warps saw.
@@ -272,12 +275,13 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
     const uint32_t ks = smem_u32(sb);
     const uint32_t vs = ks + tile_bytes;
     const float* lse_s = reinterpret_cast<const float*>(sb + 2 * tile_bytes);
-    const int blk = sel_s[rank + i * CS];
-    const int ntok = min(B, L - blk * B);
-    if (ntok < B) {
+    const int jt = rank + i * CS;
+    const int blk = sel_s[jt / TPB];
+    const int ntok = max(0, min(TB, L - blk * B - (jt % TPB) * TB));   // (0: a tile of the open block wholly past the end)
+    if (ntok < TB) {
       // the open block of the sequence: rows past its end hold whatever the cache memory holds; the value rows
       // must be zero so that (probability 0) x (garbage) cannot produce a NaN
-      for (int idx = gtid; idx < (B - ntok) * (D / 8) && !dead; idx += kAttendThreads) {
+      for (int idx = gtid; idx < (TB - ntok) * (D / 8) && !dead; idx += kAttendThreads) {
         const int row = ntok + idx / (D / 8), ch = idx % (D / 8);
         *reinterpret_cast<uint4*>(sb + tile_bytes + (ch >> 3) * half_bytes + row * 128 + (((ch & 7) ^ (row & 7)) << 4)) =
             make_uint4(0u, 0u, 0u, 0u);
@@ -416,7 +420,7 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
   // count their bytes on that CTA's merge barrier.
   constexpr int kRecvEntries = 16;
   float* recv = recv_raw ? reinterpret_cast<float*>(recv_raw)
-                         : reinterpret_cast<float*>(smem_raw + attend_mma_ring_bytes(B, D, NG));   // [16][2][D], [16][2]
+                         : reinterpret_cast<float*>(smem_raw + attend_mma_ring_bytes(TB, D, NG));  // [16][2][D], [16][2]
   float* recv_ml = recv + kRecvEntries * 2 * D;
   const int my_heads = G > rank ? (G - rank + CS - 1) / CS : 0;         // heads this CTA merges
   if (tid == 0 && my_heads > 0) mbar_expect_tx(mbar_merge, (uint32_t)(my_heads * CS * (2 * D * 4 + 8)));

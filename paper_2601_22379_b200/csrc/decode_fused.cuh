@@ -66,7 +66,7 @@ static cudaError_t fused_launch_win(const Params& p, const AttendMaps& maps, con
   using SM = Smem<D, GP, ST, 8>;
   const int U = p.batch * p.Hkv;
   size_t smem = (size_t)SM::kEll + (size_t)p.G * p.chunk * sizeof(float);
-  const size_t smem_attend = attend_mma_ring_bytes(p.B, D, 1);     // (the merge's receive area lies in phase 1's layout)
+  const size_t smem_attend = attend_mma_ring_bytes(p.tile_rows, D, 1);     // (the merge's receive area lies in phase 1's layout)
   if (smem_attend > smem) smem = smem_attend;
   auto kern = decode_fused_kernel<D, GP, WIN, EARLY, ST>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

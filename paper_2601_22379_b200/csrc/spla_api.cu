@@ -196,13 +196,15 @@ extern "C" int spla_init_cache(const spla_config_t* config, const spla_buffers_t
   p.state_part = (float*)(ws + w.state_part); p.state_ticket = (int*)(ws + w.state_ticket);
   p.status = (int*)(ws + w.status);
   p.max_chunks = w.max_chunks;
+  p.tile_rows = (p.B * p.d * 2 > 16384 && p.B % 32 == 0) ? p.B / 2 : p.B;
   p.acs = 0;
 
   c->maps.valid = false;
   c->state_maps.valid = false;
   if (p.kv_bf16) {
     const unsigned long long rows = (unsigned long long)p.batch * p.Hkv * p.max_blocks * p.B;
-    c->maps.valid = make_kv_map(c->maps.k, b->k_cache, p.d, p.B, rows) && make_kv_map(c->maps.v, b->v_cache, p.d, p.B, rows);
+    c->maps.valid = make_kv_map(c->maps.k, b->k_cache, p.d, p.tile_rows, rows) &&
+                    make_kv_map(c->maps.v, b->v_cache, p.d, p.tile_rows, rows);
     c->state_maps.valid = p.d == 128 && rows >= 64 && rows < (1ull << 31) && !(config->flags & SPLA_GENERAL_KERNELS) &&
                           make_kv_map(c->state_maps.k, b->k_cache, p.d, 64, rows) &&
                           make_kv_map(c->state_maps.v, b->v_cache, p.d, 64, rows);
@@ -300,7 +302,7 @@ static void plan_score_grid(spla_cache* c, Params* p, bool fused = false) {
 // phase is built for) whenever the cluster score plan exists.
 static bool fused_eligible(const spla_cache* c) {
   return !(c->cfg.flags & SPLA_GENERAL_KERNELS) && c->p.kv_bf16 && c->cfg.q_dtype == SPLA_BF16 &&
-         c->p.G <= 8 && c->maps.valid && attend_mma_smem_bytes(c->p.B, c->p.d, 1) + 4096 <= (size_t)113 * 1024;
+         c->p.G <= 8 && c->maps.valid && attend_mma_smem_bytes(c->p.tile_rows, c->p.d, 1) + 4096 <= (size_t)113 * 1024;
 }
 
 
@@ -315,7 +317,7 @@ static void plan_attend(spla_cache* c, Params* p) {
   p->acs = 0;
   if (c->cfg.flags & SPLA_GENERAL_KERNELS) return;
   const long long U = (long long)c->p.batch * c->p.Hkv;
-  const size_t smem = attend_mma_smem_bytes(c->p.B, c->p.d, 1) + 2048;
+  const size_t smem = attend_mma_smem_bytes(c->p.tile_rows, c->p.d, 1) + 2048;
   long long per_sm = (227 * 1024) / (long long)smem;
   if (per_sm > 2) per_sm = 2;                     // the kernel is compiled for two CTAs per SM (no register spills)
   if (per_sm < 1) return;                         // the tiles do not fit: use the general kernel

@@ -37,6 +37,7 @@ struct Params {
   int n_chunks_cap;                     // score-kernel chunks launched per unit
   int chunk;                            // block records per score CTA
   int cs;                               // score kernel, cluster edition: CTAs per unit (0 = general kernel)
+  int tile_rows;                        // tensor-core attend: rows of a K/V tile (the block size, or half of it where a block exceeds 16 KB)
   int acs;                              // tensor-core attend kernel: CTAs (cluster size) per unit
   // caller buffers
   void* k_cache;
