@@ -79,8 +79,8 @@ struct Smem {
   static constexpr int kStageRec = NWP * kRecPerWarp;              // statistics records per ring stage
   static constexpr int kRecBytes = 2 * D * (int)sizeof(ST);        // ST: element type of the statistics records
   static constexpr int kStageBytes = kStageRec * kRecBytes;
-  // tensor-core streaming (groups of up to four heads): the ring is cut into slots of 16 records, one MMA tile each
-  static constexpr bool kMma = GP <= 4 && sizeof(ST) == 2;         // 16-bit records, groups of up to four heads
+  // tensor-core streaming (16-bit records): the ring is cut into slots of 16 records, one MMA row tile each
+  static constexpr bool kMma = sizeof(ST) == 2;
   static constexpr int kSlotBytes = kSlotRec * kRecBytes;
   static constexpr int kSlots = NWP;                               // one ring position per warp
   static constexpr int kStreamBytes = kMma ? kSlots * kSlotBytes : kStages * kStageBytes;
@@ -219,49 +219,53 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
   const int hl = lane % W, grp = lane / W;
   constexpr int CW = VECW >= 4 ? 4 : VECW;      // floats per vector load
   constexpr int NC = VECW / CW;
-  // Tensor-core streaming (16-bit records, groups of up to four heads): a slot of 16 records is the A operand of
-  // mma.m16n8k16 (16 x d, row-major, as stored), the B operand's eight columns are the group's scaled queries, each
-  // split in two bf16 parts, bf16(q) and bf16(q - bf16(q)) (column n: head n / 2, part n % 2), whose products are
+  // Tensor-core streaming (16-bit records): a slot of 16 records is the A operand of mma.m16n8k16 (16 x d, row-major,
+  // as stored), the B operand's eight columns are four heads' scaled queries, each split in two bf16 parts, bf16(q) and
+  // bf16(q - bf16(q)) (column n: head n / 2, part n % 2; a second column tile serves heads 4..7), whose products are
   // added after the MMA: the query enters with 16 significant bits, the statistics exactly, the sums are fp32.
   // Thread (g8, t4) owns 16 consecutive bytes of every 64 of a record half (mean or variance), which it fetches with
   // one 128-bit load per row; the k index inside an MMA is a permutation of the channels, the same for A and B.
   constexpr bool MMA = SM::kMma;
   constexpr int NJ = D * (int)sizeof(ST) / 64;   // 16-byte chunks per thread and record half
   const int g8 = lane >> 2, t4 = lane & 3;
-  uint32_t bq[MMA ? NJ : 1][4], bv[MMA ? NJ : 1][4];
+  constexpr int NT2 = GP > 4 ? 2 : 1;            // column tiles of eight: four heads x two query parts each
+  uint32_t bq[MMA ? NT2 : 1][MMA ? NJ : 1][4], bv[MMA ? NT2 : 1][MMA ? NJ : 1][4];
   float qm[GP][VECW], qv[GP][VECW];
   if constexpr (MMA) {
-    const int head = g8 >> 1, part = g8 & 1;
 #pragma unroll
-    for (int j = 0; j < NJ; ++j) {
-      float x[8];                                // channels 32 j + 8 t4 .. + 7
-      if (head < G) {
-        const size_t qoff = ((size_t)b * p.Hq + (size_t)h * G + head) * D + (size_t)j * 32 + t4 * 8;
+    for (int nt = 0; nt < NT2; ++nt) {
+      const int head = nt * 4 + (g8 >> 1), part = g8 & 1;
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          float y[4];
-          if (q_is_bf16) load_vec<4>(reinterpret_cast<const __nv_bfloat16*>(q_raw) + qoff + c * 4, y);
-          else load_vec<4>(reinterpret_cast<const float*>(q_raw) + qoff + c * 4, y);
+      for (int j = 0; j < NJ; ++j) {
+        float x[8];                                // channels 32 j + 8 t4 .. + 7
+        if (head < G) {
+          const size_t qoff = ((size_t)b * p.Hq + (size_t)h * G + head) * D + (size_t)j * 32 + t4 * 8;
 #pragma unroll
-          for (int v = 0; v < 4; ++v) x[c * 4 + v] = y[v];
+          for (int c = 0; c < 2; ++c) {
+            float y[4];
+            if (q_is_bf16) load_vec<4>(reinterpret_cast<const __nv_bfloat16*>(q_raw) + qoff + c * 4, y);
+            else load_vec<4>(reinterpret_cast<const float*>(q_raw) + qoff + c * 4, y);
+#pragma unroll
+            for (int v = 0; v < 4; ++v) x[c * 4 + v] = y[v];
+          }
+        } else {
+#pragma unroll
+          for (int v = 0; v < 8; ++v) x[v] = 0.f;
         }
-      } else {
+        float qa[8], qb2[8];                       // this thread's part of q_hat and of q_hat^2 / 2
 #pragma unroll
-        for (int v = 0; v < 8; ++v) x[v] = 0.f;
-      }
-      float qa[8], qb2[8];                       // this thread's part of q_hat and of q_hat^2 / 2
+        for (int v = 0; v < 8; ++v) {
+          const float qh = x[v] * p.sm_scale;
+          const float qq = (p.flags & 2u) ? 0.f : 0.5f * qh * qh;
+          const float h1 = __bfloat162float(__float2bfloat16_rn(qh)), h2 = __bfloat162float(__float2bfloat16_rn(qq));
+          qa[v] = part ? qh - h1 : h1;
+          qb2[v] = part ? qq - h2 : h2;
+        }
 #pragma unroll
-      for (int v = 0; v < 8; ++v) {
-        const float qh = x[v] * p.sm_scale;
-        const float qq = (p.flags & 2u) ? 0.f : 0.5f * qh * qh;
-        const float h1 = __bfloat162float(__float2bfloat16_rn(qh)), h2 = __bfloat162float(__float2bfloat16_rn(qq));
-        qa[v] = part ? qh - h1 : h1;
-        qb2[v] = part ? qq - h2 : h2;
-      }
-#pragma unroll
-      for (int v = 0; v < 4; ++v) {
-        bq[j][v] = pack_bf16(qa[2 * v], qa[2 * v + 1]);
-        bv[j][v] = pack_bf16(qb2[2 * v], qb2[2 * v + 1]);
+        for (int v = 0; v < 4; ++v) {
+          bq[nt][j][v] = pack_bf16(qa[2 * v], qa[2 * v + 1]);
+          bv[nt][j][v] = pack_bf16(qb2[2 * v], qb2[2 * v + 1]);
+        }
       }
     }
   }
@@ -360,12 +364,15 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
     const float ln_win = logf((float)p.win_C);
     const unsigned nw_magic = 0xffffffffu / (unsigned)NW + 1u;   // floor(x / NW) = umulhi(x, magic) for x < 2^16, NW <= 8
     float run_max = -INFINITY, run_sum = 0.f;
+    float run_max2 = -INFINITY, run_sum2 = 0.f;  // (tensor-core path, groups of more than four heads: head 4 + t4)
 
-    // Tensor-core path: one slot of 16 records -> dots of head t4 with records g8 and g8 + 8 of the slot -> log
-    // masses.  `li0` is the CTA-local index of the slot's first record, `limit` the number of local records that
-    // exist for this call.  Rows past the limit hold stale bytes; every row is independent and theirs are dropped.
+    // Tensor-core path: one slot of 16 records -> dots of heads t4 (and 4 + t4) with records g8 and g8 + 8 of the
+    // slot -> log masses.  `li0` is the CTA-local index of the slot's first record, `limit` the number of local records
+    // that exist for this call.  Rows past the limit hold stale bytes; every row is independent and theirs are dropped.
     auto consume_slot = [&](const unsigned char* slot, int li0, int limit) {
-      float cm[4] = {0.f, 0.f, 0.f, 0.f}, cv[4] = {0.f, 0.f, 0.f, 0.f};
+      float cm[NT2][4], cv[NT2][4];
+#pragma unroll
+      for (int nt = 0; nt < NT2; ++nt) { cm[nt][0] = cm[nt][1] = cm[nt][2] = cm[nt][3] = 0.f; cv[nt][0] = cv[nt][1] = cv[nt][2] = cv[nt][3] = 0.f; }
       const unsigned char* r0 = slot + (size_t)g8 * SM::kRecBytes + t4 * 16;
       const unsigned char* r1 = r0 + 8 * SM::kRecBytes;
       constexpr int HALF = SM::kRecBytes / 2;                      // the variance follows the mean
@@ -373,33 +380,42 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
       for (int j = 0; j < (MMA ? NJ : 0); ++j) {
         const uint4 m0 = *reinterpret_cast<const uint4*>(r0 + j * 64), m1 = *reinterpret_cast<const uint4*>(r1 + j * 64);
         const uint4 v0 = *reinterpret_cast<const uint4*>(r0 + HALF + j * 64), v1 = *reinterpret_cast<const uint4*>(r1 + HALF + j * 64);
-        mma_bf16(cm, m0.x, m1.x, m0.y, m1.y, bq[j][0], bq[j][1]);
-        mma_bf16(cv, v0.x, v1.x, v0.y, v1.y, bv[j][0], bv[j][1]);
-        mma_bf16(cm, m0.z, m1.z, m0.w, m1.w, bq[j][2], bq[j][3]);
-        mma_bf16(cv, v0.z, v1.z, v0.w, v1.w, bv[j][2], bv[j][3]);
-      }
-      // columns 2 t4 and 2 t4 + 1 are the two query parts of head t4
 #pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-        const float dm = cm[2 * hf] + cm[2 * hf + 1], dv = cv[2 * hf] + cv[2 * hf + 1];
-        const int li = li0 + g8 + 8 * hf;
-        if (t4 < G && li < limit) {
-          if (!WIN) {
-            const float ell = (rec_begin + li == nblk_fin - 1 ? ln_last : ln_full) + dm + __logf(1.f + dv);
-            ell_s[t4 * chunk + li] = ell;
-            const float nm = fmaxf(run_max, ell);
-            run_sum = run_sum * __expf(run_max - nm) + __expf(ell - nm);
-            run_max = nm;
-          } else {
-            // strided windows (Section 3.1, "Strided Block Selection"): log mass of window w of a block,
-            // max-pooled into the block's slot right away through an order-preserving integer key
-            const int lb = (int)__umulhi((unsigned)li, nw_magic), w = li - lb * NW;   // li / NW without a division
-            float ln_n = ln_win;
-            if (cta_blk0 + lb == nblk_fin - 1) {
-              const int cnt = min(p.win_C, n_last - w * p.win_s);
-              ln_n = cnt > 0 ? logf((float)cnt) : -INFINITY;
+        for (int nt = 0; nt < (MMA ? NT2 : 0); ++nt) {
+          mma_bf16(cm[nt], m0.x, m1.x, m0.y, m1.y, bq[nt][j][0], bq[nt][j][1]);
+          mma_bf16(cv[nt], v0.x, v1.x, v0.y, v1.y, bv[nt][j][0], bv[nt][j][1]);
+          mma_bf16(cm[nt], m0.z, m1.z, m0.w, m1.w, bq[nt][j][2], bq[nt][j][3]);
+          mma_bf16(cv[nt], v0.z, v1.z, v0.w, v1.w, bv[nt][j][2], bv[nt][j][3]);
+        }
+      }
+      // columns 2 t4 and 2 t4 + 1 of column tile nt are the two query parts of head 4 nt + t4
+#pragma unroll
+      for (int nt = 0; nt < NT2; ++nt) {
+        const int hd = nt * 4 + t4;
+        float& rmax = nt == 0 ? run_max : run_max2;
+        float& rsum = nt == 0 ? run_sum : run_sum2;
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          const float dm = cm[nt][2 * hf] + cm[nt][2 * hf + 1], dv = cv[nt][2 * hf] + cv[nt][2 * hf + 1];
+          const int li = li0 + g8 + 8 * hf;
+          if (hd < G && li < limit) {
+            if (!WIN) {
+              const float ell = (rec_begin + li == nblk_fin - 1 ? ln_last : ln_full) + dm + __logf(1.f + dv);
+              ell_s[hd * chunk + li] = ell;
+              const float nm = fmaxf(rmax, ell);
+              rsum = rsum * __expf(rmax - nm) + __expf(ell - nm);
+              rmax = nm;
+            } else {
+              // strided windows (Section 3.1, "Strided Block Selection"): log mass of window w of a block,
+              // max-pooled into the block's slot right away through an order-preserving integer key
+              const int lb = (int)__umulhi((unsigned)li, nw_magic), w = li - lb * NW;   // li / NW without a division
+              float ln_n = ln_win;
+              if (cta_blk0 + lb == nblk_fin - 1) {
+                const int cnt = min(p.win_C, n_last - w * p.win_s);
+                ln_n = cnt > 0 ? logf((float)cnt) : -INFINITY;
+              }
+              atomicMax(reinterpret_cast<uint32_t*>(ell_s) + hd * chunk + lb, float_order_key(ln_n + dm + __logf(1.f + dv)));
             }
-            atomicMax(reinterpret_cast<uint32_t*>(ell_s) + t4 * chunk + lb, float_order_key(ln_n + dm + __logf(1.f + dv)));
           }
         }
       }
@@ -567,15 +583,25 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
       }
     }
     if constexpr (MMA) {
-      // lanes with the same t4 hold partial normalisers of head t4: fold over g8
+      // lanes with the same t4 hold partial normalisers of head t4 (and 4 + t4): fold over g8
 #pragma unroll
       for (int o = 4; o < 32; o <<= 1) {
         const float m2 = __shfl_xor_sync(0xffffffffu, run_max, o), s2 = __shfl_xor_sync(0xffffffffu, run_sum, o);
         lse_merge(run_max, run_sum, m2, s2);
+        if constexpr (NT2 == 2) {
+          const float m3 = __shfl_xor_sync(0xffffffffu, run_max2, o), s3 = __shfl_xor_sync(0xffffffffu, run_sum2, o);
+          lse_merge(run_max2, run_sum2, m3, s3);
+        }
       }
-      if (!WIN && lane < G) {
-        wred[(warp * GP + lane) * 2 + 0] = run_max;
-        wred[(warp * GP + lane) * 2 + 1] = run_sum;
+      if (!WIN && lane < 4) {
+        if (lane < G) {
+          wred[(warp * GP + lane) * 2 + 0] = run_max;
+          wred[(warp * GP + lane) * 2 + 1] = run_sum;
+        }
+        if (NT2 == 2 && 4 + lane < G) {
+          wred[(warp * GP + 4 + lane) * 2 + 0] = run_max2;
+          wred[(warp * GP + 4 + lane) * 2 + 1] = run_sum2;
+        }
       }
     }
     // fold the finalising lanes of a head: copy lanes (xor < LPV), then the record groups of the warp (xor W)

@@ -141,6 +141,13 @@ def test_bf16_statistics_long_128k_full_size_sampled_units():
     _stepped_full(synth.CONFIGS[2].scaled(n_steps=3), n_units=3, check_steps={0, 2}, flags=F16)
 
 
+@pytest.mark.parametrize("hq", [40, 64])
+def test_bf16_statistics_long_128k_full_size_groups_of_five_and_eight(hq):
+    """Groups of five (the paper's model) and eight heads at the full 128K context: the tensor-core score path with two
+    column tiles, inside the fused decode kernel."""
+    _stepped_full(synth.CONFIGS[2].scaled(n_q_heads=hq, n_steps=2), n_units=2, check_steps={0, 1}, flags=F16)
+
+
 def test_bf16_statistics_windows_long_128k_full_size_sampled_units():
     _stepped_full(synth.CONFIGS[2].scaled(n_steps=2), n_units=2, check_steps={1}, window=WIN, flags=F16)
 
