@@ -79,10 +79,11 @@ struct Smem {
   static constexpr int kStageRec = NWP * kRecPerWarp;              // statistics records per ring stage
   static constexpr int kRecBytes = 2 * D * (int)sizeof(ST);        // ST: element type of the statistics records
   static constexpr int kStageBytes = kStageRec * kRecBytes;
-  // tensor-core streaming (16-bit records): the ring is cut into slots of 16 records, one MMA row tile each
-  static constexpr bool kMma = sizeof(ST) == 2;
+  // tensor-core streaming (16-bit records; fp32 records for groups of more than four heads, where the FMA pipe cannot
+  // keep up): the ring is cut into slots of 16 records, one MMA row tile each
+  static constexpr bool kMma = sizeof(ST) == 2 || GP > 4;
   static constexpr int kSlotBytes = kSlotRec * kRecBytes;
-  static constexpr int kSlots = NWP;                               // one ring position per warp
+  static constexpr int kSlots = sizeof(ST) == 2 ? NWP : 6;         // one ring position per streaming warp (6 x 16 KB with fp32 records)
   static constexpr int kStreamBytes = kMma ? kSlots * kSlotBytes : kStages * kStageBytes;
   // after streaming the ring is dead and holds the selection's work arrays:
   static constexpr int kKeys = 0;                                   // uint32 [16 x 1024]   the keys of the whole unit, by block index
@@ -112,7 +113,7 @@ struct Smem {
   static constexpr int kLse = kAllPart + kMaxCluster * GP * 2 * 4;  // float [GP]
   static constexpr int kWred = kLse + GP * 4;                       // float [NWP][GP][2]
   static constexpr int kBars = (kWred + NWP * GP * 2 * 4 + 7) / 8 * 8;            // uint64: full / empty per stage, or one per slot
-  static constexpr int kRingBars = kMma ? NWP : 2 * kStages;
+  static constexpr int kRingBars = kMma ? kSlots : 2 * kStages;
   static constexpr int kNumBars = kRingBars + 2;                    // ... and one each for the two exchanges of the cluster
   static constexpr int kEll = (kBars + kNumBars * 8 + 15) / 16 * 16;               // float [G][chunk]
 };
@@ -226,10 +227,15 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
   // Thread (g8, t4) owns 16 consecutive bytes of every 64 of a record half (mean or variance), which it fetches with
   // one 128-bit load per row; the k index inside an MMA is a permutation of the channels, the same for A and B.
   constexpr bool MMA = SM::kMma;
+  // With fp32 records each element is split the same way, bf16(x) + bf16(x - bf16(x)) (16 significant bits, the
+  // rounding of the second part 2^-17 relative), and each part gets its own MMA against the same columns.
+  constexpr bool MMAF = MMA && sizeof(ST) == 4;
   constexpr int NJ = D * (int)sizeof(ST) / 64;   // 16-byte chunks per thread and record half
+  constexpr int CPC = 16 / (int)sizeof(ST);      // channels per chunk: 8 (two MMA k-steps) or 4 (one)
+  constexpr int BW = MMAF ? 2 : 4;               // B-fragment words per chunk
   const int g8 = lane >> 2, t4 = lane & 3;
   constexpr int NT2 = GP > 4 ? 2 : 1;            // column tiles of eight: four heads x two query parts each
-  uint32_t bq[MMA ? NT2 : 1][MMA ? NJ : 1][4], bv[MMA ? NT2 : 1][MMA ? NJ : 1][4];
+  uint32_t bq[MMA ? NT2 : 1][MMA ? NJ : 1][BW], bv[MMA ? NT2 : 1][MMA ? NJ : 1][BW];
   float qm[GP][VECW], qv[GP][VECW];
   if constexpr (MMA) {
 #pragma unroll
@@ -237,11 +243,11 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
       const int head = nt * 4 + (g8 >> 1), part = g8 & 1;
 #pragma unroll
       for (int j = 0; j < NJ; ++j) {
-        float x[8];                                // channels 32 j + 8 t4 .. + 7
+        float x[CPC];                              // channels j * 4 * CPC + t4 * CPC .. + CPC - 1
         if (head < G) {
-          const size_t qoff = ((size_t)b * p.Hq + (size_t)h * G + head) * D + (size_t)j * 32 + t4 * 8;
+          const size_t qoff = ((size_t)b * p.Hq + (size_t)h * G + head) * D + (size_t)j * 4 * CPC + t4 * CPC;
 #pragma unroll
-          for (int c = 0; c < 2; ++c) {
+          for (int c = 0; c < CPC / 4; ++c) {
             float y[4];
             if (q_is_bf16) load_vec<4>(reinterpret_cast<const __nv_bfloat16*>(q_raw) + qoff + c * 4, y);
             else load_vec<4>(reinterpret_cast<const float*>(q_raw) + qoff + c * 4, y);
@@ -250,11 +256,11 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
           }
         } else {
 #pragma unroll
-          for (int v = 0; v < 8; ++v) x[v] = 0.f;
+          for (int v = 0; v < CPC; ++v) x[v] = 0.f;
         }
-        float qa[8], qb2[8];                       // this thread's part of q_hat and of q_hat^2 / 2
+        float qa[CPC], qb2[CPC];                   // this thread's part of q_hat and of q_hat^2 / 2
 #pragma unroll
-        for (int v = 0; v < 8; ++v) {
+        for (int v = 0; v < CPC; ++v) {
           const float qh = x[v] * p.sm_scale;
           const float qq = (p.flags & 2u) ? 0.f : 0.5f * qh * qh;
           const float h1 = __bfloat162float(__float2bfloat16_rn(qh)), h2 = __bfloat162float(__float2bfloat16_rn(qq));
@@ -262,7 +268,7 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
           qb2[v] = part ? qq - h2 : h2;
         }
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
+        for (int v = 0; v < BW; ++v) {
           bq[nt][j][v] = pack_bf16(qa[2 * v], qa[2 * v + 1]);
           bv[nt][j][v] = pack_bf16(qb2[2 * v], qb2[2 * v + 1]);
         }
@@ -376,16 +382,39 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
       const unsigned char* r0 = slot + (size_t)g8 * SM::kRecBytes + t4 * 16;
       const unsigned char* r1 = r0 + 8 * SM::kRecBytes;
       constexpr int HALF = SM::kRecBytes / 2;                      // the variance follows the mean
+      if constexpr (MMA && !MMAF) {
 #pragma unroll
-      for (int j = 0; j < (MMA ? NJ : 0); ++j) {
-        const uint4 m0 = *reinterpret_cast<const uint4*>(r0 + j * 64), m1 = *reinterpret_cast<const uint4*>(r1 + j * 64);
-        const uint4 v0 = *reinterpret_cast<const uint4*>(r0 + HALF + j * 64), v1 = *reinterpret_cast<const uint4*>(r1 + HALF + j * 64);
+        for (int j = 0; j < NJ; ++j) {
+          const uint4 m0 = *reinterpret_cast<const uint4*>(r0 + j * 64), m1 = *reinterpret_cast<const uint4*>(r1 + j * 64);
+          const uint4 v0 = *reinterpret_cast<const uint4*>(r0 + HALF + j * 64), v1 = *reinterpret_cast<const uint4*>(r1 + HALF + j * 64);
 #pragma unroll
-        for (int nt = 0; nt < (MMA ? NT2 : 0); ++nt) {
-          mma_bf16(cm[nt], m0.x, m1.x, m0.y, m1.y, bq[nt][j][0], bq[nt][j][1]);
-          mma_bf16(cv[nt], v0.x, v1.x, v0.y, v1.y, bv[nt][j][0], bv[nt][j][1]);
-          mma_bf16(cm[nt], m0.z, m1.z, m0.w, m1.w, bq[nt][j][2], bq[nt][j][3]);
-          mma_bf16(cv[nt], v0.z, v1.z, v0.w, v1.w, bv[nt][j][2], bv[nt][j][3]);
+          for (int nt = 0; nt < NT2; ++nt) {
+            mma_bf16(cm[nt], m0.x, m1.x, m0.y, m1.y, bq[nt][j][0], bq[nt][j][1]);
+            mma_bf16(cv[nt], v0.x, v1.x, v0.y, v1.y, bv[nt][j][0], bv[nt][j][1]);
+            mma_bf16(cm[nt], m0.z, m1.z, m0.w, m1.w, bq[nt][j][2], bq[nt][j][3]);
+            mma_bf16(cv[nt], v0.z, v1.z, v0.w, v1.w, bv[nt][j][2], bv[nt][j][3]);
+          }
+        }
+      }
+      if constexpr (MMAF) {
+        // fp32 records: this thread's four channels of the chunk, rows g8 and g8 + 8, are the A fragment of one k-step
+        // (k indices 2 t4, 2 t4 + 1, 2 t4 + 8, 2 t4 + 9); first the mean, then the variance, each as two bf16 parts
+        auto split_mma = [&](const unsigned char* a_lo, const unsigned char* a_hi, float (&acc)[NT2][4], const uint32_t (&bf)[NT2][NJ][BW],
+                             int j) {
+          const float4 x0 = *reinterpret_cast<const float4*>(a_lo + j * 64), x1 = *reinterpret_cast<const float4*>(a_hi + j * 64);
+          const uint32_t h0 = pack_bf16(x0.x, x0.y), h1 = pack_bf16(x1.x, x1.y), h2 = pack_bf16(x0.z, x0.w), h3 = pack_bf16(x1.z, x1.w);
+          const uint32_t l0 = pack_bf16(x0.x - bf16_lo(h0), x0.y - bf16_hi(h0)), l1 = pack_bf16(x1.x - bf16_lo(h1), x1.y - bf16_hi(h1));
+          const uint32_t l2 = pack_bf16(x0.z - bf16_lo(h2), x0.w - bf16_hi(h2)), l3 = pack_bf16(x1.z - bf16_lo(h3), x1.w - bf16_hi(h3));
+#pragma unroll
+          for (int nt = 0; nt < NT2; ++nt) {
+            mma_bf16(acc[nt], h0, h1, h2, h3, bf[nt][j][0], bf[nt][j][1]);
+            mma_bf16(acc[nt], l0, l1, l2, l3, bf[nt][j][0], bf[nt][j][1]);
+          }
+        };
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) {
+          split_mma(r0, r1, cm, bq, j);
+          split_mma(r0 + HALF, r1 + HALF, cv, bv, j);
         }
       }
       // columns 2 t4 and 2 t4 + 1 of column tile nt are the two query parts of head 4 nt + t4
@@ -422,7 +451,7 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
     };
     if constexpr (MMA) {
 #pragma unroll 1
-      for (int r = warp; r < n_slots; r += SM::kSlots) {          // warp w owns ring position w
+      for (int r = warp; warp < SM::kSlots && r < n_slots; r += SM::kSlots) {   // warp w < kSlots owns ring position w
         const int pos = r % SM::kSlots;
         if (!mbar_wait(&full[pos], (r / SM::kSlots) & 1, p.wait_limit)) { if (lane == 0) atomicExch(&err_s, 1); break; }
         consume_slot(smem_raw + (size_t)pos * SM::kSlotBytes, r * kSlotRec, n_stream);

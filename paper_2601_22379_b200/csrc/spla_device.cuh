@@ -216,6 +216,10 @@ __device__ __forceinline__ void st_dsmem_v4(uint32_t addr, uint32_t a, uint32_t 
   asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
+// the two bf16 halves of a packed word, as floats
+__device__ __forceinline__ float bf16_lo(uint32_t x) { return __uint_as_float(x << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
+
 // ---- warp-level tensor-core product D += A B with fp32 accumulators (mma.m16n8k16, bf16 inputs) -------------------
 // Fragment layout (PTX ISA; g = lane / 4, t = lane % 4): A rows g and g + 8, B column g, D rows g and g + 8 at
 // columns 2t, 2t + 1.
