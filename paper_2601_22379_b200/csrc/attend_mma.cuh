@@ -42,10 +42,11 @@ namespace {
 
 constexpr int kMaxSlots = 4;       // ring positions at most (two per warp group)
 
-// Tiled TMA load of one box (never multicast): coordinates {x = element column, y = row}.
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-               "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+// Tiled TMA load of one K or V tile (never multicast): the map sees the cache as [column halves][rows][64 columns]; the
+// box starts at column 0 of `row` and takes every half.
+__device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* map, int row, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+               "l"(map), "r"(0), "r"(row), "r"(0), "r"(smem_u32(bar))
                : "memory");
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
@@ -96,7 +97,7 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
                                                 unsigned char* recv_raw = nullptr, const float* obar_local = nullptr) {
   constexpr int KS = D / 16;        // k-steps of the two QK-type products
   constexpr int NT = D / 8;         // n-tiles of the PV-type product
-  constexpr int NH = D / 64;        // 64-column halves of a tile (one TMA box each)
+  constexpr int NH = D / 64;        // 64-column halves of a tile
   constexpr int NTHR = NG * kAttendThreads;
   constexpr int NWARP = NTHR / 32;
   __shared__ __align__(8) uint64_t full_own[kMaxSlots + 1];
@@ -223,10 +224,10 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
   const int nb = n_tiles > rank ? (n_tiles - rank + CS - 1) / CS : 0;   // my tiles: j = rank + i * CS
   const int tile_bytes = TB * D * 2;
   const int slot_bytes = (2 * tile_bytes + TB * 4 + 1023) & ~1023;  // K tile, V tile, per-token lse; the swizzle needs 1 KB alignment
-  // The copies of tile i of this CTA (K and V in 64-column halves, the tokens' log-sum-exp): `part` < 0 issues all of
-  // them from one thread; otherwise the caller spreads the parts 0 .. kTileParts - 1 over lanes (part 0 also announces
-  // the bytes; the barrier's transaction count may run ahead of that announcement).
-  constexpr int kTileParts = 2 * NH + 1;
+  // The copies of tile i of this CTA (K, V, the tokens' log-sum-exp): `part` < 0 issues all of them from one thread;
+  // otherwise the caller spreads the parts 0 .. kTileParts - 1 over lanes (part 0 also announces the bytes; the
+  // barrier's transaction count may run ahead of that announcement).
+  constexpr int kTileParts = 3;
   auto issue = [&](int i, int part = -1) {
     const int slot = i % ns;
     const int j = rank + i * CS;
@@ -234,12 +235,9 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
     const uint32_t base = smem_u32(smem_raw + (size_t)slot * slot_bytes);
     const int row0 = (int)(((size_t)u * p.max_blocks + blk) * B) + (j % TPB) * TB;
     if (part <= 0) mbar_expect_tx(&full[slot], (uint32_t)(2 * tile_bytes + TB * 4 + p.dbg_tx_extra));
-#pragma unroll
-    for (int hh = 0; hh < NH; ++hh) {
-      if (part < 0 || part == 2 * hh) tma_load_2d(base + hh * (TB * 128), &map_k, hh * 64, row0, &full[slot]);
-      if (part < 0 || part == 2 * hh + 1) tma_load_2d(base + tile_bytes + hh * (TB * 128), &map_v, hh * 64, row0, &full[slot]);
-    }
-    if (part < 0 || part == 2 * NH)
+    if (part <= 0) tma_load_tile(base, &map_k, row0, &full[slot]);
+    if (part < 0 || part == 1) tma_load_tile(base + tile_bytes, &map_v, row0, &full[slot]);
+    if (part < 0 || part == 2)
       bulk_g2s(smem_raw + (size_t)slot * slot_bytes + 2 * tile_bytes, p.tok_lse + (size_t)row0, (uint32_t)(TB * 4), &full[slot]);
   };
   if (tid < ns * kTileParts && tid / kTileParts < nb) issue(tid / kTileParts, tid % kTileParts);   // the first tiles, one copy per lane

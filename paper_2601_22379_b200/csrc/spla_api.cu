@@ -45,22 +45,44 @@ static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // TMA tensor map over a K or V cache seen as a 2-D bf16 matrix [batch * H_kv * max_blocks * B rows][d columns]:
 // boxes of B rows x 64 columns (128 bytes, the widest the 128-byte swizzle allows).
-static bool make_kv_map(void* out128, void* base, int d, int B, unsigned long long rows) {
-  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-  static EncodeFn encode = nullptr;
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                      const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static TensorMapEncodeFn tensor_map_encoder() {
+  static TensorMapEncodeFn encode = nullptr;
   if (!encode) {
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult st;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &st) != cudaSuccess || !fn) return false;
-    encode = (EncodeFn)fn;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &st) != cudaSuccess || !fn) return nullptr;
+    encode = (TensorMapEncodeFn)fn;
   }
+  return encode;
+}
+
+// A K or V cache as a bf16 matrix [rows][d] with boxes of B rows x 64 columns (128-byte swizzle).
+static bool make_kv_map(void* out128, void* base, int d, int B, unsigned long long rows) {
+  TensorMapEncodeFn encode = tensor_map_encoder();
+  if (!encode) return false;
   const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)d * 2};
   const cuuint32_t box[2] = {64u, (cuuint32_t)B};
   const cuuint32_t estr[2] = {1u, 1u};
   return encode(reinterpret_cast<CUtensorMap*>(out128), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The same cache seen as [d / 64 column halves][rows][64 columns], so that ONE copy brings a whole tile of `tile_rows`
+// rows: its box is all halves x tile_rows x 64, which lands in shared memory half by half, each half [rows][128 bytes]
+// with the 128-byte swizzle - the layout the attend phase reads.  (An issue costs the issuing thread about 0.1 us.)
+static bool make_kv_tile_map(void* out128, void* base, int d, int tile_rows, unsigned long long rows) {
+  TensorMapEncodeFn encode = tensor_map_encoder();
+  if (!encode || d % 64 != 0) return false;
+  const cuuint64_t dims[3] = {64u, (cuuint64_t)rows, (cuuint64_t)(d / 64)};
+  const cuuint64_t strides[2] = {(cuuint64_t)d * 2, 128u};
+  const cuuint32_t box[3] = {64u, (cuuint32_t)tile_rows, (cuuint32_t)(d / 64)};
+  const cuuint32_t estr[3] = {1u, 1u, 1u};
+  return encode(reinterpret_cast<CUtensorMap*>(out128), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -203,8 +225,8 @@ extern "C" int spla_init_cache(const spla_config_t* config, const spla_buffers_t
   c->state_maps.valid = false;
   if (p.kv_bf16) {
     const unsigned long long rows = (unsigned long long)p.batch * p.Hkv * p.max_blocks * p.B;
-    c->maps.valid = make_kv_map(c->maps.k, b->k_cache, p.d, p.tile_rows, rows) &&
-                    make_kv_map(c->maps.v, b->v_cache, p.d, p.tile_rows, rows);
+    c->maps.valid = make_kv_tile_map(c->maps.k, b->k_cache, p.d, p.tile_rows, rows) &&
+                    make_kv_tile_map(c->maps.v, b->v_cache, p.d, p.tile_rows, rows);
     c->state_maps.valid = p.d == 128 && rows >= 64 && rows < (1ull << 31) && !(config->flags & SPLA_GENERAL_KERNELS) &&
                           make_kv_map(c->state_maps.k, b->k_cache, p.d, 64, rows) &&
                           make_kv_map(c->state_maps.v, b->v_cache, p.d, 64, rows);
