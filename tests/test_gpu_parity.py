@@ -272,6 +272,18 @@ def test_long_128k_full_size_with_the_group_size_of_the_papers_model():
     _stepped_full(w, n_units=2, check_steps={0, 5}, all_selections=True)
 
 
+def test_sequences_of_more_than_8192_blocks_on_the_cluster_kernels():
+    """More blocks than the selection's per-thread bit masks cover (128 x 64): the cluster kernels then select with the
+    histogram method over the whole key table.  One sequence, two KV heads, 9000 blocks of 64 tokens: index sets of both
+    units, outputs of one."""
+    w = synth.BY_NAME["long_128k"].scaled(batch=1, n_q_heads=4, n_kv_heads=2, context=64 * 9000 + 17, n_needles=6)
+    cache, K, V, lens = runner.build_cache(w, DEV)
+    gamma = synth.gamma(w).to(DEV)
+    q = synth.step_queries(w, 0, DEV)
+    _check_all_selections(w, cache, q, K, V, lens.cpu().numpy())
+    _check_units(w, cache, q, gamma, K, V, lens.cpu().numpy(), [(0, 1)], w.n_sink, w.n_local)
+
+
 def test_config4_very_long_1m_full():
     w = synth.CONFIGS[3]
     cache, K, V, lens = runner.build_cache(w, DEV)
