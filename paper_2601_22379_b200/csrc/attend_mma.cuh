@@ -97,7 +97,6 @@ __device__ __forceinline__ void attend_mma_body(const Params& p, const CUtensorM
                                                 unsigned char* recv_raw = nullptr, const float* obar_local = nullptr) {
   constexpr int KS = D / 16;        // k-steps of the two QK-type products
   constexpr int NT = D / 8;         // n-tiles of the PV-type product
-  constexpr int NH = D / 64;        // 64-column halves of a tile
   constexpr int NTHR = NG * kAttendThreads;
   constexpr int NWARP = NTHR / 32;
   __shared__ __align__(8) uint64_t full_own[kMaxSlots + 1];

@@ -108,10 +108,8 @@ struct Smem {
   static constexpr int kRingBytes = kStreamBytes > kMergeRecv + kMergeRecvBytes ? kStreamBytes : kMergeRecv + kMergeRecvBytes;
   static_assert(kStateScratch >= 68 * 1024, "the attend phase's tile ring must end below the o_bar scratch");
   // fixed region after the ring:
-  static constexpr int kPart = kRingBytes;                          // float [GP][2]  this CTA's (max, sum)
-  static constexpr int kAllPart = kPart + GP * 2 * 4;               // float [16][GP][2]
-  static constexpr int kLse = kAllPart + kMaxCluster * GP * 2 * 4;  // float [GP]
-  static constexpr int kWred = kLse + GP * 4;                       // float [NWP][GP][2]
+  static constexpr int kAllPart = kRingBytes;                       // float [16][GP][2]  every CTA's (max, sum exp) per head
+  static constexpr int kWred = kAllPart + kMaxCluster * GP * 2 * 4; // float [NWP][GP][2] the warps' partials
   static constexpr int kBars = (kWred + NWP * GP * 2 * 4 + 7) / 8 * 8;            // uint64: full / empty per stage, or one per slot
   static constexpr int kRingBars = kMma ? kSlots : 2 * kStages;
   static constexpr int kNumBars = kRingBars + 2;                    // ... and one each for the two exchanges of the cluster
@@ -184,9 +182,7 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
   const int u = blockIdx.y;
   const int b = u / p.Hkv, h = u % p.Hkv;
 
-  float* part_s = reinterpret_cast<float*>(smem_raw + SM::kPart);
   float* all_part = reinterpret_cast<float*>(smem_raw + SM::kAllPart);
-  float* lse_s = reinterpret_cast<float*>(smem_raw + SM::kLse);
   float* wred = reinterpret_cast<float*>(smem_raw + SM::kWred);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw + SM::kBars);
   uint64_t* empty = full + kStages;
