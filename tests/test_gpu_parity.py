@@ -272,6 +272,18 @@ def test_long_128k_full_size_with_the_group_size_of_the_papers_model():
     _stepped_full(w, n_units=2, check_steps={0, 5}, all_selections=True)
 
 
+@pytest.mark.parametrize("hq,flags", [(64, 0), (40, 0), (64, binding.SPLA_STATS_BF16), (24, 0)])
+def test_more_heads_per_group_than_ctas_per_unit(hq, flags):
+    """64 units share the device, so a unit gets a cluster of four CTAs or fewer; with groups of up to eight heads a CTA
+    then merges two heads (and computes o_bar of both), and the partial results of a head arrive in the second row of
+    its receive area."""
+    w = synth.BY_NAME["gqa_32k"].scaled(batch=8, n_q_heads=hq, n_kv_heads=8, context=64 * 44 + 9, n_needles=3)
+    cache, K, V, lens = runner.build_cache(w, DEV, flags=flags)
+    gamma = synth.gamma(w).to(DEV)
+    q = synth.step_queries(w, 0, DEV)
+    _check_units(w, cache, q, gamma, K, V, lens.cpu().numpy(), _sample_units(w, 6, 3), w.n_sink, w.n_local)
+
+
 def test_sequences_of_more_than_8192_blocks_on_the_cluster_kernels():
     """More blocks than the selection's per-thread bit masks cover (128 x 64): the cluster kernels then select with the
     histogram method over the whole key table.  One sequence, two KV heads, 9000 blocks of 64 tokens: index sets of both
