@@ -113,7 +113,11 @@ struct Smem {
   static constexpr int kBars = (kWred + NWP * GP * 2 * 4 + 7) / 8 * 8;            // uint64: full / empty per stage, or one per slot
   static constexpr int kRingBars = kMma ? kSlots : 2 * kStages;
   static constexpr int kNumBars = kRingBars + 2;                    // ... and one each for the two exchanges of the cluster
-  static constexpr int kEll = (kBars + kNumBars * 8 + 15) / 16 * 16;               // float [G][chunk]
+  // (tensor-core path with two column tiles: the B fragments of the variance dots, one word per lane and (tile, chunk,
+  // word), kept here instead of in 32 more registers per thread)
+  static constexpr int kBfrag = (kBars + kNumBars * 8 + 15) / 16 * 16;
+  static constexpr int kBfragBytes = (sizeof(ST) == 2 && GP > 4) ? 2 * (D * 2 / 64) * 4 * 32 * 4 : 0;
+  static constexpr int kEll = kBfrag + kBfragBytes;                                // float [G][chunk]
 };
 
 }  // namespace
@@ -231,7 +235,12 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
   constexpr int BW = MMAF ? 2 : 4;               // B-fragment words per chunk
   const int g8 = lane >> 2, t4 = lane & 3;
   constexpr int NT2 = GP > 4 ? 2 : 1;            // column tiles of eight: four heads x two query parts each
-  uint32_t bq[MMA ? NT2 : 1][MMA ? NJ : 1][BW], bv[MMA ? NT2 : 1][MMA ? NJ : 1][BW];
+  // 16-bit records with two column tiles: the variance fragments live in shared memory (the same for every warp).
+  // (With fp32 records they stay in registers although that costs the GP = 8 builds a few spilled words: fetching them
+  // per MMA made the already latency-bound slot loop 2 us slower per decode.)
+  constexpr bool BVS = MMA && NT2 == 2 && !MMAF;
+  uint32_t bq[MMA ? NT2 : 1][MMA ? NJ : 1][BW], bv[(MMA && !BVS) ? NT2 : 1][(MMA && !BVS) ? NJ : 1][BW];
+  uint32_t* bv_s = reinterpret_cast<uint32_t*>(smem_raw + SM::kBfrag);   // [NT2][NJ][BW][32 lanes]
   float qm[GP][VECW], qv[GP][VECW];
   if constexpr (MMA) {
 #pragma unroll
@@ -266,7 +275,8 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
 #pragma unroll
         for (int v = 0; v < BW; ++v) {
           bq[nt][j][v] = pack_bf16(qa[2 * v], qa[2 * v + 1]);
-          bv[nt][j][v] = pack_bf16(qb2[2 * v], qb2[2 * v + 1]);
+          if constexpr (BVS) { if (warp == 0) bv_s[((nt * NJ + j) * BW + v) * 32 + lane] = pack_bf16(qb2[2 * v], qb2[2 * v + 1]); }
+          else bv[nt][j][v] = pack_bf16(qb2[2 * v], qb2[2 * v + 1]);
         }
       }
     }
@@ -386,31 +396,41 @@ __device__ __forceinline__ void score_cluster_body(const Params& p, const void* 
 #pragma unroll
           for (int nt = 0; nt < NT2; ++nt) {
             mma_bf16(cm[nt], m0.x, m1.x, m0.y, m1.y, bq[nt][j][0], bq[nt][j][1]);
-            mma_bf16(cv[nt], v0.x, v1.x, v0.y, v1.y, bv[nt][j][0], bv[nt][j][1]);
+            uint32_t w0, w1, w2, w3;
+            if constexpr (BVS) {
+              const uint32_t* t = bv_s + ((nt * NJ + j) * BW) * 32 + lane;
+              w0 = t[0]; w1 = t[32]; w2 = t[64]; w3 = t[96];
+            } else {
+              w0 = bv[nt][j][0]; w1 = bv[nt][j][1]; w2 = bv[nt][j][2]; w3 = bv[nt][j][3];
+            }
+            mma_bf16(cv[nt], v0.x, v1.x, v0.y, v1.y, w0, w1);
             mma_bf16(cm[nt], m0.z, m1.z, m0.w, m1.w, bq[nt][j][2], bq[nt][j][3]);
-            mma_bf16(cv[nt], v0.z, v1.z, v0.w, v1.w, bv[nt][j][2], bv[nt][j][3]);
+            mma_bf16(cv[nt], v0.z, v1.z, v0.w, v1.w, w2, w3);
           }
         }
       }
       if constexpr (MMAF) {
         // fp32 records: this thread's four channels of the chunk, rows g8 and g8 + 8, are the A fragment of one k-step
         // (k indices 2 t4, 2 t4 + 1, 2 t4 + 8, 2 t4 + 9); first the mean, then the variance, each as two bf16 parts
-        auto split_mma = [&](const unsigned char* a_lo, const unsigned char* a_hi, float (&acc)[NT2][4], const uint32_t (&bf)[NT2][NJ][BW],
-                             int j) {
+        auto split_mma = [&](const unsigned char* a_lo, const unsigned char* a_hi, float (&acc)[NT2][4], const bool var, int j) {
           const float4 x0 = *reinterpret_cast<const float4*>(a_lo + j * 64), x1 = *reinterpret_cast<const float4*>(a_hi + j * 64);
           const uint32_t h0 = pack_bf16(x0.x, x0.y), h1 = pack_bf16(x1.x, x1.y), h2 = pack_bf16(x0.z, x0.w), h3 = pack_bf16(x1.z, x1.w);
           const uint32_t l0 = pack_bf16(x0.x - bf16_lo(h0), x0.y - bf16_hi(h0)), l1 = pack_bf16(x1.x - bf16_lo(h1), x1.y - bf16_hi(h1));
           const uint32_t l2 = pack_bf16(x0.z - bf16_lo(h2), x0.w - bf16_hi(h2)), l3 = pack_bf16(x1.z - bf16_lo(h3), x1.w - bf16_hi(h3));
 #pragma unroll
           for (int nt = 0; nt < NT2; ++nt) {
-            mma_bf16(acc[nt], h0, h1, h2, h3, bf[nt][j][0], bf[nt][j][1]);
-            mma_bf16(acc[nt], l0, l1, l2, l3, bf[nt][j][0], bf[nt][j][1]);
+            uint32_t w0, w1;
+            if (!var) { w0 = bq[nt][j][0]; w1 = bq[nt][j][1]; }
+            else if constexpr (BVS) { const uint32_t* t = bv_s + ((nt * NJ + j) * BW) * 32 + lane; w0 = t[0]; w1 = t[32]; }
+            else { w0 = bv[nt][j][0]; w1 = bv[nt][j][1]; }
+            mma_bf16(acc[nt], h0, h1, h2, h3, w0, w1);
+            mma_bf16(acc[nt], l0, l1, l2, l3, w0, w1);
           }
         };
 #pragma unroll
         for (int j = 0; j < NJ; ++j) {
-          split_mma(r0, r1, cm, bq, j);
-          split_mma(r0 + HALF, r1 + HALF, cv, bv, j);
+          split_mma(r0, r1, cm, false, j);
+          split_mma(r0 + HALF, r1 + HALF, cv, true, j);
         }
       }
       // columns 2 t4 and 2 t4 + 1 of column tile nt are the two query parts of head 4 nt + t4

@@ -58,7 +58,7 @@ __device__ __forceinline__ void lse_merge(float& m, float& s, float m2, float s2
 }  // namespace
 
 template <int D, int GP>
-__global__ void __launch_bounds__(kScoreThreads, GP >= 8 ? 1 : 2) score_select_kernel(const Params p, const void* __restrict__ q_raw,
+__global__ void __launch_bounds__(kScoreThreads, GP >= 2 ? 1 : 2) score_select_kernel(const Params p, const void* __restrict__ q_raw,
                                                                         int q_is_bf16, int* __restrict__ sel_user) {
   constexpr int VEC = D / 32;
   constexpr int NV = 2 * GP;             // values reduced per record: GP mean dots, GP variance dots
