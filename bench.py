@@ -35,7 +35,8 @@ L2_BYTES = 126 * 1024 * 1024
 GRAPH_STEPS = 64
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from ncu captures of this command
 # on a small case (one cache, a few launches), per workload
-NCU_TRAFFIC = {"long_128k": 106.4e6, "long_128k+windows(C=32,s=16)": 241.2e6, "long_128k+stats_bf16": 70.4e6, "gqa_32k": 72.6e6}
+NCU_TRAFFIC = {"long_128k": 106.4e6, "long_128k+windows(C=32,s=16)": 241.2e6, "long_128k+stats_bf16": 70.4e6, "gqa_32k": 72.6e6, "very_long_1m": 86.2e6,
+               "long_128k+n_q_heads=40": 108.2e6}
 
 
 # ------------------------------------------------------------------------------------------------------------
