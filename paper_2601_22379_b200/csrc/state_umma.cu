@@ -28,7 +28,7 @@
 // result does not depend on the order in which CTAs ran.  With a single split the CTA adds to S_bar itself.
 //
 // Every wait is an mbarrier poll with an iteration limit; on expiry the CTA raises its abort flag, all roles
-// leave their loops, tensor memory is released and status -3 is latched.  No multicast anywhere.
+// leave their loops, tensor memory is released and the time-out status is latched.  No multicast anywhere.
 #include <cuda.h>
 
 #include "spla_internal.h"
